@@ -1,0 +1,197 @@
+"""Seeded synthetic inputs for the CAST draft-and-verify step.
+
+This module only draws random tensors with the shapes, dtypes and value
+distributions of Llama/Qwen-style serving workloads and describes the five
+benchmark configurations.  It contains none of the method's arithmetic and
+imports neither the CUDA binding nor the CPU oracle; both sides of a parity
+test receive the very same tensors from here.
+
+The paper evaluates trained draft/target models on public datasets; the hot
+path only ever sees logits, Q, K, V tensors and a cost table, so seeded
+Gaussian tensors of the right shapes stand in for them.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, replace
+from typing import Dict, List, Optional, Tuple
+
+import numpy as np
+import torch
+
+BASE_SEED = 2510_26577 * 10
+
+_TORCH_DTYPE = {"f32": torch.float32, "bf16": torch.bfloat16}
+
+
+@dataclass(frozen=True)
+class Workload:
+    name: str
+    config_id: int
+    batch: int
+    kv_dtype: str  # dtype of Q, K, V and the attention output: "f32" | "bf16"
+    logit_dtype: str  # dtype of draft and target logits
+    q_heads: int
+    kv_heads: int
+    head_dim: int
+    kv_len_lo: int  # prefix lengths are integers uniform in [lo, hi]
+    kv_len_hi: int
+    page_size: int  # 0 = contiguous cache [B, Lmax, Hkv, D]
+    vocab: int
+    logit_std: float
+    depth: int  # H
+    top_k: int  # K
+    total_token: int  # m (root included)
+    cost_model: bool  # breadth pruning + dynamic rerank driven by the synthetic cost table
+    n_layers: int  # verification layers timed per step (distinct KV buffers)
+    max_tree: int = 128
+    tau: float = 1.4e-4  # slope of the synthetic cost table in B*n
+
+    @property
+    def seed(self) -> int:
+        return BASE_SEED + self.config_id
+
+    @property
+    def gqa(self) -> int:
+        return self.q_heads // self.kv_heads
+
+
+def _c3(batch: int, sub: int) -> Workload:
+    return Workload(f"c3_llama8b_b{batch}", 30 + sub, batch, "bf16", "f32", 32, 8, 128, 512, 4096, 16,
+                    128256, 3.0, 6, 8, 64, True, max(2, 64 // batch))
+
+
+def _c4(m: int, sub: int) -> Workload:
+    return Workload(f"c4_llama70b_n{m}", 40 + sub, 8, "bf16", "f32", 64, 8, 128, 4096, 4096, 0,
+                    32000, 3.0, 7, 8, m, False, 4)
+
+
+CONFIGS: Dict[str, Workload] = {
+    w.name: w
+    for w in [
+        Workload("c1_tiny", 1, 1, "f32", "f32", 8, 8, 64, 256, 256, 0, 4096, 2.0, 4, 4, 16, False, 2),
+        Workload("c2_llama8b", 2, 1, "bf16", "f32", 32, 8, 128, 2048, 2048, 0, 128256, 3.0, 6, 10, 60, False, 32),
+        _c3(1, 0), _c3(4, 1), _c3(16, 2), _c3(64, 3),
+        _c4(16, 0), _c4(32, 1), _c4(64, 2), _c4(128, 3),
+        Workload("c5_qwen_long", 5, 4, "bf16", "f32", 28, 4, 128, 32768, 32768, 16, 152064, 3.0, 8, 8, 96, False, 2),
+    ]
+}
+
+
+def shrink(w: Workload, **kw) -> Workload:
+    """A smaller variant of a configuration (for CPU-seconds parity cases)."""
+    return replace(w, **kw)
+
+
+def _gen(w: Workload, stream: int, device) -> torch.Generator:
+    g = torch.Generator(device=device)
+    g.manual_seed(w.seed * 1000 + stream)
+    return g
+
+
+def _randn(shape, std, dtype, gen, device) -> torch.Tensor:
+    x = torch.randn(shape, generator=gen, device=device, dtype=torch.float32)
+    if std != 1.0:
+        x = x * std
+    return x.to(_TORCH_DTYPE[dtype])
+
+
+def root_tokens(w: Workload, device="cpu") -> torch.Tensor:
+    g = torch.Generator(device="cpu")
+    g.manual_seed(w.seed * 1000 + 1)
+    return torch.randint(0, w.vocab, (w.batch,), generator=g, dtype=torch.int32).to(device)
+
+
+def kv_lengths(w: Workload, device="cpu") -> torch.Tensor:
+    g = torch.Generator(device="cpu")
+    g.manual_seed(w.seed * 1000 + 2)
+    return torch.randint(w.kv_len_lo, w.kv_len_hi + 1, (w.batch,), generator=g, dtype=torch.int32).to(device)
+
+
+def draft_logits(w: Workload, layer: int, device="cpu", peaked: bool = False) -> torch.Tensor:
+    """[B, W, V] draft logits of one layer (W = K rows per batch row).  With
+    `peaked`, one token per row is raised by 8 so that scores decay slowly with
+    depth, as those of a trained draft head do."""
+    g = _gen(w, 100 + layer, device)
+    x = _randn((w.batch, w.top_k, w.vocab), w.logit_std, "f32", g, device)
+    if peaked:
+        idx = torch.randint(0, w.vocab, (w.batch, w.top_k, 1), generator=g, device=device)
+        x.scatter_add_(2, idx, torch.full_like(idx, 8.0, dtype=torch.float32))
+    return x.to(_TORCH_DTYPE[w.logit_dtype])
+
+
+def query(w: Workload, layer: int, device="cpu") -> torch.Tensor:
+    return _randn((w.batch, w.max_tree, w.q_heads, w.head_dim), 1.0, w.kv_dtype, _gen(w, 300 + layer, device), device)
+
+
+def seq_capacity(w: Workload) -> int:
+    """Positions reserved per sequence: the longest prefix plus the tree."""
+    cap = w.kv_len_hi + w.max_tree
+    if w.page_size:
+        cap = (cap + w.page_size - 1) // w.page_size * w.page_size
+    return cap
+
+
+def page_table(w: Workload, device="cpu") -> Tuple[Optional[torch.Tensor], int]:
+    """(page_table [B, max_pages] int32, num_pages).  Pages are handed out in a
+    seeded random permutation of the pool, so sequences are not contiguous."""
+    if w.page_size == 0:
+        return None, 0
+    per_seq = seq_capacity(w) // w.page_size
+    num_pages = per_seq * w.batch
+    g = torch.Generator(device="cpu")
+    g.manual_seed(w.seed * 1000 + 3)
+    perm = torch.randperm(num_pages, generator=g, dtype=torch.int64).to(torch.int32)
+    return perm.view(w.batch, per_seq).contiguous().to(device), num_pages
+
+
+def kv_cache(w: Workload, layer: int, device="cpu") -> Tuple[torch.Tensor, torch.Tensor]:
+    """K and V ~ N(0,1) for one layer; the tree tokens' rows are part of it
+    (positions L_b .. L_b+N-1 are 'already written')."""
+    if w.page_size:
+        shape = (seq_capacity(w) // w.page_size * w.batch, w.page_size, w.kv_heads, w.head_dim)
+    else:
+        shape = (w.batch, seq_capacity(w), w.kv_heads, w.head_dim)
+    g = _gen(w, 500 + layer, device)
+    return _randn(shape, 1.0, w.kv_dtype, g, device), _randn(shape, 1.0, w.kv_dtype, g, device)
+
+
+def target_logits(w: Workload, device="cpu") -> torch.Tensor:
+    return _randn((w.batch, w.max_tree, w.vocab), w.logit_std, w.logit_dtype, _gen(w, 700, device), device)
+
+
+def plant_acceptance(w: Workload, logits: torch.Tensor, tokens, parent, n_tree, p_plant=0.7, p_geo=0.6) -> None:
+    """Make a random tree accept non-trivially: for every tree node that has
+    children, with probability p_plant raise the target logit of one child's
+    token (child rank geometric with parameter p_geo) to (row max + 1).  The
+    tree (tokens, parent, n_tree: host arrays) is an input of this recipe."""
+    rng = np.random.Generator(np.random.Philox(w.seed * 1000 + 900))
+    tokens = np.asarray(tokens)
+    parent = np.asarray(parent)
+    for b in range(tokens.shape[0]):
+        N = int(n_tree[b])
+        kids: Dict[int, List[int]] = {}
+        for t in range(1, N):
+            kids.setdefault(int(parent[b, t]), []).append(t)
+        for t in range(N):
+            draw = rng.random()
+            rank = int(rng.geometric(p_geo)) - 1
+            if t not in kids or draw >= p_plant:
+                continue
+            child = kids[t][min(rank, len(kids[t]) - 1)]
+            row = logits[b, t]
+            row[int(tokens[b, child])] = (row.float().max() + 1.0).to(row.dtype)
+
+
+def cost_table_arrays(w: Workload, B: int, L: int = 512, M: int = 64, Ntab: int = 128,
+                      stepped: bool = False) -> Tuple[int, int, int, np.ndarray, np.ndarray]:
+    """Synthetic stand-in for the profiled latency tables (the real ones need
+    the models): f_T(B, c, n) = 1 + 0.25*B*c/(64*4096) + tau*B*n on the grid
+    c = g*L, n = 1..Ntab, and f_D = 0.05 * f_T; strictly increasing in n.  The
+    `stepped` variant adds 0.02*ceil(B*n/64) (tile quantisation)."""
+    c = (np.arange(1, M + 1, dtype=np.float64) * L)[:, None]
+    n = np.arange(1, Ntab + 1, dtype=np.float64)[None, :]
+    fT = 1.0 + 0.25 * (B * c) / (64.0 * 4096.0) + w.tau * B * n
+    if stepped:
+        fT = fT + 0.02 * np.ceil(B * n / 64.0)
+    fD = 0.05 * fT
+    return L, M, Ntab, fT, fD
