@@ -1,0 +1,235 @@
+/*
+ * cast.h - C-ABI of the B200-native CAST hot path.
+ *
+ * One batched draft-and-verify step of cost-aware tree speculative decoding
+ * (paper: "Inference-Cost-Aware Dynamic Tree Construction for Efficient
+ * Inference in Large Language Models"):
+ *
+ *   cast_step_begin      root node, value 1                (Sec. "Tree Expansion Phase")
+ *   cast_tree_expand     one draft layer: top-K children, path values,
+ *                        breadth pruning (Eq. 1, Eq. 2, Algorithm 1),
+ *                        depth pruning (Sec. "Dynamic Expansion Stage")
+ *   cast_select_nodes    dynamic rerank (Sec. "Dynamic Reranking Stage"),
+ *                        linearisation + ancestor mask (Sec. "Tree Reranking Phase")
+ *   cast_tree_attention  verification attention under that mask
+ *   cast_accept          greedy acceptance (Sec. "Speculative Decoding", T = 0)
+ *   cast_compact_kv      accepted KV rows made contiguous
+ *
+ * Conventions
+ *  - Plain C. Every tensor pointer is a DEVICE pointer owned by the caller
+ *    unless its comment says "host". The library owns only what cast_create
+ *    allocates (freed by cast_destroy).
+ *  - `stream` is a cudaStream_t passed as void*. Compute calls only enqueue
+ *    work: they never synchronise the host. Tree sizes (n_i, go/no-go, N) are
+ *    decided on the device and stay there.
+ *  - Compute calls allocate nothing, with one exception: cast_tree_attention
+ *    grows a context-owned workspace the first time it sees a larger shape
+ *    (do that call once before capturing a CUDA graph).
+ *  - The return value reports errors the host can see (bad arguments, caps).
+ *    Errors only the device can see (non-finite logits, a malformed tree, a
+ *    page index out of range) are written to a device status word; read it with
+ *    cast_poll_status, which synchronises `stream`.
+ *  - A context must not be used from two streams at once.
+ *  - Row-major layouts, innermost index last, written as [d0, d1, ...].
+ */
+#ifndef CAST_H
+#define CAST_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  CAST_OK = 0,
+  CAST_ERR_INVALID_ARG = 1, /* null pointer, negative size, wrong call order          */
+  CAST_ERR_SHAPE = 2,       /* head/group/dimension combination the kernels do not take */
+  CAST_ERR_CAPACITY = 3,    /* a cap of this build or of the context is exceeded       */
+  CAST_ERR_DTYPE = 4,
+  CAST_ERR_COST_TABLE = 5,  /* no table for this batch size, or f not strictly increasing in n */
+  CAST_ERR_BAD_TREE = 6,    /* device: parent[t] >= t, depth beyond max_depth, index out of range */
+  CAST_ERR_BAD_PAGE = 7,    /* device: page-table entry out of range                     */
+  CAST_ERR_NONFINITE = 8,   /* device: NaN or +inf logit, or a row without K finite logits */
+  CAST_ERR_TIMEOUT = 9,     /* device: a bounded wait ran out                            */
+  CAST_ERR_CUDA = 10        /* a CUDA runtime call failed                                */
+} cast_status;
+
+typedef enum { CAST_F32 = 0, CAST_BF16 = 1 } cast_dtype;
+
+/* Caps of this build. */
+#define CAST_MAX_TOP_K 16
+#define CAST_MAX_WIDTH 16
+#define CAST_MAX_DEPTH 16
+#define CAST_MAX_TREE 128
+#define CAST_MAX_BATCH 64
+
+typedef struct cast_ctx cast_ctx;
+
+#if defined(__GNUC__)
+#define CAST_API __attribute__((visibility("default")))
+#else
+#define CAST_API
+#endif
+
+/*
+ * Hyper-parameters (paper notation in brackets).
+ *   top_k [K]        children generated per retained node, 1..CAST_MAX_TOP_K
+ *   max_depth [H]    draft layers below the root = number of cast_tree_expand calls
+ *   max_width [W]    most nodes retained per layer (0 means K); Algorithm 1 for
+ *                    layer i runs on the first min(N_i, W, Ntab) sorted candidates
+ *   max_tree [Ncap]  row stride of every per-tree-token array, <= CAST_MAX_TREE
+ *   total_token [m]  cap on verified tokens, root included, <= max_tree
+ *   C1, C2, C3       thresholds of breadth pruning, depth pruning, rerank
+ *   fifo_len [R]     length of the depth-pruning buffers A_i
+ *   enable_bp/dp/dr  breadth pruning / depth pruning / dynamic rerank. All three
+ *                    off gives the fixed EAGLE-2 shape: n_i = min(K, N_i), all H
+ *                    layers, N = min(pool, m).
+ *   pool_mode        0: rerank over root + every generated candidate;
+ *                    1: rerank over root + retained nodes only (N <= sum n_i)
+ *   ctx_base_mode    0: context of Eq. 2 is sum_{j<i} n_j; 1: add n_0
+ */
+typedef struct {
+  double C1, C2, C3;
+  int32_t max_batch, vocab, top_k, max_depth, max_width, max_tree, total_token;
+  int32_t fifo_len, enable_bp, enable_dp, enable_dr, pool_mode, ctx_base_mode;
+  int32_t reserved;
+} cast_config;
+
+/* Allocates the context and its device scratch on the current device.
+ * Errors: INVALID_ARG, CAPACITY (a field beyond the caps above), CUDA. */
+CAST_API cast_status cast_create(const cast_config* cfg, cast_ctx** out);
+CAST_API cast_status cast_destroy(cast_ctx* ctx);
+CAST_API const char* cast_status_string(cast_status s);
+
+/*
+ * Cost tables S_T(B), S_D(B) (Sec. "Method"): f(B, c, n) for c = g*L, g = 1..M and
+ * n = 1..Ntab, as host arrays [M][Ntab] of doubles (copied; one pair per batch
+ * size B, replacing an earlier pair for the same B). Synchronises the device.
+ * Errors: COST_TABLE if a value is not finite and positive or a row is not
+ * strictly increasing in n (precondition of Algorithm 1).
+ */
+CAST_API cast_status cast_set_cost_tables(cast_ctx* ctx, int B, int L, int M, int Ntab,
+                                 const double* fT /* host */, const double* fD /* host */);
+
+/*
+ * Depth-pruning state (buffers A_1..A_{H-1}): the only state that outlives a
+ * step. Blob layout: int32 H-1, int32 R, then for each buffer int32 count and R
+ * doubles, oldest first. Call with blob = NULL to get the size. Both calls
+ * synchronise the device.
+ */
+CAST_API cast_status cast_state_export(cast_ctx* ctx, void* blob /* host */, size_t* bytes);
+CAST_API cast_status cast_state_import(cast_ctx* ctx, const void* blob /* host */, size_t bytes);
+
+/*
+ * Begin a step for B sequences: the pool of every row becomes {root}, root
+ * value 1 (log-value 0), depth 0. root_token [B] int32: last accepted token.
+ * kv_len [B] int32: prefix lengths; the padded context n_0 is their maximum.
+ * Errors: CAPACITY (B > max_batch), COST_TABLE (a switch is on and B has no table).
+ */
+CAST_API cast_status cast_step_begin(cast_ctx* ctx, int B, const int32_t* root_token, const int32_t* kv_len,
+                            void* stream);
+
+/*
+ * Expansion layer `layer` (1..H, in order). draft_logits [B, W, V]: row r of
+ * sequence b is the draft distribution after the rank-r node retained by the
+ * previous layer (layer 1: row 0 = root); rows >= n_{layer-1} are not read.
+ * Children: the K tokens first in (logit descending, token id ascending); child
+ * log-value = parent log-value + log-softmax. Then per sequence the N_i
+ * candidates are sorted by (value desc, token asc, creation order), u (Eq. 1)
+ * and c (Eq. 2) are formed, n_i = Algorithm 1(u, c, C1), and the depth test
+ * Avg(A_i) * u_{n_i} / c_{n_i} >= C2 decides whether a further layer follows.
+ * Outputs (device): next_tokens [B, W], next_parent_row [B, W] (which logits row
+ * of this layer produced each retained node), -1 beyond n_i; next_count [1]:
+ * n_i if a further layer follows, else 0 (layer H, or the depth test failed).
+ * Once a layer was refused, later calls of the step only write next_count = 0.
+ * -inf logits are legal (probability 0). Errors: INVALID_ARG when `layer` is
+ * not the next layer of the step; device: NONFINITE.
+ */
+CAST_API cast_status cast_tree_expand(cast_ctx* ctx, int layer, const void* draft_logits, cast_dtype dtype,
+                             int32_t* next_tokens, int32_t* next_parent_row, int32_t* next_count,
+                             void* stream);
+
+/*
+ * Rerank and linearise. Pool nodes are sorted per sequence by (value desc,
+ * depth asc, token asc, creation order); with v(s) the batch mean of the
+ * rank-s values, u_k = sum_{s<=k} v(s), c_k = S_T[select(n_0)][k] / S_T[select(n_0)][1],
+ * N = Algorithm 1(u, c, C3) capped by min(pool, m) (N = that cap if enable_dr = 0).
+ * Each sequence keeps its own N best nodes, ordered by creation (root first,
+ * parents before children). Outputs, all [B, Ncap] unless noted, entries >= N
+ * are -1 (0 for anc_mask and scores):
+ *   tokens, parent (linear index, -1 for the root), depth, pool_idx (int32);
+ *   anc_mask [B, Ncap, ceil(Ncap/32)] uint32: bit j of row t set iff j is t or
+ *   an ancestor of t; scores (double log-values; may be NULL); n_tree [B] int32.
+ */
+CAST_API cast_status cast_select_nodes(cast_ctx* ctx, int32_t* tokens, int32_t* parent, int32_t* depth,
+                              uint32_t* anc_mask, int32_t* pool_idx, double* scores, int32_t* n_tree,
+                              void* stream);
+
+/*
+ * One layer of verification attention (the mask of Sec. "Tree Reranking Phase"):
+ * out[b,t,h] = softmax over {prefix positions 0..kv_len[b]-1} U {tree positions
+ * kv_len[b]+j : bit j of anc_mask[b,t]} of (q . k) * scale, times v, for
+ * t < n_tree[b]; rows t >= n_tree[b] are written as zeros.
+ *   q, out        [B, Ncap, Hq, D], dtype `dtype`
+ *   k_cache, v_cache  paged: [num_pages, page_size, Hkv, D]; the cache rows of
+ *                 the tree tokens are already stored at positions kv_len[b]+j.
+ *                 page_size = 0: contiguous [B, seq_capacity, Hkv, D].
+ *   page_table    [B, seq_capacity] int32 page ids in [0, num_pages) (paged only;
+ *                 seq_capacity is then the number of entries per sequence)
+ *   scale         0 selects 1/sqrt(D)
+ * Accumulation is fp32. Needs Hq % Hkv == 0, D in {64, 128}, 16-byte aligned
+ * pointers. Device errors: BAD_PAGE.
+ */
+CAST_API cast_status cast_tree_attention(cast_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
+                                cast_dtype dtype, int B, int Hq, int Hkv, int D, int page_size,
+                                const int32_t* page_table, int seq_capacity, int num_pages,
+                                const int32_t* kv_len, const uint32_t* anc_mask, const int32_t* n_tree,
+                                float scale, void* out, void* stream);
+
+/*
+ * Greedy acceptance: g[t] = argmax of target_logits[b,t,:] (ties: lower id).
+ * Starting at the root, step to the child c of the current node with
+ * tokens[c] == g[current] (lowest index if several) until there is none.
+ *   target_logits [B, Ncap, V]; tokens, parent [B, Ncap]; n_tree [B]
+ *   accept_len [B]   drafts accepted (root excluded)
+ *   accept_path [B, H+1]  linear tree indices, root first, -1 padded
+ *   bonus_token [B]  g at the last accepted node
+ * `depth` and `anc_mask` may be NULL (not needed by the walk).
+ * Device errors: BAD_TREE (parent[t] >= t or a path longer than H+1).
+ */
+CAST_API cast_status cast_accept(cast_ctx* ctx, const void* target_logits, cast_dtype dtype, int B,
+                        const int32_t* tokens, const int32_t* parent, const int32_t* depth,
+                        const uint32_t* anc_mask, const int32_t* n_tree, int32_t* accept_len,
+                        int32_t* accept_path, int32_t* bonus_token, void* stream);
+
+/*
+ * KV compaction (not in the paper; the plain gather): for every layer, kv-head
+ * and j = 0..accept_len[b], cache row kv_len[b]+j := old row kv_len[b]+accept_path[b,j],
+ * K and V, with out-of-place semantics; then kv_len[b] += accept_len[b] + 1.
+ * Layer l of a cache starts layer_stride_bytes * l after the base pointer.
+ * Cache layout, page_size, page_table, seq_capacity, num_pages as for
+ * cast_tree_attention. Device errors: BAD_PAGE (also for a path entry < 0).
+ */
+CAST_API cast_status cast_compact_kv(cast_ctx* ctx, void* k_cache, void* v_cache, cast_dtype dtype, int B,
+                            int n_layers, size_t layer_stride_bytes, int Hkv, int D, int page_size,
+                            const int32_t* page_table, int seq_capacity, int num_pages,
+                            const int32_t* accept_path, const int32_t* accept_len,
+                            int32_t* kv_len /* in/out */, void* stream);
+
+/* Synchronises `stream`, returns the device status word and clears it.
+ * detail: an index that identifies the offending row/entry (meaning per status). */
+CAST_API cast_status cast_poll_status(cast_ctx* ctx, void* stream, cast_status* device_status, int32_t* detail);
+
+/*
+ * Synchronises `stream` and copies the step counters to host int32 info[4 + H]:
+ * info[0] layers generated, info[1] pool size, info[2] n_0, info[3] N of the
+ * last cast_select_nodes (0 before), info[4 + i - 1] = n_i.
+ */
+CAST_API cast_status cast_step_info(cast_ctx* ctx, void* stream, int32_t* info /* host */);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CAST_H */

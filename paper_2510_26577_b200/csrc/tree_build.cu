@@ -1,0 +1,765 @@
+// Draft-tree construction: cast_step_begin, cast_tree_expand, cast_select_nodes.
+//
+// cast_tree_expand is ONE kernel per draft layer:
+//   1. vocabulary sweep - every logits row is cut into chunks, one CTA per chunk: streaming
+//      16-byte loads, online max / sum-exp, and an exact top-K by threshold filtering
+//      (the K-th largest of the per-thread maxima bounds the K-th largest of the chunk);
+//   2. the last CTA to finish a row merges the chunk partials (log-sum-exp in fp64, exact
+//      top-K of the chunk winners) and appends the K children to the node pool;
+//   3. the last CTA to finish the layer sorts each sequence's candidates, forms the
+//      utility u (Eq. 1) and the cost c (Eq. 2), runs Algorithm 1 (breadth pruning), the
+//      depth-pruning test and the FIFO update, and publishes the retained nodes.
+// "Last CTA" is decided by an atomic ticket; nothing spins.
+#include <math.h>
+
+#include "cast_internal.h"
+
+using namespace cast;
+
+namespace {
+
+// ------------------------------------------------------------------ step begin
+__global__ void step_begin_kernel(DevState* st, int B, int P, int W, const int32_t* root_token,
+                                  const int32_t* kv_len, double* pool_score, int32_t* pool_token,
+                                  int32_t* pool_parent, int32_t* pool_depth, uint8_t* pool_kept,
+                                  int32_t* retained, int32_t* row_ticket, int32_t* layer_ticket, int n_rows) {
+  __shared__ int s_max;
+  const int tid = threadIdx.x;
+  if (tid == 0) s_max = 0;
+  __syncthreads();
+  for (int b = tid; b < B; b += blockDim.x) {
+    const size_t o = (size_t)b * P;
+    pool_score[o] = 0.0;  // root: value 1
+    pool_token[o] = root_token[b];
+    pool_parent[o] = -1;
+    pool_depth[o] = 0;
+    pool_kept[o] = 1;
+    retained[b * W] = 0;
+    atomicMax(&s_max, kv_len[b]);
+  }
+  for (int i = tid; i < n_rows; i += blockDim.x) row_ticket[i] = 0;
+  __syncthreads();
+  if (tid == 0) {
+    *layer_ticket = 0;
+    st->B = B;
+    st->pool_size = 1;
+    st->ctx_sum = 0;
+    st->n0 = s_max;
+    st->layers_done = 0;
+    st->n_tree = 0;
+    st->kept_total = 1;
+    st->u_last = 1.0;
+    st->n_hist[0] = 1;
+    for (int i = 1; i <= CAST_MAX_DEPTH; ++i) st->n_hist[i] = 0;
+    for (int i = 0; i < CAST_MAX_DEPTH + 2; ++i) st->rows[i] = 0;
+    st->rows[1] = 1;
+  }
+}
+
+// ------------------------------------------------------------------ expand
+struct ExpandParams {
+  const void* logits;
+  int V, K, W, H, P, layer, nchunks, chunk_elems;
+  double* pool_score;
+  int32_t* pool_token;
+  int32_t* pool_parent;
+  int32_t* pool_depth;
+  uint8_t* pool_kept;
+  int32_t* retained;
+  DevState* st;
+  unsigned long long* part_keys;
+  float* part_max;
+  double* part_sum;
+  int32_t* row_ticket;
+  int32_t* layer_ticket;
+  double* fifo_vals;
+  int32_t* fifo_cnt;
+  int R;
+  DevTable tab;
+  double C1, C2;
+  int enable_bp, enable_dp, ctx_base_mode;
+  int32_t* next_tokens;
+  int32_t* next_parent_row;
+  int32_t* next_count;
+};
+
+template <typename T> struct Vec;
+template <> struct Vec<float> {
+  static constexpr int N = 4;
+  static __device__ __forceinline__ void load(const float* p, float* out) {
+    const float4 a = __ldcs(reinterpret_cast<const float4*>(p));
+    out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w;
+  }
+};
+template <> struct Vec<__nv_bfloat16> {
+  static constexpr int N = 8;
+  static __device__ __forceinline__ void load(const __nv_bfloat16* p, float* out) {
+    const uint4 a = __ldcs(reinterpret_cast<const uint4*>(p));
+    const uint32_t w[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {  // bf16 -> fp32 is a 16-bit shift
+      out[2 * i] = __uint_as_float(w[i] << 16);
+      out[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  }
+};
+
+// Exact top-K (descending) of n distinct keys in shared memory, written to out[0..K).
+// Missing entries (n < K) become 0. All threads of the CTA call it; `keys` is clobbered
+// when n > 512.
+__device__ void block_top_k(unsigned long long* keys, int n, int K, unsigned long long* out) {
+  const int tid = threadIdx.x, nt = blockDim.x;
+  if (tid < K) out[tid] = 0ull;
+  __syncthreads();
+  if (n <= 512) {  // rank by counting: keys are distinct, so ranks are too
+    for (int i = tid; i < n; i += nt) {
+      const unsigned long long k = keys[i];
+      int rank = 0;
+      for (int j = 0; j < n; ++j) rank += (keys[j] > k);
+      if (rank < K) out[rank] = k;
+    }
+  } else {  // bitonic sort, descending, on the next power of two
+    int n2 = 1024;
+    while (n2 < n) n2 <<= 1;
+    for (int i = n + tid; i < n2; i += nt) keys[i] = 0ull;
+    __syncthreads();
+    for (int k = 2; k <= n2; k <<= 1)
+      for (int j = k >> 1; j > 0; j >>= 1) {
+        for (int i = tid; i < n2; i += nt) {
+          const int l = i ^ j;
+          if (l > i) {
+            const unsigned long long a = keys[i], b = keys[l];
+            const bool desc = ((i & k) == 0);
+            if (desc ? (a < b) : (a > b)) { keys[i] = b; keys[l] = a; }
+          }
+        }
+        __syncthreads();
+      }
+    if (tid < K) out[tid] = keys[tid];
+  }
+  __syncthreads();
+}
+
+// Layer tail (Eq. 1, Eq. 2, Algorithm 1, depth pruning), run by the last CTA of the layer.
+__device__ void layer_tail(const ExpandParams& p, int B, int n_prev, int base, unsigned char* scratch,
+                           int* sorted /* [CAST_MAX_BATCH * CAST_MAX_WIDTH] */) {
+  __shared__ double vbar[CAST_MAX_WIDTH], u[CAST_MAX_WIDTH], c[CAST_MAX_WIDTH];
+  __shared__ int mark[CAST_MAX_WIDTH];
+  __shared__ int s_ni, s_next;
+  const int tid = threadIdx.x, nt = blockDim.x;
+  DevState* st = p.st;
+  const int K = p.K, W = p.W, P = p.P;
+  const int Ni = n_prev * K;
+  const bool need_cost = p.enable_bp || p.enable_dp;
+  int n = Ni < W ? Ni : W;
+  if (need_cost && p.tab.Ntab < n) n = p.tab.Ntab;
+
+  double* sc = reinterpret_cast<double*>(scratch);              // 2048 scores
+  int* tk = reinterpret_cast<int*>(scratch + 16384);            // 2048 tokens
+  double* vs = reinterpret_cast<double*>(scratch + 24576);      // [B][CAST_MAX_WIDTH] sorted values
+  const int group = 2048 / Ni;                                  // sequences sorted per pass
+  for (int b0 = 0; b0 < B; b0 += group) {
+    const int nb = (B - b0) < group ? (B - b0) : group;
+    for (int i = tid; i < nb * Ni; i += nt) {
+      const size_t o = (size_t)(b0 + i / Ni) * P + base + (i % Ni);
+      sc[i] = __ldcg(p.pool_score + o);
+      tk[i] = __ldcg(p.pool_token + o);
+    }
+    __syncthreads();
+    // rank by counting under the order (value desc, token asc, creation order)
+    for (int i = tid; i < nb * Ni; i += nt) {
+      const int bl = i / Ni, ci = i % Ni;
+      const double s = sc[i];
+      const int t = tk[i];
+      const double* ss = sc + bl * Ni;
+      const int* tt = tk + bl * Ni;
+      int rank = 0;
+      for (int j = 0; j < Ni; ++j) {
+        const double sj = ss[j];
+        rank += (sj > s) || (sj == s && (tt[j] < t || (tt[j] == t && j < ci)));
+      }
+      if (rank < n) {
+        sorted[(b0 + bl) * CAST_MAX_WIDTH + rank] = base + ci;
+        vs[(b0 + bl) * CAST_MAX_WIDTH + rank] = exp(s);
+      }
+    }
+    __syncthreads();
+  }
+  // Eq. 1: batch mean of the rank-wise values, then prefix sums
+  if (tid < n) {
+    double a = 0.0;
+    for (int b = 0; b < B; ++b) a += vs[b * CAST_MAX_WIDTH + tid];
+    vbar[tid] = a / (double)B;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    double a = 0.0;
+    for (int k = 0; k < n; ++k) { a += vbar[k]; u[k] = a; }
+  }
+  // Eq. 2: draft cost of k nodes relative to one target token, at context select(sum n_j)
+  if (need_cost && tid < n) {
+    const int ctx = st->ctx_sum + (p.ctx_base_mode ? st->n0 : 0);
+    const int g = select_grid(ctx, p.tab.L, p.tab.M);
+    c[tid] = p.tab.fD[(size_t)(g - 1) * p.tab.Ntab + tid] / p.tab.fT[(size_t)(g - 1) * p.tab.Ntab];
+  }
+  __syncthreads();
+  // Algorithm 1: mark[j] survives iff no earlier i has (u_j - u_i) < C1 (c_j - c_i)
+  if (tid < n) {
+    int ok = 1;
+    if (p.enable_bp)
+      for (int i = 0; i < tid; ++i)
+        if ((u[tid] - u[i]) < p.C1 * (c[tid] - c[i])) ok = 0;
+    mark[tid] = ok;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int n_i = 1;
+    for (int j = 0; j < n; ++j)
+      if (mark[j]) n_i = j + 1;
+    bool go = true;
+    if (p.enable_dp) {
+      if (p.layer >= 2) {  // gain ratio of the previous layer goes into its buffer, FIFO
+        const double phi = u[n_i - 1] / st->u_last;
+        double* A = p.fifo_vals + (size_t)(p.layer - 2) * p.R;
+        int cnt = p.fifo_cnt[p.layer - 2];
+        if (cnt < p.R) {
+          A[cnt++] = phi;
+        } else {
+          for (int k = 1; k < p.R; ++k) A[k - 1] = A[k];
+          A[p.R - 1] = phi;
+        }
+        p.fifo_cnt[p.layer - 2] = cnt;
+      }
+      if (p.layer < p.H) {  // generate layer i+1 only if Avg(A_i) * u / c >= C2
+        const double* A = p.fifo_vals + (size_t)(p.layer - 1) * p.R;
+        const int cnt = p.fifo_cnt[p.layer - 1];
+        double a = 0.0;
+        for (int k = 0; k < cnt; ++k) a += A[k];
+        const double alpha = a / (double)cnt;
+        go = (alpha * u[n_i - 1] / c[n_i - 1]) >= p.C2;
+      }
+    }
+    s_ni = n_i;
+    s_next = (p.layer < p.H && go) ? n_i : 0;
+  }
+  __syncthreads();
+  const int n_i = s_ni;
+  for (int i = tid; i < B * W; i += nt) {
+    const int b = i / W, s = i % W;
+    int tok = -1, prow = -1;
+    if (s < n_i) {
+      const int idx = sorted[b * CAST_MAX_WIDTH + s];
+      tok = __ldcg(p.pool_token + (size_t)b * P + idx);
+      prow = (idx - base) / K;
+      p.retained[b * W + s] = idx;
+      p.pool_kept[(size_t)b * P + idx] = 1;
+    }
+    p.next_tokens[i] = tok;
+    p.next_parent_row[i] = prow;
+  }
+  if (tid == 0) {
+    st->rows[p.layer + 1] = s_next;
+    st->n_hist[p.layer] = n_i;
+    st->ctx_sum += n_i;
+    st->kept_total += n_i;
+    st->u_last = u[n_i - 1];
+    st->pool_size = base + Ni;
+    st->layers_done = p.layer;
+    *p.next_count = s_next;
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParams p) {
+  __shared__ __align__(16) unsigned long long cand[kCandCap];
+  __shared__ unsigned long long topk[CAST_MAX_TOP_K];
+  __shared__ unsigned long long warp_thr[kSweepThreads / 32];
+  __shared__ float red_f[kSweepThreads / 32];
+  __shared__ double red_d[kSweepThreads / 32];
+  __shared__ int sorted[CAST_MAX_BATCH * CAST_MAX_WIDTH];
+  __shared__ int cand_cnt, s_flag;
+  __shared__ double s_lse;
+
+  const int chunk = blockIdx.x, r = blockIdx.y, b = blockIdx.z, B = gridDim.z;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  DevState* st = p.st;
+  const int n_prev = st->rows[p.layer];
+  if (n_prev == 0) {
+    if (chunk == 0 && r == 0 && b == 0 && tid == 0) *p.next_count = 0;
+    return;
+  }
+  if (r >= n_prev) return;
+  const int K = p.K;
+  const int row = b * p.W + r;
+  const T* x = reinterpret_cast<const T*>(p.logits) + (size_t)row * p.V;
+  const int begin = chunk * p.chunk_elems;
+  const int end = min(begin + p.chunk_elems, p.V);
+  constexpr int VEC = Vec<T>::N;
+  constexpr int NV = kSweepEpt / VEC;
+  const bool aligned = (reinterpret_cast<uintptr_t>(x) & 15) == 0;  // chunk starts are multiples of 8 logits
+
+  float m_run = -INFINITY, s_run = 0.f;
+  unsigned long long thr_prev = 0ull;
+  if (tid == 0) cand_cnt = 0;
+  __syncthreads();
+
+  for (int sub = begin; sub < end; sub += kSweepSub) {
+    float xv[kSweepEpt];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+      const int idx = sub + (v * kSweepThreads + tid) * VEC;
+      if (aligned && idx + VEC <= end) {
+        Vec<T>::load(x + idx, xv + v * VEC);
+      } else {
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) xv[v * VEC + e] = (idx + e < end) ? to_float(x[idx + e]) : -INFINITY;
+      }
+    }
+    // per-thread maximum (first maximum = lowest token id) and online sum-exp
+    float tmax = -INFINITY;
+    int targ = -1;
+#pragma unroll
+    for (int i = 0; i < kSweepEpt; ++i)
+      if (xv[i] > tmax) {
+        tmax = xv[i];
+        targ = sub + ((i / VEC) * kSweepThreads + tid) * VEC + (i % VEC);
+      }
+    if (tmax > m_run) {
+      s_run *= expf(m_run - tmax);
+      m_run = tmax;
+    }
+    if (m_run > -INFINITY) {
+#pragma unroll
+      for (int i = 0; i < kSweepEpt; ++i) s_run += expf(xv[i] - m_run);
+    }
+    // K-th largest of the warp's 32 thread maxima (bitonic sort over lanes, descending)
+    unsigned long long key = targ >= 0 ? make_key(tmax, targ) : 0ull;
+#pragma unroll
+    for (int k = 2; k <= 32; k <<= 1)
+#pragma unroll
+      for (int j = k >> 1; j > 0; j >>= 1) {
+        const unsigned long long o = __shfl_xor_sync(0xffffffffu, key, j);
+        const bool desc = ((lane & k) == 0), low = ((lane & j) == 0);
+        key = (desc == low) ? (key > o ? key : o) : (key < o ? key : o);
+      }
+    const unsigned long long wk = __shfl_sync(0xffffffffu, key, K - 1);
+    if (lane == 0) warp_thr[warp] = wk;
+    __syncthreads();
+    // at least K logits of this pass are >= each warp's K-th maximum, and at least K seen so
+    // far are >= thr_prev: nothing below the largest of these bounds can be in the top K.
+    unsigned long long thr = thr_prev;
+#pragma unroll
+    for (int w = 0; w < kSweepThreads / 32; ++w) thr = warp_thr[w] > thr ? warp_thr[w] : thr;
+    const float thr_val = thr ? key_value(thr) : -INFINITY;
+#pragma unroll
+    for (int i = 0; i < kSweepEpt; ++i) {
+      if (xv[i] >= thr_val) {
+        const int id = sub + ((i / VEC) * kSweepThreads + tid) * VEC + (i % VEC);
+        if (id < end) {
+          const unsigned long long k2 = make_key(xv[i], id);
+          if (k2 >= thr) {
+            const int pos = atomicAdd(&cand_cnt, 1);
+            if (pos < kCandCap) cand[pos] = k2;
+          }
+        }
+      }
+    }
+    __syncthreads();
+    const int n = cand_cnt < kCandCap ? cand_cnt : kCandCap;
+    if (n > K) {
+      block_top_k(cand, n, K, topk);
+      if (tid < K) cand[tid] = topk[tid];
+      thr_prev = topk[K - 1];
+      if (tid == 0) cand_cnt = K;
+    } else {
+      thr_prev = 0ull;
+    }
+    __syncthreads();
+  }
+
+  // chunk partials: top-K keys, maximum, sum of exp(x - maximum) in fp64
+  {
+    const int have = cand_cnt;
+    if (tid < K) p.part_keys[((size_t)row * kSweepMaxChunks + chunk) * CAST_MAX_TOP_K + tid] = tid < have ? cand[tid] : 0ull;
+    float M = m_run;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    if (lane == 0) red_f[warp] = M;
+    __syncthreads();
+    M = red_f[0];
+#pragma unroll
+    for (int w = 1; w < kSweepThreads / 32; ++w) M = fmaxf(M, red_f[w]);
+    double sd = (m_run > -INFINITY) ? (double)s_run * (double)expf(m_run - M) : 0.0;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sd += __shfl_xor_sync(0xffffffffu, sd, o);
+    if (lane == 0) red_d[warp] = sd;
+    __syncthreads();
+    if (tid == 0) {
+      double S = 0.0;
+      for (int w = 0; w < kSweepThreads / 32; ++w) S += red_d[w];
+      p.part_max[(size_t)row * kSweepMaxChunks + chunk] = M;
+      p.part_sum[(size_t)row * kSweepMaxChunks + chunk] = S;
+    }
+  }
+
+  // ---- row merge by the last CTA of this logits row
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const int t = p.nchunks > 1 ? atomicAdd(&p.row_ticket[row], 1) : 0;
+    s_flag = (t == p.nchunks - 1);
+  }
+  __syncthreads();
+  if (!s_flag) return;
+  __threadfence();
+  if (tid == 0) p.row_ticket[row] = 0;
+  const int nk = p.nchunks * K;
+  for (int i = tid; i < nk; i += kSweepThreads)
+    cand[i] = __ldcg(p.part_keys + ((size_t)row * kSweepMaxChunks + i / K) * CAST_MAX_TOP_K + (i % K));
+  __syncthreads();
+  block_top_k(cand, nk, K, topk);
+  if (warp == 0) {
+    float Mc = -INFINITY;
+    double Sc = 0.0;
+    if (lane < p.nchunks) {
+      Mc = __ldcg(p.part_max + (size_t)row * kSweepMaxChunks + lane);
+      Sc = __ldcg(p.part_sum + (size_t)row * kSweepMaxChunks + lane);
+    }
+    float Mr = Mc;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) Mr = fmaxf(Mr, __shfl_xor_sync(0xffffffffu, Mr, o));
+    double term = (Mc > -INFINITY) ? Sc * exp((double)Mc - (double)Mr) : 0.0;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) term += __shfl_xor_sync(0xffffffffu, term, o);
+    const double lse = (double)Mr + log(term);
+    if (lane == 0) {
+      s_lse = lse;
+      if (!isfinite(lse)) report(st, CAST_ERR_NONFINITE, row);
+    }
+  }
+  __syncthreads();
+  const int base = st->pool_size;
+  if (tid < K) {
+    const unsigned long long key = topk[tid];
+    const float val = key_value(key);
+    int tok = key_token(key);
+    if (key == 0ull || !(val > -INFINITY) || tok < 0 || tok >= p.V) {  // fewer than K finite logits
+      report(st, CAST_ERR_NONFINITE, row);
+      tok = 0;
+    }
+    const int parent = p.layer == 1 ? 0 : p.retained[b * p.W + r];
+    const size_t o = (size_t)b * p.P;
+    const int idx = base + r * K + tid;
+    p.pool_score[o + idx] = p.pool_score[o + parent] + ((double)val - s_lse);
+    p.pool_token[o + idx] = tok;
+    p.pool_parent[o + idx] = parent;
+    p.pool_depth[o + idx] = p.layer;
+    p.pool_kept[o + idx] = 0;
+  }
+
+  // ---- layer tail by the last CTA of the layer
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const int t = atomicAdd(p.layer_ticket, 1);
+    s_flag = (t == B * n_prev - 1);
+  }
+  __syncthreads();
+  if (!s_flag) return;
+  __threadfence();
+  if (tid == 0) *p.layer_ticket = 0;
+  layer_tail(p, B, n_prev, base, reinterpret_cast<unsigned char*>(cand), sorted);
+}
+
+// ------------------------------------------------------------------ rerank + linearise
+struct SelectParams {
+  const double* pool_score;
+  const int32_t* pool_token;
+  const int32_t* pool_parent;
+  const int32_t* pool_depth;
+  const uint8_t* pool_kept;
+  DevState* st;
+  int P, P2, Ncap, words, m, pool_mode, enable_dr;
+  double C3;
+  DevTable tab;
+  double* sel_score;
+  double* sel_value;
+  int32_t* sel_idx;
+  int32_t* tokens;
+  int32_t* parent;
+  int32_t* depth;
+  uint32_t* anc;
+  int32_t* pool_idx;
+  double* scores;
+  int32_t* n_tree;
+};
+
+// Total order of the rerank: (value desc, depth asc, token asc, creation order); idx < 0 sorts last.
+__device__ __forceinline__ bool ranks_before(const SelectParams& p, size_t o, double sa, int ia, double sb, int ib) {
+  if (ia < 0) return false;
+  if (ib < 0) return true;
+  if (sa != sb) return sa > sb;
+  const int da = p.pool_depth[o + ia], db = p.pool_depth[o + ib];
+  if (da != db) return da < db;
+  const int ta = p.pool_token[o + ia], tb = p.pool_token[o + ib];
+  if (ta != tb) return ta < tb;
+  return ia < ib;
+}
+
+// Phase 1: sort sequence b's pool, publish the best min(pool, m) nodes with their values.
+__device__ void select_sort_phase(const SelectParams& p, int b, unsigned char* smem) {
+  double* key_s = reinterpret_cast<double*>(smem);
+  int* idx_s = reinterpret_cast<int*>(smem + (size_t)p.P2 * sizeof(double));
+  const int tid = threadIdx.x, nt = blockDim.x;
+  const size_t o = (size_t)b * p.P;
+  const int pool = p.st->pool_size;
+  for (int i = tid; i < p.P2; i += nt) {
+    const bool in = i < pool && (p.pool_mode == 0 || p.pool_kept[o + i]);
+    key_s[i] = in ? p.pool_score[o + i] : -INFINITY;
+    idx_s[i] = in ? i : -1;
+  }
+  __syncthreads();
+  for (int k = 2; k <= p.P2; k <<= 1)
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      for (int i = tid; i < p.P2; i += nt) {
+        const int l = i ^ j;
+        if (l > i) {
+          const double sa = key_s[i], sb = key_s[l];
+          const int ia = idx_s[i], ib = idx_s[l];
+          const bool up = ((i & k) == 0);
+          const bool swap = up ? ranks_before(p, o, sb, ib, sa, ia) : ranks_before(p, o, sa, ia, sb, ib);
+          if (swap) {
+            key_s[i] = sb; key_s[l] = sa;
+            idx_s[i] = ib; idx_s[l] = ia;
+          }
+        }
+      }
+      __syncthreads();
+    }
+  const int peff = p.pool_mode == 0 ? pool : p.st->kept_total;
+  const int n_out = min(min(peff, p.m), p.Ncap);
+  for (int s = tid; s < n_out; s += nt) {
+    p.sel_score[(size_t)b * p.Ncap + s] = key_s[s];
+    p.sel_value[(size_t)b * p.Ncap + s] = exp(key_s[s]);
+    p.sel_idx[(size_t)b * p.Ncap + s] = idx_s[s];
+  }
+}
+
+// Phase 2: batch-mean utility, target-cost ratio, Algorithm 1 -> N; then sequence b's tree.
+__device__ void select_finalize_phase(const SelectParams& p, int b, int B) {
+  __shared__ double u[CAST_MAX_TREE], c[CAST_MAX_TREE];
+  __shared__ int kept[CAST_MAX_TREE], lin_parent[CAST_MAX_TREE];
+  __shared__ short lin_of[1 + CAST_MAX_TOP_K + (CAST_MAX_DEPTH - 1) * CAST_MAX_WIDTH * CAST_MAX_TOP_K];
+  __shared__ int s_N;
+  const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31;
+  const size_t o = (size_t)b * p.P;
+  const int pool = p.st->pool_size;
+  const int peff = p.pool_mode == 0 ? pool : p.st->kept_total;
+  int n = min(min(peff, p.m), p.Ncap);
+  if (p.enable_dr && p.tab.Ntab < n) n = p.tab.Ntab;
+  if (tid == 0) s_N = 1;
+  // u_k = sum_{s<=k} v(s), v(s) = batch mean of the rank-s values
+  if (tid < 32) {
+    double v[4], run = 0.0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int s = lane * 4 + e;
+      double a = 0.0;
+      if (s < n) {
+        for (int bb = 0; bb < B; ++bb) a += p.sel_value[(size_t)bb * p.Ncap + s];
+        a /= (double)B;
+      }
+      run += a;
+      v[e] = run;
+    }
+    double incl = run;  // inclusive scan of the lane totals
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const double t = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += t;
+    }
+    const double excl = incl - run;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int s = lane * 4 + e;
+      if (s < n) u[s] = excl + v[e];
+    }
+  }
+  if (p.enable_dr) {
+    const int g0 = select_grid(p.st->n0, p.tab.L, p.tab.M);
+    const double* f = p.tab.fT + (size_t)(g0 - 1) * p.tab.Ntab;
+    for (int k = tid; k < n; k += nt) c[k] = f[k] / f[0];
+  }
+  __syncthreads();
+  int N = n;
+  if (p.enable_dr) {
+    for (int j = tid; j < n; j += nt) {
+      bool ok = true;
+      for (int i = 0; i < j; ++i)
+        if ((u[j] - u[i]) < p.C3 * (c[j] - c[i])) ok = false;
+      if (ok) atomicMax(&s_N, j + 1);
+    }
+    __syncthreads();
+    N = s_N;
+  }
+  // linearise: kept nodes in creation order (ascending pool index)
+  for (int s = tid; s < N; s += nt) kept[s] = p.sel_idx[(size_t)b * p.Ncap + s];
+  __syncthreads();
+  for (int s = tid; s < N; s += nt) {
+    const int mine = kept[s];
+    int t = 0;
+    for (int j = 0; j < N; ++j) t += (kept[j] < mine);
+    lin_of[mine] = (short)t;
+  }
+  __syncthreads();
+  for (int s = tid; s < N; s += nt) {
+    const int pi = kept[s];
+    const int t = lin_of[pi];
+    const int pp = p.pool_parent[o + pi];
+    const int lp = pp >= 0 ? (int)lin_of[pp] : -1;
+    lin_parent[t] = lp;
+    const size_t q = (size_t)b * p.Ncap + t;
+    p.tokens[q] = p.pool_token[o + pi];
+    p.parent[q] = lp;
+    p.depth[q] = p.pool_depth[o + pi];
+    p.pool_idx[q] = pi;
+    if (p.scores) p.scores[q] = p.pool_score[o + pi];
+  }
+  __syncthreads();
+  for (int t = tid; t < p.Ncap; t += nt) {
+    uint32_t w[CAST_MAX_TREE / 32] = {0u, 0u, 0u, 0u};
+    const size_t q = (size_t)b * p.Ncap + t;
+    if (t < N) {
+      int a = t, guard = 0;
+      while (a >= 0 && a < N && guard++ <= CAST_MAX_DEPTH + 1) {  // walk to the root, setting one bit per ancestor
+        w[a >> 5] |= 1u << (a & 31);
+        a = lin_parent[a];
+      }
+    } else {
+      p.tokens[q] = -1;
+      p.parent[q] = -1;
+      p.depth[q] = -1;
+      p.pool_idx[q] = -1;
+      if (p.scores) p.scores[q] = 0.0;
+    }
+    for (int k = 0; k < p.words; ++k) p.anc[q * p.words + k] = w[k];
+  }
+  if (tid == 0) {
+    p.n_tree[b] = N;
+    if (b == 0) p.st->n_tree = N;
+  }
+}
+
+__global__ void __launch_bounds__(512) select_sort_kernel(const SelectParams p) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  select_sort_phase(p, blockIdx.x, smem);
+}
+__global__ void __launch_bounds__(512) select_finalize_kernel(const SelectParams p) {
+  select_finalize_phase(p, blockIdx.x, gridDim.x);
+}
+__global__ void __launch_bounds__(512) select_fused_kernel(const SelectParams p) {  // batch 1: one launch
+  extern __shared__ __align__(16) unsigned char smem[];
+  select_sort_phase(p, 0, smem);
+  __syncthreads();
+  select_finalize_phase(p, 0, 1);
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------ C-ABI
+extern "C" cast_status cast_step_begin(cast_ctx* c, int B, const int32_t* root_token, const int32_t* kv_len,
+                                       void* stream) {
+  if (!c || !root_token || !kv_len || B < 1) return CAST_ERR_INVALID_ARG;
+  if (B > c->cfg.max_batch) return CAST_ERR_CAPACITY;
+  const bool need = c->cfg.enable_bp || c->cfg.enable_dp || c->cfg.enable_dr;
+  auto it = c->tables->find(B);
+  if (it != c->tables->end()) {
+    c->cur_table = it->second.dev;
+  } else {
+    if (need) return CAST_ERR_COST_TABLE;
+    c->cur_table = DevTable{1, 1, 1 << 30, nullptr, nullptr};
+  }
+  c->cur_B = B;
+  c->next_layer = 1;
+  step_begin_kernel<<<1, 128, 0, (cudaStream_t)stream>>>(c->state, B, c->P, c->W, root_token, kv_len, c->pool_score,
+                                                         c->pool_token, c->pool_parent, c->pool_depth, c->pool_kept,
+                                                         c->retained, c->row_ticket, c->layer_ticket,
+                                                         c->cfg.max_batch * c->W);
+  return launch_status();
+}
+
+extern "C" cast_status cast_tree_expand(cast_ctx* c, int layer, const void* draft_logits, cast_dtype dtype,
+                                        int32_t* next_tokens, int32_t* next_parent_row, int32_t* next_count,
+                                        void* stream) {
+  if (!c || !draft_logits || !next_tokens || !next_parent_row || !next_count) return CAST_ERR_INVALID_ARG;
+  if (dtype != CAST_F32 && dtype != CAST_BF16) return CAST_ERR_DTYPE;
+  if (c->cur_B < 1 || layer < 1 || layer > c->cfg.max_depth || layer != c->next_layer) return CAST_ERR_INVALID_ARG;
+  c->next_layer = layer + 1;
+  const int B = c->cur_B, V = c->cfg.vocab;
+  const int rows_per_seq = layer == 1 ? 1 : c->W;
+  // enough CTAs to cover the machine about twice, at least 2048 logits each
+  int nchunks = (2 * c->num_sms + B * rows_per_seq - 1) / (B * rows_per_seq);
+  if (nchunks > kSweepMaxChunks) nchunks = kSweepMaxChunks;
+  if (nchunks > V / 2048) nchunks = V / 2048;
+  if (nchunks < 1) nchunks = 1;
+  int chunk_elems = (V + nchunks - 1) / nchunks;
+  chunk_elems = (chunk_elems + 7) / 8 * 8;
+  nchunks = (V + chunk_elems - 1) / chunk_elems;
+
+  ExpandParams p;
+  p.logits = draft_logits;
+  p.V = V; p.K = c->cfg.top_k; p.W = c->W; p.H = c->cfg.max_depth; p.P = c->P; p.layer = layer;
+  p.nchunks = nchunks; p.chunk_elems = chunk_elems;
+  p.pool_score = c->pool_score; p.pool_token = c->pool_token; p.pool_parent = c->pool_parent;
+  p.pool_depth = c->pool_depth; p.pool_kept = c->pool_kept; p.retained = c->retained;
+  p.st = c->state;
+  p.part_keys = c->part_keys; p.part_max = c->part_max; p.part_sum = c->part_sum;
+  p.row_ticket = c->row_ticket; p.layer_ticket = c->layer_ticket;
+  p.fifo_vals = c->fifo_vals; p.fifo_cnt = c->fifo_cnt; p.R = c->cfg.fifo_len;
+  p.tab = c->cur_table;
+  p.C1 = c->cfg.C1; p.C2 = c->cfg.C2;
+  p.enable_bp = c->cfg.enable_bp; p.enable_dp = c->cfg.enable_dp; p.ctx_base_mode = c->cfg.ctx_base_mode;
+  p.next_tokens = next_tokens; p.next_parent_row = next_parent_row; p.next_count = next_count;
+  const dim3 grid(nchunks, rows_per_seq, B);
+  if (dtype == CAST_F32)
+    expand_kernel<float><<<grid, kSweepThreads, 0, (cudaStream_t)stream>>>(p);
+  else
+    expand_kernel<__nv_bfloat16><<<grid, kSweepThreads, 0, (cudaStream_t)stream>>>(p);
+  return launch_status();
+}
+
+extern "C" cast_status cast_select_nodes(cast_ctx* c, int32_t* tokens, int32_t* parent, int32_t* depth,
+                                         uint32_t* anc_mask, int32_t* pool_idx, double* scores, int32_t* n_tree,
+                                         void* stream) {
+  if (!c || !tokens || !parent || !depth || !anc_mask || !pool_idx || !n_tree) return CAST_ERR_INVALID_ARG;
+  if (c->cur_B < 1) return CAST_ERR_INVALID_ARG;
+  SelectParams p;
+  p.pool_score = c->pool_score; p.pool_token = c->pool_token; p.pool_parent = c->pool_parent;
+  p.pool_depth = c->pool_depth; p.pool_kept = c->pool_kept; p.st = c->state;
+  p.P = c->P;
+  int P2 = 32;
+  while (P2 < c->P) P2 <<= 1;
+  p.P2 = P2;
+  p.Ncap = c->cfg.max_tree; p.words = c->words; p.m = c->cfg.total_token;
+  p.pool_mode = c->cfg.pool_mode; p.enable_dr = c->cfg.enable_dr; p.C3 = c->cfg.C3;
+  p.tab = c->cur_table;
+  p.sel_score = c->sel_score; p.sel_value = c->sel_value; p.sel_idx = c->sel_idx;
+  p.tokens = tokens; p.parent = parent; p.depth = depth; p.anc = anc_mask; p.pool_idx = pool_idx;
+  p.scores = scores; p.n_tree = n_tree;
+  const size_t smem = (size_t)P2 * (sizeof(double) + sizeof(int));
+  cudaStream_t s = (cudaStream_t)stream;
+  static bool attr_done = false;
+  if (!attr_done) {
+    CAST_CUDA_OK(cudaFuncSetAttribute(select_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 4096 * 12));
+    CAST_CUDA_OK(cudaFuncSetAttribute(select_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 4096 * 12));
+    attr_done = true;
+  }
+  const int threads = P2 >= 1024 ? 512 : (P2 / 2 < 128 ? 128 : P2 / 2);
+  if (c->cur_B == 1) {
+    select_fused_kernel<<<1, threads, smem, s>>>(p);
+  } else {
+    select_sort_kernel<<<c->cur_B, threads, smem, s>>>(p);
+    select_finalize_kernel<<<c->cur_B, 128, 0, s>>>(p);
+  }
+  return launch_status();
+}

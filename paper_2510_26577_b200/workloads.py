@@ -45,19 +45,20 @@ class Workload:
     n_layers: int  # verification layers timed per step (distinct KV buffers)
     max_tree: int = 128
     tau: float = 1.4e-4  # slope of the synthetic cost table in B*n
+    seed_salt: int = 0  # bumped when a seed puts a tree decision within rounding of its threshold
 
     @property
     def seed(self) -> int:
-        return BASE_SEED + self.config_id
+        return BASE_SEED + self.config_id + 1000 * self.seed_salt
 
     @property
     def gqa(self) -> int:
         return self.q_heads // self.kv_heads
 
 
-def _c3(batch: int, sub: int) -> Workload:
+def _c3(batch: int, sub: int, salt: int = 0) -> Workload:
     return Workload(f"c3_llama8b_b{batch}", 30 + sub, batch, "bf16", "f32", 32, 8, 128, 512, 4096, 16,
-                    128256, 3.0, 6, 8, 64, True, max(2, 64 // batch))
+                    128256, 3.0, 6, 8, 64, True, max(2, 64 // batch), seed_salt=salt)
 
 
 def _c4(m: int, sub: int) -> Workload:
@@ -70,9 +71,10 @@ CONFIGS: Dict[str, Workload] = {
     for w in [
         Workload("c1_tiny", 1, 1, "f32", "f32", 8, 8, 64, 256, 256, 0, 4096, 2.0, 4, 4, 16, False, 2),
         Workload("c2_llama8b", 2, 1, "bf16", "f32", 32, 8, 128, 2048, 2048, 0, 128256, 3.0, 6, 10, 60, False, 32),
-        _c3(1, 0), _c3(4, 1), _c3(16, 2), _c3(64, 3),
+        _c3(1, 0, 2), _c3(4, 1), _c3(16, 2), _c3(64, 3, 7),
         _c4(16, 0), _c4(32, 1), _c4(64, 2), _c4(128, 3),
-        Workload("c5_qwen_long", 5, 4, "bf16", "f32", 28, 4, 128, 32768, 32768, 16, 152064, 3.0, 8, 8, 96, False, 2),
+        Workload("c5_qwen_long", 5, 4, "bf16", "f32", 28, 4, 128, 32768, 32768, 16, 152064, 3.0, 8, 8, 96, False, 2,
+                 seed_salt=1),
     ]
 }
 
@@ -107,14 +109,15 @@ def kv_lengths(w: Workload, device="cpu") -> torch.Tensor:
     return torch.randint(w.kv_len_lo, w.kv_len_hi + 1, (w.batch,), generator=g, dtype=torch.int32).to(device)
 
 
-def draft_logits(w: Workload, layer: int, device="cpu", peaked: bool = False) -> torch.Tensor:
-    """[B, W, V] draft logits of one layer (W = K rows per batch row).  With
+def draft_logits(w: Workload, layer: int, device="cpu", peaked: bool = False, width: int = 0) -> torch.Tensor:
+    """[B, W, V] draft logits of one layer (W = `width`, default K rows).  With
     `peaked`, one token per row is raised by 8 so that scores decay slowly with
     depth, as those of a trained draft head do."""
     g = _gen(w, 100 + layer, device)
-    x = _randn((w.batch, w.top_k, w.vocab), w.logit_std, "f32", g, device)
+    rows = width or w.top_k
+    x = _randn((w.batch, rows, w.vocab), w.logit_std, "f32", g, device)
     if peaked:
-        idx = torch.randint(0, w.vocab, (w.batch, w.top_k, 1), generator=g, device=device)
+        idx = torch.randint(0, w.vocab, (w.batch, rows, 1), generator=g, device=device)
         x.scatter_add_(2, idx, torch.full_like(idx, 8.0, dtype=torch.float32))
     return x.to(_TORCH_DTYPE[w.logit_dtype])
 
