@@ -1,0 +1,406 @@
+"""Benchmark of the CAST draft-and-verify step on B200.
+
+One "step" is one pass of the whole hot path over one batch of synthetic input:
+cast_step_begin, H x cast_tree_expand, cast_select_nodes, n_layers x
+cast_tree_attention (distinct KV buffers per layer), cast_accept,
+cast_compact_kv - captured in one CUDA graph and replayed.  The headline value
+is tree tokens verified per second; the per-phase timings, the attention
+roofline and the CPU oracle baseline ride along in the same JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME]
+  python bench.py --impl reference ...      (the CPU oracle, bounded sample)
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC, UNIT = "tree_verify_tokens_per_s", "tokens/s"
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled during the timed region."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in out.splitlines():
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------ CPU oracle arm
+def oracle_step_seconds(w, attn_pairs=256):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload and
+    extrapolates to one full step.  Returns (seconds_per_step, description, threads)."""
+    import numpy as np
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from helpers import cfg_kwargs, make_tables, oracle_tree, to_f64
+    from oracle import CostTable, compact_kv, greedy_accept, tree_attention
+    from paper_2510_26577_b200 import workloads as wl
+
+    kw = cfg_kwargs(w)
+    B = w.batch
+    tables = None
+    if w.cost_model:
+        L, M, Ntab, fT, fD = make_tables(w, B)
+        tables = {B: CostTable(B, L, M, Ntab, fT, fD)}
+    root, kv = wl.root_tokens(w), wl.kv_lengths(w)
+    logits = [wl.draft_logits(w, l) for l in range(1, w.depth + 1)]
+    t0 = time.perf_counter()
+    o = oracle_tree(kw, tables, root, kv, logits)
+    t_tree = time.perf_counter() - t0
+    n_tree = o["n_tree"]
+    q = wl.query(w, 0).float().numpy()
+    k, v = (t.float().numpy() for t in wl.kv_cache(w, 0))
+    table, _ = wl.page_table(w)
+    tab = table.numpy() if table is not None else None
+    rng = np.random.default_rng(0)
+    total_pairs = int(sum(int(n) for n in n_tree)) * w.q_heads
+    only = set()
+    while len(only) < min(attn_pairs, total_pairs):
+        b = int(rng.integers(0, B))
+        only.add((b, int(rng.integers(0, n_tree[b])), int(rng.integers(0, w.q_heads))))
+    t0 = time.perf_counter()
+    tree_attention(q, k, v, w.page_size, tab, kv.numpy(), o["anc"], n_tree, None, only)
+    t_attn_layer = (time.perf_counter() - t0) * total_pairs / len(only)
+    nmax = int(n_tree.max())
+    rows = min(nmax, 8)
+    tl = to_f64(wl.target_logits(w)[:, :nmax])
+    t0 = time.perf_counter()
+    ol, op, _ = greedy_accept(tl, o["tokens"], o["parent"], n_tree, w.depth)
+    t_accept = time.perf_counter() - t0
+    kk, vv = k[None], v[None]
+    t0 = time.perf_counter()
+    compact_kv(kk, vv, w.page_size, tab, kv.numpy(), op, ol)
+    t_compact = (time.perf_counter() - t0) * w.n_layers
+    total = t_tree + w.n_layers * t_attn_layer + t_accept + t_compact
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = 1
+    desc = (f"tree build + accept in full; attention: {len(only)} of {total_pairs} (token, head) outputs of one layer, "
+            f"scaled to {w.n_layers} layers; compaction of one layer scaled to {w.n_layers}")
+    del rows
+    return total, desc, threads, int(sum(int(n) for n in n_tree))
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    times = []
+    for i in range(args.warmup + args.steps):
+        sec, desc, threads, ntok = oracle_step_seconds(w, attn_pairs=64)
+        if i >= args.warmup:
+            times.append(sec)
+    sec = sum(times) / len(times)
+    val = ntok / sec
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "batch": w.batch, "tree_tokens": ntok, "kv_prefix": [w.kv_len_lo, w.kv_len_hi],
+                   "n_layers": w.n_layers},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------ CUDA arm
+def run_ours(args, w):
+    import numpy as np
+    import torch
+    from paper_2510_26577_b200 import build as _build
+    _build.build()
+    from paper_2510_26577_b200 import binding, workloads as wl
+
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+
+    B, H, K, Ncap, m = w.batch, w.depth, w.top_k, w.max_tree, w.total_token
+    Hq, Hkv, D, nl = w.q_heads, w.kv_heads, w.head_dim, w.n_layers
+    kw = dict(vocab=w.vocab, top_k=K, max_depth=H, total_token=m, max_tree=Ncap)
+    if w.cost_model:
+        kw.update(enable_bp=1, enable_dr=1)
+    ctx = binding.CastContext(max_batch=B, **kw)
+    if w.cost_model:
+        ctx.cast_set_cost_tables(B, *wl.cost_table_arrays(w, B))
+
+    # ---- synthetic inputs, resident in HBM
+    root, kv0 = wl.root_tokens(w, dev), wl.kv_lengths(w, dev)
+    kv_len = kv0.clone()
+    logits = [wl.draft_logits(w, l, dev) for l in range(1, H + 1)]
+    q = torch.stack([wl.query(w, l, dev) for l in range(nl)])
+    kc = torch.empty((nl,) + tuple(wl.kv_cache(w, 0, dev)[0].shape), dtype=q.dtype, device=dev)
+    vc = torch.empty_like(kc)
+    for l in range(nl):
+        kc[l], vc[l] = wl.kv_cache(w, l, dev)
+    table, num_pages = wl.page_table(w, dev)
+    seq_cap = wl.seq_capacity(w) // (w.page_size or 1)
+    tl = wl.target_logits(w, dev)
+    out = torch.zeros_like(q)
+    nt = [torch.empty((B, K), dtype=torch.int32, device=dev) for _ in range(H)]
+    npr = [torch.empty((B, K), dtype=torch.int32, device=dev) for _ in range(H)]
+    cnt = [torch.empty((1,), dtype=torch.int32, device=dev) for _ in range(H)]
+    tr = dict(tokens=torch.empty((B, Ncap), dtype=torch.int32, device=dev),
+              parent=torch.empty((B, Ncap), dtype=torch.int32, device=dev),
+              depth=torch.empty((B, Ncap), dtype=torch.int32, device=dev),
+              anc=torch.empty((B, Ncap, ctx.words), dtype=torch.int32, device=dev),
+              pool_idx=torch.empty((B, Ncap), dtype=torch.int32, device=dev),
+              scores=torch.empty((B, Ncap), dtype=torch.float64, device=dev),
+              n_tree=torch.empty((B,), dtype=torch.int32, device=dev))
+    alen = torch.empty((B,), dtype=torch.int32, device=dev)
+    apath = torch.empty((B, H + 1), dtype=torch.int32, device=dev)
+    bonus = torch.empty((B,), dtype=torch.int32, device=dev)
+    layer_stride = kc[0].numel() * kc.element_size()
+
+    def tree_build():
+        ctx.cast_step_begin(B, root, kv_len)
+        for i in range(H):
+            ctx.cast_tree_expand(i + 1, logits[i], nt[i], npr[i], cnt[i])
+        ctx.cast_select_nodes(tr["tokens"], tr["parent"], tr["depth"], tr["anc"], tr["pool_idx"], tr["scores"],
+                              tr["n_tree"])
+
+    def attention():
+        for l in range(nl):
+            ctx.cast_tree_attention(q[l], kc[l], vc[l], B, Hq, Hkv, D, w.page_size, table, seq_cap, num_pages, kv_len,
+                                    tr["anc"], tr["n_tree"], 0.0, out[l])
+
+    def accept():
+        ctx.cast_accept(tl, B, tr["tokens"], tr["parent"], tr["depth"], tr["anc"], tr["n_tree"], alen, apath, bonus)
+
+    def compact():
+        ctx.cast_compact_kv(kc, vc, B, nl, layer_stride, Hkv, D, w.page_size, table, seq_cap, num_pages, apath, alen,
+                            kv_len)
+
+    def step():
+        kv_len.copy_(kv0)  # compaction advanced the lengths; every step starts from the same prefix
+        tree_build(); attention(); accept(); compact()
+
+    # first pass: sizes the attention workspace, gives the tree for planting acceptance
+    tree_build()
+    torch.cuda.synchronize()
+    st, detail = ctx.cast_poll_status()
+    assert st == 0, f"device status {st} ({detail})"
+    n_tree = tr["n_tree"].cpu().numpy()
+    wl.plant_acceptance(w, tl, tr["tokens"].cpu().numpy(), tr["parent"].cpu().numpy(), n_tree)
+    step()
+    torch.cuda.synchronize()
+    assert ctx.cast_poll_status()[0] == 0
+    tokens_per_step = int(n_tree.sum())
+    accept_mean = float(alen.float().mean().item())
+
+    stream = torch.cuda.Stream(device=dev)
+
+    def capture(fn):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(stream):
+            fn()  # warm the stream
+            stream.synchronize()
+            with torch.cuda.graph(g, stream=stream):
+                fn()
+        return g
+
+    def time_graph(g, reps, warm):
+        with torch.cuda.stream(stream):
+            for _ in range(warm):
+                g.replay()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            stream.synchronize()
+            e0.record(stream)
+            for _ in range(reps):
+                g.replay()
+            e1.record(stream)
+            stream.synchronize()
+        return e0.elapsed_time(e1) / reps  # ms per replay
+
+    g_step = capture(step)
+    g_tree, g_attn, g_acc, g_cmp = capture(tree_build), capture(attention), capture(accept), capture(compact)
+
+    # ---- phase timings (each phase alone; KV working set of the attention graph exceeds 2x L2)
+    sub_reps = max(args.steps, 20)
+    ms_tree = time_graph(g_tree, sub_reps * 5, 5)
+    ms_attn = time_graph(g_attn, sub_reps, args.warmup)
+    ms_acc = time_graph(g_acc, sub_reps, args.warmup)
+    kv_len.copy_(kv0)
+    ms_cmp = time_graph(g_cmp, 3, 1)
+    kv_len.copy_(kv0)
+
+    # ---- the timed region: K replays of the whole step
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local) if rank == 0 else None
+    ms_step = time_graph(g_step, args.steps, args.warmup)
+    if dist is not None:
+        t = torch.tensor([ms_step], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.barrier()
+        ms_step = float(t.item())
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if sampler else None
+    assert ctx.cast_poll_status()[0] == 0
+
+    # ---- end to end: per-step inputs start in pinned host memory, results are read back
+    h_logits = [x.cpu().pin_memory() for x in logits]
+    h_q = q[:, :, :m].contiguous().cpu().pin_memory()
+    h_tl = tl[:, :m].contiguous().cpu().pin_memory()
+    h_out = torch.empty_like(h_q).pin_memory()
+    h_res = torch.empty((B, H + 3), dtype=torch.int32).pin_memory()
+    d_res = torch.empty((B, H + 3), dtype=torch.int32, device=dev)
+    h2d = sum(x.numel() * x.element_size() for x in h_logits) + h_q.numel() * 2 + h_tl.numel() * h_tl.element_size()
+    d2h = h_out.numel() * h_out.element_size() + h_res.numel() * 4
+
+    def e2e_step():
+        for i in range(H):
+            logits[i].copy_(h_logits[i], non_blocking=True)
+        q[:, :, :m].copy_(h_q, non_blocking=True)
+        tl[:, :m].copy_(h_tl, non_blocking=True)
+        step()
+        h_out.copy_(out[:, :, :m], non_blocking=True)
+        d_res[:, 0] = alen; d_res[:, 1] = bonus; d_res[:, 2:] = apath
+        h_res.copy_(d_res, non_blocking=True)
+
+    with torch.cuda.stream(stream):
+        for _ in range(max(args.warmup, 3)):
+            e2e_step()
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.steps):
+            e2e_step()
+        e1.record(stream)
+        stream.synchronize()
+    ms_e2e = e0.elapsed_time(e1) / args.steps
+    if dist is not None:
+        t = torch.tensor([ms_e2e], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (tree attention, one layer per launch)
+    e = 2 if w.kv_dtype == "bf16" else 4
+    kvl = kv0.cpu().numpy().astype(np.int64)
+    attn_bytes = int(sum(2 * (int(kvl[b]) + int(n_tree[b])) * Hkv * D * e + 2 * int(n_tree[b]) * Hq * D * e
+                         for b in range(B)))
+    peak, which = peaks()
+    attn_us = ms_attn * 1e3 / nl
+    achieved = attn_bytes / (attn_us * 1e-6) / 1e9
+    logits_bytes = sum(int(x.numel() * x.element_size()) for x in logits) // K * 1  # layer 1 reads one row
+    sel_launches = 1 if B == 1 else 2
+    launches = args.steps * (1 + H + sel_launches + 2 * nl + 2 + 1)
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        sec, desc, threads, ntok = oracle_step_seconds(w)
+        cpu = {"value": ntok / sec, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc,
+               "ms_per_step": sec * 1e3}
+
+    line = {
+        "metric": METRIC, "value": world * tokens_per_step / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": w.kv_dtype, "data": "synthetic",
+        "config": {"workload": w.name, "batch": B, "tree_tokens_per_step": tokens_per_step, "depth": H, "top_k": K,
+                   "vocab": w.vocab, "q_heads": Hq, "kv_heads": Hkv, "head_dim": D,
+                   "kv_prefix": [w.kv_len_lo, w.kv_len_hi], "page_size": w.page_size, "n_layers": nl,
+                   "logit_dtype": w.logit_dtype, "parallelism": "replicas" if world > 1 else "single",
+                   "l2": "distinct KV buffers per layer; step working set exceeds 2x L2", "cuda_graph": True,
+                   "accept_len_mean": accept_mean},
+        "e2e": {"value": world * tokens_per_step / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e,
+                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
+        "gpu_launches": launches,
+        "clocks": clocks,
+        "phases": {"tree_build_us": ms_tree * 1e3, "attention_us_per_layer": attn_us, "accept_us": ms_acc * 1e3,
+                   "compact_us": ms_cmp * 1e3},
+        "roofline": {"kernel": "cast_tree_attention (one layer)", "bound": "hbm", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_source": which, "traffic": None,
+                     "algorithmic_bytes": attn_bytes},
+        "cpu_baseline": cpu,
+    }
+    del logits_bytes
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2_llama8b")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    from paper_2510_26577_b200 import workloads as wl
+    w = wl.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()
