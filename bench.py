@@ -275,8 +275,8 @@ def run_ours(args, w):
     g_tree, g_attn, g_acc, g_cmp = capture(tree_build), capture(attention), capture(accept), capture(compact)
 
     # ---- phase timings (each phase alone; KV working set of the attention graph exceeds 2x L2)
-    sub_reps = max(args.steps, 20)
-    ms_tree = time_graph(g_tree, sub_reps * 5, 5)
+    sub_reps = args.steps if args.quick else max(args.steps, 20)
+    ms_tree = time_graph(g_tree, sub_reps if args.quick else sub_reps * 5, 5)
     ms_attn = time_graph(g_attn, sub_reps, args.warmup)
     ms_acc = time_graph(g_acc, sub_reps, args.warmup)
     kv_len.copy_(kv0)
@@ -319,16 +319,16 @@ def run_ours(args, w):
         h_res.copy_(d_res, non_blocking=True)
 
     with torch.cuda.stream(stream):
-        for _ in range(max(args.warmup, 3)):
+        for _ in range(0 if args.quick else max(args.warmup, 3)):
             e2e_step()
         stream.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
-        for _ in range(args.steps):
+        for _ in range(1 if args.quick else args.steps):
             e2e_step()
         e1.record(stream)
         stream.synchronize()
-    ms_e2e = e0.elapsed_time(e1) / args.steps
+    ms_e2e = e0.elapsed_time(e1) / (1 if args.quick else args.steps)
     if dist is not None:
         t = torch.tensor([ms_e2e], device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -352,7 +352,7 @@ def run_ours(args, w):
     launches = args.steps * (1 + H + sel_launches + 2 * nl + 2 + 1)
 
     cpu = None
-    if not args.no_cpu_baseline:
+    if not (args.no_cpu_baseline or args.quick):
         sec, desc, threads, ntok = oracle_step_seconds(w)
         cpu = {"value": ntok / sec, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc,
                "ms_per_step": sec * 1e3}
@@ -392,6 +392,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2_llama8b")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--quick", action="store_true",
+                    help="profiling mode: few replays per phase, one end-to-end step, no CPU baseline")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     from paper_2510_26577_b200 import workloads as wl

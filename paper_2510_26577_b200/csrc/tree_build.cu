@@ -16,6 +16,22 @@
 
 using namespace cast;
 
+// Development aid, compiled only with -DCAST_PHASE_CLOCKS: thread 0 of the CTA that ends up running
+// the layer tail / the rerank records clock64() at phase boundaries.
+#ifdef CAST_PHASE_CLOCKS
+__device__ long long g_phase_clock[64];
+#define CAST_STAMP(k) do { if (threadIdx.x == 0) stamp_s[k] = clock64(); } while (0)
+#define CAST_STAMP_DECL __shared__ long long stamp_s[32];
+#define CAST_STAMP_FLUSH(off, n) do { if (threadIdx.x == 0) for (int _i = 0; _i < (n); ++_i) g_phase_clock[(off) + _i] = stamp_s[_i]; } while (0)
+extern "C" __attribute__((visibility("default"))) int cast_debug_read_clocks(long long* out) {
+  return (int)cudaMemcpyFromSymbol(out, g_phase_clock, sizeof(long long) * 64);
+}
+#else
+#define CAST_STAMP(k) do {} while (0)
+#define CAST_STAMP_DECL
+#define CAST_STAMP_FLUSH(off, n) do {} while (0)
+#endif
+
 namespace {
 
 // ------------------------------------------------------------------ step begin
@@ -279,6 +295,8 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
   __shared__ int sorted[CAST_MAX_BATCH * CAST_MAX_WIDTH];
   __shared__ int cand_cnt, s_flag;
   __shared__ double s_lse;
+  CAST_STAMP_DECL
+  CAST_STAMP(0);
 
   const int chunk = blockIdx.x, r = blockIdx.y, b = blockIdx.z, B = gridDim.z;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -302,6 +320,7 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
   unsigned long long thr_prev = 0ull;
   if (tid == 0) cand_cnt = 0;
   __syncthreads();
+  CAST_STAMP(1);
 
   for (int sub = begin; sub < end; sub += kSweepSub) {
     float xv[kSweepEpt];
@@ -377,6 +396,7 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
     __syncthreads();
   }
 
+  CAST_STAMP(2);
   // chunk partials: top-K keys, maximum, sum of exp(x - maximum) in fp64
   {
     const int have = cand_cnt;
@@ -402,6 +422,7 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
     }
   }
 
+  CAST_STAMP(3);
   // ---- row merge by the last CTA of this logits row
   __threadfence();
   __syncthreads();
@@ -411,6 +432,7 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
   }
   __syncthreads();
   if (!s_flag) return;
+  CAST_STAMP(4);
   __threadfence();
   if (tid == 0) p.row_ticket[row] = 0;
   const int nk = p.nchunks * K;
@@ -457,6 +479,7 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
     p.pool_kept[o + idx] = 0;
   }
 
+  CAST_STAMP(5);
   // ---- layer tail by the last CTA of the layer
   __threadfence();
   __syncthreads();
@@ -468,7 +491,10 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
   if (!s_flag) return;
   __threadfence();
   if (tid == 0) *p.layer_ticket = 0;
+  CAST_STAMP(6);
   layer_tail(p, B, n_prev, base, reinterpret_cast<unsigned char*>(cand), sorted);
+  CAST_STAMP(7);
+  CAST_STAMP_FLUSH(0, 8);
 }
 
 // ------------------------------------------------------------------ rerank + linearise
@@ -659,9 +685,14 @@ __global__ void __launch_bounds__(512) select_finalize_kernel(const SelectParams
 }
 __global__ void __launch_bounds__(512) select_fused_kernel(const SelectParams p) {  // batch 1: one launch
   extern __shared__ __align__(16) unsigned char smem[];
+  CAST_STAMP_DECL
+  CAST_STAMP(0);
   select_sort_phase(p, 0, smem);
   __syncthreads();
+  CAST_STAMP(1);
   select_finalize_phase(p, 0, 1);
+  CAST_STAMP(2);
+  CAST_STAMP_FLUSH(16, 3);
 }
 
 }  // namespace

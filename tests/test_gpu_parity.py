@@ -301,6 +301,18 @@ def test_attention_arbitrary_trees_ragged(binding, dtype, D, Hq, Hkv, page):
     k, v = (t.cuda() for t in wl.kv_cache(w, 0, "cpu"))
     table, num_pages = wl.page_table(w, "cuda")
     nt = torch.from_numpy(n_tree).cuda()
+    # cache rows past a sequence's last tree token may hold anything: poison them with NaN
+    cap = wl.seq_capacity(w)
+    for b in range(B):
+        end = int(kv[b]) + int(n_tree[b])
+        if page:
+            for pos in range(end, cap):
+                pg = int(table[b, pos // page])
+                k[pg, pos % page] = float("nan")
+                v[pg, pos % page] = float("nan")
+        else:
+            k[b, end:] = float("nan")
+            v[b, end:] = float("nan")
     out = gpu_attention(ctx, w, q, k, v, table, num_pages, kv, anc, nt, scale=0.0)
     assert ctx.cast_poll_status()[0] == 0
     f32 = lambda t: t.float().cpu().numpy()
