@@ -271,16 +271,36 @@ def run_ours(args, w):
             stream.synchronize()
         return e0.elapsed_time(e1) / reps  # ms per replay
 
+    if args.only:  # profiling aid: replay one phase only (no graph), print its time, stop
+        fn = {"tree": tree_build, "attention": attention, "accept": accept, "compact": compact}[args.only]
+        with torch.cuda.stream(stream):
+            for _ in range(args.warmup):
+                fn()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(args.steps):
+                fn()
+            e1.record(stream)
+            stream.synchronize()
+        st = ctx.cast_poll_status()
+        print(json.dumps({"only": args.only, "workload": w.name, "us_per_call": e0.elapsed_time(e1) * 1e3 / args.steps,
+                          "device_status": st[0]}))
+        return
+
     g_step = capture(step)
-    g_tree, g_attn, g_acc, g_cmp = capture(tree_build), capture(attention), capture(accept), capture(compact)
+    def compact_phase():
+        kv_len.copy_(kv0)  # each replay compacts from the same prefix lengths
+        compact()
+
+    g_tree, g_attn, g_acc, g_cmp = capture(tree_build), capture(attention), capture(accept), capture(compact_phase)
 
     # ---- phase timings (each phase alone; KV working set of the attention graph exceeds 2x L2)
+    kv_len.copy_(kv0)  # the capture passes ran the compaction
     sub_reps = args.steps if args.quick else max(args.steps, 20)
     ms_tree = time_graph(g_tree, sub_reps if args.quick else sub_reps * 5, 5)
     ms_attn = time_graph(g_attn, sub_reps, args.warmup)
     ms_acc = time_graph(g_acc, sub_reps, args.warmup)
-    kv_len.copy_(kv0)
-    ms_cmp = time_graph(g_cmp, 3, 1)
+    ms_cmp = time_graph(g_cmp, sub_reps, args.warmup)
     kv_len.copy_(kv0)
 
     # ---- the timed region: K replays of the whole step
@@ -296,7 +316,8 @@ def run_ours(args, w):
         ms_step = float(t.item())
     torch.cuda.synchronize()
     clocks = sampler.stop() if sampler else None
-    assert ctx.cast_poll_status()[0] == 0
+    st = ctx.cast_poll_status()
+    assert st[0] == 0, f"device status {st}"
 
     # ---- end to end: per-step inputs start in pinned host memory, results are read back
     h_logits = [x.cpu().pin_memory() for x in logits]
@@ -392,6 +413,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2_llama8b")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--only", default="", choices=["", "tree", "attention", "accept", "compact"],
+                    help="profiling aid: run one phase only, without graphs")
     ap.add_argument("--quick", action="store_true",
                     help="profiling mode: few replays per phase, one end-to-end step, no CPU baseline")
     args = ap.parse_args()

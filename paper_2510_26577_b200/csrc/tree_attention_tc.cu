@@ -2,40 +2,60 @@
 //
 // One CTA owns (sequence b, kv-head, block of 128 query rows, KV split). A query row is a
 // (tree token, head of the GQA group) pair, so every K/V tile is fetched once for all tree
-// tokens and all heads of the group. Per tile of 128 positions:
-//   control warp : TMA loads K and V (128B-swizzled, two 64-column halves each) into a 2-stage
-//                  ring; S = Q K^T by tcgen05.mma (M=128 rows, N=128 positions, K=128) into TMEM;
-//                  after the softmax warps have written P, O += P V (B operand MN-major, so V
-//                  is used exactly as it lies in the cache: no transpose).
-//   8 softmax warps: thread (row, column half) reads its 64 scores with tcgen05.ld, applies the
+// tokens and all heads of the group. Tiles are 64 positions. Roles:
+//   control warp : TMA loads of K and V (128B-swizzled, two 64-column halves each) into a 4-stage
+//                  ring; S = Q K^T by tcgen05.mma (M=128 rows, N=64 positions, K=128) into one of
+//                  two TMEM buffers; once the softmax warps have written P, O += P V (V is the
+//                  MN-major B operand: used exactly as it lies in the cache, no transpose).
+//                  QK^T of tile i+1 is issued before P of tile i is awaited, so the tensor pipe
+//                  works on the next scores while the softmax of the current tile runs.
+//   8 softmax warps: thread (row, column half) reads its 32 scores with tcgen05.ld, applies the
 //                  prefix/ancestor mask (only tiles that reach past the prefix need one), keeps a
 //                  lazily updated row maximum (O in TMEM is rescaled only when the maximum grows
-//                  by more than 2^8), writes P as bf16 into swizzled shared memory.
-// All mbarrier waits are bounded: on expiry the CTA records CAST_ERR_TIMEOUT, drains its
-// copies, frees its TMEM and returns.
+//                  by more than 2^8), writes P as bf16 into one of two swizzled smem buffers.
+// The number of KV splits is decided on the device from the actual tree sizes and prefix
+// lengths (the host only fixes its upper bound), so the grid fills the machine whatever N the
+// cost model picked. All mbarrier waits are bounded: on expiry the CTA records
+// CAST_ERR_TIMEOUT, drains its copies, frees its TMEM and returns.
 #include <cuda.h>
 #include <math.h>
 
 #include "cast_internal.h"
 
+#ifdef CAST_PHASE_CLOCKS
+__device__ long long g_attn_clock[256];
+extern "C" __attribute__((visibility("default"))) int cast_debug_read_attn_clocks(long long* out) {
+  return (int)cudaMemcpyFromSymbol(out, g_attn_clock, sizeof(long long) * 256);
+}
+#define TC_STAMP(role, it, k) do { if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (it) >= 4 && (it) < 8 && \
+    (threadIdx.x == ((role) ? 288 : 0))) g_attn_clock[(role) * 128 + ((it) - 4) * 16 + (k)] = clock64(); } while (0)
+#define TC_MARK(k) do { if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) g_attn_clock[240 + (k)] = clock64(); } while (0)
+#else
+#define TC_STAMP(role, it, k) do {} while (0)
+#define TC_MARK(k) do {} while (0)
+#endif
+
 namespace cast {
 
 namespace {
 
-constexpr int kBM = 128;          // query rows per CTA
-constexpr int kBN = 128;          // positions per tile
+constexpr int kBM = 128;          // query rows per CTA (UMMA M)
+constexpr int kBN = 64;           // positions per tile
 constexpr int kHD = 128;          // head dim
-constexpr int kStages = 2;
+constexpr int kStages = 4;        // K/V ring
 constexpr int kSoftmaxThreads = 256;
-constexpr int kThreadsTC = kSoftmaxThreads + 32;
-constexpr int kRegion = kBM * 128;                 // one [128][64] bf16 region: 16 KB
-constexpr int kSmemQ = 0;
-constexpr int kSmemP = 2 * kRegion;
-constexpr int kSmemKV = 4 * kRegion;               // stage s: K at +s*4*kRegion, V at +2*kRegion after K
-constexpr int kSmemBytes = 4 * kRegion + kStages * 4 * kRegion;  // 192 KB
-constexpr int kTmemCols = 256;                     // S: columns [0,128), O: columns [128,256)
+constexpr int kThreadsTC = kSoftmaxThreads + 64;  // + TMA producer warp + MMA issuer warp
+constexpr int kRegionQ = kBM * 128;                // [128 rows][64] bf16, 128B rows: 16 KB
+constexpr int kRegionKV = kBN * 128;               // [64 positions][64] bf16: 8 KB
+constexpr int kSmemQ = 0;                          // 2 regions (d 0-63, d 64-127)
+constexpr int kSmemP = 2 * kRegionQ;               // 2 buffers of one region [128 rows][64 positions]
+constexpr int kSmemKV = 4 * kRegionQ;              // stage s: K (2 regions) then V (2 regions)
+constexpr int kStageBytes = 4 * kRegionKV;         // 32 KB
+constexpr int kSmemBytes = kSmemKV + kStages * kStageBytes;  // 192 KB
+constexpr int kTmemCols = 256;                     // S0: [0,64), S1: [64,128), O: [128,256)
 constexpr float kRescaleThreshold = 8.0f;          // log2 units
 constexpr long long kWaitCycles = 4000000000ll;    // about two seconds
+constexpr int kMaxSplit = 16;
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -44,7 +64,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 struct TcParams {
   const __nv_bfloat16* q;
   __nv_bfloat16* out;
-  int B, Ncap, Hq, Hkv, G, page_size, seq_capacity, num_pages, words, nsplit;
+  int B, Ncap, Hq, Hkv, G, page_size, seq_capacity, num_pages, words, nsplit_max, num_sms;
   const int32_t* page_table;
   const int32_t* kv_len;
   const int32_t* n_tree;
@@ -159,16 +179,54 @@ __device__ __forceinline__ void softmax_bar() { asm volatile("bar.sync 1, %0;" :
 // Byte offset of 16-byte chunk `c` (0..7) of row `r` inside a 128B-swizzled [rows][64 bf16] region.
 __device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4)); }
 
+// KV splits actually used, from the tree sizes and prefix lengths on the device: enough CTAs for
+// about four waves, at least eight tiles each where the sequences are long enough, and never fewer
+// CTAs than SMs when the work allows. Every warp computes the same value.
+__device__ __forceinline__ int effective_splits(const TcParams& p) {
+  const int lane = threadIdx.x & 31;
+  const int max_pos = p.page_size == 0 ? p.seq_capacity : p.seq_capacity * p.page_size;
+  int active = 0, tiles = 0;
+  for (int b = lane; b < p.B; b += 32) {
+    int N = p.n_tree[b];
+    N = N < 0 ? 0 : (N > p.Ncap ? p.Ncap : N);
+    int L = p.kv_len[b];
+    L = L < 0 ? 0 : L;
+    int total = L + N;
+    total = total > max_pos ? max_pos : total;
+    const int nrb = (N * p.G + kBM - 1) / kBM;
+    active += p.Hkv * nrb;
+    tiles += p.Hkv * nrb * ((total + kBN - 1) / kBN);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    active += __shfl_xor_sync(0xffffffffu, active, o);
+    tiles += __shfl_xor_sync(0xffffffffu, tiles, o);
+  }
+  if (active == 0) return 1;
+  const int per = tiles / active;  // mean tiles per (sequence, kv-head, row block)
+  int want = active * per / 8;
+  want = want > 4 * p.num_sms ? 4 * p.num_sms : want;
+  want = want < p.num_sms ? p.num_sms : want;
+  int ns = (want + active - 1) / active;
+  ns = ns > p.nsplit_max ? p.nsplit_max : ns;
+  ns = ns > per ? per : ns;
+  return ns < 1 ? 1 : ns;
+}
+
 __global__ void __launch_bounds__(kThreadsTC, 1)
 tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) uint64_t bar_full[kStages], bar_free[kStages], bar_s, bar_p;
+  __shared__ __align__(8) uint64_t bar_full[kStages], bar_free[kStages], bar_s[2], bar_p[2];
   __shared__ uint32_t tmem_base_s;
   __shared__ float xch[2][kBM * 2];
   __shared__ uint32_t anc_s[kBM][CAST_MAX_TREE / 32];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int split = blockIdx.x % p.nsplit, rb = blockIdx.x / p.nsplit;
+  TC_MARK(0);
+  const int nsplit = effective_splits(p);
+  TC_MARK(1);
+  const int split = blockIdx.x % p.nsplit_max, rb = blockIdx.x / p.nsplit_max;
+  if (split >= nsplit) return;
   const int kvh = blockIdx.y, b = blockIdx.z;
   int N = p.n_tree[b];
   N = N < 0 ? 0 : (N > p.Ncap ? p.Ncap : N);
@@ -183,13 +241,13 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     total = max_pos;
   }
   const int ntiles = (total + kBN - 1) / kBN;
-  const int t0 = (int)((long long)split * ntiles / p.nsplit), t1 = (int)((long long)(split + 1) * ntiles / p.nsplit);
+  const int t0 = (int)((long long)split * ntiles / nsplit), t1 = (int)((long long)(split + 1) * ntiles / nsplit);
   const int ntile = t1 - t0;
-  const int half = warp >> 2, quarter = warp & 3, r = quarter * 32 + lane;  // softmax-role coordinates
+  const int half = (warp >> 2) & 1, quarter = warp & 3, r = quarter * 32 + lane;  // softmax-role coordinates
   const int row = row0 + r;
   const bool row_ok = warp < 8 && row < rows_total;
   const int t_tok = row_ok ? row / G : 0, h_q = kvh * G + (row_ok ? row % G : 0);
-  const size_t pr = (((size_t)b * p.Hq + h_q) * p.Ncap + t_tok) * p.nsplit + split;
+  const size_t pr = (((size_t)b * p.Hq + h_q) * p.Ncap + t_tok) * p.nsplit_max + split;
   if (ntile <= 0) {  // nothing to attend to in this split: an empty partial
     if (row_ok && half == 0) {
       p.part_ml[pr * 2] = -INFINITY;
@@ -199,28 +257,84 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
   }
   unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
 
-  if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(&bar_full[s], 1);
-      mbar_init(&bar_free[s], 1);
+  // tile j of this CTA -> ring stage j % kStages (producer warp only; all 32 lanes call it)
+  auto issue_load = [&](int j) -> bool {
+    const int stage = j % kStages;
+    unsigned char* kdst = smem + kSmemKV + stage * kStageBytes;
+    unsigned char* vdst = kdst + 2 * kRegionKV;
+    const int pos0 = (t0 + j) * kBN;
+    const int ps = p.page_size;
+    int npages = 0, page = 0;
+    if (ps != 0) {  // page ids are fetched before the stage is awaited: their latency hides behind the wait
+      const int ppt = kBN / ps;
+      npages = (total - pos0 + ps - 1) / ps;
+      npages = npages > ppt ? ppt : npages;
+      if (lane < npages * 4) {
+        page = p.page_table[(size_t)b * p.seq_capacity + pos0 / ps + (lane >> 2)];
+        if (page < 0 || page >= p.num_pages) {
+          report(p.st, CAST_ERR_BAD_PAGE, b);
+          page = 0;
+        }
+      }
     }
-    mbar_init(&bar_s, 1);
-    mbar_init(&bar_p, kSoftmaxThreads);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (warp == 0) {  // TMEM: 256 columns for S and O
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)),
-                 "n"(kTmemCols));
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
-  }
-  if (warp < 8) {
+    if (j >= kStages) {
+      const bool w = mbar_wait(&bar_free[stage], ((j / kStages) - 1) & 1);
+      if (!__all_sync(0xffffffffu, w)) return false;
+    }
+    if (ps == 0) {
+      if (lane == 0) mbar_expect_tx(&bar_full[stage], kStageBytes);
+      __syncwarp();
+      if (lane < 4) {
+        const int hsel = lane & 1;
+        tma_load_3d(lane < 2 ? &map_k : &map_v, (lane < 2 ? kdst : vdst) + hsel * kRegionKV, &bar_full[stage], hsel * 64,
+                    kvh, b * p.seq_capacity + pos0);
+      }
+    } else {  // at most 8 pages per tile (page size >= 8): one (page, tensor, half) per lane
+      if (lane == 0) mbar_expect_tx(&bar_full[stage], (uint32_t)npages * ps * 128 * 4);
+      __syncwarp();
+      if (lane < npages * 4) {
+        const int slot = lane >> 2, which = lane & 3, hsel = which & 1;
+        tma_load_4d(which < 2 ? &map_k : &map_v, (which < 2 ? kdst : vdst) + hsel * kRegionKV + slot * ps * 128,
+                    &bar_full[stage], hsel * 64, kvh, 0, page);
+      }
+    }
+    __syncwarp();
+    return true;
+  };
+
+  int armed = 0;
+  bool prod_ok = true;
+  if (warp == 8) {
+    if (lane == 0) {
+      for (int s = 0; s < kStages; ++s) {
+        mbar_init(&bar_full[s], 1);
+        mbar_init(&bar_free[s], 1);
+      }
+      for (int s = 0; s < 2; ++s) {
+        mbar_init(&bar_s[s], 1);
+        mbar_init(&bar_p[s], kSoftmaxThreads);
+      }
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      fence_proxy_async();
+    }
+    __syncwarp();
+    for (int j = 0; j < kStages && j < ntile; ++j) {  // the ring fills while the other warps stage Q
+      prod_ok = issue_load(j);
+      armed = j + 1;
+    }
+  } else if (warp < 8) {
+    if (warp == 0) {  // TMEM: two S buffers and O
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)),
+                   "n"(kTmemCols));
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+    }
     // Q rows -> swizzled shared memory (rows past the tree are zero); ancestor masks
     const __nv_bfloat16* qrow = p.q + (((size_t)b * p.Ncap + t_tok) * p.Hq + h_q) * kHD + half * 64;
 #pragma unroll
     for (int c = 0; c < 8; ++c) {
       uint4 v = make_uint4(0u, 0u, 0u, 0u);
       if (row_ok) v = *reinterpret_cast<const uint4*>(qrow + c * 8);
-      *reinterpret_cast<uint4*>(smem + kSmemQ + half * kRegion + swz(r, c)) = v;
+      *reinterpret_cast<uint4*>(smem + kSmemQ + half * kRegionQ + swz(r, c)) = v;
     }
     if (half == 0) {
       for (int w = 0; w < CAST_MAX_TREE / 32; ++w)
@@ -228,101 +342,20 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     }
     fence_proxy_async();
   }
+  TC_MARK(2);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  TC_MARK(3);
   const uint32_t tmem_base = tmem_base_s;
-  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + kBN;
+  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 2 * kBN;
 
   if (warp == 8) {
-    // =========================== control warp: TMA + MMA issue ===========================
-    const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
-    const uint32_t idesc_pv = idesc_qk | (1u << 16);  // B operand (V) is MN-major
-    const uint32_t q_addr = smem_u32(smem + kSmemQ), p_addr = smem_u32(smem + kSmemP);
-    auto issue_load = [&](int j) -> bool {  // tile j of this CTA into stage j % kStages
-      const int stage = j % kStages;
-      if (j >= kStages && !mbar_wait(&bar_free[stage], ((j / kStages) - 1) & 1)) return false;
-      unsigned char* kdst = smem + kSmemKV + stage * 4 * kRegion;
-      unsigned char* vdst = kdst + 2 * kRegion;
-      const int pos0 = (t0 + j) * kBN;
-      if (p.page_size == 0) {
-        if (lane == 0) mbar_expect_tx(&bar_full[stage], 4 * kRegion);
-        __syncwarp();
-        if (lane < 4) {
-          const int hsel = lane & 1;
-          tma_load_3d(lane < 2 ? &map_k : &map_v, (lane < 2 ? kdst : vdst) + hsel * kRegion, &bar_full[stage], hsel * 64,
-                      kvh, b * p.seq_capacity + pos0);
-        }
-      } else {
-        const int ps = p.page_size, ppt = kBN / ps;
-        int npages = (total - pos0 + ps - 1) / ps;
-        npages = npages > ppt ? ppt : npages;
-        if (lane == 0) mbar_expect_tx(&bar_full[stage], (uint32_t)npages * ps * 128 * 4);
-        __syncwarp();
-        for (int op = lane; op < npages * 4; op += 32) {
-          const int slot = op >> 2, which = op & 3, hsel = which & 1;
-          int page = p.page_table[(size_t)b * p.seq_capacity + pos0 / ps + slot];
-          if (page < 0 || page >= p.num_pages) {
-            report(p.st, CAST_ERR_BAD_PAGE, b);
-            page = 0;
-          }
-          tma_load_4d(which < 2 ? &map_k : &map_v, (which < 2 ? kdst : vdst) + hsel * kRegion + slot * ps * 128,
-                      &bar_full[stage], hsel * 64, kvh, 0, page);
-        }
-      }
-      __syncwarp();
-      return true;
-    };
-    auto mma_qk = [&](int stage) {  // S = Q K^T
-      if (lane == 0) {
-        const uint32_t k_addr = smem_u32(smem + kSmemKV + stage * 4 * kRegion);
-#pragma unroll
-        for (int ks = 0; ks < kHD / 16; ++ks) {
-          const uint32_t off = (ks >> 2) * kRegion + (ks & 3) * 32;
-          umma_bf16(tmem_s, umma_desc(q_addr + off, 16, 1024), umma_desc(k_addr + off, 16, 1024), idesc_qk, ks > 0);
-        }
-        umma_commit(&bar_s);
-      }
-      __syncwarp();
-    };
-    auto mma_pv = [&](int stage, bool first) {  // O (+)= P V
-      if (lane == 0) {
-        const uint32_t v_addr = smem_u32(smem + kSmemKV + stage * 4 * kRegion + 2 * kRegion);
-#pragma unroll
-        for (int ks = 0; ks < kBN / 16; ++ks) {
-          const uint32_t aoff = (ks >> 2) * kRegion + (ks & 3) * 32;
-          umma_bf16(tmem_o, umma_desc(p_addr + aoff, 16, 1024), umma_desc(v_addr + ks * 2048, kRegion, 1024), idesc_pv,
-                    (!first || ks > 0) ? 1u : 0u);
-        }
-        umma_commit(&bar_free[stage]);
-      }
-      __syncwarp();
-    };
-    int armed = 0;
-    bool ok = issue_load(0);
-    armed = 1;
-    if (ok && ntile > 1) { ok = issue_load(1); armed = 2; }
-    if (ok) ok = mbar_wait(&bar_full[0], 0);
-    if (ok) {
-      tc_fence_after();
-      mma_qk(0);
-    }
-    for (int it = 0; ok && it < ntile; ++it) {
-      const int stage = it % kStages;
-      ok = mbar_wait(&bar_p, it & 1);
-      if (!ok) break;
-      tc_fence_after();
-      mma_pv(stage, it == 0);
-      if (it + 1 < ntile) {
-        ok = mbar_wait(&bar_full[(it + 1) % kStages], ((it + 1) / kStages) & 1);
-        if (!ok) break;
-        tc_fence_after();
-        mma_qk((it + 1) % kStages);
-      }
-      if (it + 2 < ntile) {
-        ok = issue_load(it + 2);
-        if (ok) armed = it + 3;
-      }
+    // =========================== TMA producer ===========================
+    bool ok = prod_ok;
+    for (int j = armed; ok && j < ntile; ++j) {
+      ok = issue_load(j);
+      if (ok) armed = j + 1;
     }
     if (!ok) {  // drain: copies in flight must land before the CTA's shared memory is released
       if (lane == 0) report(p.st, CAST_ERR_TIMEOUT, b);
@@ -331,116 +364,207 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
         while (!mbar_test(&bar_full[j % kStages], (j / kStages) & 1) && clock64() - tw < kWaitCycles) {}
       }
     }
-  } else {
-    // =========================== softmax warps ===========================
-    const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
-    float m_used = -INFINITY, l_run = 0.f;
-    bool ok = true;
-    for (int it = 0; it < ntile; ++it) {
-      const int stage = it % kStages;
-      const int pos0 = (t0 + it) * kBN;
-      ok = mbar_wait(&bar_s, it & 1);
-      if (!ok) break;
-      tc_fence_after();
-      uint32_t sr[64];
-      tmem_ld32(tmem_s + lane_sel + half * 64, sr);
-      tmem_ld32(tmem_s + lane_sel + half * 64 + 32, sr + 32);
-      tmem_wait_ld();
-      // visibility of this thread's 64 columns: prefix positions always, tree positions by the ancestor mask
-      const int cbase = pos0 + half * 64;
-      unsigned long long vis = 0ull;
-      if (row_ok) {
-        if (cbase + 64 <= L) {
-          vis = ~0ull;
-        } else {
-          for (int c = 0; c < 64; ++c) {
-            const int pos = cbase + c;
-            bool v = pos < L;
-            if (!v && pos < total) {
-              const int j = pos - L;
-              v = (anc_s[r][j >> 5] >> (j & 31)) & 1u;
-            }
-            vis |= (unsigned long long)v << c;
-          }
-        }
-      }
-      float mx = -INFINITY;
+  } else if (warp == 9) {
+    // =========================== MMA issuer ===========================
+    const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+    const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(kHD >> 3) << 17) |
+                              ((uint32_t)(kBM >> 4) << 24);  // B operand (V) is MN-major, N = head dim
+    // descriptors differ only in the start-address field (16-byte units), so they are built once
+    const uint64_t dq = umma_desc(smem_u32(smem + kSmemQ), 16, 1024);
+    const uint64_t dk = umma_desc(smem_u32(smem + kSmemKV), 16, 1024);
+    const uint64_t dv = umma_desc(smem_u32(smem + kSmemKV + 2 * kRegionKV), kRegionKV, 1024);
+    const uint64_t dp = umma_desc(smem_u32(smem + kSmemP), 16, 1024);
+    auto mma_qk = [&](int stage, int buf) {  // S[buf] = Q K^T
+      if (lane == 0) {
+        const uint64_t dks = dk + (uint64_t)(stage * (kStageBytes >> 4));
 #pragma unroll
-      for (int c = 0; c < 64; ++c) {
-        const float s2 = ((vis >> c) & 1ull) ? __uint_as_float(sr[c]) * p.scale_log2 : -INFINITY;
-        sr[c] = __float_as_uint(s2);
-        mx = fmaxf(mx, s2);
+        for (int ks = 0; ks < kHD / 16; ++ks)
+          umma_bf16(tmem_s + buf * kBN, dq + (uint64_t)((ks >> 2) * (kRegionQ >> 4) + (ks & 3) * 2),
+                    dks + (uint64_t)((ks >> 2) * (kRegionKV >> 4) + (ks & 3) * 2), idesc_qk, ks > 0);
+        umma_commit(&bar_s[buf]);
       }
-      xch[it & 1][half * kBM + r] = mx;
-      softmax_bar();
-      mx = fmaxf(mx, xch[it & 1][(half ^ 1) * kBM + r]);
-      // lazy maximum: move the reference only when the row maximum outgrows it by 2^8
-      float alpha = 1.f;
-      const bool grow = mx > m_used + kRescaleThreshold || (m_used == -INFINITY && mx > -INFINITY);
-      if (grow) {
-        alpha = fast_exp2(m_used - mx);  // 0 when m_used = -inf
-        m_used = mx;
-        l_run *= alpha;
-      }
-      if (it > 0 && __any_sync(0xffffffffu, grow)) {  // rescale this thread's 64 columns of O
-        uint32_t orr[32];
+      __syncwarp();
+    };
+    auto mma_pv = [&](int stage, int buf, bool first) {  // O (+)= P[buf] V
+      if (lane == 0) {
+        const uint64_t dvs = dv + (uint64_t)(stage * (kStageBytes >> 4));
+        const uint64_t dpb = dp + (uint64_t)(buf * (kRegionQ >> 4));
 #pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {
-          const uint32_t ta = tmem_o + lane_sel + half * 64 + hh * 32;
-          tmem_ld32(ta, orr);
-          tmem_wait_ld();
-#pragma unroll
-          for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
-          tmem_st32(ta, orr);
-        }
-        tmem_wait_st();
+        for (int ks = 0; ks < kBN / 16; ++ks)
+          umma_bf16(tmem_o, dpb + (uint64_t)(ks * 2), dvs + (uint64_t)(ks * (2048 >> 4)), idesc_pv,
+                    (!first || ks > 0) ? 1u : 0u);
+        umma_commit(&bar_free[stage]);
       }
-      // P = 2^(s - m) as bf16 into the swizzled A-operand buffer; row sum in fp32
-      float lsum = 0.f;
-      unsigned char* prow = smem + kSmemP + half * kRegion;
-#pragma unroll
-      for (int c8 = 0; c8 < 8; ++c8) {
-        uint32_t pk[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          float p0 = 0.f, p1 = 0.f;
-          if (m_used > -INFINITY) {
-            p0 = fast_exp2(__uint_as_float(sr[c8 * 8 + 2 * e]) - m_used);
-            p1 = fast_exp2(__uint_as_float(sr[c8 * 8 + 2 * e + 1]) - m_used);
-          }
-          lsum += p0 + p1;
-          const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
-          pk[e] = *reinterpret_cast<const uint32_t*>(&pb);
-        }
-        *reinterpret_cast<uint4*>(prow + swz(r, c8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-      }
-      l_run += lsum;
-      // V rows past the end of the sequence may hold anything (0 * NaN would poison O): zero them
-      const int valid = total - pos0;
-      if (valid < kBN) {
-        unsigned char* vbase = smem + kSmemKV + stage * 4 * kRegion + 2 * kRegion;
-        for (int i = tid; i < (kBN - valid) * 16; i += kSoftmaxThreads) {
-          const int rr = valid + (i >> 4), reg = (i >> 3) & 1, c = i & 7;
-          *reinterpret_cast<uint4*>(vbase + reg * kRegion + rr * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
-        }
-      }
-      fence_proxy_async();
-      tc_fence_before();
-      mbar_arrive(&bar_p);
-    }
-    // epilogue: wait for the last P V, read O, normalise or emit the partial
-    if (ok) ok = mbar_wait(&bar_free[(ntile - 1) % kStages], ((ntile - 1) / kStages) & 1);
+      __syncwarp();
+    };
+    auto wait_all = [&](uint64_t* bar, uint32_t parity) -> bool {
+      const bool w = mbar_wait(bar, parity);
+      return __all_sync(0xffffffffu, w);
+    };
+    bool ok = wait_all(&bar_full[0], 0);
     if (ok) {
       tc_fence_after();
-      xch[0][half * kBM + r] = l_run;
+      mma_qk(0, 0);
+    }
+    for (int it = 0; ok && it < ntile; ++it) {
+      TC_STAMP(1, it, 0);
+      if (it + 1 < ntile) {  // next scores first: they are computed while the softmax of tile `it` runs
+        ok = wait_all(&bar_full[(it + 1) % kStages], ((it + 1) / kStages) & 1);
+        if (!ok) break;
+        TC_STAMP(1, it, 1);
+        tc_fence_after();
+        mma_qk((it + 1) % kStages, (it + 1) & 1);
+        TC_STAMP(1, it, 2);
+      }
+      ok = wait_all(&bar_p[it & 1], (it >> 1) & 1);
+      if (!ok) break;
+      TC_STAMP(1, it, 3);
+      tc_fence_after();
+      mma_pv(it % kStages, it & 1, it == 0);
+      TC_STAMP(1, it, 4);
+    }
+    if (!ok && lane == 0) report(p.st, CAST_ERR_TIMEOUT, b);
+  } else {
+    // =========================== softmax warps ===========================
+    // After a wait has expired a thread keeps visiting the barriers (so nobody blocks on it) but
+    // touches neither TMEM nor the operand buffers. A warp whose 32 rows all lie past the tree
+    // only keeps the barriers in step: its P rows feed output rows nobody reads.
+    const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
+    const bool warp_live = row0 + quarter * 32 < rows_total;
+    const float sc = p.scale_log2;
+    float m_used = -INFINITY, l_run = 0.f;  // m_used: running reference maximum in raw score units
+    bool ok = true;
+    for (int it = 0; it < ntile; ++it) {
+      const int buf = it & 1, stage = it % kStages;
+      const int pos0 = (t0 + it) * kBN;
+      uint32_t sr[32];
+      float mx = -INFINITY;
+      TC_STAMP(0, it, 0);
+      if (warp_live) {
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bar_s[buf], (it >> 1) & 1));
+        TC_STAMP(0, it, 1);
+        if (ok) {
+          tc_fence_after();
+          tmem_ld32(tmem_s + buf * kBN + lane_sel + half * 32, sr);
+          tmem_wait_ld();
+          TC_STAMP(0, it, 2);
+          const int cbase = pos0 + half * 32;
+          if (cbase + 32 > L) {  // this thread's 32 columns reach past the prefix: ancestor mask
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+              const int pos = cbase + c;
+              bool v = pos < L;
+              if (!v && pos < total) {
+                const int j = pos - L;
+                v = (anc_s[r][j >> 5] >> (j & 31)) & 1u;
+              }
+              if (!v) sr[c] = 0xff800000u;  // -inf
+            }
+          }
+          float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+          for (int c = 0; c < 32; c += 4) {
+            m0 = fmaxf(m0, __uint_as_float(sr[c]));
+            m1 = fmaxf(m1, __uint_as_float(sr[c + 1]));
+            m2 = fmaxf(m2, __uint_as_float(sr[c + 2]));
+            m3 = fmaxf(m3, __uint_as_float(sr[c + 3]));
+          }
+          mx = row_ok ? fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) : -INFINITY;
+        }
+      }
+      TC_STAMP(0, it, 3);
+      xch[buf][half * kBM + r] = mx;
       softmax_bar();
+      mx = fmaxf(mx, xch[buf][(half ^ 1) * kBM + r]);
+      TC_STAMP(0, it, 4);
+      if (warp_live && ok) {
+        // lazy maximum: move the reference only when the row maximum outgrows it by 2^8
+        float alpha = 1.f;
+        const bool grow = (mx - m_used) * sc > kRescaleThreshold || (m_used == -INFINITY && mx > -INFINITY);
+        if (grow) {
+          alpha = fast_exp2((m_used - mx) * sc);  // 0 when m_used = -inf
+          m_used = mx;
+          l_run *= alpha;
+        }
+        if (it > 0 && __any_sync(0xffffffffu, grow)) {  // rescale this thread's 64 columns of O
+          ok = __all_sync(0xffffffffu, mbar_wait(&bar_free[(it - 1) % kStages], ((it - 1) / kStages) & 1));
+          if (ok) {
+            tc_fence_after();
+            uint32_t orr[32];
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+              const uint32_t ta = tmem_o + lane_sel + half * 64 + hh * 32;
+              tmem_ld32(ta, orr);
+              tmem_wait_ld();
+#pragma unroll
+              for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
+              tmem_st32(ta, orr);
+            }
+            tmem_wait_st();
+          }
+        }
+        TC_STAMP(0, it, 5);
+        // the P buffer was last read by the P V product of tile it-2
+        if (ok && it >= 2)
+          ok = __all_sync(0xffffffffu, mbar_wait(&bar_free[(it - 2) % kStages], ((it - 2) / kStages) & 1));
+        TC_STAMP(0, it, 6);
+        if (ok) {
+          // P = 2^((s - m) * scale) as bf16 into the swizzled A-operand buffer; row sum in fp32
+          const bool live = m_used > -INFINITY;
+          const float neg_ms = live ? -m_used * sc : 0.f;
+          float l0 = 0.f, l1 = 0.f;
+          unsigned char* prow = smem + kSmemP + buf * kRegionQ;
+#pragma unroll
+          for (int c8 = 0; c8 < 4; ++c8) {
+            uint32_t pk[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              float p0 = fast_exp2(fmaf(__uint_as_float(sr[c8 * 8 + 2 * e]), sc, neg_ms));
+              float p1 = fast_exp2(fmaf(__uint_as_float(sr[c8 * 8 + 2 * e + 1]), sc, neg_ms));
+              if (!live) p0 = p1 = 0.f;
+              l0 += p0;
+              l1 += p1;
+              const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+              pk[e] = *reinterpret_cast<const uint32_t*>(&pb);
+            }
+            *reinterpret_cast<uint4*>(prow + swz(r, half * 4 + c8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          }
+          l_run += l0 + l1;
+        }
+      }
+      // V rows past the end of the sequence may hold anything (0 * NaN would poison O): zero them
+      if (ok && total - pos0 < kBN) {
+        if (!warp_live) ok = __all_sync(0xffffffffu, mbar_wait(&bar_s[buf], (it >> 1) & 1));  // V has landed by then
+        if (ok) {
+          const int valid = total - pos0;
+          unsigned char* vbase = smem + kSmemKV + stage * kStageBytes + 2 * kRegionKV;
+          for (int i = tid; i < (kBN - valid) * 16; i += kSoftmaxThreads) {
+            const int rr = valid + (i >> 4), reg = (i >> 3) & 1, c = i & 7;
+            *reinterpret_cast<uint4*>(vbase + reg * kRegionKV + rr * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
+          }
+        }
+      }
+      TC_STAMP(0, it, 7);
+      fence_proxy_async();
+      tc_fence_before();
+      mbar_arrive(&bar_p[buf]);
+      TC_STAMP(0, it, 9);
+    }
+    // epilogue: wait for the last P V, read O, normalise or emit the partial
+    TC_MARK(4);
+    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bar_free[(ntile - 1) % kStages], ((ntile - 1) / kStages) & 1));
+    TC_MARK(5);
+    xch[0][half * kBM + r] = l_run;
+    softmax_bar();
+    if (ok && warp_live) {
+      tc_fence_after();
       const float l_tot = l_run + xch[0][(half ^ 1) * kBM + r];
       uint32_t orr[64];
       tmem_ld32(tmem_o + lane_sel + half * 64, orr);
       tmem_ld32(tmem_o + lane_sel + half * 64 + 32, orr + 32);
       tmem_wait_ld();
       if (row_ok) {
-        if (p.nsplit == 1) {
+        if (nsplit == 1) {
           const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
           __nv_bfloat16* orow = p.out + (((size_t)b * p.Ncap + t_tok) * p.Hq + h_q) * kHD + half * 64;
 #pragma unroll
@@ -462,15 +586,17 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
                 make_float4(__uint_as_float(orr[c4 * 4]), __uint_as_float(orr[c4 * 4 + 1]),
                             __uint_as_float(orr[c4 * 4 + 2]), __uint_as_float(orr[c4 * 4 + 3]));
           if (half == 0) {
-            p.part_ml[pr * 2] = m_used * 0.69314718055994531f;  // back to natural-log units
+            p.part_ml[pr * 2] = m_used * sc * 0.69314718055994531f;  // natural-log units
             p.part_ml[pr * 2 + 1] = l_tot;
           }
         }
       }
     }
   }
+  TC_MARK(6);
   tc_fence_before();
   __syncthreads();
+  TC_MARK(7);
   if (warp == 0) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols));
@@ -487,12 +613,13 @@ __global__ void __launch_bounds__(kHD) tc_combine_kernel(const TcParams p) {
     out[d] = __float2bfloat16_rn(0.f);
     return;
   }
-  if (p.nsplit == 1) return;  // written by the attention kernel itself
-  const size_t pr = (((size_t)b * p.Hq + h) * p.Ncap + t) * p.nsplit;
+  const int nsplit = effective_splits(p);
+  if (nsplit == 1) return;  // written by the attention kernel itself
+  const size_t pr = (((size_t)b * p.Hq + h) * p.Ncap + t) * p.nsplit_max;
   float M = -INFINITY;
-  for (int s = 0; s < p.nsplit; ++s) M = fmaxf(M, p.part_ml[(pr + s) * 2]);
+  for (int s = 0; s < nsplit; ++s) M = fmaxf(M, p.part_ml[(pr + s) * 2]);
   float l = 0.f, acc = 0.f;
-  for (int s = 0; s < p.nsplit; ++s) {
+  for (int s = 0; s < nsplit; ++s) {
     const float ms = p.part_ml[(pr + s) * 2];
     if (ms > -INFINITY) {
       const float w = expf(ms - M);
@@ -545,7 +672,7 @@ bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const v
                               int page_size, const int32_t* page_table, int seq_capacity, int num_pages,
                               const int32_t* kv_len, const uint32_t* anc, const int32_t* n_tree, float scale, void* out,
                               cudaStream_t stream, cast_status* status) {
-  if (D != kHD) return false;
+  if (D != kHD || !(scale > 0.f)) return false;
   if (page_size != 0 && (page_size < 8 || page_size > kBN || (kBN % page_size) != 0 || (page_size % 8) != 0))
     return false;
   if ((((uintptr_t)k | (uintptr_t)v) & 127) != 0) return false;
@@ -555,23 +682,23 @@ bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const v
     return false;
   const int G = Hq / Hkv, Ncap = c->cfg.max_tree;
   const int nrb = (Ncap * G + kBM - 1) / kBM;
-  const int base = B * Hkv * ((c->cfg.total_token * G + kBM - 1) / kBM);
   const int max_pos = page_size == 0 ? seq_capacity : seq_capacity * page_size;
   const int max_tiles = (max_pos + kBN - 1) / kBN;
-  int nsplit = (c->num_sms + base - 1) / base;
-  if (nsplit > max_tiles) nsplit = max_tiles;
-  if (nsplit > 64) nsplit = 64;
-  if (nsplit < 1) nsplit = 1;
+  // upper bound of the KV splits; the kernel picks the actual number from the device-side sizes
+  int nsplit_max = (4 * c->num_sms + B * Hkv - 1) / (B * Hkv);
+  if (nsplit_max > max_tiles) nsplit_max = max_tiles;
+  if (nsplit_max > kMaxSplit) nsplit_max = kMaxSplit;
+  if (nsplit_max < 1) nsplit_max = 1;
   TcParams p;
   p.q = (const __nv_bfloat16*)q; p.out = (__nv_bfloat16*)out;
   p.B = B; p.Ncap = Ncap; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.page_size = page_size; p.seq_capacity = seq_capacity;
-  p.num_pages = num_pages; p.words = c->words; p.nsplit = nsplit;
+  p.num_pages = num_pages; p.words = c->words; p.nsplit_max = nsplit_max; p.num_sms = c->num_sms;
   p.page_table = page_table; p.kv_len = kv_len; p.n_tree = n_tree; p.anc = anc;
   p.scale_log2 = scale * 1.4426950408889634f;
   p.part_o = nullptr; p.part_ml = nullptr; p.st = c->state;
   *status = CAST_OK;
-  if (nsplit > 1) {
-    const size_t rows = (size_t)B * Hq * Ncap * nsplit;
+  if (nsplit_max > 1) {
+    const size_t rows = (size_t)B * Hq * Ncap * nsplit_max;
     const size_t need = rows * (kHD + 2) * sizeof(float);
     if (need > c->attn_ws_bytes) {  // grows the workspace (synchronises; not legal during graph capture)
       if (cudaDeviceSynchronize() != cudaSuccess) { *status = CAST_ERR_CUDA; return true; }
@@ -593,7 +720,7 @@ bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const v
     }
     attr_done = true;
   }
-  tree_attn_tc_kernel<<<dim3(nsplit * nrb, Hkv, B), kThreadsTC, kSmemBytes + 1024, stream>>>(p, map_k, map_v);
+  tree_attn_tc_kernel<<<dim3(nsplit_max * nrb, Hkv, B), kThreadsTC, kSmemBytes + 1024, stream>>>(p, map_k, map_v);
   tc_combine_kernel<<<dim3(Ncap, Hq, B), kHD, 0, stream>>>(p);
   *status = launch_status();
   return true;
