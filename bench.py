@@ -252,7 +252,9 @@ def run_ours(args, w):
     def capture(fn):
         g = torch.cuda.CUDAGraph()
         with torch.cuda.stream(stream):
+            kv_len.copy_(kv0)  # an earlier pass may have run the compaction
             fn()  # warm the stream
+            kv_len.copy_(kv0)
             stream.synchronize()
             with torch.cuda.graph(g, stream=stream):
                 fn()

@@ -171,7 +171,8 @@ CAST_API cast_status cast_select_nodes(cast_ctx* ctx, int32_t* tokens, int32_t* 
  * One layer of verification attention (the mask of Sec. "Tree Reranking Phase"):
  * out[b,t,h] = softmax over {prefix positions 0..kv_len[b]-1} U {tree positions
  * kv_len[b]+j : bit j of anc_mask[b,t]} of (q . k) * scale, times v, for
- * t < n_tree[b]; rows t >= n_tree[b] are written as zeros.
+ * t < n_tree[b]; rows t >= n_tree[b] of `out` are left untouched.
+ * n_tree[b] must not exceed the context's total_token (device error BAD_TREE).
  *   q, out        [B, Ncap, Hq, D], dtype `dtype`
  *   k_cache, v_cache  paged: [num_pages, page_size, Hkv, D]; the cache rows of
  *                 the tree tokens are already stored at positions kv_len[b]+j.

@@ -350,7 +350,7 @@ def _gather_kv(cache, b, npos, page_size, page_table):
 def tree_attention(q, k_cache, v_cache, page_size, page_table, kv_len, anc, n_tree, scale=None, only=None):
     """out[b,t,h] = softmax_p(q.k_p * scale) . v_p over p in [0, L_b) and the
     tree positions L_b + j for every j set in anc[b,t].  Rows t >= n_tree[b] are
-    zero.  q: [B, Ncap, Hq, D]; paged caches [num_pages, page, Hkv, D] or
+    not part of the result (returned as zeros).  q: [B, Ncap, Hq, D]; paged caches [num_pages, page, Hkv, D] or
     contiguous [B, Lmax, Hkv, D] (page_size 0); all float64.  `only`: optional
     set of (b, t, h) to compute (the other entries stay zero) - for sampled
     checks at sizes where the full loop would take minutes."""

@@ -272,17 +272,14 @@ __global__ void __launch_bounds__(kThreads) tree_attn_cc_kernel(const AttnParams
   }
 }
 
-// Merge the split partials of one (sequence, tree token, head); rows >= n_tree become zeros.
+// Merge the split partials of one (sequence, tree token, head); rows >= n_tree are left untouched.
 template <typename T, int D>
 __global__ void __launch_bounds__(D) attn_combine_kernel(const AttnParams p) {
   const int t = blockIdx.x, h = blockIdx.y, b = blockIdx.z, d = threadIdx.x;
   T* out = reinterpret_cast<T*>(p.out) + (((size_t)b * p.Ncap + t) * p.Hq + h) * D;
   int N = p.n_tree[b];
   N = N > p.Ncap ? p.Ncap : N;
-  if (t >= N) {
-    store_out(out + d, 0.f);
-    return;
-  }
+  if (t >= N) return;
   const size_t pr = (((size_t)b * p.Hq + h) * p.Ncap + t) * p.nsplit;
   float M = -INFINITY;
   for (int s = 0; s < p.nsplit; ++s) M = fmaxf(M, p.part_ml[(pr + s) * 2]);
