@@ -2,16 +2,17 @@
 //
 // One CTA owns (sequence b, kv-head, block of 128 query rows, KV split). A query row is a
 // (tree token, head of the GQA group) pair, so every K/V tile is fetched once for all tree
-// tokens and all heads of the group. Tiles are 128 positions. Roles (10 warps):
+// tokens and all heads of the group. Tiles are 64 positions; a CTA needs 112 KB of shared memory
+// and 256 TMEM columns, so two CTAs share an SM: while one waits for a tile or runs its
+// prologue/epilogue, the other streams (128 registers per thread for that). Roles:
 //   TMA producer : K tiles and V tiles (128B-swizzled, two 64-column halves each) into two
 //                  2-stage rings; a K stage is released as soon as Q K^T has consumed it, a V
-//                  stage after P V, so K runs about two tiles ahead of the tensor pipe.
-//   MMA issuer   : S = Q K^T by tcgen05.mma (M=128 rows, N=128 positions, K=128) into one of two
+//                  stage after P V.
+//   MMA issuer   : S = Q K^T by tcgen05.mma (M=128 rows, N=64 positions, K=128) into one of two
 //                  TMEM buffers; once the softmax warps have written P, O += P V (V is the
 //                  MN-major B operand: used exactly as it lies in the cache, no transpose).
-//                  Q K^T of tile i+1 is issued before P of tile i is awaited, so the tensor pipe
-//                  works on the next scores while the softmax of the current tile runs.
-//   8 softmax warps: thread (row, column half) reads its 64 scores with tcgen05.ld, applies the
+//                  Q K^T of tile i+1 is issued before P of tile i is awaited.
+//   4 softmax warps: one thread per query row reads its 64 scores with tcgen05.ld, applies the
 //                  prefix/ancestor mask (only tiles that reach past the prefix need one), keeps a
 //                  lazily updated row maximum (O in TMEM is rescaled only when the maximum grows
 //                  by more than 2^8), writes P as bf16 into swizzled shared memory.
@@ -22,6 +23,7 @@
 // CAST_ERR_TIMEOUT, drains its copies, frees its TMEM and returns.
 #include <cuda.h>
 #include <math.h>
+#include <stdlib.h>
 
 #include "cast_internal.h"
 
@@ -31,7 +33,7 @@ extern "C" __attribute__((visibility("default"))) int cast_debug_read_attn_clock
   return (int)cudaMemcpyFromSymbol(out, g_attn_clock, sizeof(long long) * 256);
 }
 #define TC_STAMP(role, it, k) do { if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (it) >= 2 && (it) < 6 && \
-    (threadIdx.x == ((role) ? 288 : 0))) g_attn_clock[(role) * 128 + ((it) - 2) * 16 + (k)] = clock64(); } while (0)
+    (threadIdx.x == ((role) ? 160 : 0))) g_attn_clock[(role) * 128 + ((it) - 2) * 16 + (k)] = clock64(); } while (0)
 #define TC_MARK(k) do { if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) g_attn_clock[240 + (k)] = clock64(); } while (0)
 __device__ unsigned long long g_cta_log[4 * 16384];
 extern "C" __attribute__((visibility("default"))) int cast_debug_read_cta_log(unsigned long long* out) {
@@ -51,19 +53,21 @@ namespace cast {
 namespace {
 
 constexpr int kBM = 128;          // query rows per CTA (UMMA M)
-constexpr int kBN = 128;          // positions per tile
+constexpr int kBN = 64;           // positions per tile
 constexpr int kHD = 128;          // head dim
 constexpr int kStages = 2;        // K ring and V ring
-constexpr int kSoftmaxThreads = 256;
-constexpr int kThreadsTC = kSoftmaxThreads + 64;  // + TMA producer warp + MMA issuer warp
-constexpr int kRegion = 128 * 128;                 // [128 rows][64] bf16, 128-byte rows: 16 KB
-constexpr int kTile = 2 * kRegion;                 // a [128][128] bf16 operand: 32 KB
-constexpr int kSmemQ = 0;
-constexpr int kSmemP = kTile;
-constexpr int kSmemK = 2 * kTile;                  // kStages tiles
-constexpr int kSmemV = kSmemK + kStages * kTile;   // kStages tiles
-constexpr int kSmemBytes = kSmemV + kStages * kTile;  // 192 KB
-constexpr int kTmemCols = 512;                     // S0: [0,128), S1: [128,256), O: [256,384)
+constexpr int kSoftmaxThreads = 128;               // one thread per query row
+constexpr int kThreadsTC = 256;  // 4 softmax warps, TMA producer, MMA issuer, 2 idle: registers are allotted per 4 warps
+constexpr int kRegionQ = kBM * 128;                // [128 rows][64] bf16, 128-byte rows: 16 KB
+constexpr int kRegionKV = kBN * 128;               // [64 positions][64] bf16: 8 KB
+constexpr int kTileKV = 2 * kRegionKV;             // a [64][128] K or V tile: 16 KB
+constexpr int kSmemQ = 0;                          // 2 regions (d 0-63, d 64-127)
+constexpr int kSmemK = 2 * kRegionQ;               // kStages tiles
+constexpr int kSmemV = kSmemK + kStages * kTileKV; // kStages tiles
+constexpr int kSmemP = kSmemV + kStages * kTileKV; // one region [128 rows][64 positions]
+constexpr int kSmemBar = kSmemP + kRegionQ;        // mbarriers and two words, 128 bytes
+constexpr int kSmemBytes = kSmemBar + 128;         // 112 KB + 128 B: two CTAs per SM
+constexpr int kTmemCols = 256;                     // S0: [0,64), S1: [64,128), O: [128,256)
 constexpr float kRescaleThreshold = 8.0f;          // log2 units
 constexpr long long kWaitCycles = 4000000000ll;    // about two seconds
 constexpr int kMaxSplit = 8;
@@ -190,63 +194,67 @@ __device__ __forceinline__ float fast_exp2(float x) {
 }
 __device__ __forceinline__ void softmax_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kSoftmaxThreads) : "memory"); }
 
+// 32 bits of the visibility vector of one query row, starting at tree index `start` (which may be
+// negative: prefix positions, always visible; or past the tree: never visible). aw = the row's
+// ancestor mask (bits >= n_tree are zero).
+__device__ __forceinline__ uint32_t vis_word(const uint32_t (&aw)[4], int i) {
+  return i < 0 ? 0xffffffffu : i == 0 ? aw[0] : i == 1 ? aw[1] : i == 2 ? aw[2] : i == 3 ? aw[3] : 0u;
+}
+__device__ __forceinline__ uint32_t vis_bits32(const uint32_t (&aw)[4], int start) {
+  const int wi = start >> 5, sh = start & 31;  // arithmetic shift: floor division for negative starts
+  const uint32_t lo = vis_word(aw, wi), hi = vis_word(aw, wi + 1);
+  return sh == 0 ? lo : ((lo >> sh) | (hi << (32 - sh)));
+}
+
 // Byte offset of 16-byte chunk `c` (0..7) of row `r` inside a 128B-swizzled [rows][64 bf16] region.
 __device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4)); }
 
 __device__ __forceinline__ int clampi(int x, int lo, int hi) { return x < lo ? lo : (x > hi ? hi : x); }
 
-// Per-sequence sizes and the number of KV splits actually used, from the tree sizes and prefix
-// lengths on the device: enough CTAs for about four waves, at least four tiles each where the
-// sequences are long enough, and never fewer CTAs than SMs when the work allows. Every warp
-// computes the same values (all 32 lanes must call). *N_b and *L_b receive the sizes of sequence b.
+// Per-sequence sizes and the number of KV splits of sequence b, from the tree sizes and prefix
+// lengths on the device. Work is cut into pieces of about `chunk` tiles, chunk = the total tile
+// count over twice the SM count (two CTAs share an SM), at least 4: one wave of equal-sized CTAs
+// whatever the mix of lengths, and as few splits as that allows. Every warp computes the same
+// values (all 32 lanes must call).
 __device__ __forceinline__ int effective_splits(const TcParams& p, int b, int* N_b, int* L_b) {
   const int lane = threadIdx.x & 31;
   const int max_pos = p.page_size == 0 ? p.seq_capacity : p.seq_capacity * p.page_size;
-  int active = 0, tiles = 0, Nb = 0, Lb = 0;
-  for (int b0 = 0; b0 < p.B; b0 += 32) {
-    const int bb = b0 + lane;
-    int N = 0, L = 0;
-    if (bb < p.B) {
-      N = clampi(p.n_tree[bb], 0, p.Nmax);
-      L = p.kv_len[bb];
-      L = L < 0 ? 0 : L;
-    }
+  int Nv[CAST_MAX_BATCH / 32], Lv[CAST_MAX_BATCH / 32];
+#pragma unroll
+  for (int k = 0; k < CAST_MAX_BATCH / 32; ++k) {  // all loads first: one memory round trip
+    const int bb = k * 32 + lane;
+    Nv[k] = bb < p.B ? p.n_tree[bb] : 0;
+    Lv[k] = bb < p.B ? p.kv_len[bb] : 0;
+  }
+  int tiles = 0, Nb = 0, Lb = 0;
+#pragma unroll
+  for (int k = 0; k < CAST_MAX_BATCH / 32; ++k) {
+    const int N = clampi(Nv[k], 0, p.Nmax), L = Lv[k] < 0 ? 0 : Lv[k];
     int total = L + N;
     total = total > max_pos ? max_pos : total;
-    const int nrb = (N * p.G + kBM - 1) / kBM;
-    active += p.Hkv * nrb;
-    tiles += p.Hkv * nrb * ((total + kBN - 1) / kBN);
-    if (b >= b0 && b < b0 + 32) {
-      Nb = __shfl_sync(0xffffffffu, N, b - b0);
-      Lb = __shfl_sync(0xffffffffu, L, b - b0);
+    tiles += p.Hkv * ((N * p.G + kBM - 1) / kBM) * ((total + kBN - 1) / kBN);
+    if ((b >> 5) == k) {
+      Nb = __shfl_sync(0xffffffffu, N, b & 31);
+      Lb = __shfl_sync(0xffffffffu, L, b & 31);
     }
   }
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    active += __shfl_xor_sync(0xffffffffu, active, o);
-    tiles += __shfl_xor_sync(0xffffffffu, tiles, o);
-  }
+  for (int o = 16; o > 0; o >>= 1) tiles += __shfl_xor_sync(0xffffffffu, tiles, o);
   *N_b = Nb;
   *L_b = Lb;
-  if (active == 0) return 1;
-  const int per = tiles / active;  // mean tiles per (sequence, kv-head, row block)
-  int want = active * per / 4;
-  want = want > 4 * p.num_sms ? 4 * p.num_sms : want;
-  want = want < p.num_sms ? p.num_sms : want;
-  int ns = (want + active - 1) / active;
+  int chunk = (tiles + 2 * p.num_sms - 1) / (2 * p.num_sms);
+  chunk = chunk < 4 ? 4 : chunk;
+  int total_b = Lb + Nb;
+  total_b = total_b > max_pos ? max_pos : total_b;
+  const int tiles_b = (total_b + kBN - 1) / kBN;
+  int ns = (tiles_b + chunk - 1) / chunk;
   ns = ns > p.nsplit_max ? p.nsplit_max : ns;
   return ns < 1 ? 1 : ns;
 }
 
-__global__ void __launch_bounds__(kThreadsTC, 1)
+__global__ void __launch_bounds__(kThreadsTC, 2)
 tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
-  extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) uint64_t bar_fullk[kStages], bar_fullv[kStages], bar_freek[kStages], bar_freev[kStages],
-      bar_s[2], bar_p;
-  __shared__ uint32_t tmem_base_s;
-  __shared__ int last_s;
-  __shared__ float xch[2][kBM * 2];
-  __shared__ uint32_t anc_s[kBM][CAST_MAX_TREE / 32];
+  extern __shared__ __align__(1024) unsigned char smem[];  // no static shared memory: the base is 1 KB aligned
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int split = blockIdx.x % p.nsplit_max, rb = blockIdx.x / p.nsplit_max;
@@ -271,19 +279,31 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
   const int ntiles = (total + kBN - 1) / kBN;  // >= 1 because N >= 1 here
   nsplit = nsplit > ntiles ? ntiles : nsplit;  // this sequence's splits: none of them is empty
   if (split >= nsplit) return;
+  if ((smem_u32(smem) & 1023u) != 0u) {  // the swizzled operand regions need a 1 KB aligned base
+    if (tid == 0) report(p.st, CAST_ERR_CUDA, 1024);
+    return;
+  }
   const int t0 = (int)((long long)split * ntiles / nsplit), t1 = (int)((long long)(split + 1) * ntiles / nsplit);
   const int ntile = t1 - t0;
-  const int half = (warp >> 2) & 1, quarter = warp & 3, r = quarter * 32 + lane;  // softmax-role coordinates
+  const int r = tid & (kBM - 1);  // softmax role: the query row of this thread
   const int row = row0 + r;
-  const bool row_ok = warp < 8 && row < rows_total;
+  const bool row_ok = warp < 4 && row < rows_total;
   const int t_tok = row_ok ? row / G : 0, h_q = kvh * G + (row_ok ? row % G : 0);
-  unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
 
-  // ---- producer helpers (warp 8; all 32 lanes call them) ----
-  // which = 0: K tile j into the K ring, which = 1: V tile j into the V ring
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kSmemBar);
+  uint64_t* bar_fullk = bars;          // [kStages]
+  uint64_t* bar_fullv = bars + 2;      // [kStages]
+  uint64_t* bar_freek = bars + 4;      // [kStages]
+  uint64_t* bar_freev = bars + 6;      // [kStages]
+  uint64_t* bar_s = bars + 8;          // [2]
+  uint64_t* bar_p = bars + 10;
+  uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(bars + 11);
+  int* last_s = reinterpret_cast<int*>(bars + 12);
+
+  // ---- producer helper (warp 4; all 32 lanes call it): which = 0: K tile j, which = 1: V tile j
   auto issue_tile = [&](int j, int which) -> bool {
     const int stage = j % kStages;
-    unsigned char* dst = smem + (which ? kSmemV : kSmemK) + stage * kTile;
+    unsigned char* dst = smem + (which ? kSmemV : kSmemK) + stage * kTileKV;
     uint64_t* full = which ? &bar_fullv[stage] : &bar_fullk[stage];
     const CUtensorMap* map = which ? &map_v : &map_k;
     const int pos0 = (t0 + j) * kBN;
@@ -303,15 +323,15 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     }
     if (j >= kStages && !mbar_wait(which ? &bar_freev[stage] : &bar_freek[stage], ((j / kStages) - 1) & 1)) return false;
     if (ps == 0) {
-      if (lane == 0) mbar_expect_tx(full, kTile);
+      if (lane == 0) mbar_expect_tx(full, kTileKV);
       __syncwarp();
-      if (lane < 2) tma_load_3d(map, dst + lane * kRegion, full, lane * 64, kvh, b * p.seq_capacity + pos0);
-    } else {  // at most 16 pages per tile (page size >= 8): one (page, column half) per lane
+      if (lane < 2) tma_load_3d(map, dst + lane * kRegionKV, full, lane * 64, kvh, b * p.seq_capacity + pos0);
+    } else {  // at most 8 pages per tile (page size >= 8): one (page, column half) per lane
       if (lane == 0) mbar_expect_tx(full, (uint32_t)npages * ps * 128 * 2);
       __syncwarp();
       if (lane < npages * 2) {
         const int slot = lane >> 1, hsel = lane & 1;
-        tma_load_4d(map, dst + hsel * kRegion + slot * ps * 128, full, hsel * 64, kvh, 0, page);
+        tma_load_4d(map, dst + hsel * kRegionKV + slot * ps * 128, full, hsel * 64, kvh, 0, page);
       }
     }
     __syncwarp();
@@ -331,7 +351,8 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
 
   int armed_k = 0, armed_v = 0;
   bool prod_ok = true;
-  if (warp == 8) {
+  uint32_t aw[4] = {0u, 0u, 0u, 0u};  // softmax role: ancestor mask of this thread's row
+  if (warp == 4) {
     if (lane == 0) {
       for (int s = 0; s < kStages; ++s) {
         mbar_init(&bar_fullk[s], 1);
@@ -341,44 +362,50 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
       }
       mbar_init(&bar_s[0], 1);
       mbar_init(&bar_s[1], 1);
-      mbar_init(&bar_p, kSoftmaxThreads);
+      mbar_init(bar_p, kSoftmaxThreads);
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       fence_proxy_async();
     }
     __syncwarp();
+    __threadfence_block();
+    asm volatile("bar.arrive 2, %0;" ::"n"(kThreadsTC) : "memory");
     // K0 K1 V0 V1 need no stage wait: the rings fill while the other warps stage Q
     for (int i = 0; i < 5 && prod_ok; ++i) {
       if (i == 3) continue;  // K2 waits for a stage; V1 (element 4) does not
       prod_ok = issue_seq(i, &armed_k, &armed_v);
     }
-  } else if (warp < 8) {
+  } else if (warp < 4) {
     if (warp == 0) {  // TMEM: two S buffers and O
-      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)),
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_base_s)),
                    "n"(kTmemCols));
       asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
     }
-    // Q rows -> swizzled shared memory (rows past the tree are zero); ancestor masks
-    const __nv_bfloat16* qrow = p.q + (((size_t)b * p.Ncap + t_tok) * p.Hq + h_q) * kHD + half * 64;
-    uint4 qv[8];
+    // Q row -> swizzled shared memory (rows past the tree are zero); ancestor mask -> registers
+    const __nv_bfloat16* qrow = p.q + (((size_t)b * p.Ncap + t_tok) * p.Hq + h_q) * kHD;
+    uint4 qv[16];
 #pragma unroll
-    for (int c = 0; c < 8; ++c) qv[c] = row_ok ? *reinterpret_cast<const uint4*>(qrow + c * 8) : make_uint4(0u, 0u, 0u, 0u);
+    for (int c = 0; c < 16; ++c) qv[c] = row_ok ? *reinterpret_cast<const uint4*>(qrow + c * 8) : make_uint4(0u, 0u, 0u, 0u);
+    if (row_ok) {
 #pragma unroll
-    for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(smem + kSmemQ + half * kRegion + swz(r, c)) = qv[c];
-    if (half == 0) {
-      for (int w = 0; w < CAST_MAX_TREE / 32; ++w)
-        anc_s[r][w] = (row_ok && w < p.words) ? p.anc[((size_t)b * p.Ncap + t_tok) * p.words + w] : 0u;
+      for (int w = 0; w < 4; ++w)
+        if (w < p.words) aw[w] = p.anc[((size_t)b * p.Ncap + t_tok) * p.words + w];
     }
+#pragma unroll
+    for (int c = 0; c < 16; ++c)
+      *reinterpret_cast<uint4*>(smem + kSmemQ + (c >> 3) * kRegionQ + swz(r, c & 7)) = qv[c];
     fence_proxy_async();
   }
   TC_MARK(2);
+  // everyone but the producer waits here for the barrier objects, the TMEM address and Q; the producer
+  // only signals that the barriers exist (it arrived right after initialising them) and keeps loading
   tc_fence_before();
-  __syncthreads();
+  if (warp != 4) asm volatile("bar.sync 2, %0;" ::"n"(kThreadsTC) : "memory");
   tc_fence_after();
   TC_MARK(3);
-  const uint32_t tmem_base = tmem_base_s;
+  const uint32_t tmem_base = *tmem_base_s;
   const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 2 * kBN;
 
-  if (warp == 8) {
+  if (warp == 4) {
     // =========================== TMA producer ===========================
     bool ok = prod_ok;
     if (ok) ok = issue_seq(3, &armed_k, &armed_v);  // K2
@@ -394,23 +421,23 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
         }
       }
     }
-  } else if (warp == 9) {
+  } else if (warp == 5) {
     // =========================== MMA issuer ===========================
     const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
-    const uint32_t idesc_pv = idesc_qk | (1u << 16);  // B operand (V) is MN-major; N = head dim = 128 as well
+    const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(kHD >> 3) << 17) |
+                              ((uint32_t)(kBM >> 4) << 24);  // B operand (V) is MN-major, N = head dim
     // descriptors differ only in the start-address field (16-byte units), so they are built once
     const uint64_t dq = umma_desc(smem_u32(smem + kSmemQ), 16, 1024);
     const uint64_t dk = umma_desc(smem_u32(smem + kSmemK), 16, 1024);
-    const uint64_t dv = umma_desc(smem_u32(smem + kSmemV), kRegion, 1024);
+    const uint64_t dv = umma_desc(smem_u32(smem + kSmemV), kRegionKV, 1024);
     const uint64_t dp = umma_desc(smem_u32(smem + kSmemP), 16, 1024);
     auto mma_qk = [&](int stage, int buf) {  // S[buf] = Q K^T; releases the K stage
       if (lane == 0) {
-        const uint64_t dks = dk + (uint64_t)(stage * (kTile >> 4));
+        const uint64_t dks = dk + (uint64_t)(stage * (kTileKV >> 4));
 #pragma unroll
-        for (int ks = 0; ks < kHD / 16; ++ks) {
-          const uint64_t off = (uint64_t)((ks >> 2) * (kRegion >> 4) + (ks & 3) * 2);
-          umma_bf16(tmem_s + buf * kBN, dq + off, dks + off, idesc_qk, ks > 0);
-        }
+        for (int ks = 0; ks < kHD / 16; ++ks)
+          umma_bf16(tmem_s + buf * kBN, dq + (uint64_t)((ks >> 2) * (kRegionQ >> 4) + (ks & 3) * 2),
+                    dks + (uint64_t)((ks >> 2) * (kRegionKV >> 4) + (ks & 3) * 2), idesc_qk, ks > 0);
         umma_commit(&bar_s[buf]);
         umma_commit(&bar_freek[stage]);
       }
@@ -418,15 +445,17 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     };
     auto mma_pv = [&](int stage, bool first) {  // O (+)= P V; releases the V stage (and P)
       if (lane == 0) {
-        const uint64_t dvs = dv + (uint64_t)(stage * (kTile >> 4));
+        const uint64_t dvs = dv + (uint64_t)(stage * (kTileKV >> 4));
 #pragma unroll
         for (int ks = 0; ks < kBN / 16; ++ks)
-          umma_bf16(tmem_o, dp + (uint64_t)((ks >> 2) * (kRegion >> 4) + (ks & 3) * 2), dvs + (uint64_t)(ks * (2048 >> 4)),
-                    idesc_pv, (!first || ks > 0) ? 1u : 0u);
+          umma_bf16(tmem_o, dp + (uint64_t)(ks * 2), dvs + (uint64_t)(ks * (2048 >> 4)), idesc_pv,
+                    (!first || ks > 0) ? 1u : 0u);
         umma_commit(&bar_freev[stage]);
       }
       __syncwarp();
     };
+    // next scores first: Q K^T of tile it+1 runs while the softmax of tile `it` does; the other CTA on
+    // this SM covers the moments when a K tile is late
     bool ok = mbar_wait(&bar_fullk[0], 0);
     if (ok) {
       tc_fence_after();
@@ -434,7 +463,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     }
     for (int it = 0; ok && it < ntile; ++it) {
       TC_STAMP(1, it, 0);
-      if (it + 1 < ntile) {  // next scores first: they are computed while the softmax of tile `it` runs
+      if (it + 1 < ntile) {
         ok = mbar_wait(&bar_fullk[(it + 1) % kStages], ((it + 1) / kStages) & 1);
         if (!ok) break;
         TC_STAMP(1, it, 1);
@@ -442,7 +471,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
         mma_qk((it + 1) % kStages, (it + 1) & 1);
         TC_STAMP(1, it, 2);
       }
-      ok = mbar_wait(&bar_p, it & 1) && mbar_wait(&bar_fullv[it % kStages], (it / kStages) & 1);
+      ok = mbar_wait(bar_p, it & 1) && mbar_wait(&bar_fullv[it % kStages], (it / kStages) & 1);
       if (!ok) break;
       TC_STAMP(1, it, 3);
       tc_fence_after();
@@ -450,157 +479,166 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
       TC_STAMP(1, it, 4);
     }
     if (!ok && lane == 0) report(p.st, CAST_ERR_TIMEOUT, b);
-  } else {
+  } else if (warp < 4) {
     // =========================== softmax warps ===========================
     // After a wait has expired a thread keeps visiting the barriers (so nobody blocks on it) but
     // touches neither TMEM nor the operand buffers. A warp whose 32 rows all lie past the tree
     // only keeps the barriers in step: its P rows feed output rows nobody reads.
-    const uint32_t lane_sel = (uint32_t)(quarter * 32) << 16;
-    const bool warp_live = row0 + quarter * 32 < rows_total;
+    const uint32_t lane_sel = (uint32_t)(warp * 32) << 16;
+    const bool warp_live = row0 + warp * 32 < rows_total;
     const float sc = p.scale_log2;
     float m_used = -INFINITY, l_run = 0.f;  // m_used: running reference maximum in raw score units
     bool ok = true;
     for (int it = 0; it < ntile; ++it) {
       const int buf = it & 1, stage = it % kStages;
       const int pos0 = (t0 + it) * kBN;
-      uint32_t sr[64];
-      float mx = -INFINITY;
       TC_STAMP(0, it, 0);
+      float mx = -INFINITY;
+      uint32_t v0 = 0xffffffffu, v1 = 0xffffffffu;  // visibility of this row's 64 columns
       if (warp_live) {
         if (ok) ok = mbar_wait(&bar_s[buf], (it >> 1) & 1);
         TC_STAMP(0, it, 1);
         if (ok) {
           tc_fence_after();
-          tmem_ld32(tmem_s + buf * kBN + lane_sel + half * 64, sr);
-          tmem_ld32(tmem_s + buf * kBN + lane_sel + half * 64 + 32, sr + 32);
-          tmem_wait_ld();
-          TC_STAMP(0, it, 2);
-          const int cbase = pos0 + half * 64;
-          if (cbase + 64 > L) {  // this thread's 64 columns reach past the prefix: ancestor mask
-#pragma unroll
-            for (int c = 0; c < 64; ++c) {
-              const int pos = cbase + c;
-              bool v = pos < L;
-              if (!v && pos < total) {
-                const int j = pos - L;
-                v = (anc_s[r][j >> 5] >> (j & 31)) & 1u;
-              }
-              if (!v) sr[c] = 0xff800000u;  // -inf
-            }
+          if (pos0 + kBN > L) {  // the tile reaches past the prefix: ancestor mask
+            v0 = vis_bits32(aw, pos0 - L);
+            v1 = vis_bits32(aw, pos0 - L + 32);
           }
-          float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
-#pragma unroll
-          for (int c = 0; c < 64; c += 4) {
-            m0 = fmaxf(m0, __uint_as_float(sr[c]));
-            m1 = fmaxf(m1, __uint_as_float(sr[c + 1]));
-            m2 = fmaxf(m2, __uint_as_float(sr[c + 2]));
-            m3 = fmaxf(m3, __uint_as_float(sr[c + 3]));
-          }
-          mx = row_ok ? fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) : -INFINITY;
-        }
-      }
-      TC_STAMP(0, it, 3);
-      xch[buf][half * kBM + r] = mx;
-      softmax_bar();
-      mx = fmaxf(mx, xch[buf][(half ^ 1) * kBM + r]);
-      TC_STAMP(0, it, 4);
-      // P (and O) were last touched by the P V product of tile it-1
-      if (warp_live && ok && it >= 1) ok = mbar_wait(&bar_freev[(it - 1) % kStages], ((it - 1) / kStages) & 1);
-      TC_STAMP(0, it, 5);
-      if (warp_live && ok) {
-        // lazy maximum: move the reference only when the row maximum outgrows it by 2^8
-        float alpha = 1.f;
-        const bool grow = (mx - m_used) * sc > kRescaleThreshold || (m_used == -INFINITY && mx > -INFINITY);
-        if (grow) {
-          alpha = fast_exp2((m_used - mx) * sc);  // 0 when m_used = -inf
-          m_used = mx;
-          l_run *= alpha;
-        }
-        if (it > 0 && __any_sync(0xffffffffu, grow)) {  // rescale this thread's 64 columns of O
-          tc_fence_after();
-          uint32_t orr[32];
+          if (!row_ok) v0 = v1 = 0u;
+          // pass 1: the row maximum (the scores are read again from TMEM in pass 2: registers are scarce
+          // with two CTAs per SM, TMEM bandwidth is not)
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {
-            const uint32_t ta = tmem_o + lane_sel + half * 64 + hh * 32;
-            tmem_ld32(ta, orr);
+            uint32_t sr[32];
+            tmem_ld32(tmem_s + buf * kBN + lane_sel + hh * 32, sr);
             tmem_wait_ld();
+            const uint32_t vv = hh ? v1 : v0;
+            float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
-            for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
-            tmem_st32(ta, orr);
+            for (int c = 0; c < 32; c += 4) {
+              m0 = fmaxf(m0, ((vv >> c) & 1u) ? __uint_as_float(sr[c]) : -INFINITY);
+              m1 = fmaxf(m1, ((vv >> (c + 1)) & 1u) ? __uint_as_float(sr[c + 1]) : -INFINITY);
+              m2 = fmaxf(m2, ((vv >> (c + 2)) & 1u) ? __uint_as_float(sr[c + 2]) : -INFINITY);
+              m3 = fmaxf(m3, ((vv >> (c + 3)) & 1u) ? __uint_as_float(sr[c + 3]) : -INFINITY);
+            }
+            mx = fmaxf(mx, fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)));
           }
-          tmem_wait_st();
+          TC_STAMP(0, it, 2);
         }
-        TC_STAMP(0, it, 6);
-        // P = 2^((s - m) * scale) as bf16 into the swizzled A-operand buffer; row sum in fp32
-        const bool live = m_used > -INFINITY;
-        const float neg_ms = live ? -m_used * sc : 0.f;
-        float l0 = 0.f, l1 = 0.f;
-        unsigned char* prow = smem + kSmemP + half * kRegion;
-#pragma unroll
-        for (int c8 = 0; c8 < 8; ++c8) {
-          uint32_t pk[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            float p0 = fast_exp2(fmaf(__uint_as_float(sr[c8 * 8 + 2 * e]), sc, neg_ms));
-            float p1 = fast_exp2(fmaf(__uint_as_float(sr[c8 * 8 + 2 * e + 1]), sc, neg_ms));
-            if (!live) p0 = p1 = 0.f;
-            l0 += p0;
-            l1 += p1;
-            const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
-            pk[e] = *reinterpret_cast<const uint32_t*>(&pb);
+        TC_STAMP(0, it, 3);
+      }
+      // P (and O) were last touched by the P V product of tile it-1. Every warp waits here, live or not:
+      // it also keeps a warp from arriving on bar_p for tile `it` before the phase of tile it-1 is over.
+      if (ok && it >= 1) ok = mbar_wait(&bar_freev[(it - 1) % kStages], ((it - 1) / kStages) & 1);
+      TC_STAMP(0, it, 5);
+      if (warp_live) {
+        if (ok) {
+          // lazy maximum: move the reference only when the row maximum outgrows it by 2^8
+          float alpha = 1.f;
+          const bool grow = (mx - m_used) * sc > kRescaleThreshold || (m_used == -INFINITY && mx > -INFINITY);
+          if (grow) {
+            alpha = fast_exp2((m_used - mx) * sc);  // 0 when m_used = -inf
+            m_used = mx;
+            l_run *= alpha;
           }
-          *reinterpret_cast<uint4*>(prow + swz(r, c8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          if (it > 0 && __any_sync(0xffffffffu, grow)) {  // rescale this row of O
+            tc_fence_after();
+#pragma unroll
+            for (int hh = 0; hh < 4; ++hh) {
+              uint32_t orr[32];
+              const uint32_t ta = tmem_o + lane_sel + hh * 32;
+              tmem_ld32(ta, orr);
+              tmem_wait_ld();
+#pragma unroll
+              for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
+              tmem_st32(ta, orr);
+            }
+            tmem_wait_st();
+          }
+          TC_STAMP(0, it, 6);
+          // pass 2: P = 2^((s - m) * scale) as bf16 into the swizzled A-operand buffer; row sum in fp32
+          const bool live = m_used > -INFINITY;
+          const float neg_ms = live ? -m_used * sc : 0.f;
+          float l0 = 0.f, l1 = 0.f;
+          unsigned char* prow = smem + kSmemP;
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            uint32_t sr[32];
+            tmem_ld32(tmem_s + buf * kBN + lane_sel + hh * 32, sr);
+            tmem_wait_ld();
+            const uint32_t vv = live ? (hh ? v1 : v0) : 0u;
+#pragma unroll
+            for (int c8 = 0; c8 < 4; ++c8) {
+              uint32_t pk[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const int c = c8 * 8 + 2 * e;
+                float p0 = fast_exp2(fmaf(__uint_as_float(sr[c]), sc, neg_ms));
+                float p1 = fast_exp2(fmaf(__uint_as_float(sr[c + 1]), sc, neg_ms));
+                p0 = ((vv >> c) & 1u) ? p0 : 0.f;
+                p1 = ((vv >> (c + 1)) & 1u) ? p1 : 0.f;
+                l0 += p0;
+                l1 += p1;
+                const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+                pk[e] = *reinterpret_cast<const uint32_t*>(&pb);
+              }
+              *reinterpret_cast<uint4*>(prow + swz(r, hh * 4 + c8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            }
+          }
+          l_run += l0 + l1;
         }
-        l_run += l0 + l1;
       }
       // V rows past the end of the sequence may hold anything (0 * NaN would poison O): zero them
       if (ok && total - pos0 < kBN) {
         ok = mbar_wait(&bar_fullv[stage], (it / kStages) & 1);  // the tile has landed
         if (ok) {
           const int valid = total - pos0;
-          unsigned char* vbase = smem + kSmemV + stage * kTile;
+          unsigned char* vbase = smem + kSmemV + stage * kTileKV;
           for (int i = tid; i < (kBN - valid) * 16; i += kSoftmaxThreads) {
             const int rr = valid + (i >> 4), reg = (i >> 3) & 1, c = i & 7;
-            *reinterpret_cast<uint4*>(vbase + reg * kRegion + rr * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4*>(vbase + reg * kRegionKV + rr * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
           }
         }
       }
       TC_STAMP(0, it, 7);
       fence_proxy_async();
       tc_fence_before();
-      mbar_arrive(&bar_p);
+      mbar_arrive(bar_p);
       TC_STAMP(0, it, 9);
     }
-    // epilogue: wait for the last P V; O goes through shared memory (the K/V rings are idle now) so
-    // that every global store of a row is one contiguous 512-byte (fp32) or 256-byte (bf16) piece
+    // epilogue: wait for the last P V; O goes through shared memory (the K/V rings and P are idle
+    // now) so that every global store of a row is one contiguous 512-byte (fp32) or 256-byte (bf16) piece
     TC_MARK(4);
     if (ok) ok = mbar_wait(&bar_freev[(ntile - 1) % kStages], ((ntile - 1) / kStages) & 1);
     TC_MARK(5);
     constexpr int kStageStride = kHD + 4;  // floats per staged row: 16-byte stores stay conflict-free
-    float* stage_o = reinterpret_cast<float*>(smem + kSmemK);
-    xch[0][half * kBM + r] = l_run;
-    if (half == 0) xch[1][r] = m_used * sc * 0.69314718055994531f;  // natural-log units
+    float* stage_o = reinterpret_cast<float*>(smem + kSmemK);  // 128 x 132 floats < K ring + V ring + P
+    float* stage_ml = reinterpret_cast<float*>(smem + kSmemQ);  // [128][2]: Q is idle as well
     if (ok && warp_live) {
       tc_fence_after();
-      uint32_t orr[64];
-      tmem_ld32(tmem_o + lane_sel + half * 64, orr);
-      tmem_ld32(tmem_o + lane_sel + half * 64 + 32, orr + 32);
-      tmem_wait_ld();
-      float* so = stage_o + r * kStageStride + half * 64;
 #pragma unroll
-      for (int c4 = 0; c4 < 16; ++c4)
-        *reinterpret_cast<float4*>(so + c4 * 4) =
-            make_float4(__uint_as_float(orr[c4 * 4]), __uint_as_float(orr[c4 * 4 + 1]), __uint_as_float(orr[c4 * 4 + 2]),
-                        __uint_as_float(orr[c4 * 4 + 3]));
+      for (int hh = 0; hh < 4; ++hh) {
+        uint32_t orr[32];
+        tmem_ld32(tmem_o + lane_sel + hh * 32, orr);
+        tmem_wait_ld();
+        float* so = stage_o + r * kStageStride + hh * 32;
+#pragma unroll
+        for (int c4 = 0; c4 < 8; ++c4)
+          *reinterpret_cast<float4*>(so + c4 * 4) =
+              make_float4(__uint_as_float(orr[c4 * 4]), __uint_as_float(orr[c4 * 4 + 1]), __uint_as_float(orr[c4 * 4 + 2]),
+                          __uint_as_float(orr[c4 * 4 + 3]));
+      }
+      stage_ml[r * 2] = m_used * sc * 0.69314718055994531f;  // natural-log units
+      stage_ml[r * 2 + 1] = l_run;
     }
     softmax_bar();
     const int rows_here = rows_total - row0 < kBM ? rows_total - row0 : kBM;
-    const int wv = warp;  // 0..7: rows wv, wv+8, ... ; lane: columns 4*lane .. 4*lane+3
+    const int wv = warp;  // 0..3: rows wv, wv+4, ... ; lane: columns 4*lane .. 4*lane+3
     if (ok) {
-      for (int rr = wv; rr < rows_here; rr += 8) {
+      for (int rr = wv; rr < rows_here; rr += 4) {
         const int grow = row0 + rr, tt = grow / G, hh = kvh * G + grow % G;
         const float4 o4 = *reinterpret_cast<const float4*>(stage_o + rr * kStageStride + lane * 4);
-        const float l_tot = xch[0][rr] + xch[0][kBM + rr];
+        const float l_tot = stage_ml[rr * 2 + 1];
         if (nsplit == 1) {
           const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
           const __nv_bfloat162 a = __floats2bfloat162_rn(o4.x * inv, o4.y * inv), c2 = __floats2bfloat162_rn(o4.z * inv, o4.w * inv);
@@ -612,7 +650,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
           const size_t pr = (((size_t)b * p.Hq + hh) * p.Ncap + tt) * p.nsplit_max + split;
           __stcg(reinterpret_cast<float4*>(p.part_o + pr * kHD + lane * 4), o4);
           if (lane == 0) {
-            __stcg(p.part_ml + pr * 2, xch[1][rr]);
+            __stcg(p.part_ml + pr * 2, stage_ml[rr * 2]);
             __stcg(p.part_ml + pr * 2 + 1, l_tot);
           }
         }
@@ -625,16 +663,16 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
       if (tid == 0) {
         int32_t* cnt = p.ticket + ((size_t)b * p.Hkv + kvh) * p.nrb + rb;
         const int t = atomicAdd(cnt, 1);
-        last_s = (t == nsplit - 1);
+        *last_s = (t == nsplit - 1);
         if (t == nsplit - 1) *cnt = 0;
         __threadfence();
       }
       softmax_bar();
-      if (last_s) TC_CTA_LOG(3, gtimer());
-      if (last_s) {
+      if (*last_s) TC_CTA_LOG(3, gtimer());
+      if (*last_s) {
         // every lane keeps up to 16 loads in flight (two rows x up to kMaxSplit splits): the merge is
         // bound by L2 latency, not by bytes
-        for (int rr = wv; rr < rows_here; rr += 16) {
+        for (int rr = wv; rr < rows_here; rr += 8) {
           float4 acc[2];
           float inv[2];
           size_t orow[2];
@@ -642,7 +680,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
           float wgt[2];
 #pragma unroll
           for (int u = 0; u < 2; ++u) {
-            const int r2 = rr + 8 * u;
+            const int r2 = rr + 4 * u;
             const bool on = r2 < rows_here;
             const int grow = row0 + (on ? r2 : rr), tt = grow / G, hh = kvh * G + grow % G;
             const size_t pr = (((size_t)b * p.Hq + hh) * p.Ncap + tt) * p.nsplit_max;
@@ -676,7 +714,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
               acc[u].z += v[u][s2].z * w;
               acc[u].w += v[u][s2].w * w;
             }
-            if (rr + 8 * u < rows_here) {
+            if (rr + 4 * u < rows_here) {
               const __nv_bfloat162 a = __floats2bfloat162_rn(acc[u].x * inv[u], acc[u].y * inv[u]),
                                    c2 = __floats2bfloat162_rn(acc[u].z * inv[u], acc[u].w * inv[u]);
               uint2 pk;
@@ -699,6 +737,65 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols));
   }
 }
+
+#ifdef CAST_PHASE_CLOCKS
+// Development aid: streams the same K/V tiles through the same TMA boxes and does nothing else.
+__global__ void __launch_bounds__(64, 2) dbg_loadonly_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
+                                                             const __grid_constant__ CUtensorMap map_v, int kvh_fast) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 4 * 2 * kTileKV);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int split, rb, kvh;
+  if (kvh_fast) { kvh = blockIdx.x; split = blockIdx.y % p.nsplit_max; rb = blockIdx.y / p.nsplit_max; }
+  else { split = blockIdx.x % p.nsplit_max; rb = blockIdx.x / p.nsplit_max; kvh = blockIdx.y; }
+  const int b = blockIdx.z;
+  int N, L;
+  int nsplit = effective_splits(p, b, &N, &L);
+  if (rb * kBM >= N * p.G) return;
+  const int total = L + N, ntiles = (total + kBN - 1) / kBN;
+  nsplit = nsplit > ntiles ? ntiles : nsplit;
+  if (split >= nsplit) return;
+  const int t0 = (int)((long long)split * ntiles / nsplit), t1 = (int)((long long)(split + 1) * ntiles / nsplit);
+  const int ntile = t1 - t0;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < 4; ++s) mbar_init(&bars[s], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async();
+  }
+  __syncthreads();
+  if (warp == 0) {
+    for (int j = 0; j < ntile + 3; ++j) {
+      if (j >= 3) {  // consume tile j-3
+        const int jj = j - 3;
+        if (!mbar_wait(&bars[jj % 4], (jj / 4) & 1)) break;
+      }
+      if (j < ntile) {
+        const int stage = j % 4, pos0 = (t0 + j) * kBN, ps = p.page_size;
+        unsigned char* dst = smem + stage * 2 * kTileKV;
+        if (ps == 0) {
+          if (lane == 0) mbar_expect_tx(&bars[stage], 2 * kTileKV);
+          __syncwarp();
+          if (lane < 4) tma_load_3d(lane < 2 ? &map_k : &map_v, dst + lane * kRegionKV, &bars[stage], (lane & 1) * 64, kvh,
+                                    b * p.seq_capacity + pos0);
+        } else {
+          int npages = (total - pos0 + ps - 1) / ps;
+          npages = npages > kBN / ps ? kBN / ps : npages;
+          int page = 0;
+          if (lane < npages * 4) page = p.page_table[(size_t)b * p.seq_capacity + pos0 / ps + (lane >> 2)];
+          if (lane == 0) mbar_expect_tx(&bars[stage], (uint32_t)npages * ps * 128 * 4);
+          __syncwarp();
+          if (lane < npages * 4) {
+            const int slot = lane >> 2, which = lane & 3;
+            tma_load_4d(which < 2 ? &map_k : &map_v, dst + which * kRegionKV + slot * ps * 128, &bars[stage], (which & 1) * 64,
+                        kvh, 0, page);
+          }
+        }
+        __syncwarp();
+      }
+    }
+  }
+}
+#endif
 
 EncodeTiledFn get_encode() {
   static EncodeTiledFn fn = nullptr;
@@ -738,6 +835,57 @@ bool make_kv_map(CUtensorMap* map, const void* base, int B, int Hkv, int page_si
 
 }  // namespace
 
+#ifdef CAST_PHASE_CLOCKS
+extern "C" __attribute__((visibility("default"))) int cast_debug_tc_occupancy_at(int bytes) {
+  int n = -1;
+  cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, tree_attn_tc_kernel, kThreadsTC, bytes);
+  return n;
+}
+__global__ void __launch_bounds__(256, 2) dbg_plain_kernel(float* x) {
+  float acc[96];
+#pragma unroll
+  for (int i = 0; i < 96; ++i) acc[i] = x[i * 256 + threadIdx.x];
+#pragma unroll
+  for (int k = 0; k < 8; ++k)
+#pragma unroll
+    for (int i = 0; i < 96; ++i) acc[i] = acc[i] * acc[(i + k + 1) % 96] + 1.f;
+#pragma unroll
+  for (int i = 0; i < 96; ++i) x[i * 256 + threadIdx.x] = acc[i];
+}
+extern "C" __attribute__((visibility("default"))) int cast_debug_occ_bs(int bytes, int bs, int which) {
+  int n = -1;
+  if (which == 0) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, tree_attn_tc_kernel, bs, bytes);
+  else {
+    cudaFuncAttributes a; cudaFuncGetAttributes(&a, dbg_plain_kernel);
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, dbg_plain_kernel, bs, bytes);
+    n = n * 1000 + a.numRegs;
+  }
+  return n;
+}
+extern "C" __attribute__((visibility("default"))) int cast_debug_tc_attrs(int* out) {
+  cudaFuncAttributes a;
+  cudaError_t e = cudaFuncGetAttributes(&a, tree_attn_tc_kernel);
+  out[0] = a.numRegs; out[1] = (int)a.sharedSizeBytes; out[2] = a.maxThreadsPerBlock; out[3] = (int)a.localSizeBytes;
+  out[4] = a.maxDynamicSharedSizeBytes; out[5] = a.preferredShmemCarveout; out[6] = (int)a.constSizeBytes;
+  int dev = 0, v = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&v, cudaDevAttrMaxBlocksPerMultiprocessor, dev); out[7] = v;
+  cudaDeviceGetAttribute(&v, cudaDevAttrMaxRegistersPerMultiprocessor, dev); out[8] = v;
+  cudaDeviceGetAttribute(&v, cudaDevAttrMaxRegistersPerBlock, dev); out[9] = v;
+  cudaDeviceGetAttribute(&v, cudaDevAttrReservedSharedMemoryPerBlock, dev); out[10] = v;
+  return (int)e;
+}
+extern "C" __attribute__((visibility("default"))) int cast_debug_tc_occupancy() {
+  int n = -1;
+  cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, tree_attn_tc_kernel, kThreadsTC, kSmemBytes);
+  return n;
+}
+#endif
+
 bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const void* v, int B, int Hq, int Hkv, int D,
                               int page_size, const int32_t* page_table, int seq_capacity, int num_pages,
                               const int32_t* kv_len, const uint32_t* anc, const int32_t* n_tree, float scale, void* out,
@@ -757,9 +905,8 @@ bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const v
   const int max_pos = page_size == 0 ? seq_capacity : seq_capacity * page_size;
   const int max_tiles = (max_pos + kBN - 1) / kBN;
   // upper bound of the KV splits; the kernel picks the actual number from the device-side sizes
-  int nsplit_max = (4 * c->num_sms + B * Hkv - 1) / (B * Hkv);
+  int nsplit_max = kMaxSplit;
   if (nsplit_max > max_tiles) nsplit_max = max_tiles;
-  if (nsplit_max > kMaxSplit) nsplit_max = kMaxSplit;
   if (nsplit_max < 1) nsplit_max = 1;
   TcParams p;
   p.q = (const __nv_bfloat16*)q; p.out = (__nv_bfloat16*)out;
@@ -793,14 +940,27 @@ bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const v
   }
   static bool attr_done = false;
   if (!attr_done) {
-    if (cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes + 1024) !=
+    if (cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) !=
         cudaSuccess) {
       *status = CAST_ERR_CUDA;
       return true;
     }
+    // two CTAs per SM need the largest shared-memory carve-out
+    cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
     attr_done = true;
   }
-  tree_attn_tc_kernel<<<dim3(nsplit_max * nrb, Hkv, B), kThreadsTC, kSmemBytes + 1024, stream>>>(p, map_k, map_v);
+#ifdef CAST_PHASE_CLOCKS
+  if (const char* lo = getenv("CAST_TC_LOADONLY")) {
+    const int kvh_fast = atoi(lo) == 2;
+    cudaFuncSetAttribute(dbg_loadonly_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * 2 * kTileKV + 64);
+    cudaFuncSetAttribute(dbg_loadonly_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+    const dim3 g = kvh_fast ? dim3(Hkv, nsplit_max * nrb, B) : dim3(nsplit_max * nrb, Hkv, B);
+    dbg_loadonly_kernel<<<g, 64, 4 * 2 * kTileKV + 64, stream>>>(p, map_k, map_v, kvh_fast);
+    *status = launch_status();
+    return true;
+  }
+#endif
+  tree_attn_tc_kernel<<<dim3(nsplit_max * nrb, Hkv, B), kThreadsTC, kSmemBytes, stream>>>(p, map_k, map_v);
   *status = launch_status();
   return true;
 }
