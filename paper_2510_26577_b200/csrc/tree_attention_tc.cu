@@ -211,45 +211,127 @@ __device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * 12
 
 __device__ __forceinline__ int clampi(int x, int lo, int hi) { return x < lo ? lo : (x > hi ? hi : x); }
 
-// Per-sequence sizes and the number of KV splits of sequence b, from the tree sizes and prefix
-// lengths on the device. Work is cut into pieces of about `chunk` tiles, chunk = the total tile
-// count over twice the SM count (two CTAs share an SM), at least 4: one wave of equal-sized CTAs
-// whatever the mix of lengths, and as few splits as that allows. Every warp computes the same
-// values (all 32 lanes must call).
-__device__ __forceinline__ int effective_splits(const TcParams& p, int b, int* N_b, int* L_b) {
+// The grid is one-dimensional: CTA i takes work item i. Items are enumerated on the device from
+// the actual tree sizes and prefix lengths: sequence b has Hkv * row_blocks(b) * splits(b) of them,
+// the kv-head running fastest so that the heads of one piece of a sequence stream the same pages at
+// the same time. splits(b) = ceil(tiles(b) / chunk); chunk (>= 4 tiles) is the smallest piece size
+// for which all items fit into W waves of 2 * num_sms CTAs, W being the number of waves that even
+// unsplit work would need. So the CTAs are of about equal size whatever the mix of lengths, there are
+// as few splits as the machine allows, and CTAs beyond the item count exit at once. Every warp
+// computes the same values (all 32 lanes must call).
+struct WorkItem {
+  int b, kvh, rb, split, nsplit, N, L;
+  bool valid;
+};
+
+__device__ __forceinline__ int warp_sum(int v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ WorkItem decode_work(const TcParams& p, int idx, int grid) {
+  constexpr int KB = CAST_MAX_BATCH / 32;
   const int lane = threadIdx.x & 31;
   const int max_pos = p.page_size == 0 ? p.seq_capacity : p.seq_capacity * p.page_size;
-  int Nv[CAST_MAX_BATCH / 32], Lv[CAST_MAX_BATCH / 32];
+  int Nv[KB], Lv[KB], tl[KB], nr[KB];
 #pragma unroll
-  for (int k = 0; k < CAST_MAX_BATCH / 32; ++k) {  // all loads first: one memory round trip
+  for (int k = 0; k < KB; ++k) {  // all loads first: one memory round trip
     const int bb = k * 32 + lane;
     Nv[k] = bb < p.B ? p.n_tree[bb] : 0;
     Lv[k] = bb < p.B ? p.kv_len[bb] : 0;
   }
-  int tiles = 0, Nb = 0, Lb = 0;
+  int base = 0, T = 0, tmax = 0;
 #pragma unroll
-  for (int k = 0; k < CAST_MAX_BATCH / 32; ++k) {
-    const int N = clampi(Nv[k], 0, p.Nmax), L = Lv[k] < 0 ? 0 : Lv[k];
-    int total = L + N;
+  for (int k = 0; k < KB; ++k) {
+    Nv[k] = clampi(Nv[k], 0, p.Nmax);
+    Lv[k] = Lv[k] < 0 ? 0 : Lv[k];
+    int total = Lv[k] + Nv[k];
     total = total > max_pos ? max_pos : total;
-    tiles += p.Hkv * ((N * p.G + kBM - 1) / kBM) * ((total + kBN - 1) / kBN);
-    if ((b >> 5) == k) {
-      Nb = __shfl_sync(0xffffffffu, N, b & 31);
-      Lb = __shfl_sync(0xffffffffu, L, b & 31);
+    nr[k] = (Nv[k] * p.G + kBM - 1) / kBM;
+    tl[k] = nr[k] > 0 ? (total + kBN - 1) / kBN : 0;
+    base += p.Hkv * nr[k];
+    T += p.Hkv * nr[k] * tl[k];
+    tmax = tl[k] > tmax ? tl[k] : tmax;
+  }
+  base = warp_sum(base);
+  T = warp_sum(T);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) tmax = max(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
+  const int slots = 2 * p.num_sms;
+  int W = (base + slots - 1) / slots;
+  W = W < 1 ? 1 : W;
+  int cap = W * slots;
+  cap = cap > grid ? grid : cap;
+  // smallest chunk (>= 4 tiles) whose item count fits: the count falls as the chunk grows, and a chunk
+  // of tmax tiles (no splits at all) always fits
+  auto items_at = [&](int chunk) {
+    int items = 0;
+#pragma unroll
+    for (int k = 0; k < KB; ++k) {
+      int n = (tl[k] + chunk - 1) / chunk;
+      n = n > p.nsplit_max ? p.nsplit_max : n;
+      items += p.Hkv * nr[k] * n;
+    }
+    return warp_sum(items);
+  };
+  int lo = (T + cap - 1) / cap, hi = tmax < 4 ? 4 : tmax;
+  lo = lo < 4 ? 4 : lo;
+  lo = lo > hi ? hi : lo;
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (items_at(mid) <= cap) hi = mid; else lo = mid + 1;
+  }
+  const int chunk = lo;
+  int ns[KB], cnt[KB], off[KB];
+#pragma unroll
+  for (int k = 0; k < KB; ++k) {
+    int n = (tl[k] + chunk - 1) / chunk;
+    n = n > p.nsplit_max ? p.nsplit_max : n;
+    ns[k] = n < 1 ? 1 : n;
+    cnt[k] = p.Hkv * nr[k] * ns[k];
+    off[k] = 0;
+  }
+  // items are numbered longest piece first (the block scheduler hands CTAs out in index order, so
+  // the long pieces start first and the short ones fill the gaps): sequence j precedes sequence b
+  // when its pieces are longer, ties by index
+  for (int j = 0; j < p.B; ++j) {
+    const int src = j & 31;
+    int pj, cj;
+    if (j < 32) {
+      pj = __shfl_sync(0xffffffffu, tl[0] * 16 / ns[0], src);
+      cj = __shfl_sync(0xffffffffu, cnt[0], src);
+    } else {
+      pj = __shfl_sync(0xffffffffu, tl[KB - 1] * 16 / ns[KB - 1], src);
+      cj = __shfl_sync(0xffffffffu, cnt[KB - 1], src);
+    }
+#pragma unroll
+    for (int k = 0; k < KB; ++k) {
+      const int mine = tl[k] * 16 / ns[k], bm = k * 32 + lane;
+      if (pj > mine || (pj == mine && j < bm)) off[k] += cj;
     }
   }
+  WorkItem w;
+  w.valid = false;
+  w.b = w.kvh = w.rb = w.split = w.N = w.L = 0;
+  w.nsplit = 1;
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) tiles += __shfl_xor_sync(0xffffffffu, tiles, o);
-  *N_b = Nb;
-  *L_b = Lb;
-  int chunk = (tiles + 2 * p.num_sms - 1) / (2 * p.num_sms);
-  chunk = chunk < 4 ? 4 : chunk;
-  int total_b = Lb + Nb;
-  total_b = total_b > max_pos ? max_pos : total_b;
-  const int tiles_b = (total_b + kBN - 1) / kBN;
-  int ns = (tiles_b + chunk - 1) / chunk;
-  ns = ns > p.nsplit_max ? p.nsplit_max : ns;
-  return ns < 1 ? 1 : ns;
+  for (int k = 0; k < KB; ++k) {
+    const unsigned hit = __ballot_sync(0xffffffffu, idx >= off[k] && idx < off[k] + cnt[k]);
+    if (hit != 0u && !w.valid) {
+      const int bl = __ffs(hit) - 1;
+      const int local = idx - __shfl_sync(0xffffffffu, off[k], bl);
+      w.nsplit = __shfl_sync(0xffffffffu, ns[k], bl);
+      w.N = __shfl_sync(0xffffffffu, Nv[k], bl);
+      w.L = __shfl_sync(0xffffffffu, Lv[k], bl);
+      w.b = k * 32 + bl;
+      w.kvh = local % p.Hkv;
+      const int rest = local / p.Hkv;
+      w.split = rest % w.nsplit;
+      w.rb = rest / w.nsplit;
+      w.valid = true;
+    }
+  }
+  return w;
 }
 
 __global__ void __launch_bounds__(kThreadsTC, 2)
@@ -257,19 +339,18 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
   extern __shared__ __align__(1024) unsigned char smem[];  // no static shared memory: the base is 1 KB aligned
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int split = blockIdx.x % p.nsplit_max, rb = blockIdx.x / p.nsplit_max;
-  const int kvh = blockIdx.y, b = blockIdx.z;
   TC_MARK(0);
   TC_CTA_LOG(0, gtimer());
   TC_CTA_LOG(1, 0ull);
   TC_CTA_LOG(3, 0ull);
   TC_CTA_LOG(2, (unsigned long long)smid());
-  int N, L;
-  int nsplit = effective_splits(p, b, &N, &L);
+  const WorkItem wk = decode_work(p, blockIdx.x, gridDim.x);
   TC_MARK(1);
+  if (blockIdx.x < p.B && tid == 0 && p.n_tree[blockIdx.x] > p.Nmax) report(p.st, CAST_ERR_BAD_TREE, blockIdx.x);
+  if (!wk.valid) return;
+  const int b = wk.b, kvh = wk.kvh, rb = wk.rb, split = wk.split, N = wk.N, L = wk.L;
+  int nsplit = wk.nsplit;
   const int G = p.G, rows_total = N * G, row0 = rb * kBM;
-  if (tid == 0 && rb == 0 && split == 0 && kvh == 0 && p.n_tree[b] > p.Nmax) report(p.st, CAST_ERR_BAD_TREE, b);
-  if (row0 >= rows_total) return;
   const int max_pos = p.page_size == 0 ? p.seq_capacity : p.seq_capacity * p.page_size;
   int total = L + N;
   if (total > max_pos) {
@@ -277,8 +358,6 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     total = max_pos;
   }
   const int ntiles = (total + kBN - 1) / kBN;  // >= 1 because N >= 1 here
-  nsplit = nsplit > ntiles ? ntiles : nsplit;  // this sequence's splits: none of them is empty
-  if (split >= nsplit) return;
   if ((smem_u32(smem) & 1023u) != 0u) {  // the swizzled operand regions need a 1 KB aligned base
     if (tid == 0) report(p.st, CAST_ERR_CUDA, 1024);
     return;
@@ -745,16 +824,11 @@ __global__ void __launch_bounds__(64, 2) dbg_loadonly_kernel(const TcParams p, c
   extern __shared__ __align__(1024) unsigned char smem[];
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 4 * 2 * kTileKV);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int split, rb, kvh;
-  if (kvh_fast) { kvh = blockIdx.x; split = blockIdx.y % p.nsplit_max; rb = blockIdx.y / p.nsplit_max; }
-  else { split = blockIdx.x % p.nsplit_max; rb = blockIdx.x / p.nsplit_max; kvh = blockIdx.y; }
-  const int b = blockIdx.z;
-  int N, L;
-  int nsplit = effective_splits(p, b, &N, &L);
-  if (rb * kBM >= N * p.G) return;
+  (void)kvh_fast;
+  const WorkItem wk = decode_work(p, blockIdx.x, gridDim.x);
+  if (!wk.valid) return;
+  const int b = wk.b, kvh = wk.kvh, split = wk.split, N = wk.N, L = wk.L, nsplit = wk.nsplit;
   const int total = L + N, ntiles = (total + kBN - 1) / kBN;
-  nsplit = nsplit > ntiles ? ntiles : nsplit;
-  if (split >= nsplit) return;
   const int t0 = (int)((long long)split * ntiles / nsplit), t1 = (int)((long long)(split + 1) * ntiles / nsplit);
   const int ntile = t1 - t0;
   if (threadIdx.x == 0) {
@@ -908,6 +982,10 @@ bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const v
   int nsplit_max = kMaxSplit;
   if (nsplit_max > max_tiles) nsplit_max = max_tiles;
   if (nsplit_max < 1) nsplit_max = 1;
+  // one-dimensional grid: whole waves of two CTAs per SM, enough of them for the unsplit work
+  const int slots = 2 * c->num_sms;
+  const int waves = (B * Hkv * nrb + slots - 1) / slots;
+  const int grid = slots * (waves < 1 ? 1 : waves);
   TcParams p;
   p.q = (const __nv_bfloat16*)q; p.out = (__nv_bfloat16*)out;
   p.B = B; p.Ncap = Ncap; p.Nmax = Nmax; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.page_size = page_size;
@@ -954,13 +1032,12 @@ bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const v
     const int kvh_fast = atoi(lo) == 2;
     cudaFuncSetAttribute(dbg_loadonly_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * 2 * kTileKV + 64);
     cudaFuncSetAttribute(dbg_loadonly_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
-    const dim3 g = kvh_fast ? dim3(Hkv, nsplit_max * nrb, B) : dim3(nsplit_max * nrb, Hkv, B);
-    dbg_loadonly_kernel<<<g, 64, 4 * 2 * kTileKV + 64, stream>>>(p, map_k, map_v, kvh_fast);
+    dbg_loadonly_kernel<<<grid, 64, 4 * 2 * kTileKV + 64, stream>>>(p, map_k, map_v, kvh_fast);
     *status = launch_status();
     return true;
   }
 #endif
-  tree_attn_tc_kernel<<<dim3(nsplit_max * nrb, Hkv, B), kThreadsTC, kSmemBytes, stream>>>(p, map_k, map_v);
+  tree_attn_tc_kernel<<<grid, kThreadsTC, kSmemBytes, stream>>>(p, map_k, map_v);
   *status = launch_status();
   return true;
 }
