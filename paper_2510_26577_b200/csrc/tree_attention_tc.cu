@@ -334,6 +334,63 @@ __device__ __forceinline__ WorkItem decode_work(const TcParams& p, int idx, int 
   return w;
 }
 
+// Merge of the split partials of a row block, run by all 8 warps of the last CTA to finish it.
+// Warp w takes rows w, w+8, ...; a lane owns 4 output columns. ROWS rows x SPL splits = 16 loads are
+// in flight per lane: the merge is bound by L2 latency, not by bytes.
+template <int ROWS, int SPL>
+__device__ __forceinline__ void merge_rows(const TcParams& p, int b, int kvh, int row0, int rows_here, int nsplit) {
+  const int lane = threadIdx.x & 31, wv = threadIdx.x >> 5, G = p.G;
+  for (int rr = wv; rr < rows_here; rr += 8 * ROWS) {
+    float4 v[ROWS][SPL];
+    float wgt[ROWS], inv[ROWS];
+    size_t orow[ROWS];
+#pragma unroll
+    for (int u = 0; u < ROWS; ++u) {
+      const int r2 = rr + 8 * u;
+      const int grow = row0 + (r2 < rows_here ? r2 : rr), tt = grow / G, hh = kvh * G + grow % G;
+      const size_t pr = (((size_t)b * p.Hq + hh) * p.Ncap + tt) * p.nsplit_max;
+      orow[u] = (((size_t)b * p.Ncap + tt) * p.Hq + hh) * kHD;
+      float ms = -INFINITY, ls = 0.f;  // lane s holds split s's (max, sum)
+      if (lane < nsplit) {
+        ms = __ldcg(p.part_ml + (pr + lane) * 2);
+        ls = __ldcg(p.part_ml + (pr + lane) * 2 + 1);
+      }
+#pragma unroll
+      for (int s2 = 0; s2 < SPL; ++s2)
+        v[u][s2] = s2 < nsplit ? __ldcg(reinterpret_cast<const float4*>(p.part_o + (pr + s2) * kHD + lane * 4))
+                               : make_float4(0.f, 0.f, 0.f, 0.f);
+      float M = ms;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+      wgt[u] = ms > -INFINITY ? expf(ms - M) : 0.f;
+      float lsum = ls * wgt[u];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
+      inv[u] = lsum > 0.f ? 1.f / lsum : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < ROWS; ++u) {
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int s2 = 0; s2 < SPL; ++s2) {
+        const float w = __shfl_sync(0xffffffffu, wgt[u], s2);
+        acc.x += v[u][s2].x * w;
+        acc.y += v[u][s2].y * w;
+        acc.z += v[u][s2].z * w;
+        acc.w += v[u][s2].w * w;
+      }
+      if (rr + 8 * u < rows_here) {
+        const __nv_bfloat162 a = __floats2bfloat162_rn(acc.x * inv[u], acc.y * inv[u]),
+                             c2 = __floats2bfloat162_rn(acc.z * inv[u], acc.w * inv[u]);
+        uint2 pk;
+        pk.x = *reinterpret_cast<const uint32_t*>(&a);
+        pk.y = *reinterpret_cast<const uint32_t*>(&c2);
+        *reinterpret_cast<uint2*>(p.out + orow[u] + lane * 4) = pk;
+      }
+    }
+  }
+}
+
 __global__ void __launch_bounds__(kThreadsTC, 2)
 tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
   extern __shared__ __align__(1024) unsigned char smem[];  // no static shared memory: the base is 1 KB aligned
@@ -735,80 +792,29 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
         }
       }
     }
-    if (nsplit > 1) {
-      // the last split of this row block to finish merges the partials (ticket; nothing spins)
-      __threadfence();
-      softmax_bar();
-      if (tid == 0) {
-        int32_t* cnt = p.ticket + ((size_t)b * p.Hkv + kvh) * p.nrb + rb;
-        const int t = atomicAdd(cnt, 1);
-        *last_s = (t == nsplit - 1);
-        if (t == nsplit - 1) *cnt = 0;
-        __threadfence();
-      }
-      softmax_bar();
-      if (*last_s) TC_CTA_LOG(3, gtimer());
-      if (*last_s) {
-        // every lane keeps up to 16 loads in flight (two rows x up to kMaxSplit splits): the merge is
-        // bound by L2 latency, not by bytes
-        for (int rr = wv; rr < rows_here; rr += 8) {
-          float4 acc[2];
-          float inv[2];
-          size_t orow[2];
-          float4 v[2][kMaxSplit];
-          float wgt[2];
-#pragma unroll
-          for (int u = 0; u < 2; ++u) {
-            const int r2 = rr + 4 * u;
-            const bool on = r2 < rows_here;
-            const int grow = row0 + (on ? r2 : rr), tt = grow / G, hh = kvh * G + grow % G;
-            const size_t pr = (((size_t)b * p.Hq + hh) * p.Ncap + tt) * p.nsplit_max;
-            orow[u] = (((size_t)b * p.Ncap + tt) * p.Hq + hh) * kHD;
-            float ms = -INFINITY, ls = 0.f;  // lane s holds split s's (max, sum)
-            if (lane < nsplit) {
-              ms = __ldcg(p.part_ml + (pr + lane) * 2);
-              ls = __ldcg(p.part_ml + (pr + lane) * 2 + 1);
-            }
-#pragma unroll
-            for (int s2 = 0; s2 < kMaxSplit; ++s2)
-              v[u][s2] = s2 < nsplit ? __ldcg(reinterpret_cast<const float4*>(p.part_o + (pr + s2) * kHD + lane * 4))
-                                     : make_float4(0.f, 0.f, 0.f, 0.f);
-            float M = ms;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-            wgt[u] = ms > -INFINITY ? expf(ms - M) : 0.f;
-            float lsum = ls * wgt[u];
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
-            inv[u] = lsum > 0.f ? 1.f / lsum : 0.f;
-          }
-#pragma unroll
-          for (int u = 0; u < 2; ++u) {
-            acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-            for (int s2 = 0; s2 < kMaxSplit; ++s2) {
-              const float w = __shfl_sync(0xffffffffu, wgt[u], s2);
-              acc[u].x += v[u][s2].x * w;
-              acc[u].y += v[u][s2].y * w;
-              acc[u].z += v[u][s2].z * w;
-              acc[u].w += v[u][s2].w * w;
-            }
-            if (rr + 4 * u < rows_here) {
-              const __nv_bfloat162 a = __floats2bfloat162_rn(acc[u].x * inv[u], acc[u].y * inv[u]),
-                                   c2 = __floats2bfloat162_rn(acc[u].z * inv[u], acc[u].w * inv[u]);
-              uint2 pk;
-              pk.x = *reinterpret_cast<const uint32_t*>(&a);
-              pk.y = *reinterpret_cast<const uint32_t*>(&c2);
-              *reinterpret_cast<uint2*>(p.out + orow[u] + lane * 4) = pk;
-            }
-          }
-        }
-      }
-    }
+    if (nsplit > 1) __threadfence();  // the partials must be visible before this CTA takes its ticket
   }
   TC_MARK(6);
   tc_fence_before();
   __syncthreads();
+  if (nsplit > 1) {
+    // the last split of this row block to finish merges the partials (ticket; nothing spins)
+    if (tid == 0) {
+      int32_t* cnt = p.ticket + ((size_t)b * p.Hkv + kvh) * p.nrb + rb;
+      const int t = atomicAdd(cnt, 1);
+      *last_s = (t == nsplit - 1);
+      if (t == nsplit - 1) *cnt = 0;
+      __threadfence();
+    }
+    __syncthreads();
+    if (*last_s) {
+      TC_CTA_LOG(3, gtimer());
+      const int rows_here = rows_total - row0 < kBM ? rows_total - row0 : kBM;
+      if (nsplit <= 2) merge_rows<8, 2>(p, b, kvh, row0, rows_here, nsplit);
+      else if (nsplit <= 4) merge_rows<4, 4>(p, b, kvh, row0, rows_here, nsplit);
+      else merge_rows<2, kMaxSplit>(p, b, kvh, row0, rows_here, nsplit);
+    }
+  }
   TC_MARK(7);
   TC_CTA_LOG(1, gtimer());
   if (warp == 0) {
