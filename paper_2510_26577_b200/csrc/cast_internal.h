@@ -26,6 +26,9 @@ struct DevState {
   // rows[i]: logits rows that expand call i reads (n_{i-1}; 0: expansion is over). Layer i's
   // kernel only reads rows[i] and writes rows[i+1], so CTAs that start late see a stable value.
   int32_t rows[CAST_MAX_DEPTH + 2];
+  // layer i's candidates sit at pool positions [layer_base[i], layer_base[i] + layer_n[i])
+  int32_t layer_base[CAST_MAX_DEPTH + 1];
+  int32_t layer_n[CAST_MAX_DEPTH + 1];
   int32_t status[2];    // first device-detected error and its detail
 };
 
@@ -42,10 +45,10 @@ struct HostTable {
 
 // Limits of the vocabulary sweep.
 constexpr int kSweepThreads = 256;
-constexpr int kSweepEpt = 32;                             // logits per thread per pass
+constexpr int kSweepEpt = 16;                             // logits per thread per pass
 constexpr int kSweepSub = kSweepThreads * kSweepEpt;      // logits per CTA per pass
-constexpr int kSweepMaxChunks = 32;                       // CTAs per logits row
-constexpr int kCandCap = 4096;                            // >= 8*(K-1)*kSweepEpt + 1 + K
+constexpr int kSweepMaxChunks = 64;                       // CTAs per logits row
+constexpr int kCandCap = 4096;                            // candidate keys per CTA (floods take the slow exact path)
 constexpr int kMaxFifo = 64;
 constexpr int kAcceptMaxChunks = 32;
 
@@ -66,6 +69,9 @@ struct cast_ctx {
   int32_t* pool_depth;
   uint8_t* pool_kept;
   int32_t* retained;   // [max_batch][W] pool indices of the last layer's retained nodes
+  // every layer's candidates in descending order: pool index and log-value at position base + rank
+  int32_t* lsort;      // [max_batch][P]
+  double* lscore;      // [max_batch][P]
 
   cast::DevState* state;
 

@@ -2,14 +2,18 @@
 //
 // cast_tree_expand is ONE kernel per draft layer:
 //   1. vocabulary sweep - every logits row is cut into chunks, one CTA per chunk: streaming
-//      16-byte loads, online max / sum-exp, and an exact top-K by threshold filtering
-//      (the K-th largest of the per-thread maxima bounds the K-th largest of the chunk);
+//      16-byte loads issued before anything else, online max / sum-exp in base 2, and an exact
+//      top-K by threshold filtering (the K-th largest of the per-thread maxima of a warp bounds
+//      the K-th largest of the chunk from below, so only a few dozen logits survive the filter);
 //   2. the last CTA to finish a row merges the chunk partials (log-sum-exp in fp64, exact
-//      top-K of the chunk winners) and appends the K children to the node pool;
-//   3. the last CTA to finish the layer sorts each sequence's candidates, forms the
-//      utility u (Eq. 1) and the cost c (Eq. 2), runs Algorithm 1 (breadth pruning), the
-//      depth-pruning test and the FIFO update, and publishes the retained nodes.
+//      top-K of the chunk winners, again threshold-filtered) and appends the K children to the
+//      node pool;
+//   3. the last CTA to finish the layer ranks each sequence's candidates, forms the utility u
+//      (Eq. 1) and the cost c (Eq. 2), runs Algorithm 1 (breadth pruning), the depth-pruning
+//      test and the FIFO update, and publishes the retained nodes and the layer's sorted list.
 // "Last CTA" is decided by an atomic ticket; nothing spins.
+// cast_select_nodes ranks the pool by merging the per-layer sorted lists (binary searches), forms
+// the batch-mean utility, runs Algorithm 1 with the target-cost ratio and linearises the tree.
 #include <math.h>
 
 #include "cast_internal.h"
@@ -38,7 +42,8 @@ namespace {
 __global__ void step_begin_kernel(DevState* st, int B, int P, int W, const int32_t* root_token,
                                   const int32_t* kv_len, double* pool_score, int32_t* pool_token,
                                   int32_t* pool_parent, int32_t* pool_depth, uint8_t* pool_kept,
-                                  int32_t* retained, int32_t* row_ticket, int32_t* layer_ticket, int n_rows) {
+                                  int32_t* retained, int32_t* lsort, double* lscore, int32_t* row_ticket,
+                                  int32_t* layer_ticket, int n_rows) {
   __shared__ int s_max;
   const int tid = threadIdx.x;
   if (tid == 0) s_max = 0;
@@ -50,6 +55,8 @@ __global__ void step_begin_kernel(DevState* st, int B, int P, int W, const int32
     pool_parent[o] = -1;
     pool_depth[o] = 0;
     pool_kept[o] = 1;
+    lsort[o] = 0;
+    lscore[o] = 0.0;
     retained[b * W] = 0;
     atomicMax(&s_max, kv_len[b]);
   }
@@ -66,7 +73,13 @@ __global__ void step_begin_kernel(DevState* st, int B, int P, int W, const int32
     st->kept_total = 1;
     st->u_last = 1.0;
     st->n_hist[0] = 1;
-    for (int i = 1; i <= CAST_MAX_DEPTH; ++i) st->n_hist[i] = 0;
+    st->layer_base[0] = 0;
+    st->layer_n[0] = 1;
+    for (int i = 1; i <= CAST_MAX_DEPTH; ++i) {
+      st->n_hist[i] = 0;
+      st->layer_base[i] = 0;
+      st->layer_n[i] = 0;
+    }
     for (int i = 0; i < CAST_MAX_DEPTH + 2; ++i) st->rows[i] = 0;
     st->rows[1] = 1;
   }
@@ -82,6 +95,8 @@ struct ExpandParams {
   int32_t* pool_depth;
   uint8_t* pool_kept;
   int32_t* retained;
+  int32_t* lsort;
+  double* lscore;
   DevState* st;
   unsigned long long* part_keys;
   float* part_max;
@@ -120,22 +135,53 @@ template <> struct Vec<__nv_bfloat16> {
   }
 };
 
-// Exact top-K (descending) of n distinct keys in shared memory, written to out[0..K).
-// Missing entries (n < K) become 0. All threads of the CTA call it; `keys` is clobbered
-// when n > 512.
+__device__ __forceinline__ float ex2f(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// log2(e) split into a float just below it and a positive residual: x * log2(e) to better than one ulp
+// of the product, and -inf logits stay -inf through both FMAs (no inf - inf)
+constexpr float kLog2eHi = 1.4426950216293335f;
+constexpr float kLog2eLo = 1.925963033500011e-08f;  // log2(e) - kLog2eHi
+
+// The ticket of the "last CTA" pattern: the caller has passed a CTA barrier after its global
+// writes; one thread fences (cumulative over the CTA's writes) and takes the ticket.
+__device__ __forceinline__ bool take_ticket(int32_t* counter, int expected, int* flag_s) {
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const int t = atomicAdd(counter, 1);
+    const int last = (t == expected - 1);
+    if (last) *counter = 0;
+    __threadfence();
+    *flag_s = last;
+  }
+  __syncthreads();
+  return *flag_s != 0;
+}
+
+// Exact top-K (descending) of n distinct keys in shared memory, written to out[0..K); missing
+// entries (n < K) become 0. All threads of the CTA call it; `keys` is clobbered when n > 1024.
 __device__ void block_top_k(unsigned long long* keys, int n, int K, unsigned long long* out) {
   const int tid = threadIdx.x, nt = blockDim.x;
   if (tid < K) out[tid] = 0ull;
   __syncthreads();
-  if (n <= 512) {  // rank by counting: keys are distinct, so ranks are too
+  if (n <= 1024) {  // rank by counting: keys are distinct, so ranks are too
     for (int i = tid; i < n; i += nt) {
       const unsigned long long k = keys[i];
-      int rank = 0;
-      for (int j = 0; j < n; ++j) rank += (keys[j] > k);
+      int r0 = 0, r1 = 0, r2 = 0, r3 = 0, j = 0;
+      for (; j + 4 <= n; j += 4) {
+        r0 += (keys[j] > k);
+        r1 += (keys[j + 1] > k);
+        r2 += (keys[j + 2] > k);
+        r3 += (keys[j + 3] > k);
+      }
+      for (; j < n; ++j) r0 += (keys[j] > k);
+      const int rank = r0 + r1 + r2 + r3;
       if (rank < K) out[rank] = k;
     }
   } else {  // bitonic sort, descending, on the next power of two
-    int n2 = 1024;
+    int n2 = 2048;
     while (n2 < n) n2 <<= 1;
     for (int i = n + tid; i < n2; i += nt) keys[i] = 0ull;
     __syncthreads();
@@ -169,11 +215,19 @@ __device__ void layer_tail(const ExpandParams& p, int B, int n_prev, int base, u
   const bool need_cost = p.enable_bp || p.enable_dp;
   int n = Ni < W ? Ni : W;
   if (need_cost && p.tab.Ntab < n) n = p.tab.Ntab;
+  // Eq. 2 needs one table row: fetch it now, its latency hides behind the ranking
+  double c_mine = 0.0;
+  if (need_cost && tid < n) {
+    const int ctx = st->ctx_sum + (p.ctx_base_mode ? st->n0 : 0);
+    const int g = select_grid(ctx, p.tab.L, p.tab.M);
+    c_mine = p.tab.fD[(size_t)(g - 1) * p.tab.Ntab + tid] / p.tab.fT[(size_t)(g - 1) * p.tab.Ntab];
+  }
+  const double u_last = st->u_last;
 
   double* sc = reinterpret_cast<double*>(scratch);              // 2048 scores
   int* tk = reinterpret_cast<int*>(scratch + 16384);            // 2048 tokens
   double* vs = reinterpret_cast<double*>(scratch + 24576);      // [B][CAST_MAX_WIDTH] sorted values
-  const int group = 2048 / Ni;                                  // sequences sorted per pass
+  const int group = 2048 / Ni;                                  // sequences ranked per pass
   for (int b0 = 0; b0 < B; b0 += group) {
     const int nb = (B - b0) < group ? (B - b0) : group;
     for (int i = tid; i < nb * Ni; i += nt) {
@@ -182,7 +236,7 @@ __device__ void layer_tail(const ExpandParams& p, int B, int n_prev, int base, u
       tk[i] = __ldcg(p.pool_token + o);
     }
     __syncthreads();
-    // rank by counting under the order (value desc, token asc, creation order)
+    // rank by counting under the order (value desc, token asc, creation order); branch-free
     for (int i = tid; i < nb * Ni; i += nt) {
       const int bl = i / Ni, ci = i % Ni;
       const double s = sc[i];
@@ -190,10 +244,15 @@ __device__ void layer_tail(const ExpandParams& p, int B, int n_prev, int base, u
       const double* ss = sc + bl * Ni;
       const int* tt = tk + bl * Ni;
       int rank = 0;
+#pragma unroll 4
       for (int j = 0; j < Ni; ++j) {
         const double sj = ss[j];
-        rank += (sj > s) || (sj == s && (tt[j] < t || (tt[j] == t && j < ci)));
+        const int tj = tt[j];
+        rank += (int)(sj > s) | ((int)(sj == s) & ((int)(tj < t) | ((int)(tj == t) & (int)(j < ci))));
       }
+      const size_t o = (size_t)(b0 + bl) * P + base + rank;
+      p.lsort[o] = base + ci;  // the layer's sorted list, for the rerank
+      p.lscore[o] = s;
       if (rank < n) {
         sorted[(b0 + bl) * CAST_MAX_WIDTH + rank] = base + ci;
         vs[(b0 + bl) * CAST_MAX_WIDTH + rank] = exp(s);
@@ -206,17 +265,17 @@ __device__ void layer_tail(const ExpandParams& p, int B, int n_prev, int base, u
     double a = 0.0;
     for (int b = 0; b < B; ++b) a += vs[b * CAST_MAX_WIDTH + tid];
     vbar[tid] = a / (double)B;
+    c[tid] = c_mine;
   }
   __syncthreads();
-  if (tid == 0) {
-    double a = 0.0;
-    for (int k = 0; k < n; ++k) { a += vbar[k]; u[k] = a; }
-  }
-  // Eq. 2: draft cost of k nodes relative to one target token, at context select(sum n_j)
-  if (need_cost && tid < n) {
-    const int ctx = st->ctx_sum + (p.ctx_base_mode ? st->n0 : 0);
-    const int g = select_grid(ctx, p.tab.L, p.tab.M);
-    c[tid] = p.tab.fD[(size_t)(g - 1) * p.tab.Ntab + tid] / p.tab.fT[(size_t)(g - 1) * p.tab.Ntab];
+  if (tid < 32) {  // inclusive scan of at most 16 values
+    double a = tid < n ? vbar[tid] : 0.0;
+#pragma unroll
+    for (int d = 1; d < CAST_MAX_WIDTH; d <<= 1) {
+      const double t = __shfl_up_sync(0xffffffffu, a, d);
+      if (tid >= d) a += t;
+    }
+    if (tid < n) u[tid] = a;
   }
   __syncthreads();
   // Algorithm 1: mark[j] survives iff no earlier i has (u_j - u_i) < C1 (c_j - c_i)
@@ -235,7 +294,7 @@ __device__ void layer_tail(const ExpandParams& p, int B, int n_prev, int base, u
     bool go = true;
     if (p.enable_dp) {
       if (p.layer >= 2) {  // gain ratio of the previous layer goes into its buffer, FIFO
-        const double phi = u[n_i - 1] / st->u_last;
+        const double phi = u[n_i - 1] / u_last;
         double* A = p.fifo_vals + (size_t)(p.layer - 2) * p.R;
         int cnt = p.fifo_cnt[p.layer - 2];
         if (cnt < p.R) {
@@ -257,6 +316,16 @@ __device__ void layer_tail(const ExpandParams& p, int B, int n_prev, int base, u
     }
     s_ni = n_i;
     s_next = (p.layer < p.H && go) ? n_i : 0;
+    st->rows[p.layer + 1] = s_next;
+    st->n_hist[p.layer] = n_i;
+    st->layer_base[p.layer] = base;
+    st->layer_n[p.layer] = Ni;
+    st->ctx_sum += n_i;
+    st->kept_total += n_i;
+    st->u_last = u[n_i - 1];
+    st->pool_size = base + Ni;
+    st->layers_done = p.layer;
+    *p.next_count = s_next;
   }
   __syncthreads();
   const int n_i = s_ni;
@@ -273,40 +342,27 @@ __device__ void layer_tail(const ExpandParams& p, int B, int n_prev, int base, u
     p.next_tokens[i] = tok;
     p.next_parent_row[i] = prow;
   }
-  if (tid == 0) {
-    st->rows[p.layer + 1] = s_next;
-    st->n_hist[p.layer] = n_i;
-    st->ctx_sum += n_i;
-    st->kept_total += n_i;
-    st->u_last = u[n_i - 1];
-    st->pool_size = base + Ni;
-    st->layers_done = p.layer;
-    *p.next_count = s_next;
-  }
 }
 
 template <typename T>
 __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParams p) {
-  __shared__ __align__(16) unsigned long long cand[kCandCap];
+  __shared__ __align__(16) unsigned char scratch[kCandCap * 8];  // candidate keys; later the tail's arrays
   __shared__ unsigned long long topk[CAST_MAX_TOP_K];
-  __shared__ unsigned long long warp_thr[kSweepThreads / 32];
+  __shared__ unsigned long long red_k[kSweepThreads / 32];
+  __shared__ float warp_thr[kSweepThreads / 32];
   __shared__ float red_f[kSweepThreads / 32];
   __shared__ double red_d[kSweepThreads / 32];
   __shared__ int sorted[CAST_MAX_BATCH * CAST_MAX_WIDTH];
   __shared__ int cand_cnt, s_flag;
+  __shared__ unsigned long long thr_s;
   __shared__ double s_lse;
   CAST_STAMP_DECL
   CAST_STAMP(0);
+  unsigned long long* cand = reinterpret_cast<unsigned long long*>(scratch);
 
   const int chunk = blockIdx.x, r = blockIdx.y, b = blockIdx.z, B = gridDim.z;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   DevState* st = p.st;
-  const int n_prev = st->rows[p.layer];
-  if (n_prev == 0) {
-    if (chunk == 0 && r == 0 && b == 0 && tid == 0) *p.next_count = 0;
-    return;
-  }
-  if (r >= n_prev) return;
   const int K = p.K;
   const int row = b * p.W + r;
   const T* x = reinterpret_cast<const T*>(p.logits) + (size_t)row * p.V;
@@ -316,14 +372,9 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
   constexpr int NV = kSweepEpt / VEC;
   const bool aligned = (reinterpret_cast<uintptr_t>(x) & 15) == 0;  // chunk starts are multiples of 8 logits
 
-  float m_run = -INFINITY, s_run = 0.f;
-  unsigned long long thr_prev = 0ull;
-  if (tid == 0) cand_cnt = 0;
-  __syncthreads();
-  CAST_STAMP(1);
-
-  for (int sub = begin; sub < end; sub += kSweepSub) {
-    float xv[kSweepEpt];
+  // the first pass of logits is requested before the state is read (every row r < W exists in memory)
+  float xv[kSweepEpt];
+  auto load_pass = [&](int sub) {
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
       const int idx = sub + (v * kSweepThreads + tid) * VEC;
@@ -334,49 +385,70 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
         for (int e = 0; e < VEC; ++e) xv[v * VEC + e] = (idx + e < end) ? to_float(x[idx + e]) : -INFINITY;
       }
     }
-    // per-thread maximum (first maximum = lowest token id) and online sum-exp
-    float tmax = -INFINITY;
-    int targ = -1;
+  };
+  load_pass(begin);
+  const int n_prev = st->rows[p.layer];
+  if (n_prev == 0) {
+    if (chunk == 0 && r == 0 && b == 0 && tid == 0) *p.next_count = 0;
+    return;
+  }
+  if (r >= n_prev) return;
+
+  float M2 = -INFINITY, s_run = 0.f;  // running maximum (log2 units) and sum of 2^(x log2e - M2)
+  unsigned long long thr_key = 0ull;  // exact K-th largest key so far (0: fewer than K seen)
+  if (tid == 0) cand_cnt = 0;
+  __syncthreads();
+  CAST_STAMP(1);
+
+  for (int sub = begin; sub < end; sub += kSweepSub) {
+    if (sub != begin) load_pass(sub);
+    const int have0 = cand_cnt;
+    float tmax = xv[0];
 #pragma unroll
-    for (int i = 0; i < kSweepEpt; ++i)
-      if (xv[i] > tmax) {
-        tmax = xv[i];
-        targ = sub + ((i / VEC) * kSweepThreads + tid) * VEC + (i % VEC);
-      }
-    if (tmax > m_run) {
-      s_run *= expf(m_run - tmax);
-      m_run = tmax;
+    for (int i = 1; i < kSweepEpt; ++i) tmax = fmaxf(tmax, xv[i]);
+    const float t2 = tmax * kLog2eHi;
+    if (t2 > M2) {
+      s_run *= ex2f(M2 - t2);
+      M2 = t2;
     }
-    if (m_run > -INFINITY) {
+    if (M2 > -INFINITY) {
+      float a0 = 0.f, a1 = 0.f;
 #pragma unroll
-      for (int i = 0; i < kSweepEpt; ++i) s_run += expf(xv[i] - m_run);
-    }
-    // K-th largest of the warp's 32 thread maxima (bitonic sort over lanes, descending)
-    unsigned long long key = targ >= 0 ? make_key(tmax, targ) : 0ull;
-#pragma unroll
-    for (int k = 2; k <= 32; k <<= 1)
-#pragma unroll
-      for (int j = k >> 1; j > 0; j >>= 1) {
-        const unsigned long long o = __shfl_xor_sync(0xffffffffu, key, j);
-        const bool desc = ((lane & k) == 0), low = ((lane & j) == 0);
-        key = (desc == low) ? (key > o ? key : o) : (key < o ? key : o);
+      for (int i = 0; i < kSweepEpt; i += 2) {
+        a0 += ex2f(fmaf(xv[i], kLog2eHi, fmaf(xv[i], kLog2eLo, -M2)));  // NaN and +inf logits poison the sum
+        a1 += ex2f(fmaf(xv[i + 1], kLog2eHi, fmaf(xv[i + 1], kLog2eLo, -M2)));
       }
-    const unsigned long long wk = __shfl_sync(0xffffffffu, key, K - 1);
-    if (lane == 0) warp_thr[warp] = wk;
-    __syncthreads();
-    // at least K logits of this pass are >= each warp's K-th maximum, and at least K seen so
-    // far are >= thr_prev: nothing below the largest of these bounds can be in the top K.
-    unsigned long long thr = thr_prev;
+      s_run += a0 + a1;
+    }
+    // filter threshold: the exact K-th key once K logits have been seen, else the largest of the
+    // warps' K-th largest thread maxima (at least K logits of this pass are >= it)
+    float thr_val;
+    if (thr_key == 0ull) {
+      float kx = tmax;
 #pragma unroll
-    for (int w = 0; w < kSweepThreads / 32; ++w) thr = warp_thr[w] > thr ? warp_thr[w] : thr;
-    const float thr_val = thr ? key_value(thr) : -INFINITY;
+      for (int k = 2; k <= 32; k <<= 1)
+#pragma unroll
+        for (int j = k >> 1; j > 0; j >>= 1) {
+          const float o = __shfl_xor_sync(0xffffffffu, kx, j);
+          const bool desc = ((lane & k) == 0), low = ((lane & j) == 0);
+          kx = (desc == low) ? fmaxf(kx, o) : fminf(kx, o);
+        }
+      const float wk = __shfl_sync(0xffffffffu, kx, K - 1);
+      if (lane == 0) warp_thr[warp] = wk;
+      __syncthreads();
+      thr_val = warp_thr[0];
+#pragma unroll
+      for (int w = 1; w < kSweepThreads / 32; ++w) thr_val = fmaxf(thr_val, warp_thr[w]);
+    } else {
+      thr_val = key_value(thr_key);
+    }
 #pragma unroll
     for (int i = 0; i < kSweepEpt; ++i) {
       if (xv[i] >= thr_val) {
         const int id = sub + ((i / VEC) * kSweepThreads + tid) * VEC + (i % VEC);
         if (id < end) {
           const unsigned long long k2 = make_key(xv[i], id);
-          if (k2 >= thr) {
+          if (k2 > thr_key) {
             const int pos = atomicAdd(&cand_cnt, 1);
             if (pos < kCandCap) cand[pos] = k2;
           }
@@ -384,24 +456,58 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
       }
     }
     __syncthreads();
-    const int n = cand_cnt < kCandCap ? cand_cnt : kCandCap;
+    int n = cand_cnt;
+    if (n > kCandCap) {
+      // flood (a mass of ties at the threshold): K rounds of "largest key below the last one taken"
+      unsigned long long bound = ~0ull;
+      n = have0;
+      for (int round = 0; round < K; ++round) {
+        unsigned long long best = 0ull;
+#pragma unroll
+        for (int i = 0; i < kSweepEpt; ++i) {
+          const int id = sub + ((i / VEC) * kSweepThreads + tid) * VEC + (i % VEC);
+          if (id < end && xv[i] == xv[i]) {
+            const unsigned long long k2 = make_key(xv[i], id);
+            if (k2 < bound && k2 > best) best = k2;
+          }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+          best = other > best ? other : best;
+        }
+        if (lane == 0) red_k[warp] = best;
+        __syncthreads();
+        best = red_k[0];
+#pragma unroll
+        for (int w = 1; w < kSweepThreads / 32; ++w) best = red_k[w] > best ? red_k[w] : best;
+        __syncthreads();
+        if (best == 0ull) break;
+        if (tid == 0) cand[n] = best;
+        ++n;
+        bound = best;
+      }
+      __syncthreads();
+    }
     if (n > K) {
       block_top_k(cand, n, K, topk);
       if (tid < K) cand[tid] = topk[tid];
-      thr_prev = topk[K - 1];
+      thr_key = topk[K - 1];
       if (tid == 0) cand_cnt = K;
     } else {
-      thr_prev = 0ull;
+      thr_key = 0ull;
+      if (tid == 0) cand_cnt = n;
     }
     __syncthreads();
   }
-
   CAST_STAMP(2);
-  // chunk partials: top-K keys, maximum, sum of exp(x - maximum) in fp64
+
+  // chunk partials: top-K keys in descending order, maximum, sum of 2^(. - maximum) in fp64
   {
     const int have = cand_cnt;
-    if (tid < K) p.part_keys[((size_t)row * kSweepMaxChunks + chunk) * CAST_MAX_TOP_K + tid] = tid < have ? cand[tid] : 0ull;
-    float M = m_run;
+    block_top_k(cand, have, K, topk);
+    if (tid < K) p.part_keys[((size_t)row * kSweepMaxChunks + chunk) * CAST_MAX_TOP_K + tid] = topk[tid];
+    float M = M2;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
     if (lane == 0) red_f[warp] = M;
@@ -409,7 +515,7 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
     M = red_f[0];
 #pragma unroll
     for (int w = 1; w < kSweepThreads / 32; ++w) M = fmaxf(M, red_f[w]);
-    double sd = (m_run > -INFINITY) ? (double)s_run * (double)expf(m_run - M) : 0.0;
+    double sd = (M2 > -INFINITY) ? (double)s_run * (double)ex2f(M2 - M) : 0.0;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) sd += __shfl_xor_sync(0xffffffffu, sd, o);
     if (lane == 0) red_d[warp] = sd;
@@ -421,45 +527,72 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
       p.part_sum[(size_t)row * kSweepMaxChunks + chunk] = S;
     }
   }
-
   CAST_STAMP(3);
+
   // ---- row merge by the last CTA of this logits row
-  __threadfence();
   __syncthreads();
-  if (tid == 0) {
-    const int t = p.nchunks > 1 ? atomicAdd(&p.row_ticket[row], 1) : 0;
-    s_flag = (t == p.nchunks - 1);
-  }
-  __syncthreads();
-  if (!s_flag) return;
+  if (p.nchunks > 1 && !take_ticket(&p.row_ticket[row], p.nchunks, &s_flag)) return;
   CAST_STAMP(4);
-  __threadfence();
-  if (tid == 0) p.row_ticket[row] = 0;
-  const int nk = p.nchunks * K;
-  for (int i = tid; i < nk; i += kSweepThreads)
-    cand[i] = __ldcg(p.part_keys + ((size_t)row * kSweepMaxChunks + i / K) * CAST_MAX_TOP_K + (i % K));
-  __syncthreads();
-  block_top_k(cand, nk, K, topk);
+  const unsigned long long* rk = p.part_keys + (size_t)row * kSweepMaxChunks * CAST_MAX_TOP_K;
   if (warp == 0) {
-    float Mc = -INFINITY;
-    double Sc = 0.0;
-    if (lane < p.nchunks) {
-      Mc = __ldcg(p.part_max + (size_t)row * kSweepMaxChunks + lane);
-      Sc = __ldcg(p.part_sum + (size_t)row * kSweepMaxChunks + lane);
+    // threshold: the K-th largest of the chunk maxima (every chunk list is in descending order)
+    unsigned long long k0 = lane < p.nchunks ? __ldcg(rk + (size_t)lane * CAST_MAX_TOP_K) : 0ull;
+    unsigned long long k1 = lane + 32 < p.nchunks ? __ldcg(rk + (size_t)(lane + 32) * CAST_MAX_TOP_K) : 0ull;
+    int r0 = 0, r1 = 0;
+    for (int j = 0; j < p.nchunks; ++j) {
+      const unsigned long long kj = __shfl_sync(0xffffffffu, j < 32 ? k0 : k1, j & 31);
+      r0 += (kj > k0);
+      r1 += (kj > k1);
     }
-    float Mr = Mc;
+    unsigned long long f = (r0 == K - 1 && k0 != 0ull) ? k0 : ((r1 == K - 1 && k1 != 0ull) ? k1 : 0ull);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const unsigned long long other = __shfl_xor_sync(0xffffffffu, f, o);
+      f = other > f ? other : f;
+    }
+    if (lane == 0) {
+      thr_s = f;
+      cand_cnt = 0;
+    }
+  } else if (warp == 1) {
+    // log-sum-exp over the chunk partials, fp64
+    float M0 = -INFINITY, M1 = -INFINITY;
+    double S0 = 0.0, S1 = 0.0;
+    if (lane < p.nchunks) {
+      M0 = __ldcg(p.part_max + (size_t)row * kSweepMaxChunks + lane);
+      S0 = __ldcg(p.part_sum + (size_t)row * kSweepMaxChunks + lane);
+    }
+    if (lane + 32 < p.nchunks) {
+      M1 = __ldcg(p.part_max + (size_t)row * kSweepMaxChunks + lane + 32);
+      S1 = __ldcg(p.part_sum + (size_t)row * kSweepMaxChunks + lane + 32);
+    }
+    float Mr = fmaxf(M0, M1);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) Mr = fmaxf(Mr, __shfl_xor_sync(0xffffffffu, Mr, o));
-    double term = (Mc > -INFINITY) ? Sc * exp((double)Mc - (double)Mr) : 0.0;
+    double term = (M0 > -INFINITY ? S0 * exp2((double)M0 - (double)Mr) : 0.0) +
+                  (M1 > -INFINITY ? S1 * exp2((double)M1 - (double)Mr) : 0.0);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) term += __shfl_xor_sync(0xffffffffu, term, o);
-    const double lse = (double)Mr + log(term);
+    const double lse = ((double)Mr + log2(term)) * 0.69314718055994530942;
     if (lane == 0) {
       s_lse = lse;
       if (!isfinite(lse)) report(st, CAST_ERR_NONFINITE, row);
     }
   }
   __syncthreads();
+  {
+    const unsigned long long thr = thr_s;
+    const int nk = p.nchunks * K;
+    for (int i = tid; i < nk; i += kSweepThreads) {
+      const unsigned long long key = __ldcg(rk + (size_t)(i / K) * CAST_MAX_TOP_K + (i % K));
+      if (key != 0ull && key >= thr) {
+        const int pos = atomicAdd(&cand_cnt, 1);
+        cand[pos] = key;  // at most nchunks * K <= 1024 keys
+      }
+    }
+  }
+  __syncthreads();
+  block_top_k(cand, cand_cnt, K, topk);
   const int base = st->pool_size;
   if (tid < K) {
     const unsigned long long key = topk[tid];
@@ -478,21 +611,13 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
     p.pool_depth[o + idx] = p.layer;
     p.pool_kept[o + idx] = 0;
   }
-
   CAST_STAMP(5);
+
   // ---- layer tail by the last CTA of the layer
-  __threadfence();
   __syncthreads();
-  if (tid == 0) {
-    const int t = atomicAdd(p.layer_ticket, 1);
-    s_flag = (t == B * n_prev - 1);
-  }
-  __syncthreads();
-  if (!s_flag) return;
-  __threadfence();
-  if (tid == 0) *p.layer_ticket = 0;
+  if (!take_ticket(p.layer_ticket, B * n_prev, &s_flag)) return;
   CAST_STAMP(6);
-  layer_tail(p, B, n_prev, base, reinterpret_cast<unsigned char*>(cand), sorted);
+  layer_tail(p, B, n_prev, base, scratch, sorted);
   CAST_STAMP(7);
   CAST_STAMP_FLUSH(0, 8);
 }
@@ -503,9 +628,10 @@ struct SelectParams {
   const int32_t* pool_token;
   const int32_t* pool_parent;
   const int32_t* pool_depth;
-  const uint8_t* pool_kept;
+  const int32_t* lsort;
+  const double* lscore;
   DevState* st;
-  int P, P2, Ncap, words, m, pool_mode, enable_dr;
+  int P, Ncap, words, m, pool_mode, enable_dr;
   double C3;
   DevTable tab;
   double* sel_score;
@@ -520,54 +646,62 @@ struct SelectParams {
   int32_t* n_tree;
 };
 
-// Total order of the rerank: (value desc, depth asc, token asc, creation order); idx < 0 sorts last.
-__device__ __forceinline__ bool ranks_before(const SelectParams& p, size_t o, double sa, int ia, double sb, int ib) {
-  if (ia < 0) return false;
-  if (ib < 0) return true;
-  if (sa != sb) return sa > sb;
-  const int da = p.pool_depth[o + ia], db = p.pool_depth[o + ib];
-  if (da != db) return da < db;
-  const int ta = p.pool_token[o + ia], tb = p.pool_token[o + ib];
-  if (ta != tb) return ta < tb;
-  return ia < ib;
-}
-
-// Phase 1: sort sequence b's pool, publish the best min(pool, m) nodes with their values.
-__device__ void select_sort_phase(const SelectParams& p, int b, unsigned char* smem) {
-  double* key_s = reinterpret_cast<double*>(smem);
-  int* idx_s = reinterpret_cast<int*>(smem + (size_t)p.P2 * sizeof(double));
+// Phase 1: rank sequence b's pool under (value desc, depth asc, token asc, creation order) and
+// publish the best min(pool, m) nodes with their values. The pool is the root plus one sorted list
+// per layer (written by the layer tails in exactly that order restricted to the layer), so the rank
+// of the k-th node of a list is k plus, for every other list, the number of its nodes that come
+// first: a binary search each. Lists are cut to their first m nodes (later ones cannot rank < m).
+__device__ void select_rank_phase(const SelectParams& p, int b, unsigned char* smem) {
+  __shared__ int lbase[CAST_MAX_DEPTH + 1], llen[CAST_MAX_DEPTH + 1], loff[CAST_MAX_DEPTH + 2];
+  double* ls = reinterpret_cast<double*>(smem);  // the lists' values, list l at loff[l]
   const int tid = threadIdx.x, nt = blockDim.x;
   const size_t o = (size_t)b * p.P;
-  const int pool = p.st->pool_size;
-  for (int i = tid; i < p.P2; i += nt) {
-    const bool in = i < pool && (p.pool_mode == 0 || p.pool_kept[o + i]);
-    key_s[i] = in ? p.pool_score[o + i] : -INFINITY;
-    idx_s[i] = in ? i : -1;
+  const int nl = p.st->layers_done + 1;  // lists: depth 0 (the root) .. layers_done
+  if (tid == 0) {
+    int acc = 0;
+    for (int l = 0; l < nl; ++l) {
+      int len = p.pool_mode == 0 ? p.st->layer_n[l] : p.st->n_hist[l];
+      len = len > p.m ? p.m : len;
+      lbase[l] = p.st->layer_base[l];
+      llen[l] = len;
+      loff[l] = acc;
+      acc += len;
+    }
+    loff[nl] = acc;
   }
   __syncthreads();
-  for (int k = 2; k <= p.P2; k <<= 1)
-    for (int j = k >> 1; j > 0; j >>= 1) {
-      for (int i = tid; i < p.P2; i += nt) {
-        const int l = i ^ j;
-        if (l > i) {
-          const double sa = key_s[i], sb = key_s[l];
-          const int ia = idx_s[i], ib = idx_s[l];
-          const bool up = ((i & k) == 0);
-          const bool swap = up ? ranks_before(p, o, sb, ib, sa, ia) : ranks_before(p, o, sa, ia, sb, ib);
-          if (swap) {
-            key_s[i] = sb; key_s[l] = sa;
-            idx_s[i] = ib; idx_s[l] = ia;
-          }
-        }
-      }
-      __syncthreads();
-    }
-  const int peff = p.pool_mode == 0 ? pool : p.st->kept_total;
+  const int total = loff[nl];
+  for (int i = tid; i < total; i += nt) {
+    int l = 0;
+    while (i >= loff[l + 1]) ++l;
+    ls[i] = p.lscore[o + lbase[l] + (i - loff[l])];
+  }
+  __syncthreads();
+  const int peff = p.pool_mode == 0 ? p.st->pool_size : p.st->kept_total;
   const int n_out = min(min(peff, p.m), p.Ncap);
-  for (int s = tid; s < n_out; s += nt) {
-    p.sel_score[(size_t)b * p.Ncap + s] = key_s[s];
-    p.sel_value[(size_t)b * p.Ncap + s] = exp(key_s[s]);
-    p.sel_idx[(size_t)b * p.Ncap + s] = idx_s[s];
+  for (int i = tid; i < total; i += nt) {
+    int l = 0;
+    while (i >= loff[l + 1]) ++l;
+    const int k = i - loff[l];
+    const double s = ls[i];
+    int rank = k;
+    for (int l2 = 0; l2 < nl; ++l2) {
+      if (l2 == l) continue;
+      // nodes of list l2 that come first: value > s, or value == s when their depth is smaller
+      const double* a = ls + loff[l2];
+      int lo = 0, hi = llen[l2];
+      if (l2 < l) {
+        while (lo < hi) { const int mid = (lo + hi) >> 1; if (a[mid] >= s) lo = mid + 1; else hi = mid; }
+      } else {
+        while (lo < hi) { const int mid = (lo + hi) >> 1; if (a[mid] > s) lo = mid + 1; else hi = mid; }
+      }
+      rank += lo;
+    }
+    if (rank < n_out) {
+      p.sel_score[(size_t)b * p.Ncap + rank] = s;
+      p.sel_value[(size_t)b * p.Ncap + rank] = exp(s);
+      p.sel_idx[(size_t)b * p.Ncap + rank] = p.lsort[o + lbase[l] + k];
+    }
   }
 }
 
@@ -633,9 +767,13 @@ __device__ void select_finalize_phase(const SelectParams& p, int b, int B) {
   __syncthreads();
   for (int s = tid; s < N; s += nt) {
     const int mine = kept[s];
-    int t = 0;
-    for (int j = 0; j < N; ++j) t += (kept[j] < mine);
-    lin_of[mine] = (short)t;
+    int t0 = 0, t1 = 0, j = 0;
+    for (; j + 2 <= N; j += 2) {
+      t0 += (kept[j] < mine);
+      t1 += (kept[j + 1] < mine);
+    }
+    for (; j < N; ++j) t0 += (kept[j] < mine);
+    lin_of[mine] = (short)(t0 + t1);
   }
   __syncthreads();
   for (int s = tid; s < N; s += nt) {
@@ -657,7 +795,7 @@ __device__ void select_finalize_phase(const SelectParams& p, int b, int B) {
     const size_t q = (size_t)b * p.Ncap + t;
     if (t < N) {
       int a = t, guard = 0;
-      while (a >= 0 && a < N && guard++ <= CAST_MAX_DEPTH + 1) {  // walk to the root, setting one bit per ancestor
+      while (a >= 0 && a < N && guard++ <= CAST_MAX_DEPTH + 1) {  // walk to the root, one bit per ancestor
         w[a >> 5] |= 1u << (a & 31);
         a = lin_parent[a];
       }
@@ -676,9 +814,9 @@ __device__ void select_finalize_phase(const SelectParams& p, int b, int B) {
   }
 }
 
-__global__ void __launch_bounds__(512) select_sort_kernel(const SelectParams p) {
+__global__ void __launch_bounds__(512) select_rank_kernel(const SelectParams p) {
   extern __shared__ __align__(16) unsigned char smem[];
-  select_sort_phase(p, blockIdx.x, smem);
+  select_rank_phase(p, blockIdx.x, smem);
 }
 __global__ void __launch_bounds__(512) select_finalize_kernel(const SelectParams p) {
   select_finalize_phase(p, blockIdx.x, gridDim.x);
@@ -687,7 +825,7 @@ __global__ void __launch_bounds__(512) select_fused_kernel(const SelectParams p)
   extern __shared__ __align__(16) unsigned char smem[];
   CAST_STAMP_DECL
   CAST_STAMP(0);
-  select_sort_phase(p, 0, smem);
+  select_rank_phase(p, 0, smem);
   __syncthreads();
   CAST_STAMP(1);
   select_finalize_phase(p, 0, 1);
@@ -714,8 +852,8 @@ extern "C" cast_status cast_step_begin(cast_ctx* c, int B, const int32_t* root_t
   c->next_layer = 1;
   step_begin_kernel<<<1, 128, 0, (cudaStream_t)stream>>>(c->state, B, c->P, c->W, root_token, kv_len, c->pool_score,
                                                          c->pool_token, c->pool_parent, c->pool_depth, c->pool_kept,
-                                                         c->retained, c->row_ticket, c->layer_ticket,
-                                                         c->cfg.max_batch * c->W);
+                                                         c->retained, c->lsort, c->lscore, c->row_ticket,
+                                                         c->layer_ticket, c->cfg.max_batch * c->W);
   return launch_status();
 }
 
@@ -728,10 +866,11 @@ extern "C" cast_status cast_tree_expand(cast_ctx* c, int layer, const void* draf
   c->next_layer = layer + 1;
   const int B = c->cur_B, V = c->cfg.vocab;
   const int rows_per_seq = layer == 1 ? 1 : c->W;
-  // enough CTAs to cover the machine about twice, at least 2048 logits each
+  // enough CTAs to cover the machine about twice; one pass (kSweepSub logits) per CTA when rows are few
   int nchunks = (2 * c->num_sms + B * rows_per_seq - 1) / (B * rows_per_seq);
+  const int one_pass = (V + kSweepSub - 1) / kSweepSub;
+  if (nchunks > one_pass) nchunks = one_pass;
   if (nchunks > kSweepMaxChunks) nchunks = kSweepMaxChunks;
-  if (nchunks > V / 2048) nchunks = V / 2048;
   if (nchunks < 1) nchunks = 1;
   int chunk_elems = (V + nchunks - 1) / nchunks;
   chunk_elems = (chunk_elems + 7) / 8 * 8;
@@ -743,6 +882,7 @@ extern "C" cast_status cast_tree_expand(cast_ctx* c, int layer, const void* draf
   p.nchunks = nchunks; p.chunk_elems = chunk_elems;
   p.pool_score = c->pool_score; p.pool_token = c->pool_token; p.pool_parent = c->pool_parent;
   p.pool_depth = c->pool_depth; p.pool_kept = c->pool_kept; p.retained = c->retained;
+  p.lsort = c->lsort; p.lscore = c->lscore;
   p.st = c->state;
   p.part_keys = c->part_keys; p.part_max = c->part_max; p.part_sum = c->part_sum;
   p.row_ticket = c->row_ticket; p.layer_ticket = c->layer_ticket;
@@ -766,30 +906,23 @@ extern "C" cast_status cast_select_nodes(cast_ctx* c, int32_t* tokens, int32_t* 
   if (c->cur_B < 1) return CAST_ERR_INVALID_ARG;
   SelectParams p;
   p.pool_score = c->pool_score; p.pool_token = c->pool_token; p.pool_parent = c->pool_parent;
-  p.pool_depth = c->pool_depth; p.pool_kept = c->pool_kept; p.st = c->state;
+  p.pool_depth = c->pool_depth; p.lsort = c->lsort; p.lscore = c->lscore; p.st = c->state;
   p.P = c->P;
-  int P2 = 32;
-  while (P2 < c->P) P2 <<= 1;
-  p.P2 = P2;
   p.Ncap = c->cfg.max_tree; p.words = c->words; p.m = c->cfg.total_token;
   p.pool_mode = c->cfg.pool_mode; p.enable_dr = c->cfg.enable_dr; p.C3 = c->cfg.C3;
   p.tab = c->cur_table;
   p.sel_score = c->sel_score; p.sel_value = c->sel_value; p.sel_idx = c->sel_idx;
   p.tokens = tokens; p.parent = parent; p.depth = depth; p.anc = anc_mask; p.pool_idx = pool_idx;
   p.scores = scores; p.n_tree = n_tree;
-  const size_t smem = (size_t)P2 * (sizeof(double) + sizeof(int));
+  // the lists' values: (H + 1) lists of at most m nodes
+  const size_t smem = (size_t)(c->cfg.max_depth + 1) * c->cfg.total_token * sizeof(double);
   cudaStream_t s = (cudaStream_t)stream;
-  static bool attr_done = false;
-  if (!attr_done) {
-    CAST_CUDA_OK(cudaFuncSetAttribute(select_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 4096 * 12));
-    CAST_CUDA_OK(cudaFuncSetAttribute(select_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 4096 * 12));
-    attr_done = true;
-  }
-  const int threads = P2 >= 1024 ? 512 : (P2 / 2 < 128 ? 128 : P2 / 2);
+  int threads = ((c->cfg.max_depth + 1) * c->cfg.total_token + 31) / 32 * 32;
+  threads = threads > 512 ? 512 : (threads < 128 ? 128 : threads);
   if (c->cur_B == 1) {
     select_fused_kernel<<<1, threads, smem, s>>>(p);
   } else {
-    select_sort_kernel<<<c->cur_B, threads, smem, s>>>(p);
+    select_rank_kernel<<<c->cur_B, threads, smem, s>>>(p);
     select_finalize_kernel<<<c->cur_B, 128, 0, s>>>(p);
   }
   return launch_status();
