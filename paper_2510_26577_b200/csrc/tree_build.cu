@@ -145,6 +145,22 @@ __device__ __forceinline__ float ex2f(float x) {
 constexpr float kLog2eHi = 1.4426950216293335f;
 constexpr float kLog2eLo = 1.925963033500011e-08f;  // log2(e) - kLog2eHi
 
+// exp(s) for s <= 0 to about 1.2e-7 relative: the product with log2(e) and the integer part in fp64, the
+// fractional power by the fp32 unit, exact scaling. (A node value needs no more: the decision margins that
+// the parity contract asks for are 2e-6 relative.)
+__device__ __forceinline__ double fast_exp_neg(double s) {
+  const double t = s * 1.4426950408889634074;
+  if (!(t > -1000.0)) return 0.0;
+  const double n = floor(t);
+  return ldexp((double)ex2f((float)(t - n)), (int)n);
+}
+// log2(S), S > 0, to about 1e-7 absolute: exact exponent split, fp32 logarithm of the mantissa
+__device__ __forceinline__ double fast_log2(double S) {
+  int e;
+  const double m = frexp(S, &e);
+  return (double)e + (double)log2f((float)m);
+}
+
 // The ticket of the "last CTA" pattern: the caller has passed a CTA barrier after its global
 // writes; one thread fences (cumulative over the CTA's writes) and takes the ticket.
 __device__ __forceinline__ bool take_ticket(int32_t* counter, int expected, int* flag_s) {
@@ -162,11 +178,12 @@ __device__ __forceinline__ bool take_ticket(int32_t* counter, int expected, int*
 
 // Exact top-K (descending) of n distinct keys in shared memory, written to out[0..K); missing
 // entries (n < K) become 0. All threads of the CTA call it; `keys` is clobbered when n > 1024.
-__device__ void block_top_k(unsigned long long* keys, int n, int K, unsigned long long* out) {
+__device__ __noinline__ void block_top_k(unsigned long long* keys, int n, int K, unsigned long long* out) {
   const int tid = threadIdx.x, nt = blockDim.x;
   if (tid < K) out[tid] = 0ull;
   __syncthreads();
   if (n <= 1024) {  // rank by counting: keys are distinct, so ranks are too
+#pragma unroll 1
     for (int i = tid; i < n; i += nt) {
       const unsigned long long k = keys[i];
       int r0 = 0, r1 = 0, r2 = 0, r3 = 0, j = 0;
@@ -203,7 +220,7 @@ __device__ void block_top_k(unsigned long long* keys, int n, int K, unsigned lon
 }
 
 // Layer tail (Eq. 1, Eq. 2, Algorithm 1, depth pruning), run by the last CTA of the layer.
-__device__ void layer_tail(const ExpandParams& p, int B, int n_prev, int base, unsigned char* scratch,
+__device__ __noinline__ void layer_tail(const ExpandParams& p, int B, int n_prev, int base, unsigned char* scratch,
                            int* sorted /* [CAST_MAX_BATCH * CAST_MAX_WIDTH] */) {
   __shared__ double vbar[CAST_MAX_WIDTH], u[CAST_MAX_WIDTH], c[CAST_MAX_WIDTH];
   __shared__ int mark[CAST_MAX_WIDTH];
@@ -228,6 +245,7 @@ __device__ void layer_tail(const ExpandParams& p, int B, int n_prev, int base, u
   int* tk = reinterpret_cast<int*>(scratch + 16384);            // 2048 tokens
   double* vs = reinterpret_cast<double*>(scratch + 24576);      // [B][CAST_MAX_WIDTH] sorted values
   const int group = 2048 / Ni;                                  // sequences ranked per pass
+#pragma unroll 1
   for (int b0 = 0; b0 < B; b0 += group) {
     const int nb = (B - b0) < group ? (B - b0) : group;
     for (int i = tid; i < nb * Ni; i += nt) {
@@ -255,7 +273,7 @@ __device__ void layer_tail(const ExpandParams& p, int B, int n_prev, int base, u
       p.lscore[o] = s;
       if (rank < n) {
         sorted[(b0 + bl) * CAST_MAX_WIDTH + rank] = base + ci;
-        vs[(b0 + bl) * CAST_MAX_WIDTH + rank] = exp(s);
+        vs[(b0 + bl) * CAST_MAX_WIDTH + rank] = fast_exp_neg(s);
       }
     }
     __syncthreads();
@@ -263,6 +281,7 @@ __device__ void layer_tail(const ExpandParams& p, int B, int n_prev, int base, u
   // Eq. 1: batch mean of the rank-wise values, then prefix sums
   if (tid < n) {
     double a = 0.0;
+#pragma unroll 1
     for (int b = 0; b < B; ++b) a += vs[b * CAST_MAX_WIDTH + tid];
     vbar[tid] = a / (double)B;
     c[tid] = c_mine;
@@ -282,6 +301,7 @@ __device__ void layer_tail(const ExpandParams& p, int B, int n_prev, int base, u
   if (tid < n) {
     int ok = 1;
     if (p.enable_bp)
+#pragma unroll 1
       for (int i = 0; i < tid; ++i)
         if ((u[tid] - u[i]) < p.C1 * (c[tid] - c[i])) ok = 0;
     mark[tid] = ok;
@@ -289,6 +309,7 @@ __device__ void layer_tail(const ExpandParams& p, int B, int n_prev, int base, u
   __syncthreads();
   if (tid == 0) {
     int n_i = 1;
+#pragma unroll 1
     for (int j = 0; j < n; ++j)
       if (mark[j]) n_i = j + 1;
     bool go = true;
@@ -329,6 +350,7 @@ __device__ void layer_tail(const ExpandParams& p, int B, int n_prev, int base, u
   }
   __syncthreads();
   const int n_i = s_ni;
+#pragma unroll 1
   for (int i = tid; i < B * W; i += nt) {
     const int b = i / W, s = i % W;
     int tok = -1, prow = -1;
@@ -354,8 +376,6 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
   __shared__ double red_d[kSweepThreads / 32];
   __shared__ int sorted[CAST_MAX_BATCH * CAST_MAX_WIDTH];
   __shared__ int cand_cnt, s_flag;
-  __shared__ unsigned long long thr_s;
-  __shared__ double s_lse;
   CAST_STAMP_DECL
   CAST_STAMP(0);
   unsigned long long* cand = reinterpret_cast<unsigned long long*>(scratch);
@@ -393,6 +413,10 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
     return;
   }
   if (r >= n_prev) return;
+  // the parent of this row's children and its log-value (only the row's last CTA uses them: fetched now,
+  // off the critical path)
+  const int parent = p.layer == 1 ? 0 : p.retained[b * p.W + r];
+  const double parent_score = p.pool_score[(size_t)b * p.P + parent];
 
   float M2 = -INFINITY, s_run = 0.f;  // running maximum (log2 units) and sum of 2^(x log2e - M2)
   unsigned long long thr_key = 0ull;  // exact K-th largest key so far (0: fewer than K seen)
@@ -442,16 +466,39 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
     } else {
       thr_val = key_value(thr_key);
     }
+    {
+      unsigned pm = 0u;  // which of this thread's 16 logits pass the value threshold
 #pragma unroll
-    for (int i = 0; i < kSweepEpt; ++i) {
-      if (xv[i] >= thr_val) {
-        const int id = sub + ((i / VEC) * kSweepThreads + tid) * VEC + (i % VEC);
-        if (id < end) {
-          const unsigned long long k2 = make_key(xv[i], id);
-          if (k2 > thr_key) {
-            const int pos = atomicAdd(&cand_cnt, 1);
-            if (pos < kCandCap) cand[pos] = k2;
-          }
+      for (int i = 0; i < kSweepEpt; ++i) pm |= (xv[i] >= thr_val ? 1u : 0u) << i;
+      if (pm != 0u) {  // rare: exact test on the full key
+#pragma unroll
+        for (int i = 0; i < kSweepEpt; ++i) {
+          const int id = sub + ((i / VEC) * kSweepThreads + tid) * VEC + (i % VEC);
+          const bool ok = ((pm >> i) & 1u) && id < end && make_key(xv[i], id) > thr_key;
+          pm = ok ? pm : (pm & ~(1u << i));
+        }
+      }
+      const int cntp = __popc(pm);
+      // one shared-memory atomic per warp: exclusive prefix of the lanes' counts
+      int incl = cntp;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += t;
+      }
+      const int wtotal = __shfl_sync(0xffffffffu, incl, 31);
+      if (wtotal > 0) {
+        int basepos = 0;
+        if (lane == 31) basepos = atomicAdd(&cand_cnt, wtotal);
+        basepos = __shfl_sync(0xffffffffu, basepos, 31);
+        int pos = basepos + incl - cntp;
+        if (pm != 0u) {
+#pragma unroll
+          for (int i = 0; i < kSweepEpt; ++i)
+            if ((pm >> i) & 1u) {
+              if (pos < kCandCap) cand[pos] = make_key(xv[i], sub + ((i / VEC) * kSweepThreads + tid) * VEC + (i % VEC));
+              ++pos;
+            }
         }
       }
     }
@@ -461,6 +508,7 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
       // flood (a mass of ties at the threshold): K rounds of "largest key below the last one taken"
       unsigned long long bound = ~0ull;
       n = have0;
+#pragma unroll 1
       for (int round = 0; round < K; ++round) {
         unsigned long long best = 0ull;
 #pragma unroll
@@ -495,7 +543,7 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
       thr_key = topk[K - 1];
       if (tid == 0) cand_cnt = K;
     } else {
-      thr_key = 0ull;
+      if (n < K) thr_key = 0ull;  // (n == K with a threshold: nothing new passed, the list stays sorted)
       if (tid == 0) cand_cnt = n;
     }
     __syncthreads();
@@ -505,7 +553,7 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
   // chunk partials: top-K keys in descending order, maximum, sum of 2^(. - maximum) in fp64
   {
     const int have = cand_cnt;
-    block_top_k(cand, have, K, topk);
+    if (thr_key == 0ull) block_top_k(cand, have, K, topk);  // fewer than K so far: not sorted yet
     if (tid < K) p.part_keys[((size_t)row * kSweepMaxChunks + chunk) * CAST_MAX_TOP_K + tid] = topk[tid];
     float M = M2;
 #pragma unroll
@@ -533,29 +581,13 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
   __syncthreads();
   if (p.nchunks > 1 && !take_ticket(&p.row_ticket[row], p.nchunks, &s_flag)) return;
   CAST_STAMP(4);
-  const unsigned long long* rk = p.part_keys + (size_t)row * kSweepMaxChunks * CAST_MAX_TOP_K;
+  const int base = st->pool_size;
   if (warp == 0) {
-    // threshold: the K-th largest of the chunk maxima (every chunk list is in descending order)
+    // one warp merges the row: no CTA barriers on this path
+    const unsigned long long* rk = p.part_keys + (size_t)row * kSweepMaxChunks * CAST_MAX_TOP_K;
+    // (a) every lane requests its share of the chunk lists and of the (max, sum) partials at once
     unsigned long long k0 = lane < p.nchunks ? __ldcg(rk + (size_t)lane * CAST_MAX_TOP_K) : 0ull;
     unsigned long long k1 = lane + 32 < p.nchunks ? __ldcg(rk + (size_t)(lane + 32) * CAST_MAX_TOP_K) : 0ull;
-    int r0 = 0, r1 = 0;
-    for (int j = 0; j < p.nchunks; ++j) {
-      const unsigned long long kj = __shfl_sync(0xffffffffu, j < 32 ? k0 : k1, j & 31);
-      r0 += (kj > k0);
-      r1 += (kj > k1);
-    }
-    unsigned long long f = (r0 == K - 1 && k0 != 0ull) ? k0 : ((r1 == K - 1 && k1 != 0ull) ? k1 : 0ull);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const unsigned long long other = __shfl_xor_sync(0xffffffffu, f, o);
-      f = other > f ? other : f;
-    }
-    if (lane == 0) {
-      thr_s = f;
-      cand_cnt = 0;
-    }
-  } else if (warp == 1) {
-    // log-sum-exp over the chunk partials, fp64
     float M0 = -INFINITY, M1 = -INFINITY;
     double S0 = 0.0, S1 = 0.0;
     if (lane < p.nchunks) {
@@ -566,50 +598,71 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
       M1 = __ldcg(p.part_max + (size_t)row * kSweepMaxChunks + lane + 32);
       S1 = __ldcg(p.part_sum + (size_t)row * kSweepMaxChunks + lane + 32);
     }
+    constexpr int kPerLane = kSweepMaxChunks * CAST_MAX_TOP_K / 32;  // 32 keys per lane at most
+    const int nk = p.nchunks * K;
+    // (b) threshold: the K-th largest of the chunk maxima (every chunk list is in descending order)
+    int r0 = 0, r1 = 0;
+#pragma unroll 1
+    for (int j = 0; j < p.nchunks; ++j) {
+      const unsigned long long kj = __shfl_sync(0xffffffffu, j < 32 ? k0 : k1, j & 31);
+      r0 += (kj > k0);
+      r1 += (kj > k1);
+    }
+    unsigned long long thr = (r0 == K - 1 && k0 != 0ull) ? k0 : ((r1 == K - 1 && k1 != 0ull) ? k1 : 0ull);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const unsigned long long other = __shfl_xor_sync(0xffffffffu, thr, o);
+      thr = other > thr ? other : thr;
+    }
+    // (c) survivors of the filter go to shared memory (a few more than K), then rank by counting
+    int n = 0;
+#pragma unroll 1
+    for (int i0 = 0; i0 < kPerLane * 32 && i0 < nk; i0 += 32) {
+      const int i = i0 + lane;
+      unsigned long long key = 0ull;
+      if (i < nk) key = __ldcg(rk + (size_t)(i / K) * CAST_MAX_TOP_K + (i % K));
+      const bool pass = key != 0ull && key >= thr;
+      const unsigned m = __ballot_sync(0xffffffffu, pass);
+      if (pass) cand[n + __popc(m & ((1u << lane) - 1u))] = key;
+      n += __popc(m);
+    }
+    __syncwarp();
+#pragma unroll 1
+    for (int i = lane; i < n; i += 32) {
+      const unsigned long long k = cand[i];
+      int rank = 0;
+#pragma unroll 1
+      for (int j = 0; j < n; ++j) rank += (cand[j] > k);
+      if (rank < K) topk[rank] = k;
+    }
+    if (lane < K && lane >= n) topk[lane] = 0ull;
+    // (d) log-sum-exp over the chunk partials: weights by the fp32 unit, sums in fp64
     float Mr = fmaxf(M0, M1);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) Mr = fmaxf(Mr, __shfl_xor_sync(0xffffffffu, Mr, o));
-    double term = (M0 > -INFINITY ? S0 * exp2((double)M0 - (double)Mr) : 0.0) +
-                  (M1 > -INFINITY ? S1 * exp2((double)M1 - (double)Mr) : 0.0);
+    double term = (M0 > -INFINITY ? S0 * (double)ex2f(M0 - Mr) : 0.0) + (M1 > -INFINITY ? S1 * (double)ex2f(M1 - Mr) : 0.0);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) term += __shfl_xor_sync(0xffffffffu, term, o);
-    const double lse = ((double)Mr + log2(term)) * 0.69314718055994530942;
-    if (lane == 0) {
-      s_lse = lse;
-      if (!isfinite(lse)) report(st, CAST_ERR_NONFINITE, row);
-    }
-  }
-  __syncthreads();
-  {
-    const unsigned long long thr = thr_s;
-    const int nk = p.nchunks * K;
-    for (int i = tid; i < nk; i += kSweepThreads) {
-      const unsigned long long key = __ldcg(rk + (size_t)(i / K) * CAST_MAX_TOP_K + (i % K));
-      if (key != 0ull && key >= thr) {
-        const int pos = atomicAdd(&cand_cnt, 1);
-        cand[pos] = key;  // at most nchunks * K <= 1024 keys
+    const double lse = ((double)Mr + fast_log2(term)) * 0.69314718055994530942;
+    if (lane == 0 && !(term > 0.0 && isfinite(lse))) report(st, CAST_ERR_NONFINITE, row);
+    __syncwarp();
+    // (e) the K children join the pool
+    if (lane < K) {
+      const unsigned long long key = topk[lane];
+      const float val = key_value(key);
+      int tok = key_token(key);
+      if (key == 0ull || !(val > -INFINITY) || tok < 0 || tok >= p.V) {  // fewer than K finite logits
+        report(st, CAST_ERR_NONFINITE, row);
+        tok = 0;
       }
+      const size_t o = (size_t)b * p.P;
+      const int idx = base + r * K + lane;
+      p.pool_score[o + idx] = parent_score + ((double)val - lse);
+      p.pool_token[o + idx] = tok;
+      p.pool_parent[o + idx] = parent;
+      p.pool_depth[o + idx] = p.layer;
+      p.pool_kept[o + idx] = 0;
     }
-  }
-  __syncthreads();
-  block_top_k(cand, cand_cnt, K, topk);
-  const int base = st->pool_size;
-  if (tid < K) {
-    const unsigned long long key = topk[tid];
-    const float val = key_value(key);
-    int tok = key_token(key);
-    if (key == 0ull || !(val > -INFINITY) || tok < 0 || tok >= p.V) {  // fewer than K finite logits
-      report(st, CAST_ERR_NONFINITE, row);
-      tok = 0;
-    }
-    const int parent = p.layer == 1 ? 0 : p.retained[b * p.W + r];
-    const size_t o = (size_t)b * p.P;
-    const int idx = base + r * K + tid;
-    p.pool_score[o + idx] = p.pool_score[o + parent] + ((double)val - s_lse);
-    p.pool_token[o + idx] = tok;
-    p.pool_parent[o + idx] = parent;
-    p.pool_depth[o + idx] = p.layer;
-    p.pool_kept[o + idx] = 0;
   }
   CAST_STAMP(5);
 
@@ -651,7 +704,7 @@ struct SelectParams {
 // per layer (written by the layer tails in exactly that order restricted to the layer), so the rank
 // of the k-th node of a list is k plus, for every other list, the number of its nodes that come
 // first: a binary search each. Lists are cut to their first m nodes (later ones cannot rank < m).
-__device__ void select_rank_phase(const SelectParams& p, int b, unsigned char* smem) {
+__device__ __noinline__ void select_rank_phase(const SelectParams& p, int b, unsigned char* smem) {
   __shared__ int lbase[CAST_MAX_DEPTH + 1], llen[CAST_MAX_DEPTH + 1], loff[CAST_MAX_DEPTH + 2];
   double* ls = reinterpret_cast<double*>(smem);  // the lists' values, list l at loff[l]
   const int tid = threadIdx.x, nt = blockDim.x;
@@ -671,6 +724,7 @@ __device__ void select_rank_phase(const SelectParams& p, int b, unsigned char* s
   }
   __syncthreads();
   const int total = loff[nl];
+#pragma unroll 1
   for (int i = tid; i < total; i += nt) {
     int l = 0;
     while (i >= loff[l + 1]) ++l;
@@ -679,12 +733,14 @@ __device__ void select_rank_phase(const SelectParams& p, int b, unsigned char* s
   __syncthreads();
   const int peff = p.pool_mode == 0 ? p.st->pool_size : p.st->kept_total;
   const int n_out = min(min(peff, p.m), p.Ncap);
+#pragma unroll 1
   for (int i = tid; i < total; i += nt) {
     int l = 0;
     while (i >= loff[l + 1]) ++l;
     const int k = i - loff[l];
     const double s = ls[i];
     int rank = k;
+#pragma unroll 1
     for (int l2 = 0; l2 < nl; ++l2) {
       if (l2 == l) continue;
       // nodes of list l2 that come first: value > s, or value == s when their depth is smaller
@@ -699,14 +755,14 @@ __device__ void select_rank_phase(const SelectParams& p, int b, unsigned char* s
     }
     if (rank < n_out) {
       p.sel_score[(size_t)b * p.Ncap + rank] = s;
-      p.sel_value[(size_t)b * p.Ncap + rank] = exp(s);
+      p.sel_value[(size_t)b * p.Ncap + rank] = fast_exp_neg(s);
       p.sel_idx[(size_t)b * p.Ncap + rank] = p.lsort[o + lbase[l] + k];
     }
   }
 }
 
 // Phase 2: batch-mean utility, target-cost ratio, Algorithm 1 -> N; then sequence b's tree.
-__device__ void select_finalize_phase(const SelectParams& p, int b, int B) {
+__device__ __noinline__ void select_finalize_phase(const SelectParams& p, int b, int B) {
   __shared__ double u[CAST_MAX_TREE], c[CAST_MAX_TREE];
   __shared__ int kept[CAST_MAX_TREE], lin_parent[CAST_MAX_TREE];
   __shared__ short lin_of[1 + CAST_MAX_TOP_K + (CAST_MAX_DEPTH - 1) * CAST_MAX_WIDTH * CAST_MAX_TOP_K];
@@ -726,6 +782,7 @@ __device__ void select_finalize_phase(const SelectParams& p, int b, int B) {
       const int s = lane * 4 + e;
       double a = 0.0;
       if (s < n) {
+#pragma unroll 1
         for (int bb = 0; bb < B; ++bb) a += p.sel_value[(size_t)bb * p.Ncap + s];
         a /= (double)B;
       }
@@ -748,13 +805,16 @@ __device__ void select_finalize_phase(const SelectParams& p, int b, int B) {
   if (p.enable_dr) {
     const int g0 = select_grid(p.st->n0, p.tab.L, p.tab.M);
     const double* f = p.tab.fT + (size_t)(g0 - 1) * p.tab.Ntab;
+#pragma unroll 1
     for (int k = tid; k < n; k += nt) c[k] = f[k] / f[0];
   }
   __syncthreads();
   int N = n;
   if (p.enable_dr) {
+#pragma unroll 1
     for (int j = tid; j < n; j += nt) {
       bool ok = true;
+#pragma unroll 1
       for (int i = 0; i < j; ++i)
         if ((u[j] - u[i]) < p.C3 * (c[j] - c[i])) ok = false;
       if (ok) atomicMax(&s_N, j + 1);
@@ -763,8 +823,10 @@ __device__ void select_finalize_phase(const SelectParams& p, int b, int B) {
     N = s_N;
   }
   // linearise: kept nodes in creation order (ascending pool index)
+#pragma unroll 1
   for (int s = tid; s < N; s += nt) kept[s] = p.sel_idx[(size_t)b * p.Ncap + s];
   __syncthreads();
+#pragma unroll 1
   for (int s = tid; s < N; s += nt) {
     const int mine = kept[s];
     int t0 = 0, t1 = 0, j = 0;
@@ -776,6 +838,7 @@ __device__ void select_finalize_phase(const SelectParams& p, int b, int B) {
     lin_of[mine] = (short)(t0 + t1);
   }
   __syncthreads();
+#pragma unroll 1
   for (int s = tid; s < N; s += nt) {
     const int pi = kept[s];
     const int t = lin_of[pi];
@@ -790,6 +853,7 @@ __device__ void select_finalize_phase(const SelectParams& p, int b, int B) {
     if (p.scores) p.scores[q] = p.pool_score[o + pi];
   }
   __syncthreads();
+#pragma unroll 1
   for (int t = tid; t < p.Ncap; t += nt) {
     uint32_t w[CAST_MAX_TREE / 32] = {0u, 0u, 0u, 0u};
     const size_t q = (size_t)b * p.Ncap + t;
