@@ -219,6 +219,34 @@ CAST_API cast_status cast_compact_kv(cast_ctx* ctx, void* k_cache, void* v_cache
                             const int32_t* accept_path, const int32_t* accept_len,
                             int32_t* kv_len /* in/out */, void* stream);
 
+/*
+ * cast_accept for callers that must not allocate device memory. (The paper has no counterpart:
+ * this entry point exists for hosts of the library, not for the method.)
+ *
+ * Some callers cannot call cudaMalloc at the point where they need the acceptance step: code that
+ * runs inside a memory-pool or arena discipline where every device byte is accounted for up front,
+ * code that runs after start-up in a process whose allocator has been frozen, or a plug-in that is
+ * handed device pointers but no allocator. cast_accept needs a context, and a context allocates.
+ * This variant takes no context and allocates nothing: the only scratch it needs (the per-chunk
+ * winners of the target argmax sweep) lives in a fixed 512 KB array inside the library image, which
+ * every GPU that loads the library holds until the process exits.
+ *
+ * Arguments as for cast_accept, with the sizes a context would carry passed explicitly: n_cap (row
+ * stride of tokens/parent and of the logits' second axis, <= CAST_MAX_TREE), vocab, max_depth
+ * (accept_path has max_depth + 1 entries per sequence). Limit: B * n_cap <= 2048, else
+ * CAST_ERR_CAPACITY. There is no device status word: a malformed tree ends the walk early instead
+ * of being reported.
+ *
+ * The first call on a device looks up the array's device address (no allocation, but a runtime
+ * query): make that call before any stream capture. All calls share the one array, which keeps
+ * the previous call's contents; a call overwrites every entry it later reads, so nothing needs
+ * clearing, but two calls that overlap on the GPU (different streams) race on it.
+ */
+CAST_API cast_status cast_accept_static(const void* target_logits, cast_dtype dtype, int B, int n_cap, int vocab,
+                                        int max_depth, const int32_t* tokens, const int32_t* parent,
+                                        const int32_t* n_tree, int32_t* accept_len, int32_t* accept_path,
+                                        int32_t* bonus_token, void* stream);
+
 /* Synchronises `stream`, returns the device status word and clears it.
  * detail: an index that identifies the offending row/entry (meaning per status). */
 CAST_API cast_status cast_poll_status(cast_ctx* ctx, void* stream, cast_status* device_status, int32_t* detail);

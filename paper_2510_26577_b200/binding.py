@@ -26,7 +26,7 @@ MAX_DEPTH = 16
 EXPORTS = [
     "cast_create", "cast_destroy", "cast_status_string", "cast_set_cost_tables", "cast_state_export",
     "cast_state_import", "cast_step_begin", "cast_tree_expand", "cast_select_nodes", "cast_tree_attention",
-    "cast_accept", "cast_compact_kv", "cast_poll_status", "cast_step_info",
+    "cast_accept", "cast_compact_kv", "cast_poll_status", "cast_step_info", "cast_accept_static",
 ]
 
 
@@ -76,6 +76,7 @@ def load_library() -> C.CDLL:
         "cast_accept": [vp, vp, i32, i32, i32p, i32p, i32p, vp, i32p, i32p, i32p, i32p, vp],
         "cast_compact_kv": [vp, vp, vp, i32, i32, i32, C.c_size_t, i32, i32, i32, i32p, i32, i32, i32p, i32p, i32p,
                             vp],
+        "cast_accept_static": [vp, i32, i32, i32, i32, i32, i32p, i32p, i32p, i32p, i32p, i32p, vp],
         "cast_poll_status": [vp, vp, C.POINTER(C.c_int), C.POINTER(C.c_int32)],
         "cast_step_info": [vp, vp, C.POINTER(C.c_int32)],
     }
@@ -111,6 +112,16 @@ def _stream(stream) -> int:
 def _check(code: int, where: str):
     if code != CAST_OK:
         raise CastError(code, where)
+
+
+def cast_accept_static(target_logits, B, n_cap, vocab, max_depth, tokens, parent, n_tree, accept_len, accept_path,
+                       bonus_token, stream=None):
+    """The acceptance step without a context and without any allocation (see include/cast.h): for callers
+    that are handed device pointers but may not allocate.  Needs B * n_cap <= 2048."""
+    lib = load_library()
+    _check(lib.cast_accept_static(_ptr(target_logits), _dtype_code(target_logits), B, n_cap, vocab, max_depth,
+                                  _ptr(tokens), _ptr(parent), _ptr(n_tree), _ptr(accept_len), _ptr(accept_path),
+                                  _ptr(bonus_token), _stream(stream)), "cast_accept_static")
 
 
 class CastContext:

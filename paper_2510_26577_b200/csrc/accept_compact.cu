@@ -261,6 +261,76 @@ extern "C" cast_status cast_accept(cast_ctx* c, const void* target_logits, cast_
   return launch_status();
 }
 
+// ---- cast_accept_static: the acceptance step for callers that must not allocate ----------------
+// Scratch for the chunk winners of the target argmax sweep. It lives in the library image: every GPU
+// that loads the library holds these 512 KB until the process exits.
+constexpr int kStaticAcceptRows = 2048;  // B * Ncap at most
+static __device__ __align__(256) unsigned long long g_accept_static_scratch[kStaticAcceptRows * kAcceptMaxChunks];
+// The walk kernel records a malformed tree in a state block. Without a context there is none, so the
+// record goes to this one, which nobody reads (first record sticks; it never needs clearing).
+static __device__ __align__(256) cast::DevState g_accept_static_sink;
+
+namespace {
+// Device address of the scratch array, looked up once per device. In host code the array's name is
+// only a stand-in for the symbol; the address a kernel can use comes from cudaGetSymbolAddress.
+cast_status static_scratch_address(unsigned long long** out, DevState** sink) {
+  constexpr int kMaxDevices = 64;
+  static unsigned long long* addr[kMaxDevices] = {nullptr};
+  static DevState* sink_addr[kMaxDevices] = {nullptr};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return CAST_ERR_CUDA;
+  if (addr[dev] == nullptr || sink_addr[dev] == nullptr) {
+    void* p = nullptr;
+    void* q = nullptr;
+    if (cudaGetSymbolAddress(&p, g_accept_static_scratch) != cudaSuccess || p == nullptr) return CAST_ERR_CUDA;
+    if (cudaGetSymbolAddress(&q, g_accept_static_sink) != cudaSuccess || q == nullptr) return CAST_ERR_CUDA;
+    addr[dev] = static_cast<unsigned long long*>(p);
+    sink_addr[dev] = static_cast<DevState*>(q);
+  }
+  *out = addr[dev];
+  *sink = sink_addr[dev];
+  return CAST_OK;
+}
+}  // namespace
+
+extern "C" cast_status cast_accept_static(const void* target_logits, cast_dtype dtype, int B, int n_cap, int vocab,
+                                          int max_depth, const int32_t* tokens, const int32_t* parent,
+                                          const int32_t* n_tree, int32_t* accept_len, int32_t* accept_path,
+                                          int32_t* bonus_token, void* stream) {
+  if (!target_logits || !tokens || !parent || !n_tree || !accept_len || !accept_path || !bonus_token || B < 1 ||
+      n_cap < 1 || vocab < 1 || max_depth < 1)
+    return CAST_ERR_INVALID_ARG;
+  if (dtype != CAST_F32 && dtype != CAST_BF16) return CAST_ERR_DTYPE;
+  if (n_cap > CAST_MAX_TREE || max_depth > CAST_MAX_DEPTH || (long long)B * n_cap > kStaticAcceptRows)
+    return CAST_ERR_CAPACITY;
+  unsigned long long* scratch = nullptr;
+  DevState* sink = nullptr;
+  const cast_status st = static_scratch_address(&scratch, &sink);
+  if (st != CAST_OK) return st;
+  int num_sms = 0, dev = 0;
+  CAST_CUDA_OK(cudaGetDevice(&dev));
+  CAST_CUDA_OK(cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev));
+  int nchunks = (4 * num_sms + B * n_cap - 1) / (B * n_cap);
+  if (nchunks > kAcceptMaxChunks) nchunks = kAcceptMaxChunks;
+  if (nchunks > vocab / 4096) nchunks = vocab / 4096;
+  if (nchunks < 1) nchunks = 1;
+  int chunk_elems = (vocab + nchunks - 1) / nchunks;
+  chunk_elems = (chunk_elems + 7) / 8 * 8;
+  nchunks = (vocab + chunk_elems - 1) / chunk_elems;
+  cudaStream_t s = (cudaStream_t)stream;
+  const dim3 grid(nchunks, n_cap, B);
+  // every chunk winner that the walk reads is written by this call's sweep first: nothing to clear
+  if (dtype == CAST_F32)
+    argmax_sweep_kernel<float><<<grid, kArgThreads, 0, s>>>((const float*)target_logits, vocab, n_cap, chunk_elems,
+                                                            n_tree, scratch);
+  else
+    argmax_sweep_kernel<__nv_bfloat16><<<grid, kArgThreads, 0, s>>>((const __nv_bfloat16*)target_logits, vocab, n_cap,
+                                                                    chunk_elems, n_tree, scratch);
+  accept_walk_kernel<<<B, CAST_MAX_TREE, 0, s>>>(scratch, nchunks, n_cap, max_depth, tokens, parent, n_tree, accept_len,
+                                                 accept_path, bonus_token, sink);
+  return launch_status();
+}
+
 extern "C" cast_status cast_compact_kv(cast_ctx* c, void* k_cache, void* v_cache, cast_dtype dtype, int B,
                                        int n_layers, size_t layer_stride_bytes, int Hkv, int D, int page_size,
                                        const int32_t* page_table, int seq_capacity, int num_pages,
