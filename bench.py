@@ -172,15 +172,12 @@ def run_ours(args, w):
     _build.build()
     from paper_2510_26577_b200 import binding, workloads as wl
 
-    rank = int(os.environ.get("RANK", "0"))
+    from paper_2510_26577_b200 import replicas
     local = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
     torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    dev = torch.device("cuda", local)
+    rep = replicas.init("nccl")  # N > 1: independent replicas, one per GPU; no data-path collective
+    rank, world, dev = rep.rank, rep.world, rep.device
+    w = replicas.workload_for_rank(w, rank)
 
     B, H, K, Ncap, m = w.batch, w.depth, w.top_k, w.max_tree, w.total_token
     Hq, Hkv, D, nl = w.q_heads, w.kv_heads, w.head_dim, w.n_layers
@@ -314,16 +311,12 @@ def run_ours(args, w):
     kv_len.copy_(kv0)
 
     # ---- the timed region: K replays of the whole step
-    if dist is not None:
-        dist.barrier()
+    replicas.barrier(rep)
     torch.cuda.synchronize()
     sampler = ClockSampler(local) if rank == 0 else None
     ms_step = time_graph(g_step, args.steps, args.warmup)
-    if dist is not None:
-        t = torch.tensor([ms_step], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dist.barrier()
-        ms_step = float(t.item())
+    total_tokens, ms_step = replicas.aggregate(rep, tokens_per_step, ms_step)
+    replicas.barrier(rep)
     torch.cuda.synchronize()
     clocks = sampler.stop() if sampler else None
     st = ctx.cast_poll_status()
@@ -360,14 +353,10 @@ def run_ours(args, w):
         e1.record(stream)
         stream.synchronize()
     ms_e2e = e0.elapsed_time(e1) / (1 if args.quick else args.steps)
-    if dist is not None:
-        t = torch.tensor([ms_e2e], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
+    _, ms_e2e = replicas.aggregate(rep, tokens_per_step, ms_e2e)
 
     if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
+        replicas.shutdown(rep)
         return
 
     # ---- roofline of the dominant kernel (tree attention, one layer per launch)
@@ -380,7 +369,8 @@ def run_ours(args, w):
     achieved = attn_bytes / (attn_us * 1e-6) / 1e9
     logits_bytes = sum(int(x.numel() * x.element_size()) for x in logits) // K * 1  # layer 1 reads one row
     sel_launches = 1 if B == 1 else 2
-    launches = args.steps * (1 + H + sel_launches + 2 * nl + 2 + 1)
+    attn_launches = 1 if (w.kv_dtype == "bf16" and D == 128) else 2  # CUDA-core path: main + combine
+    launches = args.steps * (1 + H + sel_launches + attn_launches * nl + 2 + 1)
 
     cpu = None
     if not (args.no_cpu_baseline or args.quick):
@@ -389,7 +379,7 @@ def run_ours(args, w):
                "ms_per_step": sec * 1e3}
 
     line = {
-        "metric": METRIC, "value": world * tokens_per_step / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": total_tokens / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": w.kv_dtype, "data": "synthetic",
         "config": {"workload": w.name, "batch": B, "tree_tokens_per_step": tokens_per_step, "depth": H, "top_k": K,
@@ -398,7 +388,7 @@ def run_ours(args, w):
                    "logit_dtype": w.logit_dtype, "parallelism": "replicas" if world > 1 else "single",
                    "l2": "distinct KV buffers per layer; step working set exceeds 2x L2", "cuda_graph": True,
                    "accept_len_mean": accept_mean},
-        "e2e": {"value": world * tokens_per_step / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e,
+        "e2e": {"value": total_tokens / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e,
                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
         "gpu_launches": launches,
         "clocks": clocks,
@@ -411,8 +401,7 @@ def run_ours(args, w):
     }
     del logits_bytes
     print(json.dumps(line))
-    if dist is not None:
-        dist.destroy_process_group()
+    replicas.shutdown(rep)
 
 
 def main():
