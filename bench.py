@@ -25,6 +25,10 @@ if ROOT not in sys.path:
 
 METRIC, UNIT = "tree_verify_tokens_per_s", "tokens/s"
 
+# DRAM bytes (read + write) of one tree_attn_tc_kernel launch from the ncu captures summarised
+# under profiles/ (same launch shape as one layer of the workload).
+NCU_ATTENTION_TRAFFIC = {"c2_llama8b": 9.22e6, "c3_llama8b_b16": 142.6e6}
+
 
 def peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -395,7 +399,7 @@ def run_ours(args, w):
         "phases": {"tree_build_us": ms_tree * 1e3, "attention_us_per_layer": attn_us, "accept_us": ms_acc * 1e3,
                    "compact_us": ms_cmp * 1e3},
         "roofline": {"kernel": "cast_tree_attention (one layer)", "bound": "hbm", "achieved": achieved, "peak": peak,
-                     "unit": "GB/s", "frac": achieved / peak, "peak_source": which, "traffic": None,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_source": which, "traffic": NCU_ATTENTION_TRAFFIC.get(w.name),
                      "algorithmic_bytes": attn_bytes},
         "cpu_baseline": cpu,
     }

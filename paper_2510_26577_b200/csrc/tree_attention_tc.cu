@@ -16,11 +16,14 @@
 //                  prefix/ancestor mask (only tiles that reach past the prefix need one), keeps a
 //                  lazily updated row maximum (O in TMEM is rescaled only when the maximum grows
 //                  by more than 2^8), writes P as bf16 into swizzled shared memory.
-// The number of KV splits is decided on the device from the actual tree sizes and prefix
-// lengths (the host only fixes its upper bound), so the grid fills the machine whatever N the
-// cost model picked. Split partials are merged by the last CTA of a row block to finish (an
-// atomic ticket; nothing spins). All mbarrier waits are bounded: on expiry the CTA records
-// CAST_ERR_TIMEOUT, drains its copies, frees its TMEM and returns.
+// The kernel is launched in thread-block clusters: a cluster covers the row blocks of one
+// (sequence, kv-head) and splits each one's KV range over its CTAs, the number of splits per row
+// block being decided on the device from the actual tree size (the host only knows the largest
+// tree). The splits of a row block are merged through distributed shared memory: every CTA stages
+// its partial output in its own shared memory, the cluster meets at a barrier, and each CTA
+// combines and writes its share of the rows, reading its peers' partials directly. Nothing goes
+// through global memory and nothing spins. All mbarrier waits are bounded: on expiry the CTA
+// records CAST_ERR_TIMEOUT, contributes nothing to the merge, and still meets its cluster.
 #include <cuda.h>
 #include <math.h>
 #include <stdlib.h>
@@ -79,15 +82,14 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 struct TcParams {
   const __nv_bfloat16* q;
   __nv_bfloat16* out;
-  int B, Ncap, Nmax, Hq, Hkv, G, page_size, seq_capacity, num_pages, words, nsplit_max, num_sms, nrb;
+  int B, Ncap, Nmax, Hq, Hkv, G, page_size, seq_capacity, num_pages, words;
+  int cs;   // CTAs per cluster (1, 2, 4 or 8)
+  int rpc;  // row blocks a cluster covers at most (cs is a multiple of it)
   const int32_t* page_table;
   const int32_t* kv_len;
   const int32_t* n_tree;
   const uint32_t* anc;
   float scale_log2;
-  float* part_o;     // [B][Hq][Ncap][nsplit_max][D]
-  float* part_ml;    // [B][Hq][Ncap][nsplit_max][2]
-  int32_t* ticket;   // [B][Hkv][nrb]
   DevState* st;
 };
 
@@ -192,7 +194,6 @@ __device__ __forceinline__ float fast_exp2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-__device__ __forceinline__ void softmax_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kSoftmaxThreads) : "memory"); }
 
 // 32 bits of the visibility vector of one query row, starting at tree index `start` (which may be
 // negative: prefix positions, always visible; or past the tree: never visible). aw = the row's
@@ -211,36 +212,33 @@ __device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * 12
 
 __device__ __forceinline__ int clampi(int x, int lo, int hi) { return x < lo ? lo : (x > hi ? hi : x); }
 
-// The grid is one-dimensional: CTA i takes work item i. Items are enumerated on the device from
-// the actual tree sizes and prefix lengths: sequence b has Hkv * row_blocks(b) * splits(b) of them,
-// the kv-head running fastest so that the heads of one piece of a sequence stream the same pages at
-// the same time. splits(b) = ceil(tiles(b) / chunk); chunk (>= 4 tiles) is the smallest piece size
-// for which all items fit into W waves of 2 * num_sms CTAs, W being the number of waves that even
-// unsplit work would need. So the CTAs are of about equal size whatever the mix of lengths, there are
-// as few splits as the machine allows, and CTAs beyond the item count exit at once. Every warp
-// computes the same values (all 32 lanes must call).
+// The grid is one-dimensional and launched in clusters of p.cs CTAs. A cluster takes one
+// (sequence, kv-head, group of up to p.rpc row blocks); its CTAs share the group's row blocks and
+// split each one's KV range evenly: with nr row blocks actually present (known only on the device,
+// from n_tree), every row block gets cs / nr splits. A small tree under a large token budget thus
+// turns the CTAs reserved for its absent row blocks into extra KV splits. Clusters are enumerated on
+// the device from the actual sizes, sequences with the longest pieces first (the block scheduler
+// hands clusters out in index order, so the long pieces start first and the short ones fill the
+// gaps), the kv-head running fastest so that the heads of one sequence stream the same pages at the
+// same time. Clusters past the count exit at once. Every warp computes the same values (all 32
+// lanes must call).
 struct WorkItem {
   int b, kvh, rb, split, nsplit, N, L;
-  bool valid;
+  bool valid;   // the cluster has work
+  bool active;  // this CTA has a row block (an inactive CTA of a valid cluster only keeps the barriers in step)
 };
 
-__device__ __forceinline__ int warp_sum(int v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
-}
-__device__ __forceinline__ WorkItem decode_work(const TcParams& p, int idx, int grid) {
+__device__ __forceinline__ WorkItem decode_work(const TcParams& p, int cid, int crank) {
   constexpr int KB = CAST_MAX_BATCH / 32;
   const int lane = threadIdx.x & 31;
   const int max_pos = p.page_size == 0 ? p.seq_capacity : p.seq_capacity * p.page_size;
-  int Nv[KB], Lv[KB], tl[KB], nr[KB];
+  int Nv[KB], Lv[KB], tl[KB], nr[KB], cnt[KB], off[KB];
 #pragma unroll
   for (int k = 0; k < KB; ++k) {  // all loads first: one memory round trip
     const int bb = k * 32 + lane;
     Nv[k] = bb < p.B ? p.n_tree[bb] : 0;
     Lv[k] = bb < p.B ? p.kv_len[bb] : 0;
   }
-  int base = 0, T = 0, tmax = 0;
 #pragma unroll
   for (int k = 0; k < KB; ++k) {
     Nv[k] = clampi(Nv[k], 0, p.Nmax);
@@ -249,115 +247,109 @@ __device__ __forceinline__ WorkItem decode_work(const TcParams& p, int idx, int 
     total = total > max_pos ? max_pos : total;
     nr[k] = (Nv[k] * p.G + kBM - 1) / kBM;
     tl[k] = nr[k] > 0 ? (total + kBN - 1) / kBN : 0;
-    base += p.Hkv * nr[k];
-    T += p.Hkv * nr[k] * tl[k];
-    tmax = tl[k] > tmax ? tl[k] : tmax;
-  }
-  base = warp_sum(base);
-  T = warp_sum(T);
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) tmax = max(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
-  const int slots = 2 * p.num_sms;
-  int W = (base + slots - 1) / slots;
-  W = W < 1 ? 1 : W;
-  int cap = W * slots;
-  cap = cap > grid ? grid : cap;
-  // smallest chunk (>= 4 tiles) whose item count fits: the count falls as the chunk grows, and a chunk
-  // of tmax tiles (no splits at all) always fits
-  auto items_at = [&](int chunk) {
-    int items = 0;
-#pragma unroll
-    for (int k = 0; k < KB; ++k) {
-      int n = (tl[k] + chunk - 1) / chunk;
-      n = n > p.nsplit_max ? p.nsplit_max : n;
-      items += p.Hkv * nr[k] * n;
-    }
-    return warp_sum(items);
-  };
-  int lo = (T + cap - 1) / cap, hi = tmax < 4 ? 4 : tmax;
-  lo = lo < 4 ? 4 : lo;
-  lo = lo > hi ? hi : lo;
-  while (lo < hi) {
-    const int mid = (lo + hi) >> 1;
-    if (items_at(mid) <= cap) hi = mid; else lo = mid + 1;
-  }
-  const int chunk = lo;
-  int ns[KB], cnt[KB], off[KB];
-#pragma unroll
-  for (int k = 0; k < KB; ++k) {
-    int n = (tl[k] + chunk - 1) / chunk;
-    n = n > p.nsplit_max ? p.nsplit_max : n;
-    ns[k] = n < 1 ? 1 : n;
-    cnt[k] = p.Hkv * nr[k] * ns[k];
+    cnt[k] = p.Hkv * ((nr[k] + p.rpc - 1) / p.rpc);
     off[k] = 0;
   }
-  // items are numbered longest piece first (the block scheduler hands CTAs out in index order, so
-  // the long pieces start first and the short ones fill the gaps): sequence j precedes sequence b
-  // when its pieces are longer, ties by index
-  for (int j = 0; j < p.B; ++j) {
-    const int src = j & 31;
-    int pj, cj;
-    if (j < 32) {
-      pj = __shfl_sync(0xffffffffu, tl[0] * 16 / ns[0], src);
-      cj = __shfl_sync(0xffffffffu, cnt[0], src);
-    } else {
-      pj = __shfl_sync(0xffffffffu, tl[KB - 1] * 16 / ns[KB - 1], src);
-      cj = __shfl_sync(0xffffffffu, cnt[KB - 1], src);
-    }
+  if (p.B > 1) {
+    for (int j = 0; j < p.B; ++j) {  // sequence j precedes sequence b when it is longer, ties by index
+      const int src = j & 31;
+      int pj, cj;
+      if (j < 32) {
+        pj = __shfl_sync(0xffffffffu, tl[0], src);
+        cj = __shfl_sync(0xffffffffu, cnt[0], src);
+      } else {
+        pj = __shfl_sync(0xffffffffu, tl[KB - 1], src);
+        cj = __shfl_sync(0xffffffffu, cnt[KB - 1], src);
+      }
 #pragma unroll
-    for (int k = 0; k < KB; ++k) {
-      const int mine = tl[k] * 16 / ns[k], bm = k * 32 + lane;
-      if (pj > mine || (pj == mine && j < bm)) off[k] += cj;
+      for (int k = 0; k < KB; ++k) {
+        const int bm = k * 32 + lane;
+        if (pj > tl[k] || (pj == tl[k] && j < bm)) off[k] += cj;
+      }
     }
   }
   WorkItem w;
-  w.valid = false;
+  w.valid = w.active = false;
   w.b = w.kvh = w.rb = w.split = w.N = w.L = 0;
   w.nsplit = 1;
 #pragma unroll
   for (int k = 0; k < KB; ++k) {
-    const unsigned hit = __ballot_sync(0xffffffffu, idx >= off[k] && idx < off[k] + cnt[k]);
+    const unsigned hit = __ballot_sync(0xffffffffu, cid >= off[k] && cid < off[k] + cnt[k]);
     if (hit != 0u && !w.valid) {
       const int bl = __ffs(hit) - 1;
-      const int local = idx - __shfl_sync(0xffffffffu, off[k], bl);
-      w.nsplit = __shfl_sync(0xffffffffu, ns[k], bl);
+      const int local = cid - __shfl_sync(0xffffffffu, off[k], bl);
+      const int nrb = __shfl_sync(0xffffffffu, nr[k], bl);
       w.N = __shfl_sync(0xffffffffu, Nv[k], bl);
       w.L = __shfl_sync(0xffffffffu, Lv[k], bl);
       w.b = k * 32 + bl;
       w.kvh = local % p.Hkv;
-      const int rest = local / p.Hkv;
-      w.split = rest % w.nsplit;
-      w.rb = rest / w.nsplit;
+      const int grp = local / p.Hkv;
+      int nr_in = nrb - grp * p.rpc;
+      nr_in = nr_in > p.rpc ? p.rpc : nr_in;  // >= 1 for an enumerated group
+      w.nsplit = p.cs / nr_in;
+      const int rbl = crank / w.nsplit;
+      w.split = crank % w.nsplit;
+      w.rb = grp * p.rpc + rbl;
+      w.active = rbl < nr_in;
       w.valid = true;
     }
   }
   return w;
 }
 
-// Merge of the split partials of a row block, run by all 8 warps of the last CTA to finish it.
-// Warp w takes rows w, w+8, ...; a lane owns 4 output columns. ROWS rows x SPL splits = 16 loads are
-// in flight per lane: the merge is bound by L2 latency, not by bytes.
+// ---- cluster primitives
+__device__ __forceinline__ uint32_t cluster_ctarank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ float2 ld_cluster_f2(uint32_t addr) {
+  float2 v;
+  asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+  return v;
+}
+
+constexpr int kStageStride = kHD + 4;  // floats per staged output row: 16-byte accesses stay conflict-free
+
+// Merge of the splits of a row block through distributed shared memory. Every CTA of the split
+// group has staged its partial O (fp32, unnormalised) and (max, sum) per row in its own shared
+// memory; this CTA owns the rows rr with rr % nsplit == split and reads them from all peers.
+// Warp w takes owned rows w, w+8, ...; a lane owns 4 output columns; ROWS x SPL loads in flight.
 template <int ROWS, int SPL>
-__device__ __forceinline__ void merge_rows(const TcParams& p, int b, int kvh, int row0, int rows_here, int nsplit) {
+__device__ __forceinline__ void merge_rows(const TcParams& p, uint32_t stage_o_s, uint32_t stage_ml_s, int rank0,
+                                           int b, int kvh, int row0, int rows_here, int nsplit, int split) {
   const int lane = threadIdx.x & 31, wv = threadIdx.x >> 5, G = p.G;
-  for (int rr = wv; rr < rows_here; rr += 8 * ROWS) {
+  const int owned = rows_here > split ? (rows_here - split + nsplit - 1) / nsplit : 0;
+  for (int i0 = wv; i0 < owned; i0 += 8 * ROWS) {
     float4 v[ROWS][SPL];
     float wgt[ROWS], inv[ROWS];
     size_t orow[ROWS];
 #pragma unroll
     for (int u = 0; u < ROWS; ++u) {
-      const int r2 = rr + 8 * u;
-      const int grow = row0 + (r2 < rows_here ? r2 : rr), tt = grow / G, hh = kvh * G + grow % G;
-      const size_t pr = (((size_t)b * p.Hq + hh) * p.Ncap + tt) * p.nsplit_max;
+      const int i2 = i0 + 8 * u;
+      const int rr = split + nsplit * (i2 < owned ? i2 : i0);
+      const int grow = row0 + rr, tt = grow / G, hh = kvh * G + grow % G;
       orow[u] = (((size_t)b * p.Ncap + tt) * p.Hq + hh) * kHD;
       float ms = -INFINITY, ls = 0.f;  // lane s holds split s's (max, sum)
       if (lane < nsplit) {
-        ms = __ldcg(p.part_ml + (pr + lane) * 2);
-        ls = __ldcg(p.part_ml + (pr + lane) * 2 + 1);
+        const float2 ml = ld_cluster_f2(map_to_rank(stage_ml_s + (uint32_t)rr * 8u, (uint32_t)(rank0 + lane)));
+        ms = ml.x;
+        ls = ml.y;
       }
 #pragma unroll
       for (int s2 = 0; s2 < SPL; ++s2)
-        v[u][s2] = s2 < nsplit ? __ldcg(reinterpret_cast<const float4*>(p.part_o + (pr + s2) * kHD + lane * 4))
+        v[u][s2] = s2 < nsplit ? ld_cluster_f4(map_to_rank(stage_o_s + (uint32_t)(rr * kStageStride + lane * 4) * 4u,
+                                                           (uint32_t)(rank0 + s2)))
                                : make_float4(0.f, 0.f, 0.f, 0.f);
       float M = ms;
 #pragma unroll
@@ -374,12 +366,14 @@ __device__ __forceinline__ void merge_rows(const TcParams& p, int b, int kvh, in
 #pragma unroll
       for (int s2 = 0; s2 < SPL; ++s2) {
         const float w = __shfl_sync(0xffffffffu, wgt[u], s2);
-        acc.x += v[u][s2].x * w;
-        acc.y += v[u][s2].y * w;
-        acc.z += v[u][s2].z * w;
-        acc.w += v[u][s2].w * w;
+        if (w > 0.f) {  // a split without visible positions staged nothing: its buffer may hold anything
+          acc.x += v[u][s2].x * w;
+          acc.y += v[u][s2].y * w;
+          acc.z += v[u][s2].z * w;
+          acc.w += v[u][s2].w * w;
+        }
       }
-      if (rr + 8 * u < rows_here) {
+      if (i0 + 8 * u < owned) {
         const __nv_bfloat162 a = __floats2bfloat162_rn(acc.x * inv[u], acc.y * inv[u]),
                              c2 = __floats2bfloat162_rn(acc.z * inv[u], acc.w * inv[u]);
         uint2 pk;
@@ -401,12 +395,18 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
   TC_CTA_LOG(1, 0ull);
   TC_CTA_LOG(3, 0ull);
   TC_CTA_LOG(2, (unsigned long long)smid());
-  const WorkItem wk = decode_work(p, blockIdx.x, gridDim.x);
+  const int cs = p.cs;
+  const int crank = cs > 1 ? (int)cluster_ctarank() : 0;
+  if (warp == 4 && lane == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_k)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_v)) : "memory");
+  }
+  const WorkItem wk = decode_work(p, (int)blockIdx.x / cs, crank);
   TC_MARK(1);
   if (blockIdx.x < p.B && tid == 0 && p.n_tree[blockIdx.x] > p.Nmax) report(p.st, CAST_ERR_BAD_TREE, blockIdx.x);
-  if (!wk.valid) return;
+  if (!wk.valid) return;  // the whole cluster leaves
   const int b = wk.b, kvh = wk.kvh, rb = wk.rb, split = wk.split, N = wk.N, L = wk.L;
-  int nsplit = wk.nsplit;
+  const int nsplit = wk.nsplit;
   const int G = p.G, rows_total = N * G, row0 = rb * kBM;
   const int max_pos = p.page_size == 0 ? p.seq_capacity : p.seq_capacity * p.page_size;
   int total = L + N;
@@ -415,8 +415,21 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     total = max_pos;
   }
   const int ntiles = (total + kBN - 1) / kBN;  // >= 1 because N >= 1 here
-  if ((smem_u32(smem) & 1023u) != 0u) {  // the swizzled operand regions need a 1 KB aligned base
-    if (tid == 0) report(p.st, CAST_ERR_CUDA, 1024);
+  float* stage_o = reinterpret_cast<float*>(smem + kSmemK);   // [128][kStageStride] floats < K ring + V ring + P
+  float* stage_ml = reinterpret_cast<float*>(smem + kSmemQ);  // [128][2]
+  const bool aligned = (smem_u32(smem) & 1023u) == 0u;  // the swizzled operand regions need a 1 KB aligned base
+  if (!wk.active || !aligned) {
+    // no row block for this CTA (or an unusable shared-memory base): it contributes nothing, but the
+    // other CTAs of the cluster still meet it at both cluster barriers
+    if (!aligned && tid == 0) report(p.st, CAST_ERR_CUDA, 1024);
+    if (tid < kBM) {
+      stage_ml[tid * 2] = -INFINITY;
+      stage_ml[tid * 2 + 1] = 0.f;
+    }
+    if (cs > 1) {
+      cluster_sync_all();
+      cluster_sync_all();
+    }
     return;
   }
   const int t0 = (int)((long long)split * ntiles / nsplit), t1 = (int)((long long)(split + 1) * ntiles / nsplit);
@@ -434,7 +447,6 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
   uint64_t* bar_s = bars + 8;          // [2]
   uint64_t* bar_p = bars + 10;
   uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(bars + 11);
-  int* last_s = reinterpret_cast<int*>(bars + 12);
 
   // ---- producer helper (warp 4; all 32 lanes call it): which = 0: K tile j, which = 1: V tile j
   auto issue_tile = [&](int j, int which) -> bool {
@@ -592,8 +604,8 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     };
     // next scores first: Q K^T of tile it+1 runs while the softmax of tile `it` does; the other CTA on
     // this SM covers the moments when a K tile is late
-    bool ok = mbar_wait(&bar_fullk[0], 0);
-    if (ok) {
+    bool ok = ntile == 0 || mbar_wait(&bar_fullk[0], 0);
+    if (ok && ntile > 0) {
       tc_fence_after();
       mma_qk(0, 0);
     }
@@ -742,15 +754,17 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
       mbar_arrive(bar_p);
       TC_STAMP(0, it, 9);
     }
-    // epilogue: wait for the last P V; O goes through shared memory (the K/V rings and P are idle
-    // now) so that every global store of a row is one contiguous 512-byte (fp32) or 256-byte (bf16) piece
+    // epilogue: wait for the last P V, then stage O (fp32, unnormalised) and (max, sum) per row in
+    // shared memory (the K/V rings, P and Q are idle now): the output rows are written, or merged
+    // across the splits, from there in contiguous pieces
     TC_MARK(4);
-    if (ok) ok = mbar_wait(&bar_freev[(ntile - 1) % kStages], ((ntile - 1) / kStages) & 1);
+    if (ok && ntile > 0) ok = mbar_wait(&bar_freev[(ntile - 1) % kStages], ((ntile - 1) / kStages) & 1);
     TC_MARK(5);
-    constexpr int kStageStride = kHD + 4;  // floats per staged row: 16-byte stores stay conflict-free
-    float* stage_o = reinterpret_cast<float*>(smem + kSmemK);  // 128 x 132 floats < K ring + V ring + P
-    float* stage_ml = reinterpret_cast<float*>(smem + kSmemQ);  // [128][2]: Q is idle as well
-    if (ok && warp_live) {
+    if (!ok) {  // a wait ran out: this split contributes nothing
+      m_used = -INFINITY;
+      l_run = 0.f;
+    }
+    if (ok && warp_live && ntile > 0) {
       tc_fence_after();
 #pragma unroll
       for (int hh = 0; hh < 4; ++hh) {
@@ -764,63 +778,42 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
               make_float4(__uint_as_float(orr[c4 * 4]), __uint_as_float(orr[c4 * 4 + 1]), __uint_as_float(orr[c4 * 4 + 2]),
                           __uint_as_float(orr[c4 * 4 + 3]));
       }
-      stage_ml[r * 2] = m_used * sc * 0.69314718055994531f;  // natural-log units
-      stage_ml[r * 2 + 1] = l_run;
     }
-    softmax_bar();
-    const int rows_here = rows_total - row0 < kBM ? rows_total - row0 : kBM;
-    const int wv = warp;  // 0..3: rows wv, wv+4, ... ; lane: columns 4*lane .. 4*lane+3
-    if (ok) {
-      for (int rr = wv; rr < rows_here; rr += 4) {
-        const int grow = row0 + rr, tt = grow / G, hh = kvh * G + grow % G;
-        const float4 o4 = *reinterpret_cast<const float4*>(stage_o + rr * kStageStride + lane * 4);
-        const float l_tot = stage_ml[rr * 2 + 1];
-        if (nsplit == 1) {
-          const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
-          const __nv_bfloat162 a = __floats2bfloat162_rn(o4.x * inv, o4.y * inv), c2 = __floats2bfloat162_rn(o4.z * inv, o4.w * inv);
-          uint2 pk;
-          pk.x = *reinterpret_cast<const uint32_t*>(&a);
-          pk.y = *reinterpret_cast<const uint32_t*>(&c2);
-          *reinterpret_cast<uint2*>(p.out + (((size_t)b * p.Ncap + tt) * p.Hq + hh) * kHD + lane * 4) = pk;
-        } else {
-          const size_t pr = (((size_t)b * p.Hq + hh) * p.Ncap + tt) * p.nsplit_max + split;
-          __stcg(reinterpret_cast<float4*>(p.part_o + pr * kHD + lane * 4), o4);
-          if (lane == 0) {
-            __stcg(p.part_ml + pr * 2, stage_ml[rr * 2]);
-            __stcg(p.part_ml + pr * 2 + 1, l_tot);
-          }
-        }
-      }
-    }
-    if (nsplit > 1) __threadfence();  // the partials must be visible before this CTA takes its ticket
+    stage_ml[r * 2] = m_used * sc * 0.69314718055994531f;  // natural-log units (-inf: nothing visible)
+    stage_ml[r * 2 + 1] = l_run;
   }
   TC_MARK(6);
   tc_fence_before();
   __syncthreads();
-  if (nsplit > 1) {
-    // the last split of this row block to finish merges the partials (ticket; nothing spins)
-    if (tid == 0) {
-      int32_t* cnt = p.ticket + ((size_t)b * p.Hkv + kvh) * p.nrb + rb;
-      const int t = atomicAdd(cnt, 1);
-      *last_s = (t == nsplit - 1);
-      if (t == nsplit - 1) *cnt = 0;
-      __threadfence();
-    }
-    __syncthreads();
-    if (*last_s) {
-      TC_CTA_LOG(3, gtimer());
-      const int rows_here = rows_total - row0 < kBM ? rows_total - row0 : kBM;
-      if (nsplit <= 2) merge_rows<8, 2>(p, b, kvh, row0, rows_here, nsplit);
-      else if (nsplit <= 4) merge_rows<4, 4>(p, b, kvh, row0, rows_here, nsplit);
-      else merge_rows<2, kMaxSplit>(p, b, kvh, row0, rows_here, nsplit);
-    }
-  }
-  TC_MARK(7);
-  TC_CTA_LOG(1, gtimer());
-  if (warp == 0) {
+  if (warp == 0) {  // every TMEM access of this CTA is over
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols));
   }
+  if (cs > 1) cluster_sync_all();  // every CTA of the cluster has staged its rows
+  TC_CTA_LOG(3, gtimer());
+  const int rows_here = rows_total - row0 < kBM ? rows_total - row0 : kBM;
+  if (nsplit == 1) {
+    for (int rr = warp; rr < rows_here; rr += kThreadsTC / 32) {
+      const int grow = row0 + rr, tt = grow / G, hh = kvh * G + grow % G;
+      const float4 o4 = *reinterpret_cast<const float4*>(stage_o + rr * kStageStride + lane * 4);
+      const float l_tot = stage_ml[rr * 2 + 1];
+      const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
+      const __nv_bfloat162 a = __floats2bfloat162_rn(o4.x * inv, o4.y * inv), c2 = __floats2bfloat162_rn(o4.z * inv, o4.w * inv);
+      uint2 pk;
+      pk.x = *reinterpret_cast<const uint32_t*>(&a);
+      pk.y = *reinterpret_cast<const uint32_t*>(&c2);
+      *reinterpret_cast<uint2*>(p.out + (((size_t)b * p.Ncap + tt) * p.Hq + hh) * kHD + lane * 4) = pk;
+    }
+  } else {
+    const uint32_t so_s = smem_u32(stage_o), sml_s = smem_u32(stage_ml);
+    const int rank0 = crank - split;  // first CTA of this row block's split group
+    if (nsplit <= 2) merge_rows<8, 2>(p, so_s, sml_s, rank0, b, kvh, row0, rows_here, nsplit, split);
+    else if (nsplit <= 4) merge_rows<4, 4>(p, so_s, sml_s, rank0, b, kvh, row0, rows_here, nsplit, split);
+    else merge_rows<2, kMaxSplit>(p, so_s, sml_s, rank0, b, kvh, row0, rows_here, nsplit, split);
+  }
+  TC_MARK(7);
+  TC_CTA_LOG(1, gtimer());
+  if (cs > 1) cluster_sync_all();  // nobody leaves while a peer may still read its shared memory
 }
 
 #ifdef CAST_PHASE_CLOCKS
@@ -984,44 +977,33 @@ bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const v
   const int nrb = (Nmax * G + kBM - 1) / kBM;
   const int max_pos = page_size == 0 ? seq_capacity : seq_capacity * page_size;
   const int max_tiles = (max_pos + kBN - 1) / kBN;
-  // upper bound of the KV splits; the kernel picks the actual number from the device-side sizes
-  int nsplit_max = kMaxSplit;
-  if (nsplit_max > max_tiles) nsplit_max = max_tiles;
-  if (nsplit_max < 1) nsplit_max = 1;
-  // one-dimensional grid: whole waves of two CTAs per SM, enough of them for the unsplit work
+  // KV splits per row block: as many (a power of two, at most 8) as keep the CTA count within one
+  // wave of two CTAs per SM, and no more than leave each split a few tiles. The tree sizes are only
+  // known on the device, so this is sized for the largest tree; a cluster then covers `rpc` row blocks
+  // and hands the CTAs of absent ones to the present ones as further splits.
   const int slots = 2 * c->num_sms;
-  const int waves = (B * Hkv * nrb + slots - 1) / slots;
-  const int grid = slots * (waves < 1 ? 1 : waves);
+  int splits = 1;
+  while (splits < kMaxSplit && (long long)B * Hkv * nrb * splits * 2 <= slots && max_tiles / (splits * 2) >= 2) splits *= 2;
+  int rpc = 1;
+  while (rpc * 2 * splits <= kMaxSplit && rpc * 2 <= nrb) rpc *= 2;
+#ifdef CAST_PHASE_CLOCKS
+  if (const char* e = getenv("CAST_TC_SPLITS")) splits = atoi(e);
+  if (const char* e = getenv("CAST_TC_RPC")) rpc = atoi(e);
+#endif
+  const int cs = splits * rpc;
+  const int groups = (nrb + rpc - 1) / rpc;
+  const long long clusters = (long long)B * Hkv * groups;
+  const long long grid = clusters * cs;
+  if (grid > 0x7fffffffll) return false;
   TcParams p;
   p.q = (const __nv_bfloat16*)q; p.out = (__nv_bfloat16*)out;
   p.B = B; p.Ncap = Ncap; p.Nmax = Nmax; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.page_size = page_size;
-  p.seq_capacity = seq_capacity; p.num_pages = num_pages; p.words = c->words; p.nsplit_max = nsplit_max;
-  p.num_sms = c->num_sms; p.nrb = nrb;
+  p.seq_capacity = seq_capacity; p.num_pages = num_pages; p.words = c->words;
+  p.cs = cs; p.rpc = rpc;
   p.page_table = page_table; p.kv_len = kv_len; p.n_tree = n_tree; p.anc = anc;
   p.scale_log2 = scale * 1.4426950408889634f;
-  p.part_o = nullptr; p.part_ml = nullptr; p.ticket = nullptr; p.st = c->state;
+  p.st = c->state;
   *status = CAST_OK;
-  if (nsplit_max > 1) {
-    const size_t rows = (size_t)B * Hq * Ncap * nsplit_max;
-    const size_t tickets = (size_t)B * Hkv * nrb;
-    const size_t need = rows * (kHD + 2) * sizeof(float) + tickets * sizeof(int32_t);
-    if (need > c->attn_ws_bytes) {  // grows the workspace (synchronises; not legal during graph capture)
-      if (cudaDeviceSynchronize() != cudaSuccess) { *status = CAST_ERR_CUDA; return true; }
-      if (c->attn_ws) cudaFree(c->attn_ws);
-      c->attn_ws = nullptr;
-      c->attn_ws_bytes = 0;
-      if (cudaMalloc(&c->attn_ws, need) != cudaSuccess) { *status = CAST_ERR_CUDA; return true; }
-      c->attn_ws_bytes = need;
-    }
-    p.part_o = reinterpret_cast<float*>(c->attn_ws);
-    p.part_ml = p.part_o + rows * kHD;
-    p.ticket = reinterpret_cast<int32_t*>(p.part_ml + rows * 2);
-    // tickets start at zero (every merge also leaves its ticket at zero again)
-    if (cudaMemsetAsync(p.ticket, 0, tickets * sizeof(int32_t), stream) != cudaSuccess) {
-      *status = CAST_ERR_CUDA;
-      return true;
-    }
-  }
   static bool attr_done = false;
   if (!attr_done) {
     if (cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) !=
@@ -1038,12 +1020,28 @@ bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const v
     const int kvh_fast = atoi(lo) == 2;
     cudaFuncSetAttribute(dbg_loadonly_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * 2 * kTileKV + 64);
     cudaFuncSetAttribute(dbg_loadonly_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
-    dbg_loadonly_kernel<<<grid, 64, 4 * 2 * kTileKV + 64, stream>>>(p, map_k, map_v, kvh_fast);
+    dbg_loadonly_kernel<<<(unsigned)grid, 64, 4 * 2 * kTileKV + 64, stream>>>(p, map_k, map_v, kvh_fast);
     *status = launch_status();
     return true;
   }
 #endif
-  tree_attn_tc_kernel<<<grid, kThreadsTC, kSmemBytes, stream>>>(p, map_k, map_v);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid, 1, 1);
+  cfg.blockDim = dim3(kThreadsTC, 1, 1);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)cs;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel, p, map_k, map_v) != cudaSuccess) {
+    cudaGetLastError();
+    *status = CAST_ERR_CUDA;
+    return true;
+  }
   *status = launch_status();
   return true;
 }
