@@ -36,7 +36,7 @@ void free_all(cast_ctx* c) {
   cudaFree(c->pool_kept); cudaFree(c->retained); cudaFree(c->lsort); cudaFree(c->lscore); cudaFree(c->state); cudaFree(c->part_keys);
   cudaFree(c->part_max); cudaFree(c->part_sum); cudaFree(c->row_ticket); cudaFree(c->layer_ticket);
   cudaFree(c->fifo_vals); cudaFree(c->fifo_cnt); cudaFree(c->sel_score); cudaFree(c->sel_value);
-  cudaFree(c->sel_idx); cudaFree(c->acc_part); cudaFree(c->compact_ticket); cudaFree(c->attn_ws);
+  cudaFree(c->sel_idx); cudaFree(c->acc_part); cudaFree(c->compact_ticket); cudaFree(c->attn_ws); cudaFree(c->attn_tc_ws);
   if (c->tables) {
     for (auto& kv : *c->tables) cudaFree(kv.second.storage);
     delete c->tables;

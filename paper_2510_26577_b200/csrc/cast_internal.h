@@ -98,6 +98,9 @@ struct cast_ctx {
   // attention workspace (grown on demand)
   void* attn_ws;
   size_t attn_ws_bytes;
+  // workspace of the tensor-core attention's global-merge mode: tickets, then split partials
+  void* attn_tc_ws;
+  size_t attn_tc_ws_bytes;
 
   std::map<int, cast::HostTable>* tables;
   cast::DevTable cur_table;   // table of the current step's batch size (zeros if none)

@@ -83,8 +83,12 @@ struct TcParams {
   const __nv_bfloat16* q;
   __nv_bfloat16* out;
   int B, Ncap, Nmax, Hq, Hkv, G, page_size, seq_capacity, num_pages, words;
-  int cs;   // CTAs per cluster (1, 2, 4 or 8)
-  int rpc;  // row blocks a cluster covers at most (cs is a multiple of it)
+  int cs;   // CTAs per cluster (1..8); 0: no clusters, splits sized on the device and merged through global memory
+  int rpc;  // cluster mode: row blocks a cluster covers at most (cs is a multiple of it)
+  int nsplit_max, num_sms, nrb;  // global-merge mode
+  float* part_o;     // [B][Hq][Ncap][nsplit_max][D]
+  float* part_ml;    // [B][Hq][Ncap][nsplit_max][2]
+  int32_t* ticket;   // [B][Hkv][nrb]
   const int32_t* page_table;
   const int32_t* kv_len;
   const int32_t* n_tree;
@@ -251,6 +255,7 @@ __device__ __forceinline__ WorkItem decode_work(const TcParams& p, int cid, int 
     off[k] = 0;
   }
   if (p.B > 1) {
+#pragma unroll 8
     for (int j = 0; j < p.B; ++j) {  // sequence j precedes sequence b when it is longer, ties by index
       const int src = j & 31;
       int pj, cj;
@@ -385,6 +390,188 @@ __device__ __forceinline__ void merge_rows(const TcParams& p, uint32_t stage_o_s
   }
 }
 
+// ---- global-merge mode -------------------------------------------------------------------------
+// For launches with long CTAs or many ragged sequences, where an even load matters more than the
+// cost of the merge: no clusters; CTA i takes work item i. Sequence b has Hkv * row_blocks(b) *
+// splits(b) items, splits(b) = ceil(tiles(b) / chunk), chunk (>= 4 tiles) being the smallest piece
+// size for which all items fit into the launched waves of 2 * num_sms CTAs; when the unsplit work
+// already fills a wave, nothing is split. The pieces are of about equal size whatever the mix of
+// lengths. Partials go to a workspace; the last CTA of a row block to finish (an atomic ticket,
+// nothing spins) merges them.
+__device__ __forceinline__ int warp_sum(int v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ WorkItem decode_work_chunked(const TcParams& p, int idx, int grid) {
+  constexpr int KB = CAST_MAX_BATCH / 32;
+  const int lane = threadIdx.x & 31;
+  const int max_pos = p.page_size == 0 ? p.seq_capacity : p.seq_capacity * p.page_size;
+  int Nv[KB], Lv[KB], tl[KB], nr[KB];
+#pragma unroll
+  for (int k = 0; k < KB; ++k) {  // all loads first: one memory round trip
+    const int bb = k * 32 + lane;
+    Nv[k] = bb < p.B ? p.n_tree[bb] : 0;
+    Lv[k] = bb < p.B ? p.kv_len[bb] : 0;
+  }
+  int base = 0, T = 0, tmax = 0;
+#pragma unroll
+  for (int k = 0; k < KB; ++k) {
+    Nv[k] = clampi(Nv[k], 0, p.Nmax);
+    Lv[k] = Lv[k] < 0 ? 0 : Lv[k];
+    int total = Lv[k] + Nv[k];
+    total = total > max_pos ? max_pos : total;
+    nr[k] = (Nv[k] * p.G + kBM - 1) / kBM;
+    tl[k] = nr[k] > 0 ? (total + kBN - 1) / kBN : 0;
+    base += p.Hkv * nr[k];
+    T += p.Hkv * nr[k] * tl[k];
+    tmax = tl[k] > tmax ? tl[k] : tmax;
+  }
+  base = warp_sum(base);
+  T = warp_sum(T);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) tmax = max(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
+  const int slots = 2 * p.num_sms;
+  int W = (base + slots - 1) / slots;
+  W = W < 1 ? 1 : W;
+  int cap = W * slots;
+  cap = cap > grid ? grid : cap;
+  // smallest chunk (>= 4 tiles) whose item count fits: the count falls as the chunk grows, and a chunk
+  // of tmax tiles (no splits at all) always fits
+  auto items_at = [&](int chunk) {
+    int items = 0;
+#pragma unroll
+    for (int k = 0; k < KB; ++k) {
+      int n = (tl[k] + chunk - 1) / chunk;
+      n = n > p.nsplit_max ? p.nsplit_max : n;
+      items += p.Hkv * nr[k] * n;
+    }
+    return warp_sum(items);
+  };
+  int lo = (T + cap - 1) / cap, hi = tmax < 4 ? 4 : tmax;
+  lo = lo < 4 ? 4 : lo;
+  lo = lo > hi ? hi : lo;
+  if (base >= slots) lo = hi;  // the unsplit work fills a wave already: no splits
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (items_at(mid) <= cap) hi = mid; else lo = mid + 1;
+  }
+  const int chunk = lo;
+  int ns[KB], cnt[KB], off[KB];
+#pragma unroll
+  for (int k = 0; k < KB; ++k) {
+    int n = (tl[k] + chunk - 1) / chunk;
+    n = n > p.nsplit_max ? p.nsplit_max : n;
+    ns[k] = n < 1 ? 1 : n;
+    cnt[k] = p.Hkv * nr[k] * ns[k];
+    off[k] = 0;
+  }
+  // items are numbered longest piece first (the block scheduler hands CTAs out in index order, so
+  // the long pieces start first and the short ones fill the gaps): sequence j precedes sequence b
+  // when its pieces are longer, ties by index
+  int key[KB];
+#pragma unroll
+  for (int k = 0; k < KB; ++k) key[k] = tl[k] * 16 / ns[k];
+  if (p.B > 1) {
+#pragma unroll 8
+    for (int j = 0; j < p.B; ++j) {
+      const int src = j & 31;
+      int pj, cj;
+      if (j < 32) {
+        pj = __shfl_sync(0xffffffffu, key[0], src);
+        cj = __shfl_sync(0xffffffffu, cnt[0], src);
+      } else {
+        pj = __shfl_sync(0xffffffffu, key[KB - 1], src);
+        cj = __shfl_sync(0xffffffffu, cnt[KB - 1], src);
+      }
+#pragma unroll
+      for (int k = 0; k < KB; ++k) {
+        const int bm = k * 32 + lane;
+        if (pj > key[k] || (pj == key[k] && j < bm)) off[k] += cj;
+      }
+    }
+  }
+  WorkItem w;
+  w.valid = w.active = false;
+  w.b = w.kvh = w.rb = w.split = w.N = w.L = 0;
+  w.nsplit = 1;
+#pragma unroll
+  for (int k = 0; k < KB; ++k) {
+    const unsigned hit = __ballot_sync(0xffffffffu, idx >= off[k] && idx < off[k] + cnt[k]);
+    if (hit != 0u && !w.valid) {
+      const int bl = __ffs(hit) - 1;
+      const int local = idx - __shfl_sync(0xffffffffu, off[k], bl);
+      w.nsplit = __shfl_sync(0xffffffffu, ns[k], bl);
+      w.N = __shfl_sync(0xffffffffu, Nv[k], bl);
+      w.L = __shfl_sync(0xffffffffu, Lv[k], bl);
+      w.b = k * 32 + bl;
+      w.kvh = local % p.Hkv;
+      const int rest = local / p.Hkv;
+      w.split = rest % w.nsplit;
+      w.rb = rest / w.nsplit;
+      w.valid = w.active = true;
+    }
+  }
+  return w;
+}
+
+// Merge of the split partials of a row block, run by all 8 warps of the last CTA to finish it.
+// Warp w takes rows w, w+8, ...; a lane owns 4 output columns. ROWS rows x SPL splits = 16 loads are
+// in flight per lane: the merge is bound by L2 latency, not by bytes.
+template <int ROWS, int SPL>
+__device__ __forceinline__ void merge_rows_global(const TcParams& p, int b, int kvh, int row0, int rows_here, int nsplit) {
+  const int lane = threadIdx.x & 31, wv = threadIdx.x >> 5, G = p.G;
+  for (int rr = wv; rr < rows_here; rr += 8 * ROWS) {
+    float4 v[ROWS][SPL];
+    float wgt[ROWS], inv[ROWS];
+    size_t orow[ROWS];
+#pragma unroll
+    for (int u = 0; u < ROWS; ++u) {
+      const int r2 = rr + 8 * u;
+      const int grow = row0 + (r2 < rows_here ? r2 : rr), tt = grow / G, hh = kvh * G + grow % G;
+      const size_t pr = (((size_t)b * p.Hq + hh) * p.Ncap + tt) * p.nsplit_max;
+      orow[u] = (((size_t)b * p.Ncap + tt) * p.Hq + hh) * kHD;
+      float ms = -INFINITY, ls = 0.f;  // lane s holds split s's (max, sum)
+      if (lane < nsplit) {
+        ms = __ldcg(p.part_ml + (pr + lane) * 2);
+        ls = __ldcg(p.part_ml + (pr + lane) * 2 + 1);
+      }
+#pragma unroll
+      for (int s2 = 0; s2 < SPL; ++s2)
+        v[u][s2] = s2 < nsplit ? __ldcg(reinterpret_cast<const float4*>(p.part_o + (pr + s2) * kHD + lane * 4))
+                               : make_float4(0.f, 0.f, 0.f, 0.f);
+      float M = ms;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+      wgt[u] = ms > -INFINITY ? expf(ms - M) : 0.f;
+      float lsum = ls * wgt[u];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
+      inv[u] = lsum > 0.f ? 1.f / lsum : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < ROWS; ++u) {
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int s2 = 0; s2 < SPL; ++s2) {
+        const float w = __shfl_sync(0xffffffffu, wgt[u], s2);
+        acc.x += v[u][s2].x * w;
+        acc.y += v[u][s2].y * w;
+        acc.z += v[u][s2].z * w;
+        acc.w += v[u][s2].w * w;
+      }
+      if (rr + 8 * u < rows_here) {
+        const __nv_bfloat162 a = __floats2bfloat162_rn(acc.x * inv[u], acc.y * inv[u]),
+                             c2 = __floats2bfloat162_rn(acc.z * inv[u], acc.w * inv[u]);
+        uint2 pk;
+        pk.x = *reinterpret_cast<const uint32_t*>(&a);
+        pk.y = *reinterpret_cast<const uint32_t*>(&c2);
+        *reinterpret_cast<uint2*>(p.out + orow[u] + lane * 4) = pk;
+      }
+    }
+  }
+}
+
 __global__ void __launch_bounds__(kThreadsTC, 2)
 tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
   extern __shared__ __align__(1024) unsigned char smem[];  // no static shared memory: the base is 1 KB aligned
@@ -401,7 +588,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_k)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_v)) : "memory");
   }
-  const WorkItem wk = decode_work(p, (int)blockIdx.x / cs, crank);
+  const WorkItem wk = cs == 0 ? decode_work_chunked(p, (int)blockIdx.x, (int)gridDim.x) : decode_work(p, (int)blockIdx.x / cs, crank);
   TC_MARK(1);
   if (blockIdx.x < p.B && tid == 0 && p.n_tree[blockIdx.x] > p.Nmax) report(p.st, CAST_ERR_BAD_TREE, blockIdx.x);
   if (!wk.valid) return;  // the whole cluster leaves
@@ -447,6 +634,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
   uint64_t* bar_s = bars + 8;          // [2]
   uint64_t* bar_p = bars + 10;
   uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(bars + 11);
+  int* last_s = reinterpret_cast<int*>(bars + 12);
 
   // ---- producer helper (warp 4; all 32 lanes call it): which = 0: K tile j, which = 1: V tile j
   auto issue_tile = [&](int j, int which) -> bool {
@@ -804,6 +992,33 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
       pk.y = *reinterpret_cast<const uint32_t*>(&c2);
       *reinterpret_cast<uint2*>(p.out + (((size_t)b * p.Ncap + tt) * p.Hq + hh) * kHD + lane * 4) = pk;
     }
+  } else if (cs == 0) {
+    // global-merge mode: partials to the workspace; the last split of this row block to finish merges
+    for (int rr = warp; rr < rows_here; rr += kThreadsTC / 32) {
+      const int grow = row0 + rr, tt = grow / G, hh = kvh * G + grow % G;
+      const size_t pr = (((size_t)b * p.Hq + hh) * p.Ncap + tt) * p.nsplit_max + split;
+      __stcg(reinterpret_cast<float4*>(p.part_o + pr * kHD + lane * 4),
+             *reinterpret_cast<const float4*>(stage_o + rr * kStageStride + lane * 4));
+      if (lane == 0) {
+        __stcg(p.part_ml + pr * 2, stage_ml[rr * 2]);
+        __stcg(p.part_ml + pr * 2 + 1, stage_ml[rr * 2 + 1]);
+      }
+    }
+    __threadfence();  // the partials must be visible before this CTA takes its ticket
+    __syncthreads();
+    if (tid == 0) {
+      int32_t* cnt = p.ticket + ((size_t)b * p.Hkv + kvh) * p.nrb + rb;
+      const int t = atomicAdd(cnt, 1);
+      *last_s = (t == nsplit - 1);
+      if (t == nsplit - 1) *cnt = 0;  // ready for the next launch
+      __threadfence();
+    }
+    __syncthreads();
+    if (*last_s) {
+      if (nsplit <= 2) merge_rows_global<8, 2>(p, b, kvh, row0, rows_here, nsplit);
+      else if (nsplit <= 4) merge_rows_global<4, 4>(p, b, kvh, row0, rows_here, nsplit);
+      else merge_rows_global<2, kMaxSplit>(p, b, kvh, row0, rows_here, nsplit);
+    }
   } else {
     const uint32_t so_s = smem_u32(stage_o), sml_s = smem_u32(stage_ml);
     const int rank0 = crank - split;  // first CTA of this row block's split group
@@ -990,20 +1205,61 @@ bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const v
   if (const char* e = getenv("CAST_TC_SPLITS")) splits = atoi(e);
   if (const char* e = getenv("CAST_TC_RPC")) rpc = atoi(e);
 #endif
-  const int cs = splits * rpc;
-  const int groups = (nrb + rpc - 1) / rpc;
-  const long long clusters = (long long)B * Hkv * groups;
-  const long long grid = clusters * cs;
-  if (grid > 0x7fffffffll) return false;
+  // Clusters pay when CTAs are short (the merge through distributed shared memory is cheap and the
+  // splits are what fills the machine). With long CTAs, or so many sequences that nothing needs
+  // splitting on average, an even load matters more: no clusters, pieces sized on the device.
+  // (with B * Hkv items or more than the machine has slots, nothing is ever split: plain launch, cs = 1)
+  bool cluster_mode = (splits > 1 && max_tiles / splits <= 64) || (long long)B * Hkv >= slots;
+  if ((long long)B * Hkv >= slots) splits = rpc = 1;
+#ifdef CAST_PHASE_CLOCKS
+  if (const char* e = getenv("CAST_TC_FORCE_CLUSTER")) cluster_mode = atoi(e) != 0;
+#endif
   TcParams p;
   p.q = (const __nv_bfloat16*)q; p.out = (__nv_bfloat16*)out;
   p.B = B; p.Ncap = Ncap; p.Nmax = Nmax; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.page_size = page_size;
   p.seq_capacity = seq_capacity; p.num_pages = num_pages; p.words = c->words;
-  p.cs = cs; p.rpc = rpc;
   p.page_table = page_table; p.kv_len = kv_len; p.n_tree = n_tree; p.anc = anc;
   p.scale_log2 = scale * 1.4426950408889634f;
   p.st = c->state;
+  p.num_sms = c->num_sms; p.nrb = nrb;
+  p.part_o = nullptr; p.part_ml = nullptr; p.ticket = nullptr;
   *status = CAST_OK;
+  long long grid;
+  int cs;
+  if (cluster_mode) {
+    cs = splits * rpc;
+    const int groups = (nrb + rpc - 1) / rpc;
+    grid = (long long)B * Hkv * groups * cs;
+    p.cs = cs; p.rpc = rpc; p.nsplit_max = 1;
+  } else {
+    cs = 1;
+    int nsplit_max = kMaxSplit < max_tiles ? kMaxSplit : max_tiles;
+    if (nsplit_max < 1) nsplit_max = 1;
+    const long long waves = ((long long)B * Hkv * nrb + slots - 1) / slots;
+    grid = (long long)slots * (waves < 1 ? 1 : waves);
+    p.cs = 0; p.rpc = 1; p.nsplit_max = nsplit_max;
+    if (nsplit_max > 1) {
+      // workspace: a fixed ticket region (B * Hkv * nrb <= 64 * Hq entries), then the partials
+      constexpr size_t kTicketBytes = (size_t)CAST_MAX_BATCH * 256 * sizeof(int32_t);
+      const size_t rows = (size_t)B * Hq * Ncap * nsplit_max;
+      if ((size_t)B * Hkv * nrb * sizeof(int32_t) > kTicketBytes) return false;
+      const size_t need = kTicketBytes + rows * (kHD + 2) * sizeof(float);
+      if (need > c->attn_tc_ws_bytes) {  // grows the workspace (synchronises; not legal during graph capture)
+        if (cudaDeviceSynchronize() != cudaSuccess) { *status = CAST_ERR_CUDA; return true; }
+        if (c->attn_tc_ws) cudaFree(c->attn_tc_ws);
+        c->attn_tc_ws = nullptr;
+        c->attn_tc_ws_bytes = 0;
+        if (cudaMalloc(&c->attn_tc_ws, need) != cudaSuccess) { *status = CAST_ERR_CUDA; return true; }
+        // tickets start at zero; every merge leaves its ticket at zero again
+        if (cudaMemset(c->attn_tc_ws, 0, kTicketBytes) != cudaSuccess) { *status = CAST_ERR_CUDA; return true; }
+        c->attn_tc_ws_bytes = need;
+      }
+      p.ticket = reinterpret_cast<int32_t*>(c->attn_tc_ws);
+      p.part_o = reinterpret_cast<float*>(reinterpret_cast<char*>(c->attn_tc_ws) + kTicketBytes);
+      p.part_ml = p.part_o + rows * kHD;
+    }
+  }
+  if (grid > 0x7fffffffll) return false;
   static bool attr_done = false;
   if (!attr_done) {
     if (cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) !=
