@@ -33,8 +33,8 @@ cudaError_t dev_alloc(T** p, size_t n) {
 
 void free_all(cast_ctx* c) {
   cudaFree(c->pool_score); cudaFree(c->pool_token); cudaFree(c->pool_parent); cudaFree(c->pool_depth);
-  cudaFree(c->pool_kept); cudaFree(c->retained); cudaFree(c->lsort); cudaFree(c->lscore); cudaFree(c->state); cudaFree(c->part_keys);
-  cudaFree(c->part_max); cudaFree(c->part_sum); cudaFree(c->row_ticket); cudaFree(c->layer_ticket);
+  cudaFree(c->pool_kept); cudaFree(c->retained); cudaFree(c->lsort); cudaFree(c->lscore); cudaFree(c->state);
+  cudaFree(c->layer_ticket);
   cudaFree(c->fifo_vals); cudaFree(c->fifo_cnt); cudaFree(c->sel_score); cudaFree(c->sel_value);
   cudaFree(c->sel_idx); cudaFree(c->acc_part); cudaFree(c->compact_ticket); cudaFree(c->attn_ws); cudaFree(c->attn_tc_ws);
   if (c->tables) {
@@ -101,10 +101,6 @@ extern "C" cast_status cast_create(const cast_config* cfg, cast_ctx** out) {
   if (e == cudaSuccess) e = dev_alloc(&c->lsort, BP);
   if (e == cudaSuccess) e = dev_alloc(&c->lscore, BP);
   if (e == cudaSuccess) e = dev_alloc(&c->state, 1);
-  if (e == cudaSuccess) e = dev_alloc(&c->part_keys, rows * kSweepMaxChunks * CAST_MAX_TOP_K);
-  if (e == cudaSuccess) e = dev_alloc(&c->part_max, rows * kSweepMaxChunks);
-  if (e == cudaSuccess) e = dev_alloc(&c->part_sum, rows * kSweepMaxChunks);
-  if (e == cudaSuccess) e = dev_alloc(&c->row_ticket, rows);
   if (e == cudaSuccess) e = dev_alloc(&c->layer_ticket, 1);
   if (e == cudaSuccess) e = dev_alloc(&c->fifo_vals, (size_t)nbuf * cfg->fifo_len);
   if (e == cudaSuccess) e = dev_alloc(&c->fifo_cnt, nbuf);

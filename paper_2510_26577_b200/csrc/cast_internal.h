@@ -44,10 +44,10 @@ struct HostTable {
 };
 
 // Limits of the vocabulary sweep.
-constexpr int kSweepThreads = 256;
-constexpr int kSweepEpt = 16;                             // logits per thread per pass
+constexpr int kSweepThreads = 512;
+constexpr int kSweepEpt = 32;                             // logits per thread per pass
 constexpr int kSweepSub = kSweepThreads * kSweepEpt;      // logits per CTA per pass
-constexpr int kSweepMaxChunks = 64;                       // CTAs per logits row
+constexpr int kSweepMaxChunks = 8;                        // CTAs per logits row: one thread-block cluster
 constexpr int kCandCap = 4096;                            // candidate keys per CTA (floods take the slow exact path)
 constexpr int kMaxFifo = 64;
 constexpr int kAcceptMaxChunks = 32;
@@ -75,11 +75,6 @@ struct cast_ctx {
 
   cast::DevState* state;
 
-  // vocabulary-sweep partials
-  unsigned long long* part_keys;  // [max_batch*W][kSweepMaxChunks][CAST_MAX_TOP_K]
-  float* part_max;                // [max_batch*W][kSweepMaxChunks]
-  double* part_sum;               // [max_batch*W][kSweepMaxChunks]
-  int32_t* row_ticket;            // [max_batch*W]
   int32_t* layer_ticket;          // [1]
 
   // depth-pruning buffers

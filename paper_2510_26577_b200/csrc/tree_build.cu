@@ -25,7 +25,8 @@ using namespace cast;
 #ifdef CAST_PHASE_CLOCKS
 __device__ long long g_phase_clock[64];
 #define CAST_STAMP(k) do { if (threadIdx.x == 0) stamp_s[k] = clock64(); } while (0)
-#define CAST_STAMP_DECL __shared__ long long stamp_s[32];
+#define CAST_STAMP_DECL
+__shared__ long long stamp_s[32];
 #define CAST_STAMP_FLUSH(off, n) do { if (threadIdx.x == 0) for (int _i = 0; _i < (n); ++_i) g_phase_clock[(off) + _i] = stamp_s[_i]; } while (0)
 extern "C" __attribute__((visibility("default"))) int cast_debug_read_clocks(long long* out) {
   return (int)cudaMemcpyFromSymbol(out, g_phase_clock, sizeof(long long) * 64);
@@ -42,8 +43,7 @@ namespace {
 __global__ void step_begin_kernel(DevState* st, int B, int P, int W, const int32_t* root_token,
                                   const int32_t* kv_len, double* pool_score, int32_t* pool_token,
                                   int32_t* pool_parent, int32_t* pool_depth, uint8_t* pool_kept,
-                                  int32_t* retained, int32_t* lsort, double* lscore, int32_t* row_ticket,
-                                  int32_t* layer_ticket, int n_rows) {
+                                  int32_t* retained, int32_t* lsort, double* lscore, int32_t* layer_ticket) {
   __shared__ int s_max;
   const int tid = threadIdx.x;
   if (tid == 0) s_max = 0;
@@ -60,7 +60,6 @@ __global__ void step_begin_kernel(DevState* st, int B, int P, int W, const int32
     retained[b * W] = 0;
     atomicMax(&s_max, kv_len[b]);
   }
-  for (int i = tid; i < n_rows; i += blockDim.x) row_ticket[i] = 0;
   __syncthreads();
   if (tid == 0) {
     *layer_ticket = 0;
@@ -98,10 +97,6 @@ struct ExpandParams {
   int32_t* lsort;
   double* lscore;
   DevState* st;
-  unsigned long long* part_keys;
-  float* part_max;
-  double* part_sum;
-  int32_t* row_ticket;
   int32_t* layer_ticket;
   double* fifo_vals;
   int32_t* fifo_cnt;
@@ -161,6 +156,32 @@ __device__ __forceinline__ double fast_log2(double S) {
   return (double)e + (double)log2f((float)m);
 }
 
+// ---- thread-block cluster primitives (a logits row is swept by one cluster)
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void st_cluster_u64(uint32_t addr, unsigned long long v) {
+  asm volatile("st.shared::cluster.u64 [%0], %1;" ::"r"(addr), "l"(v) : "memory");
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ void st_cluster_f64(uint32_t addr, double v) {
+  asm volatile("st.shared::cluster.f64 [%0], %1;" ::"r"(addr), "d"(v) : "memory");
+}
+__device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+
+// State fields the layer tail needs; every CTA reads them at its start (same cache lines as the row
+// count it needs anyway), so the tail itself starts without a round trip to memory.
+struct TailState {
+  int ctx_sum, n0, kept_total;
+  double u_last;
+};
+
 // The ticket of the "last CTA" pattern: the caller has passed a CTA barrier after its global
 // writes; one thread fences (cumulative over the CTA's writes) and takes the ticket.
 __device__ __forceinline__ bool take_ticket(int32_t* counter, int expected, int* flag_s) {
@@ -178,24 +199,31 @@ __device__ __forceinline__ bool take_ticket(int32_t* counter, int expected, int*
 
 // Exact top-K (descending) of n distinct keys in shared memory, written to out[0..K); missing
 // entries (n < K) become 0. All threads of the CTA call it; `keys` is clobbered when n > 1024.
-__device__ __noinline__ void block_top_k(unsigned long long* keys, int n, int K, unsigned long long* out) {
+__device__ __forceinline__ void block_top_k(unsigned long long* keys, int n, int K, unsigned long long* out) {
   const int tid = threadIdx.x, nt = blockDim.x;
   if (tid < K) out[tid] = 0ull;
   __syncthreads();
-  if (n <= 1024) {  // rank by counting: keys are distinct, so ranks are too
+  if (n <= 1024) {
+    // rank by counting (keys are distinct, so ranks are too): G lanes share a key, each counting over
+    // every G-th key; shared-memory latency, not the number of compares, is what this costs
+    int G = 1;
+    while (G < 32 && n * (G * 2) <= nt) G *= 2;
+    const int per = nt / G;
 #pragma unroll 1
-    for (int i = tid; i < n; i += nt) {
-      const unsigned long long k = keys[i];
-      int r0 = 0, r1 = 0, r2 = 0, r3 = 0, j = 0;
-      for (; j + 4 <= n; j += 4) {
+    for (int i0 = 0; i0 < n; i0 += per) {
+      const int i = i0 + tid / G, sub = tid % G;
+      const unsigned long long k = i < n ? keys[i] : ~0ull;
+      int r0 = 0, r1 = 0, r2 = 0, r3 = 0, j = sub;
+      for (; j + 3 * G < n; j += 4 * G) {
         r0 += (keys[j] > k);
-        r1 += (keys[j + 1] > k);
-        r2 += (keys[j + 2] > k);
-        r3 += (keys[j + 3] > k);
+        r1 += (keys[j + G] > k);
+        r2 += (keys[j + 2 * G] > k);
+        r3 += (keys[j + 3 * G] > k);
       }
-      for (; j < n; ++j) r0 += (keys[j] > k);
-      const int rank = r0 + r1 + r2 + r3;
-      if (rank < K) out[rank] = k;
+      for (; j < n; j += G) r0 += (keys[j] > k);
+      int rank = r0 + r1 + r2 + r3;
+      for (int o = G >> 1; o > 0; o >>= 1) rank += __shfl_xor_sync(0xffffffffu, rank, o);
+      if (sub == 0 && i < n && rank < K) out[rank] = k;
     }
   } else {  // bitonic sort, descending, on the next power of two
     int n2 = 2048;
@@ -220,8 +248,8 @@ __device__ __noinline__ void block_top_k(unsigned long long* keys, int n, int K,
 }
 
 // Layer tail (Eq. 1, Eq. 2, Algorithm 1, depth pruning), run by the last CTA of the layer.
-__device__ __noinline__ void layer_tail(const ExpandParams& p, int B, int n_prev, int base, unsigned char* scratch,
-                           int* sorted /* [CAST_MAX_BATCH * CAST_MAX_WIDTH] */) {
+__device__ __forceinline__ void layer_tail(const ExpandParams& p, const TailState& ts, int B, int n_prev, int base,
+                                        unsigned char* scratch, int* sorted /* [CAST_MAX_BATCH * CAST_MAX_WIDTH] */) {
   __shared__ double vbar[CAST_MAX_WIDTH], u[CAST_MAX_WIDTH], c[CAST_MAX_WIDTH];
   __shared__ int mark[CAST_MAX_WIDTH];
   __shared__ int s_ni, s_next;
@@ -235,49 +263,82 @@ __device__ __noinline__ void layer_tail(const ExpandParams& p, int B, int n_prev
   // Eq. 2 needs one table row: fetch it now, its latency hides behind the ranking
   double c_mine = 0.0;
   if (need_cost && tid < n) {
-    const int ctx = st->ctx_sum + (p.ctx_base_mode ? st->n0 : 0);
+    const int ctx = ts.ctx_sum + (p.ctx_base_mode ? ts.n0 : 0);
     const int g = select_grid(ctx, p.tab.L, p.tab.M);
     c_mine = p.tab.fD[(size_t)(g - 1) * p.tab.Ntab + tid] / p.tab.fT[(size_t)(g - 1) * p.tab.Ntab];
   }
-  const double u_last = st->u_last;
+  const double u_last = ts.u_last;
 
-  double* sc = reinterpret_cast<double*>(scratch);              // 2048 scores
-  int* tk = reinterpret_cast<int*>(scratch + 16384);            // 2048 tokens
-  double* vs = reinterpret_cast<double*>(scratch + 24576);      // [B][CAST_MAX_WIDTH] sorted values
-  const int group = 2048 / Ni;                                  // sequences ranked per pass
+  double* sc = reinterpret_cast<double*>(scratch);              // 1024 scores
+  int* tk = reinterpret_cast<int*>(scratch + 8192);             // 1024 tokens
+  unsigned short* r1s = reinterpret_cast<unsigned short*>(scratch + 12288);  // 1024: row of the candidate
+  unsigned short* cis = reinterpret_cast<unsigned short*>(scratch + 14336);  // 1024: index within the sequence
+  double* vs = reinterpret_cast<double*>(scratch + 16384);      // [B][CAST_MAX_WIDTH] sorted values
+  int* stok = reinterpret_cast<int*>(scratch + 24576);          // [B][CAST_MAX_WIDTH] tokens of the sorted nodes
+  const int group = 1024 / Ni;                                  // sequences ranked per pass
 #pragma unroll 1
   for (int b0 = 0; b0 < B; b0 += group) {
     const int nb = (B - b0) < group ? (B - b0) : group;
-    for (int i = tid; i < nb * Ni; i += nt) {
-      const size_t o = (size_t)(b0 + i / Ni) * P + base + (i % Ni);
+    const int tot = nb * Ni;
+    for (int i = tid; i < tot; i += nt) {
+      const int bl = i / Ni, ci = i - bl * Ni;  // (the divisions hide behind the loads)
+      const size_t o = (size_t)(b0 + bl) * P + base + ci;
       sc[i] = __ldcg(p.pool_score + o);
       tk[i] = __ldcg(p.pool_token + o);
+      r1s[i] = (unsigned short)(ci / K);
+      cis[i] = (unsigned short)ci;
     }
     __syncthreads();
-    // rank by counting under the order (value desc, token asc, creation order); branch-free
-    for (int i = tid; i < nb * Ni; i += nt) {
-      const int bl = i / Ni, ci = i % Ni;
-      const double s = sc[i];
-      const int t = tk[i];
-      const double* ss = sc + bl * Ni;
-      const int* tt = tk + bl * Ni;
-      int rank = 0;
-#pragma unroll 4
-      for (int j = 0; j < Ni; ++j) {
-        const double sj = ss[j];
-        const int tj = tt[j];
-        rank += (int)(sj > s) | ((int)(sj == s) & ((int)(tj < t) | ((int)(tj == t) & (int)(j < ci))));
+    CAST_STAMP(14);
+    // Rank under the order (value desc, token asc, creation order). Every logits row contributed its K
+    // children already in that order, so the rank of a candidate is the number of children that come
+    // first, row by row: a lower-bound search per row (in its own row it finds its own position). Four
+    // neighbouring lanes share a candidate; a lane runs the searches of up to four rows in lockstep,
+    // branch-free, so their shared-memory loads overlap.
+    const int sub = tid & 3;
+#pragma unroll 1
+    for (int i0 = 0; i0 < tot; i0 += nt / 4) {
+      const int i = i0 + (tid >> 2);
+      const bool act = i < tot;
+      const int ii = act ? i : 0;
+      const double s = sc[ii];
+      const int t = tk[ii];
+      const int r1 = r1s[ii], ci = cis[ii];
+      const int sbase = ii - ci;  // first candidate of the same sequence
+      int pos[4] = {0, 0, 0, 0};
+#pragma unroll
+      for (int half = 16; half >= 1; half >>= 1) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int r2 = sub + 4 * q;
+          const int idx = pos[q] + half - 1;
+          const bool valid = r2 < n_prev && idx < K;
+          const int at = valid ? sbase + r2 * K + idx : ii;
+          const double sj = sc[at];
+          const int tj = tk[at];
+          const bool first = valid && ((sj > s) || (sj == s && (tj < t || (tj == t && r2 < r1))));
+          pos[q] += first ? half : 0;
+        }
       }
-      const size_t o = (size_t)(b0 + bl) * P + base + rank;
-      p.lsort[o] = base + ci;  // the layer's sorted list, for the rerank
-      p.lscore[o] = s;
-      if (rank < n) {
-        sorted[(b0 + bl) * CAST_MAX_WIDTH + rank] = base + ci;
-        vs[(b0 + bl) * CAST_MAX_WIDTH + rank] = fast_exp_neg(s);
+      int cnt = pos[0] + pos[1] + pos[2] + pos[3];
+      cnt += __shfl_xor_sync(0xffffffffu, cnt, 2);
+      cnt += __shfl_xor_sync(0xffffffffu, cnt, 1);
+      if (act && sub == 0) {
+        const int bl = sbase / Ni, rank = cnt;
+        const size_t o = (size_t)(b0 + bl) * P + base + rank;
+        p.lsort[o] = base + ci;  // the layer's sorted list, for the rerank
+        p.lscore[o] = s;
+        if (rank < n) {
+          sorted[(b0 + bl) * CAST_MAX_WIDTH + rank] = base + ci;
+          stok[(b0 + bl) * CAST_MAX_WIDTH + rank] = t;
+          vs[(b0 + bl) * CAST_MAX_WIDTH + rank] = fast_exp_neg(s);
+        }
       }
     }
+    CAST_STAMP(21);
     __syncthreads();
   }
+  CAST_STAMP(15);
   // Eq. 1: batch mean of the rank-wise values, then prefix sums
   if (tid < n) {
     double a = 0.0;
@@ -297,6 +358,7 @@ __device__ __noinline__ void layer_tail(const ExpandParams& p, int B, int n_prev
     if (tid < n) u[tid] = a;
   }
   __syncthreads();
+  CAST_STAMP(16);
   // Algorithm 1: mark[j] survives iff no earlier i has (u_j - u_i) < C1 (c_j - c_i)
   if (tid < n) {
     int ok = 1;
@@ -307,6 +369,7 @@ __device__ __noinline__ void layer_tail(const ExpandParams& p, int B, int n_prev
     mark[tid] = ok;
   }
   __syncthreads();
+  CAST_STAMP(17);
   if (tid == 0) {
     int n_i = 1;
 #pragma unroll 1
@@ -341,14 +404,15 @@ __device__ __noinline__ void layer_tail(const ExpandParams& p, int B, int n_prev
     st->n_hist[p.layer] = n_i;
     st->layer_base[p.layer] = base;
     st->layer_n[p.layer] = Ni;
-    st->ctx_sum += n_i;
-    st->kept_total += n_i;
+    st->ctx_sum = ts.ctx_sum + n_i;
+    st->kept_total = ts.kept_total + n_i;
     st->u_last = u[n_i - 1];
     st->pool_size = base + Ni;
     st->layers_done = p.layer;
     *p.next_count = s_next;
   }
   __syncthreads();
+  CAST_STAMP(18);
   const int n_i = s_ni;
 #pragma unroll 1
   for (int i = tid; i < B * W; i += nt) {
@@ -356,7 +420,7 @@ __device__ __noinline__ void layer_tail(const ExpandParams& p, int B, int n_prev
     int tok = -1, prow = -1;
     if (s < n_i) {
       const int idx = sorted[b * CAST_MAX_WIDTH + s];
-      tok = __ldcg(p.pool_token + (size_t)b * P + idx);
+      tok = stok[b * CAST_MAX_WIDTH + s];
       prow = (idx - base) / K;
       p.retained[b * W + s] = idx;
       p.pool_kept[(size_t)b * P + idx] = 1;
@@ -376,6 +440,11 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
   __shared__ double red_d[kSweepThreads / 32];
   __shared__ int sorted[CAST_MAX_BATCH * CAST_MAX_WIDTH];
   __shared__ int cand_cnt, s_flag;
+  // filled in the first CTA of the row's cluster by all CTAs of the cluster: chunk c's top-K keys
+  // (descending), maximum (log2 units) and sum of 2^(. - maximum)
+  __shared__ unsigned long long row_keys[kSweepMaxChunks * CAST_MAX_TOP_K];
+  __shared__ float row_max[kSweepMaxChunks];
+  __shared__ double row_sum[kSweepMaxChunks];
   CAST_STAMP_DECL
   CAST_STAMP(0);
   unsigned long long* cand = reinterpret_cast<unsigned long long*>(scratch);
@@ -407,7 +476,14 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
     }
   };
   load_pass(begin);
+  // what the layer tail needs of the state is read now, together with the row count: one round trip
   const int n_prev = st->rows[p.layer];
+  TailState ts;
+  ts.ctx_sum = st->ctx_sum;
+  ts.n0 = st->n0;
+  ts.kept_total = st->kept_total;
+  ts.u_last = st->u_last;
+  const int base = st->pool_size;
   if (n_prev == 0) {
     if (chunk == 0 && r == 0 && b == 0 && tid == 0) *p.next_count = 0;
     return;
@@ -428,6 +504,7 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
     if (sub != begin) load_pass(sub);
     const int have0 = cand_cnt;
     float tmax = xv[0];
+    if (sub == begin) CAST_STAMP(10);
 #pragma unroll
     for (int i = 1; i < kSweepEpt; ++i) tmax = fmaxf(tmax, xv[i]);
     const float t2 = tmax * kLog2eHi;
@@ -444,6 +521,7 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
       }
       s_run += a0 + a1;
     }
+    if (sub == begin) CAST_STAMP(11);
     // filter threshold: the exact K-th key once K logits have been seen, else the largest of the
     // warps' K-th largest thread maxima (at least K logits of this pass are >= it)
     float thr_val;
@@ -466,43 +544,28 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
     } else {
       thr_val = key_value(thr_key);
     }
-    {
-      unsigned pm = 0u;  // which of this thread's 16 logits pass the value threshold
+    if (sub == begin) CAST_STAMP(12);
+    // Few logits pass. One vote per logit slot keeps the common path at a compare and a vote; a slot
+    // with a passer (rare) takes the exact test on the full key and one shared-memory atomic per warp.
 #pragma unroll
-      for (int i = 0; i < kSweepEpt; ++i) pm |= (xv[i] >= thr_val ? 1u : 0u) << i;
-      if (pm != 0u) {  // rare: exact test on the full key
-#pragma unroll
-        for (int i = 0; i < kSweepEpt; ++i) {
-          const int id = sub + ((i / VEC) * kSweepThreads + tid) * VEC + (i % VEC);
-          const bool ok = ((pm >> i) & 1u) && id < end && make_key(xv[i], id) > thr_key;
-          pm = ok ? pm : (pm & ~(1u << i));
-        }
-      }
-      const int cntp = __popc(pm);
-      // one shared-memory atomic per warp: exclusive prefix of the lanes' counts
-      int incl = cntp;
-#pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        const int t = __shfl_up_sync(0xffffffffu, incl, d);
-        if (lane >= d) incl += t;
-      }
-      const int wtotal = __shfl_sync(0xffffffffu, incl, 31);
-      if (wtotal > 0) {
-        int basepos = 0;
-        if (lane == 31) basepos = atomicAdd(&cand_cnt, wtotal);
-        basepos = __shfl_sync(0xffffffffu, basepos, 31);
-        int pos = basepos + incl - cntp;
-        if (pm != 0u) {
-#pragma unroll
-          for (int i = 0; i < kSweepEpt; ++i)
-            if ((pm >> i) & 1u) {
-              if (pos < kCandCap) cand[pos] = make_key(xv[i], sub + ((i / VEC) * kSweepThreads + tid) * VEC + (i % VEC));
-              ++pos;
-            }
+    for (int i = 0; i < kSweepEpt; ++i) {
+      const unsigned m0 = __ballot_sync(0xffffffffu, xv[i] >= thr_val);
+      if (m0 != 0u) {
+        const int id = sub + ((i / VEC) * kSweepThreads + tid) * VEC + (i % VEC);
+        const unsigned long long key = make_key(xv[i], id);
+        const bool ok = xv[i] >= thr_val && id < end && key > thr_key;
+        const unsigned m = __ballot_sync(0xffffffffu, ok);
+        if (m != 0u) {
+          int basepos = 0;
+          if (lane == 0) basepos = atomicAdd(&cand_cnt, __popc(m));
+          basepos = __shfl_sync(0xffffffffu, basepos, 0);
+          const int pos = basepos + __popc(m & ((1u << lane) - 1u));
+          if (ok && pos < kCandCap) cand[pos] = key;
         }
       }
     }
     __syncthreads();
+    if (sub == begin) CAST_STAMP(13);
     int n = cand_cnt;
     if (n > kCandCap) {
       // flood (a mass of ties at the threshold): K rounds of "largest key below the last one taken"
@@ -550,11 +613,11 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
   }
   CAST_STAMP(2);
 
-  // chunk partials: top-K keys in descending order, maximum, sum of 2^(. - maximum) in fp64
+  // chunk result: top-K keys in descending order, maximum, sum of 2^(. - maximum) in fp64; it goes
+  // straight into the shared memory of the cluster's first CTA, which merges the row
   {
     const int have = cand_cnt;
     if (thr_key == 0ull) block_top_k(cand, have, K, topk);  // fewer than K so far: not sorted yet
-    if (tid < K) p.part_keys[((size_t)row * kSweepMaxChunks + chunk) * CAST_MAX_TOP_K + tid] = topk[tid];
     float M = M2;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
@@ -568,84 +631,89 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
     for (int o = 16; o > 0; o >>= 1) sd += __shfl_xor_sync(0xffffffffu, sd, o);
     if (lane == 0) red_d[warp] = sd;
     __syncthreads();
-    if (tid == 0) {
-      double S = 0.0;
-      for (int w = 0; w < kSweepThreads / 32; ++w) S += red_d[w];
-      p.part_max[(size_t)row * kSweepMaxChunks + chunk] = M;
-      p.part_sum[(size_t)row * kSweepMaxChunks + chunk] = S;
+    if (p.nchunks == 1) {
+      if (tid < K) row_keys[tid] = topk[tid];
+      if (tid == 0) {
+        double S = 0.0;
+        for (int w = 0; w < kSweepThreads / 32; ++w) S += red_d[w];
+        row_max[0] = M;
+        row_sum[0] = S;
+      }
+    } else {
+      if (tid < K) st_cluster_u64(map_to_rank(smem_addr(&row_keys[chunk * CAST_MAX_TOP_K + tid]), 0u), topk[tid]);
+      if (tid == 0) {
+        double S = 0.0;
+        for (int w = 0; w < kSweepThreads / 32; ++w) S += red_d[w];
+        st_cluster_f32(map_to_rank(smem_addr(&row_max[chunk]), 0u), M);
+        st_cluster_f64(map_to_rank(smem_addr(&row_sum[chunk]), 0u), S);
+      }
     }
   }
   CAST_STAMP(3);
 
-  // ---- row merge by the last CTA of this logits row
-  __syncthreads();
-  if (p.nchunks > 1 && !take_ticket(&p.row_ticket[row], p.nchunks, &s_flag)) return;
+  // ---- row merge by the first CTA of the row's cluster
+  if (p.nchunks > 1) {
+    cluster_arrive_release();
+    if (chunk != 0) return;  // the results are on their way; the first CTA waits for them
+    cluster_wait_acquire();
+  } else {
+    __syncthreads();
+  }
   CAST_STAMP(4);
-  const int base = st->pool_size;
+  // the row's top K out of the chunks' lists (each in descending order): the rank of a key is its
+  // position in its own list plus, for every other list, the number of larger keys there (a binary
+  // search each; in its own list it finds its own position). Four neighbouring lanes share a key slot.
+  if (tid < K) topk[tid] = 0ull;
+  __syncthreads();
+  CAST_STAMP(22);
+  {
+    static_assert(kSweepThreads == 4 * kSweepMaxChunks * CAST_MAX_TOP_K, "one pass: four lanes per key slot");
+    const int slot = tid >> 2, sub = tid & 3;
+    const int c1 = slot >> 4, t = slot & 15;  // slot = list * CAST_MAX_TOP_K + position
+    const bool act = c1 < p.nchunks && t < K;
+    const unsigned long long key = act ? row_keys[slot] : 0ull;
+    int pos[2] = {0, 0};
+#pragma unroll
+    for (int half = 16; half >= 1; half >>= 1) {
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        const int c2 = sub + 4 * q;
+        const int idx = pos[q] + half - 1;
+        const bool valid = act && c2 < p.nchunks && idx < K;
+        const unsigned long long other = row_keys[valid ? c2 * CAST_MAX_TOP_K + idx : 0];
+        pos[q] += (valid && other > key) ? half : 0;
+      }
+    }
+    int cnt = pos[0] + pos[1];
+    cnt += __shfl_xor_sync(0xffffffffu, cnt, 2);
+    cnt += __shfl_xor_sync(0xffffffffu, cnt, 1);
+    if (act && sub == 0 && cnt < K) topk[cnt] = key;
+  }
+  CAST_STAMP(23);
+  __syncthreads();
+  CAST_STAMP(24);
   if (warp == 0) {
-    // one warp merges the row: no CTA barriers on this path
-    const unsigned long long* rk = p.part_keys + (size_t)row * kSweepMaxChunks * CAST_MAX_TOP_K;
-    // (a) every lane requests its share of the chunk lists and of the (max, sum) partials at once
-    unsigned long long k0 = lane < p.nchunks ? __ldcg(rk + (size_t)lane * CAST_MAX_TOP_K) : 0ull;
-    unsigned long long k1 = lane + 32 < p.nchunks ? __ldcg(rk + (size_t)(lane + 32) * CAST_MAX_TOP_K) : 0ull;
     float M0 = -INFINITY, M1 = -INFINITY;
     double S0 = 0.0, S1 = 0.0;
     if (lane < p.nchunks) {
-      M0 = __ldcg(p.part_max + (size_t)row * kSweepMaxChunks + lane);
-      S0 = __ldcg(p.part_sum + (size_t)row * kSweepMaxChunks + lane);
+      M0 = row_max[lane];
+      S0 = row_sum[lane];
     }
-    if (lane + 32 < p.nchunks) {
-      M1 = __ldcg(p.part_max + (size_t)row * kSweepMaxChunks + lane + 32);
-      S1 = __ldcg(p.part_sum + (size_t)row * kSweepMaxChunks + lane + 32);
-    }
-    constexpr int kPerLane = kSweepMaxChunks * CAST_MAX_TOP_K / 32;  // 32 keys per lane at most
-    const int nk = p.nchunks * K;
-    // (b) threshold: the K-th largest of the chunk maxima (every chunk list is in descending order)
-    int r0 = 0, r1 = 0;
-#pragma unroll 1
-    for (int j = 0; j < p.nchunks; ++j) {
-      const unsigned long long kj = __shfl_sync(0xffffffffu, j < 32 ? k0 : k1, j & 31);
-      r0 += (kj > k0);
-      r1 += (kj > k1);
-    }
-    unsigned long long thr = (r0 == K - 1 && k0 != 0ull) ? k0 : ((r1 == K - 1 && k1 != 0ull) ? k1 : 0ull);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const unsigned long long other = __shfl_xor_sync(0xffffffffu, thr, o);
-      thr = other > thr ? other : thr;
-    }
-    // (c) survivors of the filter go to shared memory (a few more than K), then rank by counting
-    int n = 0;
-#pragma unroll 1
-    for (int i0 = 0; i0 < kPerLane * 32 && i0 < nk; i0 += 32) {
-      const int i = i0 + lane;
-      unsigned long long key = 0ull;
-      if (i < nk) key = __ldcg(rk + (size_t)(i / K) * CAST_MAX_TOP_K + (i % K));
-      const bool pass = key != 0ull && key >= thr;
-      const unsigned m = __ballot_sync(0xffffffffu, pass);
-      if (pass) cand[n + __popc(m & ((1u << lane) - 1u))] = key;
-      n += __popc(m);
-    }
-    __syncwarp();
-#pragma unroll 1
-    for (int i = lane; i < n; i += 32) {
-      const unsigned long long k = cand[i];
-      int rank = 0;
-#pragma unroll 1
-      for (int j = 0; j < n; ++j) rank += (cand[j] > k);
-      if (rank < K) topk[rank] = k;
-    }
-    if (lane < K && lane >= n) topk[lane] = 0ull;
+    CAST_STAMP(25);
     // (d) log-sum-exp over the chunk partials: weights by the fp32 unit, sums in fp64
     float Mr = fmaxf(M0, M1);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) Mr = fmaxf(Mr, __shfl_xor_sync(0xffffffffu, Mr, o));
+    CAST_STAMP(28);
     double term = (M0 > -INFINITY ? S0 * (double)ex2f(M0 - Mr) : 0.0) + (M1 > -INFINITY ? S1 * (double)ex2f(M1 - Mr) : 0.0);
+    CAST_STAMP(29);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) term += __shfl_xor_sync(0xffffffffu, term, o);
+    CAST_STAMP(26);
     const double lse = ((double)Mr + fast_log2(term)) * 0.69314718055994530942;
     if (lane == 0 && !(term > 0.0 && isfinite(lse))) report(st, CAST_ERR_NONFINITE, row);
     __syncwarp();
+    CAST_STAMP(27);
     // (e) the K children join the pool
     if (lane < K) {
       const unsigned long long key = topk[lane];
@@ -670,9 +738,9 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
   __syncthreads();
   if (!take_ticket(p.layer_ticket, B * n_prev, &s_flag)) return;
   CAST_STAMP(6);
-  layer_tail(p, B, n_prev, base, scratch, sorted);
+  layer_tail(p, ts, B, n_prev, base, scratch, sorted);
   CAST_STAMP(7);
-  CAST_STAMP_FLUSH(0, 8);
+  CAST_STAMP_FLUSH(0, 31);
 }
 
 // ------------------------------------------------------------------ rerank + linearise
@@ -894,7 +962,7 @@ __global__ void __launch_bounds__(512) select_fused_kernel(const SelectParams p)
   CAST_STAMP(1);
   select_finalize_phase(p, 0, 1);
   CAST_STAMP(2);
-  CAST_STAMP_FLUSH(16, 3);
+  CAST_STAMP_FLUSH(32, 3);
 }
 
 }  // namespace
@@ -916,8 +984,7 @@ extern "C" cast_status cast_step_begin(cast_ctx* c, int B, const int32_t* root_t
   c->next_layer = 1;
   step_begin_kernel<<<1, 128, 0, (cudaStream_t)stream>>>(c->state, B, c->P, c->W, root_token, kv_len, c->pool_score,
                                                          c->pool_token, c->pool_parent, c->pool_depth, c->pool_kept,
-                                                         c->retained, c->lsort, c->lscore, c->row_ticket,
-                                                         c->layer_ticket, c->cfg.max_batch * c->W);
+                                                         c->retained, c->lsort, c->lscore, c->layer_ticket);
   return launch_status();
 }
 
@@ -930,10 +997,10 @@ extern "C" cast_status cast_tree_expand(cast_ctx* c, int layer, const void* draf
   c->next_layer = layer + 1;
   const int B = c->cur_B, V = c->cfg.vocab;
   const int rows_per_seq = layer == 1 ? 1 : c->W;
-  // enough CTAs to cover the machine about twice; one pass (kSweepSub logits) per CTA when rows are few
-  int nchunks = (2 * c->num_sms + B * rows_per_seq - 1) / (B * rows_per_seq);
-  const int one_pass = (V + kSweepSub - 1) / kSweepSub;
-  if (nchunks > one_pass) nchunks = one_pass;
+  // a logits row is swept by one cluster of up to 8 CTAs: as many as it takes to cover the machine
+  // about four times over all rows, and never so many that a CTA gets less than 2048 logits
+  int nchunks = (4 * c->num_sms + B * rows_per_seq - 1) / (B * rows_per_seq);
+  if (nchunks > V / 2048) nchunks = V / 2048;
   if (nchunks > kSweepMaxChunks) nchunks = kSweepMaxChunks;
   if (nchunks < 1) nchunks = 1;
   int chunk_elems = (V + nchunks - 1) / nchunks;
@@ -948,19 +1015,31 @@ extern "C" cast_status cast_tree_expand(cast_ctx* c, int layer, const void* draf
   p.pool_depth = c->pool_depth; p.pool_kept = c->pool_kept; p.retained = c->retained;
   p.lsort = c->lsort; p.lscore = c->lscore;
   p.st = c->state;
-  p.part_keys = c->part_keys; p.part_max = c->part_max; p.part_sum = c->part_sum;
-  p.row_ticket = c->row_ticket; p.layer_ticket = c->layer_ticket;
+  p.layer_ticket = c->layer_ticket;
   p.fifo_vals = c->fifo_vals; p.fifo_cnt = c->fifo_cnt; p.R = c->cfg.fifo_len;
   p.tab = c->cur_table;
   p.C1 = c->cfg.C1; p.C2 = c->cfg.C2;
   p.enable_bp = c->cfg.enable_bp; p.enable_dp = c->cfg.enable_dp; p.ctx_base_mode = c->cfg.ctx_base_mode;
   p.next_tokens = next_tokens; p.next_parent_row = next_parent_row; p.next_count = next_count;
-  const dim3 grid(nchunks, rows_per_seq, B);
-  if (dtype == CAST_F32)
-    expand_kernel<float><<<grid, kSweepThreads, 0, (cudaStream_t)stream>>>(p);
-  else
-    expand_kernel<__nv_bfloat16><<<grid, kSweepThreads, 0, (cudaStream_t)stream>>>(p);
-  return launch_status();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(nchunks, rows_per_seq, B);
+  cfg.blockDim = dim3(kSweepThreads, 1, 1);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = (cudaStream_t)stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)nchunks;  // the chunks of one row
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t e = dtype == CAST_F32 ? cudaLaunchKernelEx(&cfg, expand_kernel<float>, p)
+                                          : cudaLaunchKernelEx(&cfg, expand_kernel<__nv_bfloat16>, p);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return CAST_ERR_CUDA;
+  }
+  return CAST_OK;
 }
 
 extern "C" cast_status cast_select_nodes(cast_ctx* c, int32_t* tokens, int32_t* parent, int32_t* depth,
