@@ -175,6 +175,10 @@ __device__ __forceinline__ void st_cluster_f64(uint32_t addr, double v) {
 __device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 
+// Programmatic dependent launch (both are no-ops for a grid launched without the attribute).
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // State fields the layer tail needs; every CTA reads them at its start (same cache lines as the row
 // count it needs anyway), so the tail itself starts without a round trip to memory.
 struct TailState {
@@ -476,6 +480,10 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
     }
   };
   load_pass(begin);
+  // Programmatic dependent launch: this grid may have been started while the previous layer's grid was
+  // still finishing (its logits do not depend on it). Everything below reads what that grid wrote.
+  grid_dependency_wait();
+  grid_launch_dependents();  // the next grid may now take the SMs this one leaves idle
   // what the layer tail needs of the state is read now, together with the row count: one round trip
   const int n_prev = st->rows[p.layer];
   TailState ts;
@@ -948,6 +956,7 @@ __device__ __noinline__ void select_finalize_phase(const SelectParams& p, int b,
 
 __global__ void __launch_bounds__(512) select_rank_kernel(const SelectParams p) {
   extern __shared__ __align__(16) unsigned char smem[];
+  grid_dependency_wait();
   select_rank_phase(p, blockIdx.x, smem);
 }
 __global__ void __launch_bounds__(512) select_finalize_kernel(const SelectParams p) {
@@ -957,6 +966,7 @@ __global__ void __launch_bounds__(512) select_fused_kernel(const SelectParams p)
   extern __shared__ __align__(16) unsigned char smem[];
   CAST_STAMP_DECL
   CAST_STAMP(0);
+  grid_dependency_wait();
   select_rank_phase(p, 0, smem);
   __syncthreads();
   CAST_STAMP(1);
@@ -1026,13 +1036,16 @@ extern "C" cast_status cast_tree_expand(cast_ctx* c, int layer, const void* draf
   cfg.blockDim = dim3(kSweepThreads, 1, 1);
   cfg.dynamicSmemBytes = 0;
   cfg.stream = (cudaStream_t)stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = (unsigned)nchunks;  // the chunks of one row
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  // may start before the previous kernel of the stream has drained (the kernel waits where it must)
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   const cudaError_t e = dtype == CAST_F32 ? cudaLaunchKernelEx(&cfg, expand_kernel<float>, p)
                                           : cudaLaunchKernelEx(&cfg, expand_kernel<__nv_bfloat16>, p);
   if (e != cudaSuccess) {
@@ -1062,10 +1075,26 @@ extern "C" cast_status cast_select_nodes(cast_ctx* c, int32_t* tokens, int32_t* 
   cudaStream_t s = (cudaStream_t)stream;
   int threads = ((c->cfg.max_depth + 1) * c->cfg.total_token + 31) / 32 * 32;
   threads = threads > 512 ? 512 : (threads < 128 ? 128 : threads);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(c->cur_B, 1, 1);
+  cfg.blockDim = dim3(threads, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see cast_tree_expand
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   if (c->cur_B == 1) {
-    select_fused_kernel<<<1, threads, smem, s>>>(p);
+    if (cudaLaunchKernelEx(&cfg, select_fused_kernel, p) != cudaSuccess) {
+      cudaGetLastError();
+      return CAST_ERR_CUDA;
+    }
   } else {
-    select_rank_kernel<<<c->cur_B, threads, smem, s>>>(p);
+    if (cudaLaunchKernelEx(&cfg, select_rank_kernel, p) != cudaSuccess) {
+      cudaGetLastError();
+      return CAST_ERR_CUDA;
+    }
     select_finalize_kernel<<<c->cur_B, 128, 0, s>>>(p);
   }
   return launch_status();
