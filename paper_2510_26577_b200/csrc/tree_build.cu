@@ -201,56 +201,6 @@ __device__ __forceinline__ bool take_ticket(int32_t* counter, int expected, int*
   return *flag_s != 0;
 }
 
-// Exact top-K (descending) of n distinct keys in shared memory, written to out[0..K); missing
-// entries (n < K) become 0. All threads of the CTA call it; `keys` is clobbered when n > 1024.
-__device__ __forceinline__ void block_top_k(unsigned long long* keys, int n, int K, unsigned long long* out) {
-  const int tid = threadIdx.x, nt = blockDim.x;
-  if (tid < K) out[tid] = 0ull;
-  __syncthreads();
-  if (n <= 1024) {
-    // rank by counting (keys are distinct, so ranks are too): G lanes share a key, each counting over
-    // every G-th key; shared-memory latency, not the number of compares, is what this costs
-    int G = 1;
-    while (G < 32 && n * (G * 2) <= nt) G *= 2;
-    const int per = nt / G;
-#pragma unroll 1
-    for (int i0 = 0; i0 < n; i0 += per) {
-      const int i = i0 + tid / G, sub = tid % G;
-      const unsigned long long k = i < n ? keys[i] : ~0ull;
-      int r0 = 0, r1 = 0, r2 = 0, r3 = 0, j = sub;
-      for (; j + 3 * G < n; j += 4 * G) {
-        r0 += (keys[j] > k);
-        r1 += (keys[j + G] > k);
-        r2 += (keys[j + 2 * G] > k);
-        r3 += (keys[j + 3 * G] > k);
-      }
-      for (; j < n; j += G) r0 += (keys[j] > k);
-      int rank = r0 + r1 + r2 + r3;
-      for (int o = G >> 1; o > 0; o >>= 1) rank += __shfl_xor_sync(0xffffffffu, rank, o);
-      if (sub == 0 && i < n && rank < K) out[rank] = k;
-    }
-  } else {  // bitonic sort, descending, on the next power of two
-    int n2 = 2048;
-    while (n2 < n) n2 <<= 1;
-    for (int i = n + tid; i < n2; i += nt) keys[i] = 0ull;
-    __syncthreads();
-    for (int k = 2; k <= n2; k <<= 1)
-      for (int j = k >> 1; j > 0; j >>= 1) {
-        for (int i = tid; i < n2; i += nt) {
-          const int l = i ^ j;
-          if (l > i) {
-            const unsigned long long a = keys[i], b = keys[l];
-            const bool desc = ((i & k) == 0);
-            if (desc ? (a < b) : (a > b)) { keys[i] = b; keys[l] = a; }
-          }
-        }
-        __syncthreads();
-      }
-    if (tid < K) out[tid] = keys[tid];
-  }
-  __syncthreads();
-}
-
 // Layer tail (Eq. 1, Eq. 2, Algorithm 1, depth pruning), run by the last CTA of the layer.
 __device__ __forceinline__ void layer_tail(const ExpandParams& p, const TailState& ts, int B, int n_prev, int base,
                                         unsigned char* scratch, int* sorted /* [CAST_MAX_BATCH * CAST_MAX_WIDTH] */) {
@@ -293,7 +243,6 @@ __device__ __forceinline__ void layer_tail(const ExpandParams& p, const TailStat
       cis[i] = (unsigned short)ci;
     }
     __syncthreads();
-    CAST_STAMP(14);
     // Rank under the order (value desc, token asc, creation order). Every logits row contributed its K
     // children already in that order, so the rank of a candidate is the number of children that come
     // first, row by row: a lower-bound search per row (in its own row it finds its own position). Four
@@ -339,10 +288,8 @@ __device__ __forceinline__ void layer_tail(const ExpandParams& p, const TailStat
         }
       }
     }
-    CAST_STAMP(21);
     __syncthreads();
   }
-  CAST_STAMP(15);
   // Eq. 1: batch mean of the rank-wise values, then prefix sums
   if (tid < n) {
     double a = 0.0;
@@ -362,7 +309,6 @@ __device__ __forceinline__ void layer_tail(const ExpandParams& p, const TailStat
     if (tid < n) u[tid] = a;
   }
   __syncthreads();
-  CAST_STAMP(16);
   // Algorithm 1: mark[j] survives iff no earlier i has (u_j - u_i) < C1 (c_j - c_i)
   if (tid < n) {
     int ok = 1;
@@ -373,7 +319,6 @@ __device__ __forceinline__ void layer_tail(const ExpandParams& p, const TailStat
     mark[tid] = ok;
   }
   __syncthreads();
-  CAST_STAMP(17);
   if (tid == 0) {
     int n_i = 1;
 #pragma unroll 1
@@ -416,7 +361,6 @@ __device__ __forceinline__ void layer_tail(const ExpandParams& p, const TailStat
     *p.next_count = s_next;
   }
   __syncthreads();
-  CAST_STAMP(18);
   const int n_i = s_ni;
 #pragma unroll 1
   for (int i = tid; i < B * W; i += nt) {
@@ -438,12 +382,10 @@ template <typename T>
 __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParams p) {
   __shared__ __align__(16) unsigned char scratch[kCandCap * 8];  // candidate keys; later the tail's arrays
   __shared__ unsigned long long topk[CAST_MAX_TOP_K];
-  __shared__ unsigned long long red_k[kSweepThreads / 32];
-  __shared__ float warp_thr[kSweepThreads / 32];
   __shared__ float red_f[kSweepThreads / 32];
   __shared__ double red_d[kSweepThreads / 32];
   __shared__ int sorted[CAST_MAX_BATCH * CAST_MAX_WIDTH];
-  __shared__ int cand_cnt, s_flag;
+  __shared__ int s_flag;
   // filled in the first CTA of the row's cluster by all CTAs of the cluster: chunk c's top-K keys
   // (descending), maximum (log2 units) and sum of 2^(. - maximum)
   __shared__ unsigned long long row_keys[kSweepMaxChunks * CAST_MAX_TOP_K];
@@ -503,16 +445,19 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
   const double parent_score = p.pool_score[(size_t)b * p.P + parent];
 
   float M2 = -INFINITY, s_run = 0.f;  // running maximum (log2 units) and sum of 2^(x log2e - M2)
-  unsigned long long thr_key = 0ull;  // exact K-th largest key so far (0: fewer than K seen)
-  if (tid == 0) cand_cnt = 0;
-  __syncthreads();
+  // Every warp keeps the exact top K of the logits it has seen, as a descending list in shared memory;
+  // the warps never meet during the sweep. `have` (warp-uniform) is the list's length, thr_key its K-th
+  // key (0 while it is shorter than K).
+  constexpr int kWarpCap = 64;
+  constexpr int kWarps = kSweepThreads / 32;
+  unsigned long long* wlist = cand + warp * kWarpCap;
+  int have = 0;
+  unsigned long long thr_key = 0ull;
   CAST_STAMP(1);
 
   for (int sub = begin; sub < end; sub += kSweepSub) {
     if (sub != begin) load_pass(sub);
-    const int have0 = cand_cnt;
     float tmax = xv[0];
-    if (sub == begin) CAST_STAMP(10);
 #pragma unroll
     for (int i = 1; i < kSweepEpt; ++i) tmax = fmaxf(tmax, xv[i]);
     const float t2 = tmax * kLog2eHi;
@@ -529,9 +474,8 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
       }
       s_run += a0 + a1;
     }
-    if (sub == begin) CAST_STAMP(11);
-    // filter threshold: the exact K-th key once K logits have been seen, else the largest of the
-    // warps' K-th largest thread maxima (at least K logits of this pass are >= it)
+    // filter threshold: the warp's exact K-th key once it has K, else the K-th largest of the lanes'
+    // maxima of this pass (at least K of the warp's logits are >= it)
     float thr_val;
     if (thr_key == 0ull) {
       float kx = tmax;
@@ -543,18 +487,13 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
           const bool desc = ((lane & k) == 0), low = ((lane & j) == 0);
           kx = (desc == low) ? fmaxf(kx, o) : fminf(kx, o);
         }
-      const float wk = __shfl_sync(0xffffffffu, kx, K - 1);
-      if (lane == 0) warp_thr[warp] = wk;
-      __syncthreads();
-      thr_val = warp_thr[0];
-#pragma unroll
-      for (int w = 1; w < kSweepThreads / 32; ++w) thr_val = fmaxf(thr_val, warp_thr[w]);
+      thr_val = __shfl_sync(0xffffffffu, kx, K - 1);
     } else {
       thr_val = key_value(thr_key);
     }
-    if (sub == begin) CAST_STAMP(12);
     // Few logits pass. One vote per logit slot keeps the common path at a compare and a vote; a slot
-    // with a passer (rare) takes the exact test on the full key and one shared-memory atomic per warp.
+    // with a passer (rare) takes the exact test on the full key and appends to the warp's list.
+    const int have0 = have;
 #pragma unroll
     for (int i = 0; i < kSweepEpt; ++i) {
       const unsigned m0 = __ballot_sync(0xffffffffu, xv[i] >= thr_val);
@@ -563,22 +502,17 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
         const unsigned long long key = make_key(xv[i], id);
         const bool ok = xv[i] >= thr_val && id < end && key > thr_key;
         const unsigned m = __ballot_sync(0xffffffffu, ok);
-        if (m != 0u) {
-          int basepos = 0;
-          if (lane == 0) basepos = atomicAdd(&cand_cnt, __popc(m));
-          basepos = __shfl_sync(0xffffffffu, basepos, 0);
-          const int pos = basepos + __popc(m & ((1u << lane) - 1u));
-          if (ok && pos < kCandCap) cand[pos] = key;
-        }
+        const int pos = have + __popc(m & ((1u << lane) - 1u));
+        if (ok && pos < kWarpCap) wlist[pos] = key;
+        have += __popc(m);
       }
     }
-    __syncthreads();
-    if (sub == begin) CAST_STAMP(13);
-    int n = cand_cnt;
-    if (n > kCandCap) {
-      // flood (a mass of ties at the threshold): K rounds of "largest key below the last one taken"
-      unsigned long long bound = ~0ull;
-      n = have0;
+    __syncwarp();
+    if (have > kWarpCap) {
+      // flood (a mass of ties at the threshold): K rounds of "largest key below the last one taken" over
+      // the old list and this pass's logits; lane r keeps the r-th result
+      unsigned long long bound = ~0ull, mine = 0ull;
+      int n = 0;
 #pragma unroll 1
       for (int round = 0; round < K; ++round) {
         unsigned long long best = 0ull;
@@ -590,68 +524,111 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
             if (k2 < bound && k2 > best) best = k2;
           }
         }
+        if (lane < have0) {
+          const unsigned long long k2 = wlist[lane];
+          if (k2 < bound && k2 > best) best = k2;
+        }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
           const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
           best = other > best ? other : best;
         }
-        if (lane == 0) red_k[warp] = best;
-        __syncthreads();
-        best = red_k[0];
-#pragma unroll
-        for (int w = 1; w < kSweepThreads / 32; ++w) best = red_k[w] > best ? red_k[w] : best;
-        __syncthreads();
         if (best == 0ull) break;
-        if (tid == 0) cand[n] = best;
+        if (lane == round) mine = best;
         ++n;
         bound = best;
       }
-      __syncthreads();
+      __syncwarp();
+      if (lane < n) wlist[lane] = mine;
+      have = n;
+      __syncwarp();
+    } else if (have > have0) {
+      // exact order of the list (old entries and newcomers, at most 64): rank by counting, keys are distinct
+      const int n = have;
+      const unsigned long long k0 = lane < n ? wlist[lane] : 0ull;
+      const unsigned long long k1 = lane + 32 < n ? wlist[lane + 32] : 0ull;
+      int r0 = 0, r1 = 0;
+#pragma unroll 4
+      for (int j = 0; j < n; ++j) {
+        const unsigned long long kj = wlist[j];
+        r0 += (kj > k0);
+        r1 += (kj > k1);
+      }
+      __syncwarp();
+      if (lane < n && r0 < K) wlist[r0] = k0;
+      if (lane + 32 < n && r1 < K) wlist[r1] = k1;
+      have = n < K ? n : K;
+      __syncwarp();
     }
-    if (n > K) {
-      block_top_k(cand, n, K, topk);
-      if (tid < K) cand[tid] = topk[tid];
-      thr_key = topk[K - 1];
-      if (tid == 0) cand_cnt = K;
-    } else {
-      if (n < K) thr_key = 0ull;  // (n == K with a threshold: nothing new passed, the list stays sorted)
-      if (tid == 0) cand_cnt = n;
-    }
-    __syncthreads();
+    thr_key = have == K ? wlist[K - 1] : 0ull;
   }
   CAST_STAMP(2);
 
-  // chunk result: top-K keys in descending order, maximum, sum of 2^(. - maximum) in fp64; it goes
-  // straight into the shared memory of the cluster's first CTA, which merges the row
+  // chunk result: the top K of the warps' lists (each in descending order; the rank of a key is the
+  // number of larger keys, list by list: a lower-bound search each, two lanes per key slot), the
+  // maximum and the sum of 2^(. - maximum) in fp64. It goes straight into the shared memory of the
+  // cluster's first CTA, which merges the row.
   {
-    const int have = cand_cnt;
-    if (thr_key == 0ull) block_top_k(cand, have, K, topk);  // fewer than K so far: not sorted yet
-    float M = M2;
+    if (lane >= have && lane < CAST_MAX_TOP_K) wlist[lane] = 0ull;  // short lists end in "no entry"
+    float Mw = M2;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-    if (lane == 0) red_f[warp] = M;
-    __syncthreads();
-    M = red_f[0];
-#pragma unroll
-    for (int w = 1; w < kSweepThreads / 32; ++w) M = fmaxf(M, red_f[w]);
-    double sd = (M2 > -INFINITY) ? (double)s_run * (double)ex2f(M2 - M) : 0.0;
+    for (int o = 16; o > 0; o >>= 1) Mw = fmaxf(Mw, __shfl_xor_sync(0xffffffffu, Mw, o));
+    double sd = (M2 > -INFINITY) ? (double)s_run * (double)ex2f(M2 - Mw) : 0.0;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) sd += __shfl_xor_sync(0xffffffffu, sd, o);
-    if (lane == 0) red_d[warp] = sd;
+    if (lane == 0) {
+      red_f[warp] = Mw;
+      red_d[warp] = sd;
+    }
+    if (tid < K) topk[tid] = 0ull;
+    __syncthreads();
+    static_assert(kSweepThreads == 2 * kWarps * CAST_MAX_TOP_K, "two lanes per key slot");
+    const int slot = tid >> 1, sub2 = tid & 1;
+    const int w1 = slot >> 4, t = slot & 15;  // slot = warp list * CAST_MAX_TOP_K + position
+    const bool act = t < K;
+    const unsigned long long key = act ? cand[w1 * kWarpCap + t] : 0ull;
+    int pos[kWarps / 2];
+#pragma unroll
+    for (int q = 0; q < kWarps / 2; ++q) pos[q] = 0;
+#pragma unroll
+    for (int half = 16; half >= 1; half >>= 1) {
+#pragma unroll
+      for (int q = 0; q < kWarps / 2; ++q) {
+        const int w2 = sub2 + 2 * q;
+        const int idx = pos[q] + half - 1;
+        const bool valid = act && idx < K;
+        const unsigned long long other = cand[valid ? w2 * kWarpCap + idx : 0];
+        pos[q] += (valid && other > key) ? half : 0;
+      }
+    }
+    int cnt = 0;
+#pragma unroll
+    for (int q = 0; q < kWarps / 2; ++q) cnt += pos[q];
+    cnt += __shfl_xor_sync(0xffffffffu, cnt, 1);
+    if (act && sub2 == 0 && key != 0ull && cnt < K) topk[cnt] = key;
+    // meanwhile the last warp folds the warps' (maximum, sum) pairs
+    float M = -INFINITY;
+    double S = 0.0;
+    if (warp == kWarps - 1) {
+      const float Ml = lane < kWarps ? red_f[lane] : -INFINITY;
+      const double Sl = lane < kWarps ? red_d[lane] : 0.0;
+      M = Ml;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+      S = Ml > -INFINITY ? Sl * (double)ex2f(Ml - M) : 0.0;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) S += __shfl_xor_sync(0xffffffffu, S, o);
+    }
     __syncthreads();
     if (p.nchunks == 1) {
       if (tid < K) row_keys[tid] = topk[tid];
-      if (tid == 0) {
-        double S = 0.0;
-        for (int w = 0; w < kSweepThreads / 32; ++w) S += red_d[w];
+      if (tid == kSweepThreads - 32) {
         row_max[0] = M;
         row_sum[0] = S;
       }
     } else {
       if (tid < K) st_cluster_u64(map_to_rank(smem_addr(&row_keys[chunk * CAST_MAX_TOP_K + tid]), 0u), topk[tid]);
-      if (tid == 0) {
-        double S = 0.0;
-        for (int w = 0; w < kSweepThreads / 32; ++w) S += red_d[w];
+      if (tid == kSweepThreads - 32) {
         st_cluster_f32(map_to_rank(smem_addr(&row_max[chunk]), 0u), M);
         st_cluster_f64(map_to_rank(smem_addr(&row_sum[chunk]), 0u), S);
       }
@@ -673,7 +650,6 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
   // search each; in its own list it finds its own position). Four neighbouring lanes share a key slot.
   if (tid < K) topk[tid] = 0ull;
   __syncthreads();
-  CAST_STAMP(22);
   {
     static_assert(kSweepThreads == 4 * kSweepMaxChunks * CAST_MAX_TOP_K, "one pass: four lanes per key slot");
     const int slot = tid >> 2, sub = tid & 3;
@@ -697,9 +673,7 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
     cnt += __shfl_xor_sync(0xffffffffu, cnt, 1);
     if (act && sub == 0 && cnt < K) topk[cnt] = key;
   }
-  CAST_STAMP(23);
   __syncthreads();
-  CAST_STAMP(24);
   if (warp == 0) {
     float M0 = -INFINITY, M1 = -INFINITY;
     double S0 = 0.0, S1 = 0.0;
@@ -707,21 +681,16 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
       M0 = row_max[lane];
       S0 = row_sum[lane];
     }
-    CAST_STAMP(25);
     // (d) log-sum-exp over the chunk partials: weights by the fp32 unit, sums in fp64
     float Mr = fmaxf(M0, M1);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) Mr = fmaxf(Mr, __shfl_xor_sync(0xffffffffu, Mr, o));
-    CAST_STAMP(28);
     double term = (M0 > -INFINITY ? S0 * (double)ex2f(M0 - Mr) : 0.0) + (M1 > -INFINITY ? S1 * (double)ex2f(M1 - Mr) : 0.0);
-    CAST_STAMP(29);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) term += __shfl_xor_sync(0xffffffffu, term, o);
-    CAST_STAMP(26);
     const double lse = ((double)Mr + fast_log2(term)) * 0.69314718055994530942;
     if (lane == 0 && !(term > 0.0 && isfinite(lse))) report(st, CAST_ERR_NONFINITE, row);
     __syncwarp();
-    CAST_STAMP(27);
     // (e) the K children join the pool
     if (lane < K) {
       const unsigned long long key = topk[lane];
@@ -748,7 +717,7 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
   CAST_STAMP(6);
   layer_tail(p, ts, B, n_prev, base, scratch, sorted);
   CAST_STAMP(7);
-  CAST_STAMP_FLUSH(0, 31);
+  CAST_STAMP_FLUSH(0, 8);
 }
 
 // ------------------------------------------------------------------ rerank + linearise
