@@ -581,31 +581,48 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
       red_d[warp] = sd;
     }
     if (tid < K) topk[tid] = 0ull;
+    if (tid == 0) s_flag = 0;  // length of the CTA's short list
     __syncthreads();
-    static_assert(kSweepThreads == 2 * kWarps * CAST_MAX_TOP_K, "two lanes per key slot");
-    const int slot = tid >> 1, sub2 = tid & 1;
-    const int w1 = slot >> 4, t = slot & 15;  // slot = warp list * CAST_MAX_TOP_K + position
-    const bool act = t < K;
-    const unsigned long long key = act ? cand[w1 * kWarpCap + t] : 0ull;
-    int pos[kWarps / 2];
+    // The K-th largest of the warps' list heads bounds the CTA's top K from below (every list is in
+    // descending order), so only keys at or above it can belong: a dozen or so. Every warp finds that
+    // bound by itself (16 heads, one per lane), appends its survivors to a short list with one atomic,
+    // and the first warp ranks the short list by counting.
+    unsigned long long bound;
+    {
+      const unsigned long long head = lane < kWarps ? cand[lane * kWarpCap] : 0ull;
+      int rh = 0;
 #pragma unroll
-    for (int q = 0; q < kWarps / 2; ++q) pos[q] = 0;
+      for (int j = 0; j < kWarps; ++j) rh += (__shfl_sync(0xffffffffu, head, j) > head);
+      bound = (rh == K - 1) ? head : 0ull;  // heads are distinct unless 0 ("no entry")
 #pragma unroll
-    for (int half = 16; half >= 1; half >>= 1) {
-#pragma unroll
-      for (int q = 0; q < kWarps / 2; ++q) {
-        const int w2 = sub2 + 2 * q;
-        const int idx = pos[q] + half - 1;
-        const bool valid = act && idx < K;
-        const unsigned long long other = cand[valid ? w2 * kWarpCap + idx : 0];
-        pos[q] += (valid && other > key) ? half : 0;
+      for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long other = __shfl_xor_sync(0xffffffffu, bound, o);
+        bound = other > bound ? other : bound;
       }
     }
-    int cnt = 0;
-#pragma unroll
-    for (int q = 0; q < kWarps / 2; ++q) cnt += pos[q];
-    cnt += __shfl_xor_sync(0xffffffffu, cnt, 1);
-    if (act && sub2 == 0 && key != 0ull && cnt < K) topk[cnt] = key;
+    unsigned long long* shortlist = cand + kWarps * kWarpCap;  // at most kWarps * K keys
+    {
+      const unsigned long long key = lane < have ? wlist[lane] : 0ull;
+      const bool keep = key != 0ull && key >= bound;
+      const unsigned m = __ballot_sync(0xffffffffu, keep);
+      int basepos = 0;
+      if (lane == 0 && m != 0u) basepos = atomicAdd(&s_flag, __popc(m));
+      basepos = __shfl_sync(0xffffffffu, basepos, 0);
+      if (keep) shortlist[basepos + __popc(m & ((1u << lane) - 1u))] = key;
+    }
+    __syncthreads();
+    if (warp == 0) {
+      const int n = s_flag;  // <= kWarps * K = 256: up to 8 keys per lane
+#pragma unroll 1
+      for (int i0 = 0; i0 < n; i0 += 32) {
+        const int i = i0 + lane;
+        const unsigned long long key = i < n ? shortlist[i] : ~0ull;
+        int rk2 = 0;
+#pragma unroll 4
+        for (int j = 0; j < n; ++j) rk2 += (shortlist[j] > key);
+        if (i < n && rk2 < K) topk[rk2] = key;
+      }
+    }
     // meanwhile the last warp folds the warps' (maximum, sum) pairs
     float M = -INFINITY;
     double S = 0.0;
