@@ -664,30 +664,36 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
   CAST_STAMP(4);
   // the row's top K out of the chunks' lists (each in descending order): the rank of a key is its
   // position in its own list plus, for every other list, the number of larger keys there (a binary
-  // search each; in its own list it finds its own position). Four neighbouring lanes share a key slot.
+  // search each; in its own list it finds its own position). Neighbouring lanes share a key slot.
   if (tid < K) topk[tid] = 0ull;
   __syncthreads();
   {
-    static_assert(kSweepThreads == 4 * kSweepMaxChunks * CAST_MAX_TOP_K, "one pass: four lanes per key slot");
-    const int slot = tid >> 2, sub = tid & 3;
+    constexpr int kLps = kSweepThreads / (kSweepMaxChunks * CAST_MAX_TOP_K);  // lanes per key slot: one pass
+    constexpr int kLpl = kSweepMaxChunks / kLps;                              // lists per lane
+    static_assert(kLps >= 1 && kLps <= 8 && kLps * kLpl == kSweepMaxChunks, "lanes of a slot cover the lists");
+    const int slot = tid / kLps, sub = tid % kLps;
     const int c1 = slot >> 4, t = slot & 15;  // slot = list * CAST_MAX_TOP_K + position
     const bool act = c1 < p.nchunks && t < K;
     const unsigned long long key = act ? row_keys[slot] : 0ull;
-    int pos[2] = {0, 0};
+    int pos[kLpl];
+#pragma unroll
+    for (int q = 0; q < kLpl; ++q) pos[q] = 0;
 #pragma unroll
     for (int half = 16; half >= 1; half >>= 1) {
 #pragma unroll
-      for (int q = 0; q < 2; ++q) {
-        const int c2 = sub + 4 * q;
+      for (int q = 0; q < kLpl; ++q) {
+        const int c2 = sub + kLps * q;
         const int idx = pos[q] + half - 1;
         const bool valid = act && c2 < p.nchunks && idx < K;
         const unsigned long long other = row_keys[valid ? c2 * CAST_MAX_TOP_K + idx : 0];
         pos[q] += (valid && other > key) ? half : 0;
       }
     }
-    int cnt = pos[0] + pos[1];
-    cnt += __shfl_xor_sync(0xffffffffu, cnt, 2);
-    cnt += __shfl_xor_sync(0xffffffffu, cnt, 1);
+    int cnt = 0;
+#pragma unroll
+    for (int q = 0; q < kLpl; ++q) cnt += pos[q];
+#pragma unroll
+    for (int o = kLps >> 1; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
     if (act && sub == 0 && cnt < K) topk[cnt] = key;
   }
   __syncthreads();
