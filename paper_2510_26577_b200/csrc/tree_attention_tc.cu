@@ -831,7 +831,62 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
       TC_STAMP(0, it, 0);
       float mx = -INFINITY;
       uint32_t v0 = 0xffffffffu, v1 = 0xffffffffu;  // visibility of this row's 64 columns
-      if (warp_live) {
+      // Fast path (every tile but the first, as a rule): one pass over the scores with the reference
+      // maximum of the earlier tiles. P = 2^((s - m) * scale) is then not bounded by 1, but bf16 and the
+      // fp32 accumulators have the range for it; only a tile whose scores outgrow the reference by more
+      // than 2^60 (seen as a huge P) is redone on the slow path below, which moves the reference.
+      bool done = false;
+      if (warp_live && ok && it > 0 && __all_sync(0xffffffffu, m_used > -INFINITY || !row_ok)) {
+        ok = mbar_wait(&bar_s[buf], (it >> 1) & 1) && mbar_wait(&bar_freev[(it - 1) % kStages], ((it - 1) / kStages) & 1);
+        if (ok) {
+          tc_fence_after();
+          const bool plain = pos0 + kBN <= L && __all_sync(0xffffffffu, row_ok);  // nothing masked in this warp
+          if (!plain) {
+            if (pos0 + kBN > L) {
+              v0 = vis_bits32(aw, pos0 - L);
+              v1 = vis_bits32(aw, pos0 - L + 32);
+            }
+            if (!row_ok) v0 = v1 = 0u;
+          }
+          const float neg_ms = row_ok ? -m_used * sc : 0.f;
+          float l0 = 0.f, l1 = 0.f, pmax = 0.f;
+          unsigned char* prow = smem + kSmemP;
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            uint32_t sr[32];
+            tmem_ld32(tmem_s + buf * kBN + lane_sel + hh * 32, sr);
+            tmem_wait_ld();
+            const uint32_t vv = hh ? v1 : v0;
+#pragma unroll
+            for (int c8 = 0; c8 < 4; ++c8) {
+              uint32_t pk[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const int c = c8 * 8 + 2 * e;
+                float p0 = fast_exp2(fmaf(__uint_as_float(sr[c]), sc, neg_ms));
+                float p1 = fast_exp2(fmaf(__uint_as_float(sr[c + 1]), sc, neg_ms));
+                if (!plain) {
+                  p0 = ((vv >> c) & 1u) ? p0 : 0.f;
+                  p1 = ((vv >> (c + 1)) & 1u) ? p1 : 0.f;
+                }
+                l0 += p0;
+                l1 += p1;
+                pmax = fmaxf(pmax, fmaxf(p0, p1));
+                const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+                pk[e] = *reinterpret_cast<const uint32_t*>(&pb);
+              }
+              *reinterpret_cast<uint4*>(prow + swz(r, hh * 4 + c8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            }
+          }
+          if (!__any_sync(0xffffffffu, !(pmax < 1.15e18f))) {  // 2^60; a NaN score also takes the slow path
+            l_run += l0 + l1;
+            done = true;
+          } else {
+            v0 = v1 = 0xffffffffu;
+          }
+        }
+      }
+      if (warp_live && !done) {
         if (ok) ok = mbar_wait(&bar_s[buf], (it >> 1) & 1);
         TC_STAMP(0, it, 1);
         if (ok) {
@@ -867,7 +922,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
       // it also keeps a warp from arriving on bar_p for tile `it` before the phase of tile it-1 is over.
       if (ok && it >= 1) ok = mbar_wait(&bar_freev[(it - 1) % kStages], ((it - 1) / kStages) & 1);
       TC_STAMP(0, it, 5);
-      if (warp_live) {
+      if (warp_live && !done) {
         if (ok) {
           // lazy maximum: move the reference only when the row maximum outgrows it by 2^8
           float alpha = 1.f;
