@@ -999,10 +999,14 @@ extern "C" cast_status cast_tree_expand(cast_ctx* c, int layer, const void* draf
   c->next_layer = layer + 1;
   const int B = c->cur_B, V = c->cfg.vocab;
   const int rows_per_seq = layer == 1 ? 1 : c->W;
-  // a logits row is swept by one cluster of up to 8 CTAs: as many as it takes to cover the machine
-  // about four times over all rows, and never so many that a CTA gets less than 2048 logits
-  int nchunks = (4 * c->num_sms + B * rows_per_seq - 1) / (B * rows_per_seq);
-  if (nchunks > V / 2048) nchunks = V / 2048;
+  // A logits row is swept by one cluster of up to 8 CTAs: as many as it takes to cover the machine
+  // about four times over all rows. With few rows (small batches: latency counts) a CTA may get as
+  // little as 2048 logits; with many, at least half a pass, because a pass costs the same whether its
+  // slots are full or not.
+  const int rows = B * rows_per_seq;
+  int nchunks = (4 * c->num_sms + rows - 1) / rows;
+  const int min_chunk = rows < 16 ? 2048 : kSweepSub / 2;
+  if (nchunks > V / min_chunk) nchunks = V / min_chunk;
   if (nchunks > kSweepMaxChunks) nchunks = kSweepMaxChunks;
   if (nchunks < 1) nchunks = 1;
   int chunk_elems = (V + nchunks - 1) / nchunks;
