@@ -588,6 +588,10 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_k)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_v)) : "memory");
   }
+  // Programmatic dependent launch: this grid may become resident while the previous kernel of the
+  // stream drains; nothing written by earlier kernels is read before this point. (No-ops for a plain launch.)
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const WorkItem wk = cs == 0 ? decode_work_chunked(p, (int)blockIdx.x, (int)gridDim.x) : decode_work(p, (int)blockIdx.x / cs, crank);
   TC_MARK(1);
   if (blockIdx.x < p.B && tid == 0 && p.n_tree[blockIdx.x] > p.Nmax) report(p.st, CAST_ERR_BAD_TREE, blockIdx.x);
@@ -1341,13 +1345,16 @@ bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const v
   cfg.blockDim = dim3(kThreadsTC, 1, 1);
   cfg.dynamicSmemBytes = kSmemBytes;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = (unsigned)cs;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  // may become resident before the previous kernel of the stream has drained (the kernel waits where it must)
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   if (cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel, p, map_k, map_v) != cudaSuccess) {
     cudaGetLastError();
     *status = CAST_ERR_CUDA;
