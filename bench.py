@@ -124,7 +124,6 @@ def oracle_step_seconds(w, attn_pairs=256):
     tree_attention(q, k, v, w.page_size, tab, kv.numpy(), o["anc"], n_tree, None, only)
     t_attn_layer = (time.perf_counter() - t0) * total_pairs / len(only)
     nmax = int(n_tree.max())
-    rows = min(nmax, 8)
     tl = to_f64(wl.target_logits(w)[:, :nmax])
     t0 = time.perf_counter()
     ol, op, _ = greedy_accept(tl, o["tokens"], o["parent"], n_tree, w.depth)
@@ -141,7 +140,6 @@ def oracle_step_seconds(w, attn_pairs=256):
         threads = 1
     desc = (f"tree build + accept in full; attention: {len(only)} of {total_pairs} (token, head) outputs of one layer, "
             f"scaled to {w.n_layers} layers; compaction of one layer scaled to {w.n_layers}")
-    del rows
     return total, desc, threads, int(sum(int(n) for n in n_tree))
 
 
@@ -371,7 +369,6 @@ def run_ours(args, w):
     peak, which = peaks()
     attn_us = ms_attn * 1e3 / nl
     achieved = attn_bytes / (attn_us * 1e-6) / 1e9
-    logits_bytes = sum(int(x.numel() * x.element_size()) for x in logits) // K * 1  # layer 1 reads one row
     sel_launches = 1 if B == 1 else 2
     attn_launches = 1 if (w.kv_dtype == "bf16" and D == 128) else 2  # CUDA-core path: main + combine
     launches = args.steps * (1 + H + sel_launches + attn_launches * nl + 2 + 1)
@@ -403,7 +400,6 @@ def run_ours(args, w):
                      "algorithmic_bytes": attn_bytes},
         "cpu_baseline": cpu,
     }
-    del logits_bytes
     print(json.dumps(line))
     replicas.shutdown(rep)
 

@@ -1090,59 +1090,6 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
   if (cs > 1) cluster_sync_all();  // nobody leaves while a peer may still read its shared memory
 }
 
-#ifdef CAST_PHASE_CLOCKS
-// Development aid: streams the same K/V tiles through the same TMA boxes and does nothing else.
-__global__ void __launch_bounds__(64, 2) dbg_loadonly_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
-                                                             const __grid_constant__ CUtensorMap map_v, int kvh_fast) {
-  extern __shared__ __align__(1024) unsigned char smem[];
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 4 * 2 * kTileKV);
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  (void)kvh_fast;
-  const WorkItem wk = decode_work(p, blockIdx.x, gridDim.x);
-  if (!wk.valid) return;
-  const int b = wk.b, kvh = wk.kvh, split = wk.split, N = wk.N, L = wk.L, nsplit = wk.nsplit;
-  const int total = L + N, ntiles = (total + kBN - 1) / kBN;
-  const int t0 = (int)((long long)split * ntiles / nsplit), t1 = (int)((long long)(split + 1) * ntiles / nsplit);
-  const int ntile = t1 - t0;
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < 4; ++s) mbar_init(&bars[s], 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    fence_proxy_async();
-  }
-  __syncthreads();
-  if (warp == 0) {
-    for (int j = 0; j < ntile + 3; ++j) {
-      if (j >= 3) {  // consume tile j-3
-        const int jj = j - 3;
-        if (!mbar_wait(&bars[jj % 4], (jj / 4) & 1)) break;
-      }
-      if (j < ntile) {
-        const int stage = j % 4, pos0 = (t0 + j) * kBN, ps = p.page_size;
-        unsigned char* dst = smem + stage * 2 * kTileKV;
-        if (ps == 0) {
-          if (lane == 0) mbar_expect_tx(&bars[stage], 2 * kTileKV);
-          __syncwarp();
-          if (lane < 4) tma_load_3d(lane < 2 ? &map_k : &map_v, dst + lane * kRegionKV, &bars[stage], (lane & 1) * 64, kvh,
-                                    b * p.seq_capacity + pos0);
-        } else {
-          int npages = (total - pos0 + ps - 1) / ps;
-          npages = npages > kBN / ps ? kBN / ps : npages;
-          int page = 0;
-          if (lane < npages * 4) page = p.page_table[(size_t)b * p.seq_capacity + pos0 / ps + (lane >> 2)];
-          if (lane == 0) mbar_expect_tx(&bars[stage], (uint32_t)npages * ps * 128 * 4);
-          __syncwarp();
-          if (lane < npages * 4) {
-            const int slot = lane >> 2, which = lane & 3;
-            tma_load_4d(which < 2 ? &map_k : &map_v, dst + which * kRegionKV + slot * ps * 128, &bars[stage], (which & 1) * 64,
-                        kvh, 0, page);
-          }
-        }
-        __syncwarp();
-      }
-    }
-  }
-}
-#endif
 
 EncodeTiledFn get_encode() {
   static EncodeTiledFn fn = nullptr;
@@ -1182,56 +1129,6 @@ bool make_kv_map(CUtensorMap* map, const void* base, int B, int Hkv, int page_si
 
 }  // namespace
 
-#ifdef CAST_PHASE_CLOCKS
-extern "C" __attribute__((visibility("default"))) int cast_debug_tc_occupancy_at(int bytes) {
-  int n = -1;
-  cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-  cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
-  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, tree_attn_tc_kernel, kThreadsTC, bytes);
-  return n;
-}
-__global__ void __launch_bounds__(256, 2) dbg_plain_kernel(float* x) {
-  float acc[96];
-#pragma unroll
-  for (int i = 0; i < 96; ++i) acc[i] = x[i * 256 + threadIdx.x];
-#pragma unroll
-  for (int k = 0; k < 8; ++k)
-#pragma unroll
-    for (int i = 0; i < 96; ++i) acc[i] = acc[i] * acc[(i + k + 1) % 96] + 1.f;
-#pragma unroll
-  for (int i = 0; i < 96; ++i) x[i * 256 + threadIdx.x] = acc[i];
-}
-extern "C" __attribute__((visibility("default"))) int cast_debug_occ_bs(int bytes, int bs, int which) {
-  int n = -1;
-  if (which == 0) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, tree_attn_tc_kernel, bs, bytes);
-  else {
-    cudaFuncAttributes a; cudaFuncGetAttributes(&a, dbg_plain_kernel);
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, dbg_plain_kernel, bs, bytes);
-    n = n * 1000 + a.numRegs;
-  }
-  return n;
-}
-extern "C" __attribute__((visibility("default"))) int cast_debug_tc_attrs(int* out) {
-  cudaFuncAttributes a;
-  cudaError_t e = cudaFuncGetAttributes(&a, tree_attn_tc_kernel);
-  out[0] = a.numRegs; out[1] = (int)a.sharedSizeBytes; out[2] = a.maxThreadsPerBlock; out[3] = (int)a.localSizeBytes;
-  out[4] = a.maxDynamicSharedSizeBytes; out[5] = a.preferredShmemCarveout; out[6] = (int)a.constSizeBytes;
-  int dev = 0, v = 0;
-  cudaGetDevice(&dev);
-  cudaDeviceGetAttribute(&v, cudaDevAttrMaxBlocksPerMultiprocessor, dev); out[7] = v;
-  cudaDeviceGetAttribute(&v, cudaDevAttrMaxRegistersPerMultiprocessor, dev); out[8] = v;
-  cudaDeviceGetAttribute(&v, cudaDevAttrMaxRegistersPerBlock, dev); out[9] = v;
-  cudaDeviceGetAttribute(&v, cudaDevAttrReservedSharedMemoryPerBlock, dev); out[10] = v;
-  return (int)e;
-}
-extern "C" __attribute__((visibility("default"))) int cast_debug_tc_occupancy() {
-  int n = -1;
-  cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-  cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
-  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, tree_attn_tc_kernel, kThreadsTC, kSmemBytes);
-  return n;
-}
-#endif
 
 bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const void* v, int B, int Hq, int Hkv, int D,
                               int page_size, const int32_t* page_table, int seq_capacity, int num_pages,
@@ -1330,16 +1227,6 @@ bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const v
     cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
     attr_done = true;
   }
-#ifdef CAST_PHASE_CLOCKS
-  if (const char* lo = getenv("CAST_TC_LOADONLY")) {
-    const int kvh_fast = atoi(lo) == 2;
-    cudaFuncSetAttribute(dbg_loadonly_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * 2 * kTileKV + 64);
-    cudaFuncSetAttribute(dbg_loadonly_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
-    dbg_loadonly_kernel<<<(unsigned)grid, 64, 4 * 2 * kTileKV + 64, stream>>>(p, map_k, map_v, kvh_fast);
-    *status = launch_status();
-    return true;
-  }
-#endif
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid, 1, 1);
   cfg.blockDim = dim3(kThreadsTC, 1, 1);

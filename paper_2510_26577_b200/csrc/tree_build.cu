@@ -1,17 +1,18 @@
 // Draft-tree construction: cast_step_begin, cast_tree_expand, cast_select_nodes.
 //
-// cast_tree_expand is ONE kernel per draft layer:
-//   1. vocabulary sweep - every logits row is cut into chunks, one CTA per chunk: streaming
-//      16-byte loads issued before anything else, online max / sum-exp in base 2, and an exact
-//      top-K by threshold filtering (the K-th largest of the per-thread maxima of a warp bounds
-//      the K-th largest of the chunk from below, so only a few dozen logits survive the filter);
-//   2. the last CTA to finish a row merges the chunk partials (log-sum-exp in fp64, exact
-//      top-K of the chunk winners, again threshold-filtered) and appends the K children to the
-//      node pool;
-//   3. the last CTA to finish the layer ranks each sequence's candidates, forms the utility u
-//      (Eq. 1) and the cost c (Eq. 2), runs Algorithm 1 (breadth pruning), the depth-pruning
-//      test and the FIFO update, and publishes the retained nodes and the layer's sorted list.
-// "Last CTA" is decided by an atomic ticket; nothing spins.
+// cast_tree_expand is ONE kernel per draft layer, launched as thread-block clusters (the chunks of
+// one logits row form a cluster) with programmatic dependent launch between the layers:
+//   1. vocabulary sweep - one CTA per chunk: streaming 16-byte loads issued before anything else,
+//      online max / sum-exp in base 2, and an exact top-K kept per warp (the K-th largest of the
+//      lanes' maxima bounds the warp's K-th largest from below, so only a handful of logits
+//      survive the filter; the warps never meet during the sweep);
+//   2. the chunk's top K, maximum and sum go straight into the shared memory of the cluster's
+//      first CTA, which merges the row after the cluster barrier (log-sum-exp in fp64, lower-bound
+//      merge of the sorted chunk lists) and appends the K children to the node pool;
+//   3. the last row-merging CTA of the layer (an atomic ticket; nothing spins) ranks each
+//      sequence's candidates, forms the utility u (Eq. 1) and the cost c (Eq. 2), runs Algorithm 1
+//      (breadth pruning), the depth-pruning test and the FIFO update, and publishes the retained
+//      nodes and the layer's sorted list.
 // cast_select_nodes ranks the pool by merging the per-layer sorted lists (binary searches), forms
 // the batch-mean utility, runs Algorithm 1 with the target-cost ratio and linearises the tree.
 #include <math.h>
