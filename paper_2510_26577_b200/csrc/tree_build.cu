@@ -188,14 +188,15 @@ struct TailState {
 };
 
 // The ticket of the "last CTA" pattern: the caller has passed a CTA barrier after its global
-// writes; one thread fences (cumulative over the CTA's writes) and takes the ticket.
+// writes; one thread takes the ticket with release-acquire semantics (cumulative over the CTA's writes).
 __device__ __forceinline__ bool take_ticket(int32_t* counter, int expected, int* flag_s) {
   if (threadIdx.x == 0) {
-    __threadfence();
-    const int t = atomicAdd(counter, 1);
+    // one acquire-release atomic at device scope: releases this CTA's writes (the barrier before the
+    // call made them this thread's to release), acquires those of the CTAs that came earlier
+    int t;
+    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(t) : "l"(counter) : "memory");
     const int last = (t == expected - 1);
     if (last) *counter = 0;
-    __threadfence();
     *flag_s = last;
   }
   __syncthreads();
