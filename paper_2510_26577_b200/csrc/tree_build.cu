@@ -780,15 +780,18 @@ __device__ __noinline__ void select_rank_phase(const SelectParams& p, int b, uns
   const int tid = threadIdx.x, nt = blockDim.x;
   const size_t o = (size_t)b * p.P;
   const int nl = p.st->layers_done + 1;  // lists: depth 0 (the root) .. layers_done
+  if (tid < nl) {  // one memory round trip for all lists
+    int len = p.pool_mode == 0 ? p.st->layer_n[tid] : p.st->n_hist[tid];
+    llen[tid] = len > p.m ? p.m : len;
+    lbase[tid] = p.st->layer_base[tid];
+  }
+  const int peff = p.pool_mode == 0 ? p.st->pool_size : p.st->kept_total;  // (needed further down)
+  __syncthreads();
   if (tid == 0) {
     int acc = 0;
     for (int l = 0; l < nl; ++l) {
-      int len = p.pool_mode == 0 ? p.st->layer_n[l] : p.st->n_hist[l];
-      len = len > p.m ? p.m : len;
-      lbase[l] = p.st->layer_base[l];
-      llen[l] = len;
       loff[l] = acc;
-      acc += len;
+      acc += llen[l];
     }
     loff[nl] = acc;
   }
@@ -801,7 +804,6 @@ __device__ __noinline__ void select_rank_phase(const SelectParams& p, int b, uns
     ls[i] = p.lscore[o + lbase[l] + (i - loff[l])];
   }
   __syncthreads();
-  const int peff = p.pool_mode == 0 ? p.st->pool_size : p.st->kept_total;
   const int n_out = min(min(peff, p.m), p.Ncap);
 #pragma unroll 1
   for (int i = tid; i < total; i += nt) {
@@ -810,18 +812,30 @@ __device__ __noinline__ void select_rank_phase(const SelectParams& p, int b, uns
     const int k = i - loff[l];
     const double s = ls[i];
     int rank = k;
+    // nodes of another list l2 that come first: value > s, or value == s when their depth is smaller.
+    // Lower-bound searches, four lists in lockstep and branch-free so that their loads overlap.
 #pragma unroll 1
-    for (int l2 = 0; l2 < nl; ++l2) {
-      if (l2 == l) continue;
-      // nodes of list l2 that come first: value > s, or value == s when their depth is smaller
-      const double* a = ls + loff[l2];
-      int lo = 0, hi = llen[l2];
-      if (l2 < l) {
-        while (lo < hi) { const int mid = (lo + hi) >> 1; if (a[mid] >= s) lo = mid + 1; else hi = mid; }
-      } else {
-        while (lo < hi) { const int mid = (lo + hi) >> 1; if (a[mid] > s) lo = mid + 1; else hi = mid; }
+    for (int l0 = 0; l0 < nl; l0 += 4) {
+      int pos[4] = {0, 0, 0, 0}, len4[4], off4[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int l2 = l0 + q;
+        const bool valid = l2 < nl && l2 != l;
+        len4[q] = valid ? llen[l2] : 0;
+        off4[q] = valid ? loff[l2] : 0;
       }
-      rank += lo;
+#pragma unroll
+      for (int half = CAST_MAX_TREE; half >= 1; half >>= 1) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int idx = pos[q] + half - 1;
+          const bool inb = idx < len4[q];
+          const double a = ls[off4[q] + (inb ? idx : 0)];
+          const bool first = inb && ((l0 + q < l) ? (a >= s) : (a > s));
+          pos[q] += first ? half : 0;
+        }
+      }
+      rank += pos[0] + pos[1] + pos[2] + pos[3];
     }
     if (rank < n_out) {
       p.sel_score[(size_t)b * p.Ncap + rank] = s;
