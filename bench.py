@@ -324,37 +324,79 @@ def run_ours(args, w):
     st = ctx.cast_poll_status()
     assert st[0] == 0, f"device status {st}"
 
-    # ---- end to end: per-step inputs start in pinned host memory, results are read back
+    # ---- end to end: every step's inputs start in pinned host memory and its results are read back to
+    # the host, all inside the timed region. Copies run on their own stream into / out of a second set
+    # of device buffers, so the copy of step s+1 overlaps the compute of step s (PCIe is the bound).
     h_logits = [x.cpu().pin_memory() for x in logits]
     h_q = q[:, :, :m].contiguous().cpu().pin_memory()
     h_tl = tl[:, :m].contiguous().cpu().pin_memory()
     h_out = torch.empty_like(h_q).pin_memory()
     h_res = torch.empty((B, H + 3), dtype=torch.int32).pin_memory()
-    d_res = torch.empty((B, H + 3), dtype=torch.int32, device=dev)
     h2d = sum(x.numel() * x.element_size() for x in h_logits) + h_q.numel() * 2 + h_tl.numel() * h_tl.element_size()
     d2h = h_out.numel() * h_out.element_size() + h_res.numel() * 4
+    copy_stream = torch.cuda.Stream(device=dev)
+    stage_in = [dict(logits=[torch.empty_like(x) for x in logits], q=torch.empty_like(h_q, device=dev),
+                     tl=torch.empty_like(h_tl, device=dev)) for _ in range(2)]
+    stage_out = [dict(out=torch.empty_like(h_q, device=dev), res=torch.empty((B, H + 3), dtype=torch.int32, device=dev))
+                 for _ in range(2)]
+    ev_in = [torch.cuda.Event() for _ in range(2)]
+    ev_out = [torch.cuda.Event() for _ in range(2)]
+    ev_free = [torch.cuda.Event() for _ in range(2)]
 
-    def e2e_step():
-        for i in range(H):
-            logits[i].copy_(h_logits[i], non_blocking=True)
-        q[:, :, :m].copy_(h_q, non_blocking=True)
-        tl[:, :m].copy_(h_tl, non_blocking=True)
-        step()
-        h_out.copy_(out[:, :, :m], non_blocking=True)
-        d_res[:, 0] = alen; d_res[:, 1] = bonus; d_res[:, 2:] = apath
-        h_res.copy_(d_res, non_blocking=True)
+    def upload(k):  # copy stream: host -> staging set k
+        with torch.cuda.stream(copy_stream):
+            copy_stream.wait_event(ev_free[k])  # the compute stream has taken the previous contents
+            for i in range(H):
+                stage_in[k]["logits"][i].copy_(h_logits[i], non_blocking=True)
+            stage_in[k]["q"].copy_(h_q, non_blocking=True)
+            stage_in[k]["tl"].copy_(h_tl, non_blocking=True)
+            ev_in[k].record(copy_stream)
 
-    with torch.cuda.stream(stream):
-        for _ in range(0 if args.quick else max(args.warmup, 3)):
-            e2e_step()
+    def compute(k):  # compute stream: staging set k -> the graph's inputs, one step, results -> staging set k
+        with torch.cuda.stream(stream):
+            stream.wait_event(ev_in[k])
+            for i in range(H):
+                logits[i].copy_(stage_in[k]["logits"][i], non_blocking=True)
+            q[:, :, :m].copy_(stage_in[k]["q"], non_blocking=True)
+            tl[:, :m].copy_(stage_in[k]["tl"], non_blocking=True)
+            ev_free[k].record(stream)
+            g_step.replay()
+            stage_out[k]["out"].copy_(out[:, :, :m], non_blocking=True)
+            r = stage_out[k]["res"]
+            r[:, 0] = alen; r[:, 1] = bonus; r[:, 2:] = apath
+            ev_out[k].record(stream)
+
+    def download(k):  # copy stream: results of staging set k -> host
+        with torch.cuda.stream(copy_stream):
+            copy_stream.wait_event(ev_out[k])
+            h_out.copy_(stage_out[k]["out"], non_blocking=True)
+            h_res.copy_(stage_out[k]["res"], non_blocking=True)
+
+    def e2e_run(nsteps):
+        for k in range(2):
+            ev_free[k].record(stream)
+        upload(0)
+        for sidx in range(nsteps):
+            k = sidx & 1
+            if sidx + 1 < nsteps:
+                upload(k ^ 1)
+            compute(k)
+            download(k)
+        copy_stream.synchronize()
         stream.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(1 if args.quick else args.steps):
-            e2e_step()
-        e1.record(stream)
-        stream.synchronize()
-    ms_e2e = e0.elapsed_time(e1) / (1 if args.quick else args.steps)
+
+    e2e_steps = 2 if args.quick else args.steps
+    if not args.quick:
+        e2e_run(max(args.warmup, 3))
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    e2e_run(e2e_steps)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    wall_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
+    ms_e2e = max(e0.elapsed_time(e1) / e2e_steps, wall_ms)  # the copy stream may finish after the compute stream
     _, ms_e2e = replicas.aggregate(rep, tokens_per_step, ms_e2e)
 
     if rank != 0:
