@@ -409,7 +409,8 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
   constexpr int NV = kSweepEpt / VEC;
   const bool aligned = (reinterpret_cast<uintptr_t>(x) & 15) == 0;  // chunk starts are multiples of 8 logits
 
-  // the first pass of logits is requested before the state is read (every row r < W exists in memory)
+  // the first pass of logits is requested before the state is read (every row r < W exists in memory):
+  // one memory round trip for both
   float xv[kSweepEpt];
   auto load_pass = [&](int sub) {
 #pragma unroll
@@ -423,11 +424,12 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
       }
     }
   };
-  load_pass(begin);
-  // Programmatic dependent launch: this grid may have been started while the previous layer's grid was
-  // still finishing (its logits do not depend on it). Everything below reads what that grid wrote.
+  // Programmatic dependent launch: this grid may have become resident while the previous kernel of the
+  // stream was still finishing. Nothing that kernel may have written is read above this line - not the
+  // logits either: in a serving loop the previous kernel is the draft model's, and it writes them.
   grid_dependency_wait();
   grid_launch_dependents();  // the next grid may now take the SMs this one leaves idle
+  load_pass(begin);
   // what the layer tail needs of the state is read now, together with the row count: one round trip
   const int n_prev = st->rows[p.layer];
   TailState ts;
