@@ -192,6 +192,16 @@ def test_unaligned_vocab_and_bf16_ties(binding):
     build_tree_both(binding, wl.shrink(SMALL, logit_dtype="bf16", config_id=78, vocab=5000, logit_std=0.05))
 
 
+@pytest.mark.parametrize("over", [
+    dict(vocab=3000, top_k=16, depth=2, batch=2, total_token=64, max_tree=64, config_id=81),  # K = W = 16: the caps
+    dict(vocab=20, top_k=3, depth=3, batch=1, total_token=10, config_id=82),      # fewer logits than lanes
+    dict(vocab=70001, top_k=8, depth=2, batch=2, logit_dtype="bf16", logit_std=3.0, config_id=83),  # 8 ragged chunks
+    dict(vocab=200000, top_k=5, depth=2, batch=1, logit_std=3.0, config_id=84),   # chunks of more than one pass
+])
+def test_tree_build_shapes(binding, over):
+    build_tree_both(binding, wl.shrink(SMALL, **over))
+
+
 def test_uniform_and_neg_inf_logits(binding):
     w = wl.shrink(SMALL, batch=1, vocab=4096, config_id=79)
     kw = cfg_kwargs(w)
@@ -329,6 +339,36 @@ def test_attention_arbitrary_trees_ragged(binding, dtype, D, Hq, Hkv, page):
     assert err <= attention_tolerance(dtype), err
     for b in range(B):
         assert np.isnan(got[b, int(n_tree[b]):]).all()
+
+
+@pytest.mark.parametrize("name,n", [("c3_llama8b_b64", 9), ("c3_llama8b_b16", 12), ("c4_llama70b_n32", 32)])
+def test_attention_full_size_launch_sampled(binding, name, n):
+    """The launch shapes bench.py times (plain, global-merge and cluster mode at full cache sizes), on
+    random trees of the size the tree build produces there; the oracle computes sampled outputs."""
+    rng = np.random.default_rng(7)
+    w = wl.CONFIGS[name]
+    B, Ncap = w.batch, w.max_tree
+    ctx = binding.CastContext(max_batch=B, **cfg_kwargs(w, enable_bp=0, enable_dr=0))
+    kv = wl.kv_lengths(w, "cpu").cuda()
+    n_tree = np.full(B, n, dtype=np.int32)
+    anc = np.zeros((B, Ncap, 4), dtype=np.uint32)
+    for b in range(B):
+        anc[b, :n] = ancestor_masks(_random_tree(rng, n, "random"), n, 4)
+    q = wl.query(w, 0, "cpu").cuda()
+    k, v = (t.cuda() for t in wl.kv_cache(w, 0, "cpu"))
+    table, num_pages = wl.page_table(w, "cuda")
+    out = gpu_attention(ctx, w, q, k, v, table, num_pages, kv, anc, torch.from_numpy(n_tree).cuda(), scale=0.0)
+    assert ctx.cast_poll_status()[0] == 0
+    only = {(int(b), int(rng.integers(0, n)), int(rng.integers(0, w.q_heads))) for b in rng.integers(0, B, size=24)}
+    only |= {(b, n - 1, w.q_heads - 1) for b in (0, B - 1)}
+    f32 = lambda t: t.float().cpu().numpy()
+    tab = table.cpu().numpy() if table is not None else None
+    ref = tree_attention(f32(q), f32(k), f32(v), w.page_size, tab, kv.cpu().numpy(), anc, n_tree, None, only)
+    got = to_f64(out)
+    err = max(np.max(np.abs(got[i] - ref[i])) for i in only)
+    assert err <= attention_tolerance(w.kv_dtype), err
+    for b in (0, B - 1):
+        assert np.isnan(got[b, n:]).all()
 
 
 def test_attention_bad_page_sets_status(binding):
