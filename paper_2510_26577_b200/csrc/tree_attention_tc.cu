@@ -25,6 +25,7 @@
 // through global memory and nothing spins. All mbarrier waits are bounded: on expiry the CTA
 // records CAST_ERR_TIMEOUT, contributes nothing to the merge, and still meets its cluster.
 #include <cuda.h>
+#include <cuda_fp16.h>
 #include <math.h>
 #include <stdlib.h>
 
@@ -313,22 +314,25 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t saddr, uint32_t rank) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
   return r;
 }
-__device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr) {
-  float4 v;
-  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
-  return v;
-}
 __device__ __forceinline__ float2 ld_cluster_f2(uint32_t addr) {
   float2 v;
   asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
   return v;
 }
 
-constexpr int kStageStride = kHD + 4;  // floats per staged output row: 16-byte accesses stay conflict-free
+constexpr int kStageStride = kHD + 4;   // floats per staged output row: 16-byte accesses stay conflict-free
+constexpr int kStageStrideH = kHD + 8;  // halves per staged row of a cluster-merged partial (272 bytes)
+__device__ __forceinline__ uint2 ld_cluster_u2(uint32_t addr) {
+  uint2 v;
+  asm volatile("ld.shared::cluster.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+  return v;
+}
 
 // Merge of the splits of a row block through distributed shared memory. Every CTA of the split
-// group has staged its partial O (fp32, unnormalised) and (max, sum) per row in its own shared
-// memory; this CTA owns the rows rr with rr % nsplit == split and reads them from all peers.
+// group has staged its partial output rows, normalised by their own sum and rounded to half precision
+// (the merge moves half the bytes that way; the rounding, 2^-11 relative, is a quarter of the bf16
+// output's), and (max, sum) per row in its own shared memory. This CTA owns the rows rr with
+// rr % nsplit == split and reads them from all peers: split s weighs sum_s * e^(max_s - max).
 // Warp w takes owned rows w, w+8, ...; a lane owns 4 output columns; ROWS x SPL loads in flight.
 template <int ROWS, int SPL>
 __device__ __forceinline__ void merge_rows(const TcParams& p, uint32_t stage_o_s, uint32_t stage_ml_s, int rank0,
@@ -336,7 +340,7 @@ __device__ __forceinline__ void merge_rows(const TcParams& p, uint32_t stage_o_s
   const int lane = threadIdx.x & 31, wv = threadIdx.x >> 5, G = p.G;
   const int owned = rows_here > split ? (rows_here - split + nsplit - 1) / nsplit : 0;
   for (int i0 = wv; i0 < owned; i0 += 8 * ROWS) {
-    float4 v[ROWS][SPL];
+    uint2 v[ROWS][SPL];
     float wgt[ROWS], inv[ROWS];
     size_t orow[ROWS];
 #pragma unroll
@@ -353,14 +357,14 @@ __device__ __forceinline__ void merge_rows(const TcParams& p, uint32_t stage_o_s
       }
 #pragma unroll
       for (int s2 = 0; s2 < SPL; ++s2)
-        v[u][s2] = s2 < nsplit ? ld_cluster_f4(map_to_rank(stage_o_s + (uint32_t)(rr * kStageStride + lane * 4) * 4u,
+        v[u][s2] = s2 < nsplit ? ld_cluster_u2(map_to_rank(stage_o_s + (uint32_t)(rr * kStageStrideH + lane * 4) * 2u,
                                                            (uint32_t)(rank0 + s2)))
-                               : make_float4(0.f, 0.f, 0.f, 0.f);
+                               : make_uint2(0u, 0u);
       float M = ms;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-      wgt[u] = ms > -INFINITY ? expf(ms - M) : 0.f;
-      float lsum = ls * wgt[u];
+      wgt[u] = ms > -INFINITY ? ls * expf(ms - M) : 0.f;
+      float lsum = wgt[u];
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
       inv[u] = lsum > 0.f ? 1.f / lsum : 0.f;
@@ -372,10 +376,12 @@ __device__ __forceinline__ void merge_rows(const TcParams& p, uint32_t stage_o_s
       for (int s2 = 0; s2 < SPL; ++s2) {
         const float w = __shfl_sync(0xffffffffu, wgt[u], s2);
         if (w > 0.f) {  // a split without visible positions staged nothing: its buffer may hold anything
-          acc.x += v[u][s2].x * w;
-          acc.y += v[u][s2].y * w;
-          acc.z += v[u][s2].z * w;
-          acc.w += v[u][s2].w * w;
+          const float2 lo = __half22float2(*reinterpret_cast<const __half2*>(&v[u][s2].x));
+          const float2 hi = __half22float2(*reinterpret_cast<const __half2*>(&v[u][s2].y));
+          acc.x += lo.x * w;
+          acc.y += lo.y * w;
+          acc.z += hi.x * w;
+          acc.w += hi.y * w;
         }
       }
       if (i0 + 8 * u < owned) {
@@ -1013,17 +1019,39 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     }
     if (ok && warp_live && ntile > 0) {
       tc_fence_after();
+      if (cs > 1 && nsplit > 1) {  // cluster merge: the row normalised by its own sum, in half precision
+        const float inv_l = l_run > 0.f ? 1.f / l_run : 0.f;
+        __half* sh = reinterpret_cast<__half*>(stage_o) + r * kStageStrideH;
 #pragma unroll
-      for (int hh = 0; hh < 4; ++hh) {
-        uint32_t orr[32];
-        tmem_ld32(tmem_o + lane_sel + hh * 32, orr);
-        tmem_wait_ld();
-        float* so = stage_o + r * kStageStride + hh * 32;
+        for (int hh = 0; hh < 4; ++hh) {
+          uint32_t orr[32];
+          tmem_ld32(tmem_o + lane_sel + hh * 32, orr);
+          tmem_wait_ld();
 #pragma unroll
-        for (int c4 = 0; c4 < 8; ++c4)
-          *reinterpret_cast<float4*>(so + c4 * 4) =
-              make_float4(__uint_as_float(orr[c4 * 4]), __uint_as_float(orr[c4 * 4 + 1]), __uint_as_float(orr[c4 * 4 + 2]),
-                          __uint_as_float(orr[c4 * 4 + 3]));
+          for (int c8 = 0; c8 < 4; ++c8) {
+            uint32_t pk[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const __half2 h2 = __floats2half2_rn(__uint_as_float(orr[c8 * 8 + 2 * e]) * inv_l,
+                                                   __uint_as_float(orr[c8 * 8 + 2 * e + 1]) * inv_l);
+              pk[e] = *reinterpret_cast<const uint32_t*>(&h2);
+            }
+            *reinterpret_cast<uint4*>(sh + hh * 32 + c8 * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          }
+        }
+      } else {
+#pragma unroll
+        for (int hh = 0; hh < 4; ++hh) {
+          uint32_t orr[32];
+          tmem_ld32(tmem_o + lane_sel + hh * 32, orr);
+          tmem_wait_ld();
+          float* so = stage_o + r * kStageStride + hh * 32;
+#pragma unroll
+          for (int c4 = 0; c4 < 8; ++c4)
+            *reinterpret_cast<float4*>(so + c4 * 4) =
+                make_float4(__uint_as_float(orr[c4 * 4]), __uint_as_float(orr[c4 * 4 + 1]), __uint_as_float(orr[c4 * 4 + 2]),
+                            __uint_as_float(orr[c4 * 4 + 3]));
+        }
       }
     }
     stage_ml[r * 2] = m_used * sc * 0.69314718055994531f;  // natural-log units (-inf: nothing visible)
