@@ -87,7 +87,7 @@ struct TcParams {
   int cs;   // CTAs per cluster (1..8); 0: no clusters, splits sized on the device and merged through global memory
   int rpc;  // cluster mode: row blocks a cluster covers at most (cs is a multiple of it)
   int nsplit_max, num_sms, nrb;  // global-merge mode
-  float* part_o;     // [B][Hq][Ncap][nsplit_max][D]
+  __half* part_o;    // [B][Hq][Ncap][nsplit_max][D]: partial rows normalised by their own sum, half precision
   float* part_ml;    // [B][Hq][Ncap][nsplit_max][2]
   int32_t* ticket;   // [B][Hkv][nrb]
   const int32_t* page_table;
@@ -528,7 +528,7 @@ template <int ROWS, int SPL>
 __device__ __forceinline__ void merge_rows_global(const TcParams& p, int b, int kvh, int row0, int rows_here, int nsplit) {
   const int lane = threadIdx.x & 31, wv = threadIdx.x >> 5, G = p.G;
   for (int rr = wv; rr < rows_here; rr += 8 * ROWS) {
-    float4 v[ROWS][SPL];
+    uint2 v[ROWS][SPL];
     float wgt[ROWS], inv[ROWS];
     size_t orow[ROWS];
 #pragma unroll
@@ -544,13 +544,13 @@ __device__ __forceinline__ void merge_rows_global(const TcParams& p, int b, int 
       }
 #pragma unroll
       for (int s2 = 0; s2 < SPL; ++s2)
-        v[u][s2] = s2 < nsplit ? __ldcg(reinterpret_cast<const float4*>(p.part_o + (pr + s2) * kHD + lane * 4))
-                               : make_float4(0.f, 0.f, 0.f, 0.f);
+        v[u][s2] = s2 < nsplit ? __ldcg(reinterpret_cast<const uint2*>(p.part_o + (pr + s2) * kHD + lane * 4))
+                               : make_uint2(0u, 0u);
       float M = ms;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-      wgt[u] = ms > -INFINITY ? expf(ms - M) : 0.f;
-      float lsum = ls * wgt[u];
+      wgt[u] = ms > -INFINITY ? ls * expf(ms - M) : 0.f;  // split s weighs sum_s * e^(max_s - max)
+      float lsum = wgt[u];
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
       inv[u] = lsum > 0.f ? 1.f / lsum : 0.f;
@@ -561,10 +561,14 @@ __device__ __forceinline__ void merge_rows_global(const TcParams& p, int b, int 
 #pragma unroll
       for (int s2 = 0; s2 < SPL; ++s2) {
         const float w = __shfl_sync(0xffffffffu, wgt[u], s2);
-        acc.x += v[u][s2].x * w;
-        acc.y += v[u][s2].y * w;
-        acc.z += v[u][s2].z * w;
-        acc.w += v[u][s2].w * w;
+        if (w > 0.f) {  // a split without visible positions wrote zeros at best
+          const float2 lo = __half22float2(*reinterpret_cast<const __half2*>(&v[u][s2].x));
+          const float2 hi = __half22float2(*reinterpret_cast<const __half2*>(&v[u][s2].y));
+          acc.x += lo.x * w;
+          acc.y += lo.y * w;
+          acc.z += hi.x * w;
+          acc.w += hi.y * w;
+        }
       }
       if (rr + 8 * u < rows_here) {
         const __nv_bfloat162 a = __floats2bfloat162_rn(acc.x * inv[u], acc.y * inv[u]),
@@ -1019,7 +1023,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     }
     if (ok && warp_live && ntile > 0) {
       tc_fence_after();
-      if (cs > 1 && nsplit > 1) {  // cluster merge: the row normalised by its own sum, in half precision
+      if (nsplit > 1) {  // to be merged with other splits: the row normalised by its own sum, in half precision
         const float inv_l = l_run > 0.f ? 1.f / l_run : 0.f;
         __half* sh = reinterpret_cast<__half*>(stage_o) + r * kStageStrideH;
 #pragma unroll
@@ -1081,24 +1085,26 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     }
   } else if (cs == 0) {
     // global-merge mode: partials to the workspace; the last split of this row block to finish merges
+    const __half* sh = reinterpret_cast<const __half*>(stage_o);
     for (int rr = warp; rr < rows_here; rr += kThreadsTC / 32) {
       const int grow = row0 + rr, tt = grow / G, hh = kvh * G + grow % G;
       const size_t pr = (((size_t)b * p.Hq + hh) * p.Ncap + tt) * p.nsplit_max + split;
-      __stcg(reinterpret_cast<float4*>(p.part_o + pr * kHD + lane * 4),
-             *reinterpret_cast<const float4*>(stage_o + rr * kStageStride + lane * 4));
+      __stcg(reinterpret_cast<uint2*>(p.part_o + pr * kHD + lane * 4),
+             *reinterpret_cast<const uint2*>(sh + rr * kStageStrideH + lane * 4));
       if (lane == 0) {
         __stcg(p.part_ml + pr * 2, stage_ml[rr * 2]);
         __stcg(p.part_ml + pr * 2 + 1, stage_ml[rr * 2 + 1]);
       }
     }
-    __threadfence();  // the partials must be visible before this CTA takes its ticket
     __syncthreads();
     if (tid == 0) {
+      // one acquire-release atomic at device scope: releases this CTA's partials (the barrier above made
+      // them this thread's to release), acquires those of the splits that finished earlier
       int32_t* cnt = p.ticket + ((size_t)b * p.Hkv + kvh) * p.nrb + rb;
-      const int t = atomicAdd(cnt, 1);
+      int t;
+      asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(t) : "l"(cnt) : "memory");
       *last_s = (t == nsplit - 1);
       if (t == nsplit - 1) *cnt = 0;  // ready for the next launch
-      __threadfence();
     }
     __syncthreads();
     if (*last_s) {
@@ -1227,7 +1233,7 @@ bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const v
       constexpr size_t kTicketBytes = (size_t)CAST_MAX_BATCH * 256 * sizeof(int32_t);
       const size_t rows = (size_t)B * Hq * Ncap * nsplit_max;
       if ((size_t)B * Hkv * nrb * sizeof(int32_t) > kTicketBytes) return false;
-      const size_t need = kTicketBytes + rows * (kHD + 2) * sizeof(float);
+      const size_t need = kTicketBytes + rows * (kHD * sizeof(__half) + 2 * sizeof(float));
       if (need > c->attn_tc_ws_bytes) {  // grows the workspace (synchronises; not legal during graph capture)
         if (cudaDeviceSynchronize() != cudaSuccess) { *status = CAST_ERR_CUDA; return true; }
         if (c->attn_tc_ws) cudaFree(c->attn_tc_ws);
@@ -1239,8 +1245,8 @@ bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const v
         c->attn_tc_ws_bytes = need;
       }
       p.ticket = reinterpret_cast<int32_t*>(c->attn_tc_ws);
-      p.part_o = reinterpret_cast<float*>(reinterpret_cast<char*>(c->attn_tc_ws) + kTicketBytes);
-      p.part_ml = p.part_o + rows * kHD;
+      p.part_o = reinterpret_cast<__half*>(reinterpret_cast<char*>(c->attn_tc_ws) + kTicketBytes);
+      p.part_ml = reinterpret_cast<float*>(p.part_o + rows * kHD);
     }
   }
   if (grid > 0x7fffffffll) return false;
