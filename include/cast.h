@@ -29,6 +29,10 @@
  *    Errors only the device can see (non-finite logits, a malformed tree, a
  *    page index out of range) are written to a device status word; read it with
  *    cast_poll_status, which synchronises `stream`.
+ *  - cast_tree_expand, cast_select_nodes and cast_tree_attention are launched with programmatic
+ *    dependent launch: their thread blocks may become resident while the previous kernel of the
+ *    stream is still finishing, but they read no input (logits, Q, K/V, tree arrays, lengths) before
+ *    that kernel has completed, so stream order keeps its usual meaning for the caller.
  *  - A context must not be used from two streams at once.
  *  - Row-major layouts, innermost index last, written as [d0, d1, ...].
  */
