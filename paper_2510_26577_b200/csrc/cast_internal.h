@@ -48,7 +48,7 @@ constexpr int kSweepThreads = 512;
 constexpr int kSweepEpt = 32;                             // logits per thread per pass
 constexpr int kSweepSub = kSweepThreads * kSweepEpt;      // logits per CTA per pass
 constexpr int kSweepMaxChunks = 8;                        // CTAs per logits row: one thread-block cluster
-constexpr int kCandCap = 4096;                            // candidate keys per CTA (floods take the slow exact path)
+constexpr int kCandCap = 4096;                            // 64-bit keys of shared scratch per CTA (warp lists, short list)
 constexpr int kMaxFifo = 64;
 constexpr int kAcceptMaxChunks = 32;
 

@@ -382,12 +382,12 @@ __device__ __forceinline__ void layer_tail(const ExpandParams& p, const TailStat
 
 template <typename T>
 __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParams p) {
-  __shared__ __align__(16) unsigned char scratch[kCandCap * 8];  // candidate keys; later the tail's arrays
+  __shared__ __align__(16) unsigned char scratch[kCandCap * 8];  // the warps' key lists and the short list; later the tail's arrays
   __shared__ unsigned long long topk[CAST_MAX_TOP_K];
   __shared__ float red_f[kSweepThreads / 32];
   __shared__ double red_d[kSweepThreads / 32];
   __shared__ int sorted[CAST_MAX_BATCH * CAST_MAX_WIDTH];
-  __shared__ int s_flag;
+  __shared__ int s_flag, short_n;
   // filled in the first CTA of the row's cluster by all CTAs of the cluster: chunk c's top-K keys
   // (descending), maximum (log2 units) and sum of 2^(. - maximum)
   __shared__ unsigned long long row_keys[kSweepMaxChunks * CAST_MAX_TOP_K];
@@ -585,7 +585,7 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
       red_d[warp] = sd;
     }
     if (tid < K) topk[tid] = 0ull;
-    if (tid == 0) s_flag = 0;  // length of the CTA's short list
+    if (tid == 0) short_n = 0;  // length of the CTA's short list
     __syncthreads();
     // The K-th largest of the warps' list heads bounds the CTA's top K from below (every list is in
     // descending order), so only keys at or above it can belong: a dozen or so. Every warp finds that
@@ -610,13 +610,13 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
       const bool keep = key != 0ull && key >= bound;
       const unsigned m = __ballot_sync(0xffffffffu, keep);
       int basepos = 0;
-      if (lane == 0 && m != 0u) basepos = atomicAdd(&s_flag, __popc(m));
+      if (lane == 0 && m != 0u) basepos = atomicAdd(&short_n, __popc(m));
       basepos = __shfl_sync(0xffffffffu, basepos, 0);
       if (keep) shortlist[basepos + __popc(m & ((1u << lane) - 1u))] = key;
     }
     __syncthreads();
     if (warp == 0) {
-      const int n = s_flag;  // <= kWarps * K = 256: up to 8 keys per lane
+      const int n = short_n;  // <= kWarps * K = 256: up to 8 keys per lane
 #pragma unroll 1
       for (int i0 = 0; i0 < n; i0 += 32) {
         const int i = i0 + lane;
