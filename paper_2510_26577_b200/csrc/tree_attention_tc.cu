@@ -5,9 +5,10 @@
 // tokens and all heads of the group. Tiles are 64 positions; a CTA needs 112 KB of shared memory
 // and 256 TMEM columns, so two CTAs share an SM: while one waits for a tile or runs its
 // prologue/epilogue, the other streams (128 registers per thread for that). Roles:
-//   TMA producer : K tiles and V tiles (128B-swizzled, two 64-column halves each) into two
-//                  2-stage rings; a K stage is released as soon as Q K^T has consumed it, a V
-//                  stage after P V.
+//   TMA producers: one warp loads the K tiles, another the V tiles (128B-swizzled, two 64-column
+//                  halves each) into two rings; a K stage is released as soon as Q K^T has
+//                  consumed it, a V stage after P V. (One warp for both rings stalled the K loads
+//                  behind waits for V stages: the paged batch-64 case went from 142 to 114 us with two.)
 //   MMA issuer   : S = Q K^T by tcgen05.mma (M=128 rows, N=64 positions, K=128) into one of two
 //                  TMEM buffers; once the softmax warps have written P, O += P V (V is the
 //                  MN-major B operand: used exactly as it lies in the cache, no transpose).
@@ -59,16 +60,17 @@ namespace {
 constexpr int kBM = 128;          // query rows per CTA (UMMA M)
 constexpr int kBN = 64;           // positions per tile
 constexpr int kHD = 128;          // head dim
-constexpr int kStages = 2;        // K ring and V ring
+constexpr int kStagesK = 2;       // tiles in the K ring
+constexpr int kStagesV = 2;       // tiles in the V ring
 constexpr int kSoftmaxThreads = 128;               // one thread per query row
 constexpr int kThreadsTC = 256;  // 4 softmax warps, TMA producer, MMA issuer, 2 idle: registers are allotted per 4 warps
 constexpr int kRegionQ = kBM * 128;                // [128 rows][64] bf16, 128-byte rows: 16 KB
 constexpr int kRegionKV = kBN * 128;               // [64 positions][64] bf16: 8 KB
 constexpr int kTileKV = 2 * kRegionKV;             // a [64][128] K or V tile: 16 KB
 constexpr int kSmemQ = 0;                          // 2 regions (d 0-63, d 64-127)
-constexpr int kSmemK = 2 * kRegionQ;               // kStages tiles
-constexpr int kSmemV = kSmemK + kStages * kTileKV; // kStages tiles
-constexpr int kSmemP = kSmemV + kStages * kTileKV; // one region [128 rows][64 positions]
+constexpr int kSmemK = 2 * kRegionQ;                 // kStagesK tiles
+constexpr int kSmemV = kSmemK + kStagesK * kTileKV;  // kStagesV tiles
+constexpr int kSmemP = kSmemV + kStagesV * kTileKV;  // one region [128 rows][64 positions]
 constexpr int kSmemBar = kSmemP + kRegionQ;        // mbarriers and two words, 128 bytes
 constexpr int kSmemBytes = kSmemBar + 128;         // 112 KB + 128 B: two CTAs per SM
 constexpr int kTmemCols = 256;                     // S0: [0,64), S1: [64,128), O: [128,256)
@@ -641,18 +643,19 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
   const int t_tok = row_ok ? row / G : 0, h_q = kvh * G + (row_ok ? row % G : 0);
 
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kSmemBar);
-  uint64_t* bar_fullk = bars;          // [kStages]
-  uint64_t* bar_fullv = bars + 2;      // [kStages]
-  uint64_t* bar_freek = bars + 4;      // [kStages]
-  uint64_t* bar_freev = bars + 6;      // [kStages]
-  uint64_t* bar_s = bars + 8;          // [2]
-  uint64_t* bar_p = bars + 10;
-  uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(bars + 11);
-  int* last_s = reinterpret_cast<int*>(bars + 12);
+  static_assert(kStagesK <= 3 && kStagesV <= 2, "barrier slots");
+  uint64_t* bar_fullk = bars;          // [kStagesK]
+  uint64_t* bar_fullv = bars + 3;      // [kStagesV]
+  uint64_t* bar_freek = bars + 5;      // [kStagesK]
+  uint64_t* bar_freev = bars + 8;      // [kStagesV]
+  uint64_t* bar_s = bars + 10;         // [2]
+  uint64_t* bar_p = bars + 12;
+  uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(bars + 13);
+  int* last_s = reinterpret_cast<int*>(bars + 14);
 
   // ---- producer helper (warp 4; all 32 lanes call it): which = 0: K tile j, which = 1: V tile j
   auto issue_tile = [&](int j, int which) -> bool {
-    const int stage = j % kStages;
+    const int stages = which ? kStagesV : kStagesK, stage = j % stages;
     unsigned char* dst = smem + (which ? kSmemV : kSmemK) + stage * kTileKV;
     uint64_t* full = which ? &bar_fullv[stage] : &bar_fullk[stage];
     const CUtensorMap* map = which ? &map_v : &map_k;
@@ -671,7 +674,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
         }
       }
     }
-    if (j >= kStages && !mbar_wait(which ? &bar_freev[stage] : &bar_freek[stage], ((j / kStages) - 1) & 1)) return false;
+    if (j >= stages && !mbar_wait(which ? &bar_freev[stage] : &bar_freek[stage], ((j / stages) - 1) & 1)) return false;
     if (ps == 0) {
       if (lane == 0) mbar_expect_tx(full, kTileKV);
       __syncwarp();
@@ -687,27 +690,36 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     __syncwarp();
     return true;
   };
-  // issue order K0 K1 V0 K2 V1 K3 V2 ...: the order in which the stages come free
-  auto issue_seq = [&](int i, int* armed_k, int* armed_v) -> bool {  // i-th element of that sequence
-    int j, which;
-    if (i == 0) { j = 0; which = 0; }
-    else if (i & 1) { j = (i + 1) / 2; which = 0; }
-    else { j = i / 2 - 1; which = 1; }
-    if (j >= ntile) return true;
-    if (!issue_tile(j, which)) return false;
-    if (which) *armed_v = j + 1; else *armed_k = j + 1;
-    return true;
+  // a producer warp fills its ring tile by tile (K: warp 4, V: warp 6); after an expired wait it reports,
+  // then waits (bounded) for its copies in flight, which must land before the CTA's shared memory is released
+  auto produce = [&](int which, int first) {
+    const int stages = which ? kStagesV : kStagesK;
+    int armed = first;
+    bool ok = true;
+    for (int j = first; j < ntile && ok; ++j) {
+      ok = issue_tile(j, which);
+      if (ok) armed = j + 1;
+    }
+    if (!ok) {
+      if (lane == 0) report(p.st, CAST_ERR_TIMEOUT, b);
+      for (int j = (armed > stages ? armed - stages : 0); j < armed; ++j) {
+        const long long tw = clock64();
+        while (!mbar_test(which ? &bar_fullv[j % stages] : &bar_fullk[j % stages], (j / stages) & 1) &&
+               clock64() - tw < kWaitCycles) {}
+      }
+    }
   };
+  int k_issued = 0;  // K tiles issued before the CTA barrier (they need no stage wait)
 
-  int armed_k = 0, armed_v = 0;
-  bool prod_ok = true;
   uint32_t aw[4] = {0u, 0u, 0u, 0u};  // softmax role: ancestor mask of this thread's row
   if (warp == 4) {
     if (lane == 0) {
-      for (int s = 0; s < kStages; ++s) {
+      for (int s = 0; s < kStagesK; ++s) {
         mbar_init(&bar_fullk[s], 1);
-        mbar_init(&bar_fullv[s], 1);
         mbar_init(&bar_freek[s], 1);
+      }
+      for (int s = 0; s < kStagesV; ++s) {
+        mbar_init(&bar_fullv[s], 1);
         mbar_init(&bar_freev[s], 1);
       }
       mbar_init(&bar_s[0], 1);
@@ -719,11 +731,8 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     __syncwarp();
     __threadfence_block();
     asm volatile("bar.arrive 2, %0;" ::"n"(kThreadsTC) : "memory");
-    // K0 K1 V0 V1 need no stage wait: the rings fill while the other warps stage Q
-    for (int i = 0; i < 5 && prod_ok; ++i) {
-      if (i == 3) continue;  // K2 waits for a stage; V1 (element 4) does not
-      prod_ok = issue_seq(i, &armed_k, &armed_v);
-    }
+    // the first K tiles need no stage wait: the ring fills while the other warps stage Q
+    for (; k_issued < kStagesK && k_issued < ntile; ++k_issued) issue_tile(k_issued, 0);
   } else if (warp < 4) {
     if (warp == 0) {  // TMEM: two S buffers and O
       asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_base_s)),
@@ -756,21 +765,11 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
   const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 2 * kBN;
 
   if (warp == 4) {
-    // =========================== TMA producer ===========================
-    bool ok = prod_ok;
-    if (ok) ok = issue_seq(3, &armed_k, &armed_v);  // K2
-    for (int i = 5; ok && i <= 2 * ntile; ++i) ok = issue_seq(i, &armed_k, &armed_v);
-    if (!ok) {  // drain: copies in flight must land before the CTA's shared memory is released
-      if (lane == 0) report(p.st, CAST_ERR_TIMEOUT, b);
-      for (int w = 0; w < 2; ++w) {
-        const int armed = w ? armed_v : armed_k;
-        for (int j = (armed > kStages ? armed - kStages : 0); j < armed; ++j) {
-          const long long tw = clock64();
-          while (!mbar_test(w ? &bar_fullv[j % kStages] : &bar_fullk[j % kStages], (j / kStages) & 1) &&
-                 clock64() - tw < kWaitCycles) {}
-        }
-      }
-    }
+    // =========================== TMA producer: K ring ===========================
+    produce(0, k_issued);
+  } else if (warp == 6) {
+    // =========================== TMA producer: V ring ===========================
+    produce(1, 0);
   } else if (warp == 5) {
     // =========================== MMA issuer ===========================
     const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
@@ -814,18 +813,18 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     for (int it = 0; ok && it < ntile; ++it) {
       TC_STAMP(1, it, 0);
       if (it + 1 < ntile) {
-        ok = mbar_wait(&bar_fullk[(it + 1) % kStages], ((it + 1) / kStages) & 1);
+        ok = mbar_wait(&bar_fullk[(it + 1) % kStagesK], ((it + 1) / kStagesK) & 1);
         if (!ok) break;
         TC_STAMP(1, it, 1);
         tc_fence_after();
-        mma_qk((it + 1) % kStages, (it + 1) & 1);
+        mma_qk((it + 1) % kStagesK, (it + 1) & 1);
         TC_STAMP(1, it, 2);
       }
-      ok = mbar_wait(bar_p, it & 1) && mbar_wait(&bar_fullv[it % kStages], (it / kStages) & 1);
+      ok = mbar_wait(bar_p, it & 1) && mbar_wait(&bar_fullv[it % kStagesV], (it / kStagesV) & 1);
       if (!ok) break;
       TC_STAMP(1, it, 3);
       tc_fence_after();
-      mma_pv(it % kStages, it == 0);
+      mma_pv(it % kStagesV, it == 0);
       TC_STAMP(1, it, 4);
     }
     if (!ok && lane == 0) report(p.st, CAST_ERR_TIMEOUT, b);
@@ -840,7 +839,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     float m_used = -INFINITY, l_run = 0.f;  // m_used: running reference maximum in raw score units
     bool ok = true;
     for (int it = 0; it < ntile; ++it) {
-      const int buf = it & 1, stage = it % kStages;
+      const int buf = it & 1, stage = it % kStagesV;
       const int pos0 = (t0 + it) * kBN;
       TC_STAMP(0, it, 0);
       float mx = -INFINITY;
@@ -851,7 +850,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
       // than 2^60 (seen as a huge P) is redone on the slow path below, which moves the reference.
       bool done = false;
       if (warp_live && ok && it > 0 && __all_sync(0xffffffffu, m_used > -INFINITY || !row_ok)) {
-        ok = mbar_wait(&bar_s[buf], (it >> 1) & 1) && mbar_wait(&bar_freev[(it - 1) % kStages], ((it - 1) / kStages) & 1);
+        ok = mbar_wait(&bar_s[buf], (it >> 1) & 1) && mbar_wait(&bar_freev[(it - 1) % kStagesV], ((it - 1) / kStagesV) & 1);
         if (ok) {
           tc_fence_after();
           const bool plain = pos0 + kBN <= L && __all_sync(0xffffffffu, row_ok);  // nothing masked in this warp
@@ -934,7 +933,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
       }
       // P (and O) were last touched by the P V product of tile it-1. Every warp waits here, live or not:
       // it also keeps a warp from arriving on bar_p for tile `it` before the phase of tile it-1 is over.
-      if (ok && it >= 1) ok = mbar_wait(&bar_freev[(it - 1) % kStages], ((it - 1) / kStages) & 1);
+      if (ok && it >= 1) ok = mbar_wait(&bar_freev[(it - 1) % kStagesV], ((it - 1) / kStagesV) & 1);
       TC_STAMP(0, it, 5);
       if (warp_live && !done) {
         if (ok) {
@@ -995,7 +994,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
       }
       // V rows past the end of the sequence may hold anything (0 * NaN would poison O): zero them
       if (ok && total - pos0 < kBN) {
-        ok = mbar_wait(&bar_fullv[stage], (it / kStages) & 1);  // the tile has landed
+        ok = mbar_wait(&bar_fullv[stage], (it / kStagesV) & 1);  // the tile has landed
         if (ok) {
           const int valid = total - pos0;
           unsigned char* vbase = smem + kSmemV + stage * kTileKV;
@@ -1015,7 +1014,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     // shared memory (the K/V rings, P and Q are idle now): the output rows are written, or merged
     // across the splits, from there in contiguous pieces
     TC_MARK(4);
-    if (ok && ntile > 0) ok = mbar_wait(&bar_freev[(ntile - 1) % kStages], ((ntile - 1) / kStages) & 1);
+    if (ok && ntile > 0) ok = mbar_wait(&bar_freev[(ntile - 1) % kStagesV], ((ntile - 1) / kStagesV) & 1);
     TC_MARK(5);
     if (!ok) {  // a wait ran out: this split contributes nothing
       m_used = -INFINITY;
