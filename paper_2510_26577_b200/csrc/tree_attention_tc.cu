@@ -3,20 +3,24 @@
 // One CTA owns (sequence b, kv-head, block of 128 query rows, KV split). A query row is a
 // (tree token, head of the GQA group) pair, so every K/V tile is fetched once for all tree
 // tokens and all heads of the group. Tiles are 64 positions; a CTA needs 112 KB of shared memory
-// and 256 TMEM columns, so two CTAs share an SM: while one waits for a tile or runs its
-// prologue/epilogue, the other streams (128 registers per thread for that). Roles:
+// (Q 32 KB, a ring of three K tiles, a ring of two V tiles) and 256 TMEM columns (two score
+// buffers of 64, the output accumulator of 128), so two CTAs share an SM: while one waits for a
+// tile or runs its prologue/epilogue, the other streams (128 registers per thread for that). Roles:
 //   TMA producers: one warp loads the K tiles, another the V tiles (128B-swizzled, two 64-column
-//                  halves each) into two rings; a K stage is released as soon as Q K^T has
+//                  halves each) into the two rings; a K stage is released as soon as Q K^T has
 //                  consumed it, a V stage after P V. (One warp for both rings stalled the K loads
 //                  behind waits for V stages: the paged batch-64 case went from 142 to 114 us with two.)
 //   MMA issuer   : S = Q K^T by tcgen05.mma (M=128 rows, N=64 positions, K=128) into one of two
-//                  TMEM buffers; once the softmax warps have written P, O += P V (V is the
-//                  MN-major B operand: used exactly as it lies in the cache, no transpose).
-//                  Q K^T of tile i+1 is issued before P of tile i is awaited.
+//                  TMEM buffers; once the softmax warps have written P, O += P V with P taken
+//                  from tensor memory (A operand in TMEM) and V as the MN-major B operand: used
+//                  exactly as it lies in the cache, no transpose. Q K^T of tile i+1 is issued
+//                  before P of tile i is awaited.
 //   4 softmax warps: one thread per query row reads its 64 scores with tcgen05.ld, applies the
-//                  prefix/ancestor mask (only tiles that reach past the prefix need one), keeps a
-//                  lazily updated row maximum (O in TMEM is rescaled only when the maximum grows
-//                  by more than 2^8), writes P as bf16 into swizzled shared memory.
+//                  prefix/ancestor mask (only tiles that reach past the prefix need one) and
+//                  writes P = 2^((s - m) * scale) as bf16 over the scores, in tensor memory
+//                  (tcgen05.st). The first tile takes two passes (row maximum, then P); later
+//                  tiles one pass with the reference maximum of the earlier ones (O in TMEM is
+//                  rescaled only if a row's P outgrows 2^60, by a power of two).
 // The kernel is launched in thread-block clusters: a cluster covers the row blocks of one
 // (sequence, kv-head) and splits each one's KV range over its CTAs, the number of splits per row
 // block being decided on the device from the actual tree size (the host only knows the largest
@@ -60,19 +64,18 @@ namespace {
 constexpr int kBM = 128;          // query rows per CTA (UMMA M)
 constexpr int kBN = 64;           // positions per tile
 constexpr int kHD = 128;          // head dim
-constexpr int kStagesK = 2;       // tiles in the K ring
+constexpr int kStagesK = 3;       // tiles in the K ring
 constexpr int kStagesV = 2;       // tiles in the V ring
 constexpr int kSoftmaxThreads = 128;               // one thread per query row
-constexpr int kThreadsTC = 256;  // 4 softmax warps, TMA producer, MMA issuer, 2 idle: registers are allotted per 4 warps
+constexpr int kThreadsTC = 256;  // 4 softmax warps, K producer, MMA issuer, V producer, 1 idle: registers are allotted per 4 warps
 constexpr int kRegionQ = kBM * 128;                // [128 rows][64] bf16, 128-byte rows: 16 KB
 constexpr int kRegionKV = kBN * 128;               // [64 positions][64] bf16: 8 KB
 constexpr int kTileKV = 2 * kRegionKV;             // a [64][128] K or V tile: 16 KB
 constexpr int kSmemQ = 0;                          // 2 regions (d 0-63, d 64-127)
 constexpr int kSmemK = 2 * kRegionQ;                 // kStagesK tiles
 constexpr int kSmemV = kSmemK + kStagesK * kTileKV;  // kStagesV tiles
-constexpr int kSmemP = kSmemV + kStagesV * kTileKV;  // one region [128 rows][64 positions]
-constexpr int kSmemBar = kSmemP + kRegionQ;        // mbarriers and two words, 128 bytes
-constexpr int kSmemBytes = kSmemBar + 128;         // 112 KB + 128 B: two CTAs per SM
+constexpr int kSmemBar = kSmemV + kStagesV * kTileKV;  // mbarriers and two words, 128 bytes
+constexpr int kSmemBytes = kSmemBar + 128;           // 112 KB + 128 B: two CTAs per SM
 constexpr int kTmemCols = 256;                     // S0: [0,64), S1: [64,128), O: [128,256)
 constexpr float kRescaleThreshold = 8.0f;          // log2 units
 constexpr long long kWaitCycles = 4000000000ll;    // about two seconds
@@ -167,6 +170,16 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
       ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
       : "memory");
 }
+// D[tmem] (+)= A[tmem] * B[smem]: the A operand (128 rows, one per TMEM lane; 16 bf16 of the K extent
+// packed two to a 32-bit column, 8 columns per instruction) comes from tensor memory.
+__device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
@@ -192,6 +205,23 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
         "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
         "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
         "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
       : "memory");
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -779,7 +809,6 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     const uint64_t dq = umma_desc(smem_u32(smem + kSmemQ), 16, 1024);
     const uint64_t dk = umma_desc(smem_u32(smem + kSmemK), 16, 1024);
     const uint64_t dv = umma_desc(smem_u32(smem + kSmemV), kRegionKV, 1024);
-    const uint64_t dp = umma_desc(smem_u32(smem + kSmemP), 16, 1024);
     auto mma_qk = [&](int stage, int buf) {  // S[buf] = Q K^T; releases the K stage
       if (lane == 0) {
         const uint64_t dks = dk + (uint64_t)(stage * (kTileKV >> 4));
@@ -792,13 +821,13 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
       }
       __syncwarp();
     };
-    auto mma_pv = [&](int stage, bool first) {  // O (+)= P V; releases the V stage (and P)
+    auto mma_pv = [&](int stage, int buf, bool first) {  // O (+)= P V, P from tensor memory; releases the V stage
       if (lane == 0) {
         const uint64_t dvs = dv + (uint64_t)(stage * (kTileKV >> 4));
 #pragma unroll
         for (int ks = 0; ks < kBN / 16; ++ks)
-          umma_bf16(tmem_o, dp + (uint64_t)(ks * 2), dvs + (uint64_t)(ks * (2048 >> 4)), idesc_pv,
-                    (!first || ks > 0) ? 1u : 0u);
+          umma_bf16_ts(tmem_o, tmem_s + buf * kBN + ks * 8, dvs + (uint64_t)(ks * (2048 >> 4)), idesc_pv,
+                       (!first || ks > 0) ? 1u : 0u);
         umma_commit(&bar_freev[stage]);
       }
       __syncwarp();
@@ -824,7 +853,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
       if (!ok) break;
       TC_STAMP(1, it, 3);
       tc_fence_after();
-      mma_pv(it % kStagesV, it == 0);
+      mma_pv(it % kStagesV, it & 1, it == 0);
       TC_STAMP(1, it, 4);
     }
     if (!ok && lane == 0) report(p.st, CAST_ERR_TIMEOUT, b);
@@ -846,9 +875,12 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
       uint32_t v0 = 0xffffffffu, v1 = 0xffffffffu;  // visibility of this row's 64 columns
       // Fast path (every tile but the first, as a rule): one pass over the scores with the reference
       // maximum of the earlier tiles. P = 2^((s - m) * scale) is then not bounded by 1, but bf16 and the
-      // fp32 accumulators have the range for it; only a tile whose scores outgrow the reference by more
-      // than 2^60 (seen as a huge P) is redone on the slow path below, which moves the reference.
+      // fp32 accumulators have the range for it; a row whose P outgrows 2^60 moves its reference
+      // afterwards (P, the row sum and O are scaled by a power of two: exact).
+      // P is written over the scores it came from, in tensor memory: 64 bf16 = 32 columns of this row's
+      // lane; P V takes its A operand from there.
       bool done = false;
+      const uint32_t tp = tmem_s + buf * kBN + lane_sel;
       if (warp_live && ok && it > 0 && __all_sync(0xffffffffu, m_used > -INFINITY || !row_ok)) {
         ok = mbar_wait(&bar_s[buf], (it >> 1) & 1) && mbar_wait(&bar_freev[(it - 1) % kStagesV], ((it - 1) / kStagesV) & 1);
         if (ok) {
@@ -863,40 +895,68 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
           }
           const float neg_ms = row_ok ? -m_used * sc : 0.f;
           float l0 = 0.f, l1 = 0.f, pmax = 0.f;
-          unsigned char* prow = smem + kSmemP;
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {
-            uint32_t sr[32];
-            tmem_ld32(tmem_s + buf * kBN + lane_sel + hh * 32, sr);
+            uint32_t sr[32], pk[16];
+            tmem_ld32(tp + hh * 32, sr);
             tmem_wait_ld();
             const uint32_t vv = hh ? v1 : v0;
 #pragma unroll
-            for (int c8 = 0; c8 < 4; ++c8) {
-              uint32_t pk[4];
+            for (int e = 0; e < 16; ++e) {
+              const int c = 2 * e;
+              float p0 = fast_exp2(fmaf(__uint_as_float(sr[c]), sc, neg_ms));
+              float p1 = fast_exp2(fmaf(__uint_as_float(sr[c + 1]), sc, neg_ms));
+              if (!plain) {
+                p0 = ((vv >> c) & 1u) ? p0 : 0.f;
+                p1 = ((vv >> (c + 1)) & 1u) ? p1 : 0.f;
+              }
+              l0 += p0;
+              l1 += p1;
+              pmax = fmaxf(pmax, fmaxf(p0, p1));
+              const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+              pk[e] = *reinterpret_cast<const uint32_t*>(&pb);
+            }
+            tmem_st16(tp + hh * 16, pk);
+          }
+          if (__any_sync(0xffffffffu, pmax >= 1.15e18f)) {  // 2^60: rare. Move the reference of the rows concerned.
+            tmem_wait_st();
+            float alpha = 1.f;
+            if (pmax >= 1.15e18f && pmax < INFINITY) {
+              int e2;
+              frexpf(pmax, &e2);
+              alpha = ldexpf(1.f, 1 - e2);  // 2^-floor(log2 pmax)
+            }
+#pragma unroll 1
+            for (int hh = 0; hh < 2; ++hh) {
+              uint32_t pk[16];
+              tmem_ld16(tp + hh * 16, pk);
+              tmem_wait_ld();
 #pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const int c = c8 * 8 + 2 * e;
-                float p0 = fast_exp2(fmaf(__uint_as_float(sr[c]), sc, neg_ms));
-                float p1 = fast_exp2(fmaf(__uint_as_float(sr[c + 1]), sc, neg_ms));
-                if (!plain) {
-                  p0 = ((vv >> c) & 1u) ? p0 : 0.f;
-                  p1 = ((vv >> (c + 1)) & 1u) ? p1 : 0.f;
-                }
-                l0 += p0;
-                l1 += p1;
-                pmax = fmaxf(pmax, fmaxf(p0, p1));
-                const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+              for (int e = 0; e < 16; ++e) {
+                const float lo = __uint_as_float(pk[e] << 16) * alpha, hi = __uint_as_float(pk[e] & 0xffff0000u) * alpha;
+                const __nv_bfloat162 pb = __floats2bfloat162_rn(lo, hi);
                 pk[e] = *reinterpret_cast<const uint32_t*>(&pb);
               }
-              *reinterpret_cast<uint4*>(prow + swz(r, hh * 4 + c8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+              tmem_st16(tp + hh * 16, pk);
             }
+#pragma unroll 1
+            for (int hh = 0; hh < 4; ++hh) {  // O and the running sum follow (P V of tile it-1 is over)
+              uint32_t orr[32];
+              const uint32_t ta = tmem_o + lane_sel + hh * 32;
+              tmem_ld32(ta, orr);
+              tmem_wait_ld();
+#pragma unroll
+              for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
+              tmem_st32(ta, orr);
+            }
+            l0 *= alpha;
+            l1 *= alpha;
+            l_run *= alpha;
+            if (alpha < 1.f) m_used -= log2f(alpha) / sc;
           }
-          if (!__any_sync(0xffffffffu, !(pmax < 1.15e18f))) {  // 2^60; a NaN score also takes the slow path
-            l_run += l0 + l1;
-            done = true;
-          } else {
-            v0 = v1 = 0xffffffffu;
-          }
+          tmem_wait_st();
+          l_run += l0 + l1;
+          done = true;
         }
       }
       if (warp_live && !done) {
@@ -960,35 +1020,31 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
             tmem_wait_st();
           }
           TC_STAMP(0, it, 6);
-          // pass 2: P = 2^((s - m) * scale) as bf16 into the swizzled A-operand buffer; row sum in fp32
+          // pass 2: P = 2^((s - m) * scale) as bf16 over the scores in tensor memory; row sum in fp32
           const bool live = m_used > -INFINITY;
           const float neg_ms = live ? -m_used * sc : 0.f;
           float l0 = 0.f, l1 = 0.f;
-          unsigned char* prow = smem + kSmemP;
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {
-            uint32_t sr[32];
-            tmem_ld32(tmem_s + buf * kBN + lane_sel + hh * 32, sr);
+            uint32_t sr[32], pk[16];
+            tmem_ld32(tp + hh * 32, sr);
             tmem_wait_ld();
             const uint32_t vv = live ? (hh ? v1 : v0) : 0u;
 #pragma unroll
-            for (int c8 = 0; c8 < 4; ++c8) {
-              uint32_t pk[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const int c = c8 * 8 + 2 * e;
-                float p0 = fast_exp2(fmaf(__uint_as_float(sr[c]), sc, neg_ms));
-                float p1 = fast_exp2(fmaf(__uint_as_float(sr[c + 1]), sc, neg_ms));
-                p0 = ((vv >> c) & 1u) ? p0 : 0.f;
-                p1 = ((vv >> (c + 1)) & 1u) ? p1 : 0.f;
-                l0 += p0;
-                l1 += p1;
-                const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
-                pk[e] = *reinterpret_cast<const uint32_t*>(&pb);
-              }
-              *reinterpret_cast<uint4*>(prow + swz(r, hh * 4 + c8)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            for (int e = 0; e < 16; ++e) {
+              const int c = 2 * e;
+              float p0 = fast_exp2(fmaf(__uint_as_float(sr[c]), sc, neg_ms));
+              float p1 = fast_exp2(fmaf(__uint_as_float(sr[c + 1]), sc, neg_ms));
+              p0 = ((vv >> c) & 1u) ? p0 : 0.f;
+              p1 = ((vv >> (c + 1)) & 1u) ? p1 : 0.f;
+              l0 += p0;
+              l1 += p1;
+              const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+              pk[e] = *reinterpret_cast<const uint32_t*>(&pb);
             }
+            tmem_st16(tp + hh * 16, pk);
           }
+          tmem_wait_st();
           l_run += l0 + l1;
         }
       }
