@@ -875,7 +875,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
       uint32_t v0 = 0xffffffffu, v1 = 0xffffffffu;  // visibility of this row's 64 columns
       // Fast path (every tile but the first, as a rule): one pass over the scores with the reference
       // maximum of the earlier tiles. P = 2^((s - m) * scale) is then not bounded by 1, but bf16 and the
-      // fp32 accumulators have the range for it; a row whose P outgrows 2^60 moves its reference
+      // fp32 accumulators have the range for it; a row whose sum of P outgrows 2^60 moves its reference
       // afterwards (P, the row sum and O are scaled by a power of two: exact).
       // P is written over the scores it came from, in tensor memory: 64 bf16 = 32 columns of this row's
       // lane; P V takes its A operand from there.
@@ -894,7 +894,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
             if (!row_ok) v0 = v1 = 0u;
           }
           const float neg_ms = row_ok ? -m_used * sc : 0.f;
-          float l0 = 0.f, l1 = 0.f, pmax = 0.f;
+          float l0 = 0.f, l1 = 0.f;
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {
             uint32_t sr[32], pk[16];
@@ -912,19 +912,19 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
               }
               l0 += p0;
               l1 += p1;
-              pmax = fmaxf(pmax, fmaxf(p0, p1));
               const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
               pk[e] = *reinterpret_cast<const uint32_t*>(&pb);
             }
             tmem_st16(tp + hh * 16, pk);
           }
-          if (__any_sync(0xffffffffu, pmax >= 1.15e18f)) {  // 2^60: rare. Move the reference of the rows concerned.
+          const float lt = l0 + l1;  // every P of the row is at most this
+          if (__any_sync(0xffffffffu, lt >= 1.15e18f)) {  // 2^60: rare. Move the reference of the rows concerned.
             tmem_wait_st();
             float alpha = 1.f;
-            if (pmax >= 1.15e18f && pmax < INFINITY) {
+            if (lt >= 1.15e18f && lt < INFINITY) {
               int e2;
-              frexpf(pmax, &e2);
-              alpha = ldexpf(1.f, 1 - e2);  // 2^-floor(log2 pmax)
+              frexpf(lt, &e2);
+              alpha = ldexpf(1.f, 1 - e2);  // 2^-floor(log2 of the row sum)
             }
 #pragma unroll 1
             for (int hh = 0; hh < 2; ++hh) {
