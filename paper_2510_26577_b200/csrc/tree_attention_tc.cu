@@ -226,6 +226,26 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// Packed fp32 pairs (one instruction, two lanes of the FMA pipe): the softmax's inner loop is bound by
+// instruction issue, and its multiply-add and its running sum pair up naturally.
+__device__ __forceinline__ unsigned long long pack_f2(float a, float b) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack_f2(unsigned long long v, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long fma_f2(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ unsigned long long add_f2(unsigned long long a, unsigned long long b) {
+  unsigned long long r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -894,7 +914,8 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
             if (!row_ok) v0 = v1 = 0u;
           }
           const float neg_ms = row_ok ? -m_used * sc : 0.f;
-          float l0 = 0.f, l1 = 0.f;
+          const unsigned long long sc2 = pack_f2(sc, sc), neg2 = pack_f2(neg_ms, neg_ms);
+          unsigned long long lacc = pack_f2(0.f, 0.f);
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {
             uint32_t sr[32], pk[16];
@@ -904,19 +925,21 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
 #pragma unroll
             for (int e = 0; e < 16; ++e) {
               const int c = 2 * e;
-              float p0 = fast_exp2(fmaf(__uint_as_float(sr[c]), sc, neg_ms));
-              float p1 = fast_exp2(fmaf(__uint_as_float(sr[c + 1]), sc, neg_ms));
+              float x0, x1;
+              unpack_f2(fma_f2(pack_f2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, neg2), x0, x1);
+              float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
               if (!plain) {
                 p0 = ((vv >> c) & 1u) ? p0 : 0.f;
                 p1 = ((vv >> (c + 1)) & 1u) ? p1 : 0.f;
               }
-              l0 += p0;
-              l1 += p1;
+              lacc = add_f2(lacc, pack_f2(p0, p1));
               const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
               pk[e] = *reinterpret_cast<const uint32_t*>(&pb);
             }
             tmem_st16(tp + hh * 16, pk);
           }
+          float l0, l1;
+          unpack_f2(lacc, l0, l1);
           const float lt = l0 + l1;  // every P of the row is at most this
           if (__any_sync(0xffffffffu, lt >= 1.15e18f)) {  // 2^60: rare. Move the reference of the rows concerned.
             tmem_wait_st();
