@@ -699,9 +699,9 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
   uint64_t* bar_freek = bars + 5;      // [kStagesK]
   uint64_t* bar_freev = bars + 8;      // [kStagesV]
   uint64_t* bar_s = bars + 10;         // [2]
-  uint64_t* bar_p = bars + 12;
-  uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(bars + 13);
-  int* last_s = reinterpret_cast<int*>(bars + 14);
+  uint64_t* bar_p = bars + 12;         // [2]: tile it uses bar_p[it & 1], phase it >> 1
+  uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(bars + 14);
+  int* last_s = reinterpret_cast<int*>(bars + 15);
 
   // ---- producer helper (warp 4; all 32 lanes call it): which = 0: K tile j, which = 1: V tile j
   auto issue_tile = [&](int j, int which) -> bool {
@@ -774,7 +774,8 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
       }
       mbar_init(&bar_s[0], 1);
       mbar_init(&bar_s[1], 1);
-      mbar_init(bar_p, kSoftmaxThreads);
+      mbar_init(&bar_p[0], kSoftmaxThreads);
+      mbar_init(&bar_p[1], kSoftmaxThreads);
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       fence_proxy_async();
     }
@@ -869,7 +870,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
         mma_qk((it + 1) % kStagesK, (it + 1) & 1);
         TC_STAMP(1, it, 2);
       }
-      ok = mbar_wait(bar_p, it & 1) && mbar_wait(&bar_fullv[it % kStagesV], (it / kStagesV) & 1);
+      ok = mbar_wait(&bar_p[it & 1], (it >> 1) & 1) && mbar_wait(&bar_fullv[it % kStagesV], (it / kStagesV) & 1);
       if (!ok) break;
       TC_STAMP(1, it, 3);
       tc_fence_after();
@@ -902,7 +903,10 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
       bool done = false;
       const uint32_t tp = tmem_s + buf * kBN + lane_sel;
       if (warp_live && ok && it > 0 && __all_sync(0xffffffffu, m_used > -INFINITY || !row_ok)) {
-        ok = mbar_wait(&bar_s[buf], (it >> 1) & 1) && mbar_wait(&bar_freev[(it - 1) % kStagesV], ((it - 1) / kStagesV) & 1);
+        // Nothing but the scores is awaited: P goes into the score buffer it came from, and that buffer
+        // was last read by P V of tile it-2, which the tensor pipe finished before it produced these
+        // scores. So the softmax of this tile runs while P V of the previous one does.
+        ok = mbar_wait(&bar_s[buf], (it >> 1) & 1);
         if (ok) {
           tc_fence_after();
           const bool plain = pos0 + kBN <= L && __all_sync(0xffffffffu, row_ok);  // nothing masked in this warp
@@ -941,7 +945,9 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
           float l0, l1;
           unpack_f2(lacc, l0, l1);
           const float lt = l0 + l1;  // every P of the row is at most this
-          if (__any_sync(0xffffffffu, lt >= 1.15e18f)) {  // 2^60: rare. Move the reference of the rows concerned.
+          if (__any_sync(0xffffffffu, lt >= 1.15e18f) &&  // 2^60: rare. Move the reference of the rows concerned
+              mbar_wait(&bar_freev[(it - 1) % kStagesV], ((it - 1) / kStagesV) & 1)) {  // (O must be at rest)
+            tc_fence_after();
             tmem_wait_st();
             float alpha = 1.f;
             if (lt >= 1.15e18f && lt < INFINITY) {
@@ -1014,9 +1020,13 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
         }
         TC_STAMP(0, it, 3);
       }
-      // P (and O) were last touched by the P V product of tile it-1. Every warp waits here, live or not:
-      // it also keeps a warp from arriving on bar_p for tile `it` before the phase of tile it-1 is over.
-      if (ok && it >= 1) ok = mbar_wait(&bar_freev[(it - 1) % kStagesV], ((it - 1) / kStagesV) & 1);
+      // The two-pass path may rescale O, which P V of tile it-1 must have left. A warp without live rows
+      // only has to stay in step: it waits for this tile's scores like the others, so that it cannot
+      // arrive on bar_p[it & 1] before the phase of tile it-2 is over.
+      if (ok && it >= 1 && !(warp_live && done)) {
+        ok = warp_live ? mbar_wait(&bar_freev[(it - 1) % kStagesV], ((it - 1) / kStagesV) & 1)
+                       : mbar_wait(&bar_s[buf], (it >> 1) & 1);
+      }
       TC_STAMP(0, it, 5);
       if (warp_live && !done) {
         if (ok) {
@@ -1086,7 +1096,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
       TC_STAMP(0, it, 7);
       fence_proxy_async();
       tc_fence_before();
-      mbar_arrive(bar_p);
+      mbar_arrive(&bar_p[it & 1]);
       TC_STAMP(0, it, 9);
     }
     // epilogue: wait for the last P V, then stage O (fp32, unnormalised) and (max, sum) per row in
