@@ -27,7 +27,8 @@ METRIC, UNIT = "tree_verify_tokens_per_s", "tokens/s"
 
 # DRAM bytes (read + write) of one tree_attn_tc_kernel launch from the ncu captures summarised
 # under profiles/ (same launch shape as one layer of the workload).
-NCU_ATTENTION_TRAFFIC = {"c2_llama8b": 9.25e6, "c3_llama8b_b16": 143e6, "c3_llama8b_b64": 583e6}
+NCU_ATTENTION_TRAFFIC = {"c2_llama8b": 9.24e6, "c3_llama8b_b16": 142.4e6, "c3_llama8b_b64": 582.6e6,
+                         "c4_llama70b_n128": 181.8e6}
 
 
 def peaks():
