@@ -15,6 +15,7 @@ from .cast_oracle import (  # noqa: F401
     log_sum_exp,
     tree_attention,
     greedy_accept,
+    stochastic_accept,
     compact_kv,
     ancestor_masks,
 )

@@ -16,7 +16,10 @@ Theorem's linear-cost special case in exact rational arithmetic; select() on a
 hand table; expansion and rerank against brute-force enumeration of all paths
 on tiny vocabularies; attention against separately coded causal attention on a
 chain tree and against per-path dense attention; acceptance against sequential
-token-by-token decoding; compaction against an out-of-place gather.
+token-by-token decoding; stochastic acceptance against a hand-worked case, the
+greedy rule for a one-hot target, the all-accept case P_T = P_D and the
+output-distribution-equals-P_T property on sampled trees; compaction against an
+out-of-place gather.
 Parity unpinned: the FIFO length R, the split of the paper's single reported
 "threshold" into C1, C2, C3, and the cost-table contents - the paper prints no
 value for any of them, so they are parameters here, not results.
@@ -407,6 +410,76 @@ def greedy_accept(target_logits, tokens, parent, n_tree, max_depth):
         accept_path[b, : len(path)] = path
         bonus[b] = g[cur]
     return accept_len, accept_path, bonus
+
+
+# --------------------------------------------------------------------------
+# Stochastic acceptance at temperature T > 0 (Section "Speculative Decoding").
+# The paper states the rule for a chain: draft token x with q = P_D(x | .),
+# p = P_T(x | .) and u ~ Uniform(0,1) is accepted iff u <= min(1, p/q);
+# otherwise decoding falls back to a sample of norm(max(0, P_T - P_D)).
+# Reading for a tree (the paper only says that the siblings of a rejected token
+# stay in play): at a node the children are tried in tree order; after a
+# rejection P_T is replaced by the residual norm(max(0, P_T - P_D)) and the next
+# sibling is tried against that, P_D unchanged (children are draws from P_D);
+# when no child is left the bonus token is drawn from the distribution that
+# stands then - the target distribution at a leaf, a residual otherwise - by
+# inversion of its cumulative sum in token order.  A residual that sums to zero
+# (reachable only through a rejection of probability zero) ends the sibling
+# loop with the distribution before it.
+# The random numbers are inputs: u_accept[b, c] decides tree node c, u_bonus[b]
+# draws the bonus token.
+# Besides the results, the smallest distance of a decision from its threshold
+# is returned (relative), so that a comparison with another implementation can
+# tell a wrong result from a rounding-order coin flip.
+# --------------------------------------------------------------------------
+def _softmax_t(logits, T):
+    s = np.asarray(logits, dtype=np.float64) / T
+    e = np.exp(s - np.max(s))
+    return e / np.sum(e)
+
+
+def stochastic_accept(target_logits, draft_logits, tokens, parent, n_tree, max_depth, temperature, u_accept, u_bonus):
+    B = tokens.shape[0]
+    accept_len = np.zeros((B,), dtype=np.int32)
+    accept_path = np.full((B, max_depth + 1), -1, dtype=np.int32)
+    bonus = np.zeros((B,), dtype=np.int32)
+    margin = np.full((B,), np.inf)
+    for b in range(B):
+        N = int(n_tree[b])
+        cur, path = 0, [0]
+        while True:
+            p = _softmax_t(target_logits[b, cur], temperature)  # P_T(. | path to cur)
+            children = [c for c in range(N) if parent[b, c] == cur]
+            nxt = -1
+            if children:
+                q = _softmax_t(draft_logits[b, cur], temperature)  # P_D(. | path to cur)
+                for c in children:
+                    x = int(tokens[b, c])
+                    ratio = min(1.0, p[x] / q[x]) if q[x] > 0.0 else 1.0
+                    u = float(u_accept[b, c])
+                    if ratio < 1.0:
+                        margin[b] = min(margin[b], abs(u - ratio))
+                    if u <= ratio:
+                        nxt = c
+                        break
+                    residual = np.maximum(0.0, p - q)
+                    total = np.sum(residual)
+                    if not total > 0.0:
+                        break
+                    p = residual / total
+            if nxt < 0:
+                break
+            cur = nxt
+            path.append(cur)
+        cdf = np.cumsum(p)
+        goal = float(u_bonus[b]) * cdf[-1]
+        x = int(np.argmax(cdf >= goal))  # first token whose cumulative sum reaches the goal
+        below = cdf[x - 1] if x > 0 else 0.0
+        margin[b] = min(margin[b], (cdf[x] - goal) / cdf[-1], (goal - below) / cdf[-1])
+        accept_len[b] = len(path) - 1
+        accept_path[b, : len(path)] = path
+        bonus[b] = x
+    return accept_len, accept_path, bonus, margin
 
 
 # --------------------------------------------------------------------------

@@ -22,6 +22,7 @@ from oracle import (
     greedy_accept,
     log_sum_exp,
     select_grid,
+    stochastic_accept,
     topk_children,
     tree_attention,
 )
@@ -463,6 +464,128 @@ def test_greedy_accept_edge_cases():
     # nodes beyond n_tree are invisible
     al, ap, bo = greedy_accept(logits, tokens, parent, np.array([3]), 4)
     assert (al[0], bo[0]) == (1, 5)
+
+
+# ------------------------------------------------------ stochastic acceptance
+def test_stochastic_accept_hand_worked_chain_and_sibling():
+    """P_T = (0.5, 0.3, 0.2), P_D = (0.2, 0.5, 0.3) at the root. A child with token 1 is accepted iff
+    u <= 0.3/0.5; after its rejection the residual is norm(max(0, P_T - P_D)) = (1, 0, 0): a sibling
+    with token 0 is then accepted for every u (ratio 1/0.2 > 1), one with token 2 never, and a bonus
+    token drawn there is token 0 for every u."""
+    lt = np.log(np.array([0.5, 0.3, 0.2]))
+    ld = np.log(np.array([0.2, 0.5, 0.3]))
+    leaf = np.log(np.array([0.1, 0.2, 0.7]))  # target distribution at every non-root node
+    T = 1.0
+    tl = np.stack([lt, leaf, leaf, leaf])[None]
+    dl = np.stack([ld, ld, ld, ld])[None]
+
+    def run(tokens, parent, ua, ub):
+        al, ap, bo, _ = stochastic_accept(tl, dl, np.array([tokens], dtype=np.int32), np.array([parent]),
+                                          np.array([len(tokens)]), 3, T, np.array([ua]), np.array([ub]))
+        return int(al[0]), [int(x) for x in ap[0]], int(bo[0])
+
+    # chain root -> token 1: accepted just below the ratio 0.6, bonus from the leaf's (0.1, 0.2, 0.7) by inversion
+    assert run([9, 1], [-1, 0], [0.0, 0.59], 0.05) == (1, [0, 1, -1, -1], 0)
+    assert run([9, 1], [-1, 0], [0.0, 0.59], 0.25) == (1, [0, 1, -1, -1], 1)
+    assert run([9, 1], [-1, 0], [0.0, 0.59], 0.31) == (1, [0, 1, -1, -1], 2)
+    # rejected just above it: bonus from the residual (1, 0, 0)
+    for ub in (0.01, 0.5, 0.99):
+        assert run([9, 1], [-1, 0], [0.0, 0.61], ub) == (0, [0, -1, -1, -1], 0)
+    # siblings in tree order: token 1 rejected, then token 2 (residual probability 0) rejected, then token 0 accepted
+    assert run([9, 1, 2, 0], [-1, 0, 0, 0], [0.0, 0.7, 1e-9, 0.999], 0.95) == (1, [0, 3, -1, -1], 2)
+    # the uniform number of a node is used for that node only: token 0 first is accepted outright (ratio 2.5)
+    assert run([9, 0, 1], [-1, 0, 0], [0.0, 0.999, 0.0], 0.0001) == (1, [0, 1, -1, -1], 0)
+    # temperature: at T = 2 the root distributions are norm(sqrt(.)); token 1's ratio becomes
+    # sqrt(0.3)/sum_T over sqrt(0.5)/sum_D
+    sT, sD = np.sqrt([0.5, 0.3, 0.2]).sum(), np.sqrt([0.2, 0.5, 0.3]).sum()
+    ratio = (np.sqrt(0.3) / sT) / (np.sqrt(0.5) / sD)
+    for du, want in ((-1e-6, 1), (1e-6, 0)):
+        al, _, _, mg = stochastic_accept(tl, dl, np.array([[9, 1]], dtype=np.int32), np.array([[-1, 0]]), np.array([2]), 3,
+                                         2.0, np.array([[0.0, ratio + du]]), np.array([0.5]))
+        assert al[0] == want and mg[0] < 2e-6
+
+
+def test_stochastic_accept_one_hot_target_is_the_greedy_rule():
+    rng = np.random.default_rng(5)
+    V, H = 13, 6
+    for trial in range(60):
+        N = int(rng.integers(1, 20))
+        parent = np.array([-1] + [int(rng.integers(0, t)) for t in range(1, N)])
+        depth = np.zeros(N, dtype=int)
+        for t in range(1, N):
+            depth[t] = depth[parent[t]] + 1
+        if depth.max() > H:
+            continue
+        tokens = rng.integers(0, V, size=N).astype(np.int32)
+        tl = rng.normal(size=(1, N, V))
+        for t in range(N):  # a one-hot target: one logit far above the rest; often a child's token
+            kids = [c for c in range(N) if parent[c] == t]
+            x = int(tokens[kids[int(rng.integers(0, len(kids)))]]) if kids and rng.random() < 0.7 else int(rng.integers(0, V))
+            tl[0, t, x] = 5000.0
+        dl = rng.normal(size=(1, N, V))
+        ua, ub = rng.uniform(1e-6, 1 - 1e-6, size=(1, N)), rng.uniform(1e-6, 1 - 1e-6, size=(1,))
+        got = stochastic_accept(tl, dl, tokens[None], parent[None], np.array([N]), H, 1.0, ua, ub)
+        want = greedy_accept(tl, tokens[None], parent[None], np.array([N]), H)
+        # duplicate sibling tokens: the greedy walk takes the first match, and so does the stochastic one
+        assert got[0][0] == want[0][0] and list(got[1][0]) == list(want[1][0]) and got[2][0] == want[2][0]
+
+
+def test_stochastic_accept_equal_models_accept_every_first_child():
+    rng = np.random.default_rng(6)
+    V, N = 50, 9
+    parent = np.array([[-1, 0, 0, 1, 1, 3, 2, 5, 5]])
+    tokens = rng.integers(0, V, size=(1, N)).astype(np.int32)
+    tl = rng.normal(size=(1, N, V)) * 2
+    for T in (1.0, 0.5):
+        ua, ub = rng.uniform(size=(1, N)), rng.uniform(size=(1,))
+        al, ap, bo, _ = stochastic_accept(tl, tl.copy(), tokens, parent, np.array([N]), 5, T, ua, ub)
+        assert al[0] == 4 and list(ap[0]) == [0, 1, 3, 5, 7, -1]
+        # the bonus token: inversion of the leaf's distribution by a library routine
+        z = tl[0, 7] / T
+        pr = np.exp(z - z.max())
+        cdf = np.cumsum(pr / pr.sum())
+        assert bo[0] == int(np.searchsorted(cdf, ub[0] * cdf[-1], side="left"))
+
+
+def test_stochastic_accept_output_follows_the_target_distribution():
+    """With children drawn independently from P_D, the token the step emits at a node - an accepted
+    child's or the bonus token - is distributed exactly as P_T at that node, whatever P_D is. Checked
+    by simulation on a two-level tree over a 4-token vocabulary: first emitted token against
+    P_T(. | root), second against P_T(. | first) given that the first was an accepted child."""
+    rng = np.random.default_rng(11)
+    V, trials = 4, 24000
+    PT0, PD0 = np.array([0.45, 0.05, 0.2, 0.3]), np.array([0.1, 0.4, 0.3, 0.2])
+    PT1 = rng.dirichlet(np.ones(V), size=V)  # P_T(. | first token)
+    PD1 = rng.dirichlet(np.ones(V), size=V)
+    first = np.zeros(V)
+    second = np.zeros((V, V))
+    for _ in range(trials):
+        kids = rng.choice(V, size=3, p=PD0)
+        tokens = [0] + [int(x) for x in kids]
+        parent = [-1, 0, 0, 0]
+        for c in (1, 2, 3):
+            g = rng.choice(V, size=2, p=PD1[tokens[c]])
+            tokens += [int(x) for x in g]
+            parent += [c, c]
+        N = len(tokens)
+        tl = np.zeros((1, N, V))
+        dl = np.zeros((1, N, V))
+        tl[0, 0], dl[0, 0] = np.log(PT0), np.log(PD0)
+        for c in (1, 2, 3):
+            tl[0, c], dl[0, c] = np.log(PT1[tokens[c]]), np.log(PD1[tokens[c]])
+        for c in range(4, N):
+            tl[0, c] = np.log(PT0)  # never sampled from in what is counted below
+        al, ap, bo, _ = stochastic_accept(tl, dl, np.array([tokens], dtype=np.int32), np.array([parent]), np.array([N]), 3, 1.0,
+                                          rng.uniform(size=(1, N)), rng.uniform(size=(1,)))
+        out = [tokens[i] for i in ap[0, 1: al[0] + 1]] + [int(bo[0])]
+        first[out[0]] += 1
+        if al[0] >= 1:
+            second[out[0], out[1]] += 1
+    assert np.all(np.abs(first / trials - PT0) < 5 * np.sqrt(PT0 * (1 - PT0) / trials))
+    for x in range(V):
+        n = second[x].sum()
+        assert n > 500
+        assert np.all(np.abs(second[x] / n - PT1[x]) < 5 * np.sqrt(PT1[x] * (1 - PT1[x]) / n) + 1e-9)
 
 
 # ----------------------------------------------------------------- compaction
