@@ -13,6 +13,7 @@
  *                        linearisation + ancestor mask (Sec. "Tree Reranking Phase")
  *   cast_tree_attention  verification attention under that mask
  *   cast_accept          greedy acceptance (Sec. "Speculative Decoding", T = 0)
+ *   cast_accept_stochastic  the same section's rule at T > 0, with residual resampling
  *   cast_compact_kv      accepted KV rows made contiguous
  *
  * Conventions
@@ -208,6 +209,47 @@ CAST_API cast_status cast_accept(cast_ctx* ctx, const void* target_logits, cast_
                         const int32_t* tokens, const int32_t* parent, const int32_t* depth,
                         const uint32_t* anc_mask, const int32_t* n_tree, int32_t* accept_len,
                         int32_t* accept_path, int32_t* bonus_token, void* stream);
+
+/*
+ * Acceptance at temperature T > 0 (Sec. "Speculative Decoding"): a draft token x with draft
+ * probability q = P_D(x | .) and target probability p = P_T(x | .) is accepted iff
+ * u <= min(1, p / q); after a rejection the target distribution is replaced by the residual
+ * norm(max(0, P_T - P_D)). On the tree: starting at the root, the children of the current node are
+ * tried in tree order (ascending linear index), each against the distribution its rejected elder
+ * siblings left (P_D unchanged); the first accepted child becomes the current node. When no child
+ * is accepted (or there is none) the bonus token is drawn from the distribution that stands then -
+ * P_T at a leaf, a residual otherwise - by inversion of its cumulative sum in token order: the
+ * first token whose cumulative sum reaches u_bonus * total. A residual that sums to zero ends the
+ * sibling loop with the distribution before it. Both distributions are softmax(logits / temperature).
+ *   target_logits [B, Ncap, V]  row t: the target model's logits at tree token t
+ *   draft_logits  [B, Ncap, V]  row t: the draft model's logits at tree token t, i.e. the
+ *                               distribution t's children were drawn from; rows of leaves are not read
+ *   temperature   > 0 (host)
+ *   tokens, parent [B, Ncap]; n_tree [B]
+ *   u_accept [B, Ncap] fp64 in (0,1): the uniform number of tree token t (root's entry unused)
+ *   u_bonus  [B]       fp64 in (0,1)
+ *   accept_len, accept_path, bonus_token: as for cast_accept
+ * The random numbers are inputs so that the step is reproducible; the caller draws them.
+ * All arithmetic is fp64. One thread-block cluster per sequence; the launch reads only the rows of
+ * the nodes on the accepted path.
+ * Device errors: BAD_TREE (n_tree out of range, a token outside [0, V), a path longer than H+1),
+ * NONFINITE (a row whose exponentials do not sum to a positive finite number).
+ */
+CAST_API cast_status cast_accept_stochastic(cast_ctx* ctx, const void* target_logits, const void* draft_logits,
+                                            cast_dtype dtype, int B, double temperature, const int32_t* tokens,
+                                            const int32_t* parent, const int32_t* n_tree, const double* u_accept,
+                                            const double* u_bonus, int32_t* accept_len, int32_t* accept_path,
+                                            int32_t* bonus_token, void* stream);
+
+/*
+ * How cast_accept_stochastic organises its launch for this context's vocabulary and a logits dtype
+ * (host-side query; no device work): the thread-block cluster size per sequence (16 where the
+ * device can co-schedule that many CTAs with their shared memory, else 8, else 1) and whether a
+ * CTA's vocabulary slice fits in shared memory (1) or every sweep recomputes it from the logits (0).
+ * cast_accept_stochastic makes this query itself on its first call; call it before a stream capture.
+ */
+CAST_API cast_status cast_accept_stochastic_plan(cast_ctx* ctx, cast_dtype dtype, int* cluster_size /* host */,
+                                                 int* cached /* host */);
 
 /*
  * KV compaction (not in the paper; the plain gather): for every layer, kv-head

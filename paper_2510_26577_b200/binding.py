@@ -27,6 +27,7 @@ EXPORTS = [
     "cast_create", "cast_destroy", "cast_status_string", "cast_set_cost_tables", "cast_state_export",
     "cast_state_import", "cast_step_begin", "cast_tree_expand", "cast_select_nodes", "cast_tree_attention",
     "cast_accept", "cast_compact_kv", "cast_poll_status", "cast_step_info", "cast_accept_static",
+    "cast_accept_stochastic", "cast_accept_stochastic_plan",
 ]
 
 
@@ -77,6 +78,8 @@ def load_library() -> C.CDLL:
         "cast_compact_kv": [vp, vp, vp, i32, i32, i32, C.c_size_t, i32, i32, i32, i32p, i32, i32, i32p, i32p, i32p,
                             vp],
         "cast_accept_static": [vp, i32, i32, i32, i32, i32, i32p, i32p, i32p, i32p, i32p, i32p, vp],
+        "cast_accept_stochastic": [vp, vp, vp, i32, i32, C.c_double, i32p, i32p, i32p, vp, vp, i32p, i32p, i32p, vp],
+        "cast_accept_stochastic_plan": [vp, i32, C.POINTER(C.c_int), C.POINTER(C.c_int)],
         "cast_poll_status": [vp, vp, C.POINTER(C.c_int), C.POINTER(C.c_int32)],
         "cast_step_info": [vp, vp, C.POINTER(C.c_int32)],
     }
@@ -195,6 +198,24 @@ class CastContext:
         _check(self.lib.cast_accept(self.handle, _ptr(target_logits), _dtype_code(target_logits), B, _ptr(tokens),
                                     _ptr(parent), _ptr(depth), _ptr(anc_mask), _ptr(n_tree), _ptr(accept_len),
                                     _ptr(accept_path), _ptr(bonus_token), _stream(stream)), "cast_accept")
+
+    def cast_accept_stochastic(self, target_logits, draft_logits, B, temperature, tokens, parent, n_tree, u_accept,
+                               u_bonus, accept_len, accept_path, bonus_token, stream=None):
+        assert draft_logits.dtype == target_logits.dtype and u_accept.dtype == torch.float64 and \
+            u_bonus.dtype == torch.float64
+        _check(self.lib.cast_accept_stochastic(self.handle, _ptr(target_logits), _ptr(draft_logits),
+                                               _dtype_code(target_logits), B, float(temperature), _ptr(tokens),
+                                               _ptr(parent), _ptr(n_tree), _ptr(u_accept), _ptr(u_bonus),
+                                               _ptr(accept_len), _ptr(accept_path), _ptr(bonus_token),
+                                               _stream(stream)), "cast_accept_stochastic")
+
+    def cast_accept_stochastic_plan(self, dtype):
+        """(cluster size, slices cached in shared memory?) for logits of torch dtype `dtype`."""
+        cs, cached = C.c_int(0), C.c_int(0)
+        code = CAST_F32 if dtype == torch.float32 else CAST_BF16
+        _check(self.lib.cast_accept_stochastic_plan(self.handle, code, C.byref(cs), C.byref(cached)),
+               "cast_accept_stochastic_plan")
+        return cs.value, bool(cached.value)
 
     def cast_compact_kv(self, k_cache, v_cache, B, n_layers, layer_stride_bytes, Hkv, D, page_size, page_table,
                         seq_capacity, num_pages, accept_path, accept_len, kv_len, stream=None):

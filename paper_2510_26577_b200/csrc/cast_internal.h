@@ -97,6 +97,11 @@ struct cast_ctx {
   void* attn_tc_ws;
   size_t attn_tc_ws_bytes;
 
+  // stochastic acceptance, per logits dtype (0 fp32, 1 bf16): cluster size found to be launchable
+  // (0: not looked up yet) and whether a CTA's vocabulary slice is cached in shared memory
+  int sto_cs[2];
+  int sto_cached[2];
+
   std::map<int, cast::HostTable>* tables;
   cast::DevTable cur_table;   // table of the current step's batch size (zeros if none)
   int cur_B;

@@ -185,6 +185,34 @@ def plant_acceptance(w: Workload, logits: torch.Tensor, tokens, parent, n_tree, 
             row[int(tokens[b, child])] = (row.float().max() + 1.0).to(row.dtype)
 
 
+def stochastic_accept_inputs(w: Workload, tokens, parent, n_tree, device="cpu", noise: float = 1.0, n_cap: int = 0):
+    """Inputs of the acceptance step at T > 0 for a given tree (host arrays): per-node draft logits
+    [B, Ncap, V] whose largest entries at a node are its children's tokens in tree order (children are the
+    top of the draft distribution: row maximum + 1, then steps of 0.5 down), target logits = draft logits +
+    `noise` * N(0,1) (a draft that approximates its target), and the uniform numbers u_accept [B, Ncap],
+    u_bonus [B] (fp64, open interval)."""
+    B, Ncap = w.batch, n_cap or w.max_tree
+    g = _gen(w, 800, "cpu")
+    draft = _randn((B, Ncap, w.vocab), w.logit_std, "f32", g, "cpu")
+    tokens = np.asarray(tokens)
+    parent = np.asarray(parent)
+    for b in range(B):
+        kids: Dict[int, List[int]] = {}
+        for t in range(1, int(n_tree[b])):
+            kids.setdefault(int(parent[b, t]), []).append(t)
+        for t, cs in kids.items():
+            top = float(draft[b, t].max()) + 1.0
+            for j, c in enumerate(cs):
+                draft[b, t, int(tokens[b, c])] = top - 0.5 * j
+    target = draft + noise * torch.randn(draft.shape, generator=g, dtype=torch.float32)
+    rng = np.random.Generator(np.random.Philox(w.seed * 1000 + 801))
+    u_accept = rng.uniform(1e-12, 1.0 - 1e-12, size=(B, Ncap))
+    u_bonus = rng.uniform(1e-12, 1.0 - 1e-12, size=(B,))
+    dt = _TORCH_DTYPE[w.logit_dtype]
+    return (target.to(dt).to(device), draft.to(dt).to(device), torch.from_numpy(u_accept).to(device),
+            torch.from_numpy(u_bonus).to(device))
+
+
 def cost_table_arrays(w: Workload, B: int, L: int = 512, M: int = 64, Ntab: int = 128,
                       stepped: bool = False) -> Tuple[int, int, int, np.ndarray, np.ndarray]:
     """Synthetic stand-in for the profiled latency tables (the real ones need

@@ -6,7 +6,7 @@ import numpy as np
 import pytest
 import torch
 
-from oracle import ancestor_masks, compact_kv, greedy_accept, tree_attention
+from oracle import ancestor_masks, compact_kv, greedy_accept, stochastic_accept, tree_attention
 from paper_2510_26577_b200 import workloads as wl
 
 from helpers import (assert_tree_equal, attention_tolerance, cfg_kwargs, gpu_attention, gpu_tree, make_tables,
@@ -138,6 +138,9 @@ def test_c2_llama8b_full_step(binding):
     check_attention(binding, ctx, w, g, o, kv)
     ol = check_accept_and_compact(binding, ctx, w, g, o, kv)
     assert ol[0] >= 1  # planted acceptance gives the walk something to do
+    # the same tree through the acceptance rule at temperature 1 and 0.6
+    for T, salt in ((1.0, 0), (0.6, 1)):
+        _run_stochastic(binding, ctx, wl.shrink(w, seed_salt=salt), o["tokens"], o["parent"], o["n_tree"], w.depth, T, 0.7)
 
 
 @pytest.mark.parametrize("name", ["c3_llama8b_b1", "c3_llama8b_b4", "c3_llama8b_b16"])
@@ -172,6 +175,7 @@ def test_c4_llama70b(binding, name):
     assert list(o["n_tree"]) == [w.total_token] * 8
     check_attention(binding, ctx, w, g, o, kv, sample=16)
     check_accept_and_compact(binding, ctx, w, g, o, kv)
+    _run_stochastic(binding, ctx, w, o["tokens"], o["parent"], o["n_tree"], w.depth, 1.0, 0.7)
 
 
 def test_c5_qwen_long_context(binding):
@@ -426,3 +430,109 @@ def test_accept_edge_cases_and_overlapping_compaction(binding):
         assert np.array_equal(kv2.cpu().numpy(), nlen)
         assert np.array_equal(kk.view(torch.int32).cpu().numpy(), nk)
         assert np.array_equal(vv.view(torch.int32).cpu().numpy(), nv)
+
+
+# ------------------------------------------------------------------ acceptance at T > 0
+def _run_stochastic(binding, ctx, w, tokens, parent, n_tree, H, T, noise=1.0, inputs=None):
+    """GPU against oracle on the same inputs; the oracle's decision margin tells a rounding coin flip
+    (pick another seed) from a wrong result."""
+    B, Ncap = tokens.shape
+    tl, dl, ua, ub = inputs if inputs is not None else wl.stochastic_accept_inputs(w, tokens, parent, n_tree, "cuda", noise, Ncap)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    alen = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+    apath = torch.full((B, H + 1), -7, dtype=torch.int32, device="cuda")
+    bonus = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+    ctx.cast_accept_stochastic(tl, dl, B, T, dev(tokens.astype(np.int32)), dev(parent.astype(np.int32)),
+                               dev(n_tree.astype(np.int32)), ua, ub, alen, apath, bonus)
+    assert ctx.cast_poll_status()[0] == 0
+    nmax = int(n_tree.max())
+    ol, op, ob, margin = stochastic_accept(to_f64(tl[:, :nmax]), to_f64(dl[:, :nmax]), tokens, parent, n_tree, H, T,
+                                           ua.cpu().numpy(), ub.cpu().numpy())
+    assert margin.min() >= 1e-9, f"a decision sits within rounding of its threshold ({margin.min():.1e}): pick another seed"
+    assert np.array_equal(alen.cpu().numpy(), ol), (alen.cpu().numpy(), ol)
+    assert np.array_equal(apath.cpu().numpy(), op), (apath.cpu().numpy(), op)
+    assert np.array_equal(bonus.cpu().numpy(), ob), (bonus.cpu().numpy(), ob)
+    return ol
+
+
+def _random_token_tree(rng, B, Ncap, n_tree, V, H, kinds):
+    tokens = np.zeros((B, Ncap), dtype=np.int32)
+    parent = np.full((B, Ncap), -1, dtype=np.int32)
+    for b in range(B):
+        N = int(n_tree[b])
+        par = _random_tree(rng, N, kinds[b % len(kinds)])
+        depth = np.zeros(N, dtype=int)
+        for t in range(1, N):
+            if depth[par[t]] + 1 > H:  # keep the tree within the depth the output has room for
+                par[t] = 0
+            depth[t] = depth[par[t]] + 1
+        parent[b, :N] = par
+        tokens[b, 0] = rng.integers(0, V)
+        for t in range(1, N):
+            used = {int(tokens[b, c]) for c in range(1, t) if par[c] == par[t]}
+            x = int(rng.integers(0, V))
+            while x in used:
+                x = int(rng.integers(0, V))
+            tokens[b, t] = x
+    return tokens, parent
+
+
+@pytest.mark.parametrize("dtype,V,T,B,Ncap,noise", [
+    ("f32", 4096, 1.0, 4, 32, 1.0),        # small vocabulary: slices of 256
+    ("f32", 1000, 0.7, 3, 32, 0.5),        # slices of 64: the last CTA's slice is short
+    ("f32", 37, 1.3, 3, 16, 1.0),          # most CTAs of the cluster hold nothing
+    ("bf16", 128256, 1.0, 3, 64, 1.0),     # Llama-3 vocabulary, bf16 logits
+    ("f32", 152064, 0.8, 2, 64, 0.3),      # Qwen vocabulary: the largest cached slice
+    ("f32", 262144, 1.0, 2, 16, 1.0),      # slices too large to cache: every sweep recomputes them
+])
+def test_accept_stochastic_random_trees(binding, dtype, V, T, B, Ncap, noise):
+    rng = np.random.default_rng(1234 + V)
+    H = 6
+    w = wl.Workload("sto", 93, B, "f32", dtype, 8, 8, 64, 1, 2, 0, V, 3.0, H, 4, Ncap, False, 1, max_tree=Ncap)
+    ctx = binding.CastContext(max_batch=B, vocab=V, top_k=4, max_depth=H, total_token=Ncap, max_tree=Ncap)
+    cs, cached = ctx.cast_accept_stochastic_plan(torch.float32 if dtype == "f32" else torch.bfloat16)
+    assert cs in (8, 16) and cached == (V <= cs * 12288)
+    n_tree = np.array([Ncap, 1, max(2, Ncap // 3), Ncap - 5][:B], dtype=np.int32)
+    tokens, parent = _random_token_tree(rng, B, Ncap, n_tree, V, H, ["random", "chain", "star", "random"])
+    total = 0
+    for rep in range(3):  # three sets of inputs per case: different paths and rejection counts
+        w2 = wl.shrink(w, seed_salt=rep)
+        total += int(_run_stochastic(binding, ctx, w2, tokens, parent, n_tree, H, T, noise).sum())
+    assert total > 0  # the recipe accepts something
+
+
+def test_accept_stochastic_special_cases(binding):
+    rng = np.random.default_rng(77)
+    B, Ncap, V, H = 3, 32, 5000, 6
+    w = wl.Workload("sto", 94, B, "f32", "f32", 8, 8, 64, 1, 2, 0, V, 3.0, H, 4, Ncap, False, 1, max_tree=Ncap)
+    ctx = binding.CastContext(max_batch=B, vocab=V, top_k=4, max_depth=H, total_token=Ncap, max_tree=Ncap)
+    n_tree = np.array([Ncap, 20, 9], dtype=np.int32)
+    tokens, parent = _random_token_tree(rng, B, Ncap, n_tree, V, H, ["random"])
+    tl, dl, ua, ub = wl.stochastic_accept_inputs(w, tokens, parent, n_tree, "cuda", 1.0, Ncap)
+    # equal models: the first child is accepted at every node, down to a leaf
+    ol = _run_stochastic(binding, ctx, w, tokens, parent, n_tree, H, 1.0, inputs=(dl.clone(), dl, ua, ub))
+    for b in range(B):
+        cur, steps = 0, 0
+        while True:
+            kids = [c for c in range(int(n_tree[b])) if parent[b, c] == cur]
+            if not kids:
+                break
+            cur, steps = kids[0], steps + 1
+        assert ol[b] == steps
+    # a one-hot target: the greedy rule, whatever the uniform numbers are
+    hot = tl.clone()
+    for b in range(B):
+        for t in range(int(n_tree[b])):
+            kids = [c for c in range(int(n_tree[b])) if parent[b, c] == t]
+            x = int(tokens[b, kids[-1]]) if kids and (t % 3) else int(rng.integers(0, V))
+            hot[b, t, x] = 4000.0
+    ol = _run_stochastic(binding, ctx, w, tokens, parent, n_tree, H, 1.0, inputs=(hot, dl, ua, ub))
+    gl, gp, gb = greedy_accept(to_f64(hot), tokens, parent, n_tree, H)
+    assert np.array_equal(ol, gl)
+    # host-side checks
+    i32 = lambda *s: torch.zeros(s, dtype=torch.int32, device="cuda")
+    for bad_T in (0.0, -1.0, float("nan")):
+        with pytest.raises(binding.CastError):
+            ctx.cast_accept_stochastic(tl, dl, B, bad_T, i32(B, Ncap), i32(B, Ncap), i32(B), ua, ub, i32(B), i32(B, H + 1), i32(B))
+    with pytest.raises(binding.CastError):
+        ctx.cast_accept_stochastic(tl, dl, B + 1, 1.0, i32(B, Ncap), i32(B, Ncap), i32(B), ua, ub, i32(B), i32(B, H + 1), i32(B))
