@@ -304,6 +304,25 @@ def run_ours(args, w):
 
     g_tree, g_attn, g_acc, g_cmp = capture(tree_build), capture(attention), capture(accept), capture(compact_phase)
 
+    # acceptance at temperature 1 on the same tree (not part of the step: it replaces cast_accept when the
+    # serving loop samples). Its inputs hold two more [B, Ncap, V] logit tensors: skipped above 2^28 entries.
+    sto = None
+    if B * Ncap * w.vocab <= (1 << 28) and not args.quick:
+        s_tl, s_dl, s_ua, s_ub = wl.stochastic_accept_inputs(w, tr["tokens"].cpu().numpy(), tr["parent"].cpu().numpy(),
+                                                             n_tree, dev, 0.7, Ncap)
+        s_len = torch.empty_like(alen)
+        s_path, s_bonus = torch.empty_like(apath), torch.empty_like(bonus)
+
+        def accept_stochastic():
+            ctx.cast_accept_stochastic(s_tl, s_dl, B, 1.0, tr["tokens"], tr["parent"], tr["n_tree"], s_ua, s_ub, s_len,
+                                       s_path, s_bonus)
+
+        ms_sto = time_graph(capture(accept_stochastic), max(args.steps, 20), args.warmup)
+        plan = ctx.cast_accept_stochastic_plan(s_tl.dtype)
+        sto = {"us": ms_sto * 1e3, "temperature": 1.0, "target_minus_draft_logit_std": 0.7,
+               "mean_accept_len": float(s_len.float().mean().item()), "cluster_size": plan[0], "slices_cached": plan[1]}
+        del s_tl, s_dl
+
     # ---- phase timings (each phase alone; KV working set of the attention graph exceeds 2x L2)
     kv_len.copy_(kv0)  # the capture passes ran the compaction
     sub_reps = args.steps if args.quick else max(args.steps, 20)
@@ -437,7 +456,7 @@ def run_ours(args, w):
         "gpu_launches": launches,
         "clocks": clocks,
         "phases": {"tree_build_us": ms_tree * 1e3, "attention_us_per_layer": attn_us, "accept_us": ms_acc * 1e3,
-                   "compact_us": ms_cmp * 1e3},
+                   "compact_us": ms_cmp * 1e3, "accept_stochastic": sto},
         "roofline": {"kernel": "cast_tree_attention (one layer)", "bound": "hbm", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_source": which, "traffic": NCU_ATTENTION_TRAFFIC.get(w.name),
                      "algorithmic_bytes": attn_bytes},

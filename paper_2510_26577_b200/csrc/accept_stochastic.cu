@@ -21,6 +21,22 @@
 
 using namespace cast;
 
+// Development aid, compiled only with -DCAST_PHASE_CLOCKS: thread 0 of the first CTA of sequence 0 records
+// the global timer at phase boundaries.
+#ifdef CAST_PHASE_CLOCKS
+__device__ long long g_sto_clock[64];
+__device__ int g_sto_clock_n;
+#define STO_STAMP() do { if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && sto_n < 64) { long long _t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(_t)); g_sto_clock[sto_n++] = _t; g_sto_clock_n = sto_n; } } while (0)
+#define STO_STAMP_DECL int sto_n = 0;
+extern "C" __attribute__((visibility("default"))) int cast_debug_read_sto_clocks(long long* out, int* n) {
+  cudaMemcpyFromSymbol(n, g_sto_clock_n, sizeof(int));
+  return (int)cudaMemcpyFromSymbol(out, g_sto_clock, sizeof(long long) * 64);
+}
+#else
+#define STO_STAMP() do {} while (0)
+#define STO_STAMP_DECL
+#endif
+
 namespace {
 
 constexpr int kStoThreads = 512;
@@ -53,6 +69,39 @@ __device__ __forceinline__ void sto_st_remote_f64(const double* local, uint32_t 
 __device__ __forceinline__ void sto_cluster_sync() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+// exp(x) for x <= 0 in fp64 to about 3e-16 relative: x = n ln2 + r with n = round(x log2 e) (ln2 split in
+// two so that n ln2_hi is exact), the degree-12 Taylor polynomial of e^r on |r| <= ln2 / 2 (remainder below
+// 2e-16), scaling by 2^n through the exponent field. Arguments below -708 (results near the subnormal
+// range) give 0; NaN gives NaN. Half the instructions of the general-purpose library routine, and the
+// sweeps below are bound by fp64 issue.
+__device__ __forceinline__ double sto_exp(double x) {
+  // branch-free (a select at the end), so that the compiler can interleave several calls: one call is a
+  // chain of some twenty dependent fp64 instructions
+  const double xin = x;
+  x = fmax(x, -708.0);
+  const double kMagic = 6755399441055744.0;  // 1.5 * 2^52: adding it rounds to an integer in the low word
+  const double tn = fma(x, 1.4426950408889634074, kMagic);
+  const int n = __double2loint(tn);
+  const double nd = tn - kMagic;
+  double r = fma(nd, -6.93147180369123816490e-01, x);
+  r = fma(nd, -1.90821492927058770002e-10, r);
+  double y = 2.08767569878680989792e-09;  // 1/12!
+  y = fma(y, r, 2.50521083854417187751e-08);
+  y = fma(y, r, 2.75573192239858906526e-07);
+  y = fma(y, r, 2.75573192239858906526e-06);
+  y = fma(y, r, 2.48015873015873015873e-05);
+  y = fma(y, r, 1.98412698412698412698e-04);
+  y = fma(y, r, 1.38888888888888888889e-03);
+  y = fma(y, r, 8.33333333333333333333e-03);
+  y = fma(y, r, 4.16666666666666666667e-02);
+  y = fma(y, r, 1.66666666666666666667e-01);
+  y = fma(y, r, 0.5);
+  y = fma(y, r, 1.0);
+  y = fma(y, r, 1.0);
+  const double res = __hiloint2double(__double2hiint(y) + n * 1048576, __double2loint(y));
+  return xin >= -708.0 ? res : (xin != xin ? xin : 0.0);
 }
 
 struct StoShared {
@@ -129,6 +178,8 @@ __global__ void __launch_bounds__(kStoThreads, 1) accept_stochastic_kernel(const
   // the peers' shared memory may be written once all CTAs of the cluster run
   if (cs > 1) sto_cluster_sync(); else __syncthreads();
 
+  STO_STAMP_DECL
+  STO_STAMP();  // 0: start
   int parity = 0;
   int cur = 0, plen = 1;   // current node, nodes on the path so far
   double a = 0.0;          // the distribution that stands at `cur`: max(0, P_T - a P_D) / F(a)
@@ -139,8 +190,12 @@ __global__ void __launch_bounds__(kStoThreads, 1) accept_stochastic_kernel(const
   if (rank == 0 && tid == 0) p.accept_path[(size_t)b * (p.max_depth + 1)] = 0;
 
   // unnormalised slice entries: p~(i) * cp = P_T(begin + i), q~(i) * cq = P_D(begin + i)
-  auto pt = [&](int i) -> double { return CACHED ? ep[i] : exp((double)to_float(lp[begin + i]) * p.inv_T - Mp_loc); };
-  auto qt = [&](int i) -> double { return CACHED ? eq[i] : exp((double)to_float(lq[begin + i]) * p.inv_T - Mq_loc); };
+  auto pt = [&](int i) -> double {
+    return CACHED ? ep[i] : sto_exp((double)to_float(lp[begin + i]) * p.inv_T - (Mp_loc > -INFINITY ? Mp_loc : 0.0));
+  };
+  auto qt = [&](int i) -> double {
+    return CACHED ? eq[i] : sto_exp((double)to_float(lq[begin + i]) * p.inv_T - (Mq_loc > -INFINITY ? Mq_loc : 0.0));
+  };
 
   for (;;) {
     // ---- children of `cur` in tree order
@@ -165,10 +220,21 @@ __global__ void __launch_bounds__(kStoThreads, 1) accept_stochastic_kernel(const
     has_q = k > 0;
     lp = reinterpret_cast<const T*>(p.target_logits) + ((size_t)b * p.Ncap + cur) * p.V;
     lq = reinterpret_cast<const T*>(p.draft_logits) + ((size_t)b * p.Ncap + cur) * p.V;
+    if (k > 0) {
+      // the eldest child is the likeliest next node: its slices are asked into L2 while this node is worked on
+      const int c0 = sh.kids[0];
+      const char* np = reinterpret_cast<const char*>(reinterpret_cast<const T*>(p.target_logits) + ((size_t)b * p.Ncap + c0) * p.V + begin);
+      const char* nq = reinterpret_cast<const char*>(reinterpret_cast<const T*>(p.draft_logits) + ((size_t)b * p.Ncap + c0) * p.V + begin);
+      for (int off = tid * 128; off < len * (int)sizeof(T); off += kStoThreads * 128) {
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(np + off));
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(nq + off));
+      }
+    }
 
     // ---- softmax statistics of the node's rows: slice maxima, then slice sums of exp(. - slice maximum)
     {
       double mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll 8
       for (int i = tid; i < len; i += kStoThreads) {
         const double sp = (double)to_float(lp[begin + i]) * p.inv_T;
         if (CACHED) ep[i] = sp;
@@ -180,34 +246,56 @@ __global__ void __launch_bounds__(kStoThreads, 1) accept_stochastic_kernel(const
         }
       }
       sto_block_reduce<true, 2>(sh, mx);
+    STO_STAMP();
       Mp_loc = mx[0];
       Mq_loc = mx[1];
       double sm[2] = {0.0, 0.0};
-      for (int i = tid; i < len; i += kStoThreads) {
-        const double e0 = Mp_loc > -INFINITY ? exp((CACHED ? ep[i] : (double)to_float(lp[begin + i]) * p.inv_T) - Mp_loc) : 0.0;
-        if (CACHED) ep[i] = e0;
-        sm[0] += e0;
-        if (has_q) {
-          const double e1 = Mq_loc > -INFINITY ? exp((CACHED ? eq[i] : (double)to_float(lq[begin + i]) * p.inv_T) - Mq_loc) : 0.0;
-          if (CACHED) eq[i] = e1;
+      // an all -inf slice (a masked range of the vocabulary) takes reference 0: its entries become exp(-inf) = 0
+      const double ref_p = Mp_loc > -INFINITY ? Mp_loc : 0.0, ref_q = Mq_loc > -INFINITY ? Mq_loc : 0.0;
+      if (has_q) {
+#pragma unroll 4
+        for (int i = tid; i < len; i += kStoThreads) {
+          const double e0 = sto_exp((CACHED ? ep[i] : (double)to_float(lp[begin + i]) * p.inv_T) - ref_p);
+          const double e1 = sto_exp((CACHED ? eq[i] : (double)to_float(lq[begin + i]) * p.inv_T) - ref_q);
+          if (CACHED) {
+            ep[i] = e0;
+            eq[i] = e1;
+          }
+          sm[0] += e0;
           sm[1] += e1;
+        }
+      } else {
+#pragma unroll 4
+        for (int i = tid; i < len; i += kStoThreads) {
+          const double e0 = sto_exp((CACHED ? ep[i] : (double)to_float(lp[begin + i]) * p.inv_T) - ref_p);
+          if (CACHED) ep[i] = e0;
+          sm[0] += e0;
         }
       }
       sto_block_reduce<false, 2>(sh, sm);
+    STO_STAMP();
       const double rec[4] = {Mp_loc, sm[0], Mq_loc, sm[1]};
       sto_exchange(sh, parity, rank, cs, rec);
-      Mp = -INFINITY;
-      Mq = -INFINITY;
-      for (int r = 0; r < cs; ++r) {
-        Mp = fmax(Mp, sh.xch[parity][r][0]);
-        Mq = fmax(Mq, sh.xch[parity][r][2]);
-      }
-      Sp = 0.0;
-      Sq = 0.0;
-      for (int r = 0; r < cs; ++r) {
-        const double m0 = sh.xch[parity][r][0], m1 = sh.xch[parity][r][2];
-        if (m0 > -INFINITY) Sp += sh.xch[parity][r][1] * exp(m0 - Mp);
-        if (m1 > -INFINITY) Sq += sh.xch[parity][r][3] * exp(m1 - Mq);
+    STO_STAMP();
+      // fold of the ranks' records, the same in every warp of every CTA: lanes 0-15 take the target row's
+      // records by rank, lanes 16-31 the draft row's; maxima and sums through a fixed shuffle tree
+      {
+        const int rr = lane & 15, col = (lane >> 4) * 2;
+        const double m_r = rr < cs ? sh.xch[parity][rr][col] : -INFINITY;
+        const double s_r = rr < cs ? sh.xch[parity][rr][col + 1] : 0.0;
+        double M = m_r;
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) M = fmax(M, __shfl_xor_sync(0xffffffffu, M, o));
+        const double w_r = m_r > -INFINITY ? sto_exp(m_r - M) : 0.0;  // this rank's weight
+        double S = s_r * w_r;
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) S += __shfl_xor_sync(0xffffffffu, S, o);
+        Mp = __shfl_sync(0xffffffffu, M, 0);
+        Mq = __shfl_sync(0xffffffffu, M, 16);
+        Sp = __shfl_sync(0xffffffffu, S, 0);
+        Sq = __shfl_sync(0xffffffffu, S, 16);
+        cp = __shfl_sync(0xffffffffu, w_r, rank);        // exp(Mp_loc - Mp)
+        cq = __shfl_sync(0xffffffffu, w_r, 16 + rank);   // exp(Mq_loc - Mq)
       }
       parity ^= 1;
       if (!(Sp > 0.0) || !isfinite(Sp) || (has_q && (!(Sq > 0.0) || !isfinite(Sq)))) {
@@ -217,8 +305,8 @@ __global__ void __launch_bounds__(kStoThreads, 1) accept_stochastic_kernel(const
         k = 0;
         has_q = false;
       }
-      cp = Mp_loc > -INFINITY ? exp(Mp_loc - Mp) / Sp : 0.0;
-      cq = has_q && Mq_loc > -INFINITY ? exp(Mq_loc - Mq) / Sq : 0.0;
+      cp = cp / Sp;
+      cq = has_q ? cq / Sq : 0.0;
     }
 
     // ---- the children, one after the other, each against the residual its elder siblings left
@@ -232,9 +320,10 @@ __global__ void __launch_bounds__(kStoThreads, 1) accept_stochastic_kernel(const
         if (rank == 0 && tid == 0) report(p.st, CAST_ERR_BAD_TREE, b);
         continue;  // not a token: never accepted
       }
-      const double px = exp((double)to_float(lp[x]) * p.inv_T - Mp) / Sp;
-      const double qx = exp((double)to_float(lq[x]) * p.inv_T - Mq) / Sq;
       const double u = p.u_accept[(size_t)b * p.Ncap + c];
+      const double v01 = (lane & 1) ? sto_exp((double)to_float(lq[x]) * p.inv_T - Mq) / Sq
+                                    : sto_exp((double)to_float(lp[x]) * p.inv_T - Mp) / Sp;
+      const double px = __shfl_sync(0xffffffffu, v01, 0), qx = __shfl_sync(0xffffffffu, v01, 1);
       const double rx = fmax(0.0, px - a * qx);
       if (u * qx * F <= rx) {
         next = c;
@@ -243,10 +332,13 @@ __global__ void __launch_bounds__(kStoThreads, 1) accept_stochastic_kernel(const
       // rejected: the residual of the residual
       const double a2 = a + F;
       double part[1] = {0.0};
+#pragma unroll 4
       for (int i = tid; i < len; i += kStoThreads) part[0] += fmax(0.0, pt(i) * cp - a2 * (qt(i) * cq));
       sto_block_reduce<false, 1>(sh, part);
+    STO_STAMP();
       const double rec[4] = {part[0], 0.0, 0.0, 0.0};
       sto_exchange(sh, parity, rank, cs, rec);
+      STO_STAMP();
       double F2 = 0.0;
       for (int r = 0; r < cs; ++r) F2 += sh.xch[parity][r][0];
       parity ^= 1;
@@ -262,6 +354,7 @@ __global__ void __launch_bounds__(kStoThreads, 1) accept_stochastic_kernel(const
 
   // ---- bonus token: inversion of the cumulative sum, in token order, of max(0, P_T - a P_D) at `cur`
   double part[1] = {0.0};
+#pragma unroll 4
   for (int i = tid; i < len; i += kStoThreads) part[0] += fmax(0.0, pt(i) * cp - (has_q ? a * (qt(i) * cq) : 0.0));
   sto_block_reduce<false, 1>(sh, part);
   {
@@ -270,6 +363,7 @@ __global__ void __launch_bounds__(kStoThreads, 1) accept_stochastic_kernel(const
   }
   double total = 0.0;
   for (int r = 0; r < cs; ++r) total += sh.xch[parity][r][0];
+  STO_STAMP();
   const double goal = p.u_bonus[b] * total;
   // the slice in which the cumulative sum reaches the goal (rounding may leave none: the last non-empty one)
   int owner = -1, last_nonempty = 0;

@@ -192,8 +192,8 @@ def stochastic_accept_inputs(w: Workload, tokens, parent, n_tree, device="cpu", 
     `noise` * N(0,1) (a draft that approximates its target), and the uniform numbers u_accept [B, Ncap],
     u_bonus [B] (fp64, open interval)."""
     B, Ncap = w.batch, n_cap or w.max_tree
-    g = _gen(w, 800, "cpu")
-    draft = _randn((B, Ncap, w.vocab), w.logit_std, "f32", g, "cpu")
+    g = _gen(w, 800, device)
+    draft = _randn((B, Ncap, w.vocab), w.logit_std, "f32", g, device)
     tokens = np.asarray(tokens)
     parent = np.asarray(parent)
     for b in range(B):
@@ -204,13 +204,13 @@ def stochastic_accept_inputs(w: Workload, tokens, parent, n_tree, device="cpu", 
             top = float(draft[b, t].max()) + 1.0
             for j, c in enumerate(cs):
                 draft[b, t, int(tokens[b, c])] = top - 0.5 * j
-    target = draft + noise * torch.randn(draft.shape, generator=g, dtype=torch.float32)
+    target = torch.randn(draft.shape, generator=g, device=device, dtype=torch.float32)
+    target.mul_(noise).add_(draft)
     rng = np.random.Generator(np.random.Philox(w.seed * 1000 + 801))
     u_accept = rng.uniform(1e-12, 1.0 - 1e-12, size=(B, Ncap))
     u_bonus = rng.uniform(1e-12, 1.0 - 1e-12, size=(B,))
     dt = _TORCH_DTYPE[w.logit_dtype]
-    return (target.to(dt).to(device), draft.to(dt).to(device), torch.from_numpy(u_accept).to(device),
-            torch.from_numpy(u_bonus).to(device))
+    return (target.to(dt), draft.to(dt), torch.from_numpy(u_accept).to(device), torch.from_numpy(u_bonus).to(device))
 
 
 def cost_table_arrays(w: Workload, B: int, L: int = 512, M: int = 64, Ntab: int = 128,
