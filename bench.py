@@ -281,8 +281,23 @@ def run_ours(args, w):
             stream.synchronize()
         return e0.elapsed_time(e1) / reps  # ms per replay
 
+    def make_accept_stochastic():
+        """Acceptance at temperature 1 on the step's tree: inputs (two more [B, Ncap, V] logit tensors) and call."""
+        s_tl, s_dl, s_ua, s_ub = wl.stochastic_accept_inputs(w, tr["tokens"].cpu().numpy(), tr["parent"].cpu().numpy(),
+                                                             n_tree, dev, 0.7, Ncap)
+        s_len = torch.empty_like(alen)
+        s_path, s_bonus = torch.empty_like(apath), torch.empty_like(bonus)
+
+        def call():
+            ctx.cast_accept_stochastic(s_tl, s_dl, B, 1.0, tr["tokens"], tr["parent"], tr["n_tree"], s_ua, s_ub, s_len,
+                                       s_path, s_bonus)
+        return call, s_len, s_tl.dtype
+
     if args.only:  # profiling aid: replay one phase only (no graph), print its time, stop
-        fn = {"tree": tree_build, "attention": attention, "accept": accept, "compact": compact}[args.only]
+        if args.only == "accept_stochastic":
+            fn = make_accept_stochastic()[0]
+        else:
+            fn = {"tree": tree_build, "attention": attention, "accept": accept, "compact": compact}[args.only]
         with torch.cuda.stream(stream):
             for _ in range(args.warmup):
                 fn()
@@ -308,20 +323,12 @@ def run_ours(args, w):
     # serving loop samples). Its inputs hold two more [B, Ncap, V] logit tensors: skipped above 2^28 entries.
     sto = None
     if B * Ncap * w.vocab <= (1 << 28) and not args.quick:
-        s_tl, s_dl, s_ua, s_ub = wl.stochastic_accept_inputs(w, tr["tokens"].cpu().numpy(), tr["parent"].cpu().numpy(),
-                                                             n_tree, dev, 0.7, Ncap)
-        s_len = torch.empty_like(alen)
-        s_path, s_bonus = torch.empty_like(apath), torch.empty_like(bonus)
-
-        def accept_stochastic():
-            ctx.cast_accept_stochastic(s_tl, s_dl, B, 1.0, tr["tokens"], tr["parent"], tr["n_tree"], s_ua, s_ub, s_len,
-                                       s_path, s_bonus)
-
+        accept_stochastic, s_len, s_dtype = make_accept_stochastic()
         ms_sto = time_graph(capture(accept_stochastic), max(args.steps, 20), args.warmup)
-        plan = ctx.cast_accept_stochastic_plan(s_tl.dtype)
+        plan = ctx.cast_accept_stochastic_plan(s_dtype)
         sto = {"us": ms_sto * 1e3, "temperature": 1.0, "target_minus_draft_logit_std": 0.7,
                "mean_accept_len": float(s_len.float().mean().item()), "cluster_size": plan[0], "slices_cached": plan[1]}
-        del s_tl, s_dl
+        del accept_stochastic
 
     # ---- phase timings (each phase alone; KV working set of the attention graph exceeds 2x L2)
     kv_len.copy_(kv0)  # the capture passes ran the compaction
@@ -474,7 +481,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2_llama8b")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--only", default="", choices=["", "tree", "attention", "accept", "compact"],
+    ap.add_argument("--only", default="", choices=["", "tree", "attention", "accept", "accept_stochastic", "compact"],
                     help="profiling aid: run one phase only, without graphs")
     ap.add_argument("--layers", type=int, default=0,
                     help="profiling aid: override the number of attention layers (smaller device footprint)")

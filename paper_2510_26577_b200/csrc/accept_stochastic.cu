@@ -231,6 +231,15 @@ __global__ void __launch_bounds__(kStoThreads, 1) accept_stochastic_kernel(const
       }
     }
 
+    // the eldest child's test needs two logits and its uniform number: asked for now, used after the sweeps
+    float raw0 = 0.f;
+    double u0 = 0.0;
+    if (k > 0) {
+      const int c0 = sh.kids[0], x0 = sh.tok[c0];
+      if (x0 >= 0 && x0 < p.V) raw0 = (lane & 1) ? to_float(lq[x0]) : to_float(lp[x0]);
+      u0 = p.u_accept[(size_t)b * p.Ncap + c0];
+    }
+
     // ---- softmax statistics of the node's rows: slice maxima, then slice sums of exp(. - slice maximum)
     {
       double mx[2] = {-INFINITY, -INFINITY};
@@ -320,9 +329,9 @@ __global__ void __launch_bounds__(kStoThreads, 1) accept_stochastic_kernel(const
         if (rank == 0 && tid == 0) report(p.st, CAST_ERR_BAD_TREE, b);
         continue;  // not a token: never accepted
       }
-      const double u = p.u_accept[(size_t)b * p.Ncap + c];
-      const double v01 = (lane & 1) ? sto_exp((double)to_float(lq[x]) * p.inv_T - Mq) / Sq
-                                    : sto_exp((double)to_float(lp[x]) * p.inv_T - Mp) / Sp;
+      const double u = j == 0 ? u0 : p.u_accept[(size_t)b * p.Ncap + c];
+      const float raw = j == 0 ? raw0 : ((lane & 1) ? to_float(lq[x]) : to_float(lp[x]));  // odd lanes: draft
+      const double v01 = (lane & 1) ? sto_exp((double)raw * p.inv_T - Mq) / Sq : sto_exp((double)raw * p.inv_T - Mp) / Sp;
       const double px = __shfl_sync(0xffffffffu, v01, 0), qx = __shfl_sync(0xffffffffu, v01, 1);
       const double rx = fmax(0.0, px - a * qx);
       if (u * qx * F <= rx) {
