@@ -94,12 +94,17 @@ typedef struct cast_ctx cast_ctx;
  *   pool_mode        0: rerank over root + every generated candidate;
  *                    1: rerank over root + retained nodes only (N <= sum n_i)
  *   ctx_base_mode    0: context of Eq. 2 is sum_{j<i} n_j; 1: add n_0
+ *   rerank_per_row   0: the rerank sizes the tree from the batch mean of the rank-wise values, as
+ *                    Eq. 1 is printed: every sequence gets the same N. 1: every sequence runs the
+ *                    rerank's Algorithm 1 on its own cumulative values (same cost row), so n_tree
+ *                    differs per sequence; the per-layer sizing stays a batch decision (the next
+ *                    draft forward is one rectangular batch). Needs enable_dr.
  */
 typedef struct {
   double C1, C2, C3;
   int32_t max_batch, vocab, top_k, max_depth, max_width, max_tree, total_token;
   int32_t fifo_len, enable_bp, enable_dp, enable_dr, pool_mode, ctx_base_mode;
-  int32_t reserved;
+  int32_t rerank_per_row;
 } cast_config;
 
 /* Allocates the context and its device scratch on the current device.

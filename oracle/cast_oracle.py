@@ -140,6 +140,7 @@ class OracleConfig:
     enable_dr: int = 0
     pool_mode: int = 0  # 0: every generated candidate + root; 1: root + retained nodes only
     ctx_base_mode: int = 0  # 0: Eq. 2 context = sum_{j<i} n_j; 1: add n_0
+    rerank_per_row: int = 0  # 1: every sequence runs the rerank on its own values (N differs per sequence)
 
     @property
     def width(self) -> int:
@@ -299,18 +300,25 @@ class CastOracle:
         n = min(P, cfg.total_token, Ncap)
         if cfg.enable_dr:
             n = min(n, self._table().Ntab)
-        v = np.array([[np.exp(self.score[b][order[b][s]]) for s in range(n)] for b in range(B)]).mean(axis=0)
-        u = np.cumsum(v)
+        vb = np.array([[np.exp(self.score[b][order[b][s]]) for s in range(n)] for b in range(B)])
+        u_mean = np.cumsum(vb.mean(axis=0))  # Eq. 1: batch mean of the rank-wise values
         for b in range(B):
             self._note_gaps(np.array([self.score[b][p] for p in order[b]]), n)
         if cfg.enable_dr:
             tab = self._table()
             g0 = select_grid(self.n0, tab.L, tab.M)
             c = tab.fT[g0 - 1, :n] / tab.fT[g0 - 1, 0]
-            N = alg1_select_max_valid_index(u, c, cfg.C3)
-            self.stable &= alg1_is_stable(u, c, cfg.C3)
+            if cfg.rerank_per_row:  # u from the sequence's own values instead of the batch mean of Eq. 1
+                Nb = []
+                for b in range(B):
+                    u = np.cumsum(vb[b])
+                    Nb.append(alg1_select_max_valid_index(u, c, cfg.C3))
+                    self.stable &= alg1_is_stable(u, c, cfg.C3)
+            else:
+                Nb = [alg1_select_max_valid_index(u_mean, c, cfg.C3)] * B
+                self.stable &= alg1_is_stable(u_mean, c, cfg.C3)
         else:
-            N = n
+            Nb = [n] * B
         out = {
             "tokens": np.full((B, Ncap), -1, dtype=np.int32),
             "parent": np.full((B, Ncap), -1, dtype=np.int32),
@@ -318,9 +326,10 @@ class CastOracle:
             "anc": np.zeros((B, Ncap, words), dtype=np.uint32),
             "pool_idx": np.full((B, Ncap), -1, dtype=np.int32),
             "scores": np.zeros((B, Ncap), dtype=np.float64),
-            "n_tree": np.full((B,), N, dtype=np.int32),
+            "n_tree": np.array(Nb, dtype=np.int32),
         }
         for b in range(B):
+            N = Nb[b]
             kept = sorted(order[b][:N])  # ascending pool index: root first, parents before children
             lin = {p: t for t, p in enumerate(kept)}
             for t, p in enumerate(kept):
@@ -333,7 +342,7 @@ class CastOracle:
                 out["pool_idx"][b, t] = p
                 out["scores"][b, t] = self.score[b][p]
             out["anc"][b] = ancestor_masks(out["parent"][b], N, words)
-        self.last_u_sel = u
+        self.last_u_sel = u_mean
         return out
 
 

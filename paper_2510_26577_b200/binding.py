@@ -37,7 +37,7 @@ class CastConfig(C.Structure):
         ("max_batch", C.c_int32), ("vocab", C.c_int32), ("top_k", C.c_int32), ("max_depth", C.c_int32),
         ("max_width", C.c_int32), ("max_tree", C.c_int32), ("total_token", C.c_int32),
         ("fifo_len", C.c_int32), ("enable_bp", C.c_int32), ("enable_dp", C.c_int32), ("enable_dr", C.c_int32),
-        ("pool_mode", C.c_int32), ("ctx_base_mode", C.c_int32), ("reserved", C.c_int32),
+        ("pool_mode", C.c_int32), ("ctx_base_mode", C.c_int32), ("rerank_per_row", C.c_int32),
     ]
 
 
@@ -132,10 +132,10 @@ class CastContext:
 
     def __init__(self, *, max_batch, vocab, top_k, max_depth, total_token, max_width=0, max_tree=128,
                  C1=1.0, C2=1.0, C3=1.0, fifo_len=8, enable_bp=0, enable_dp=0, enable_dr=0, pool_mode=0,
-                 ctx_base_mode=0):
+                 ctx_base_mode=0, rerank_per_row=0):
         self.lib = load_library()
         self.cfg = CastConfig(C1, C2, C3, max_batch, vocab, top_k, max_depth, max_width, max_tree, total_token,
-                              fifo_len, enable_bp, enable_dp, enable_dr, pool_mode, ctx_base_mode, 0)
+                              fifo_len, enable_bp, enable_dp, enable_dr, pool_mode, ctx_base_mode, rerank_per_row)
         self.handle = C.c_void_p()
         _check(self.lib.cast_create(C.byref(self.cfg), C.byref(self.handle)), "cast_create")
         self.width = max_width if max_width > 0 else top_k

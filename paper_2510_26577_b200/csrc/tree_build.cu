@@ -756,7 +756,7 @@ struct SelectParams {
   const int32_t* lsort;
   const double* lscore;
   DevState* st;
-  int P, Ncap, words, m, pool_mode, enable_dr;
+  int P, Ncap, words, m, pool_mode, enable_dr, per_row;
   double C3;
   DevTable tab;
   double* sel_score;
@@ -860,7 +860,8 @@ __device__ __noinline__ void select_finalize_phase(const SelectParams& p, int b,
   int n = min(min(peff, p.m), p.Ncap);
   if (p.enable_dr && p.tab.Ntab < n) n = p.tab.Ntab;
   if (tid == 0) s_N = 1;
-  // u_k = sum_{s<=k} v(s), v(s) = batch mean of the rank-s values
+  // u_k = sum_{s<=k} v(s), v(s) = batch mean of the rank-s values (Eq. 1), or this sequence's own
+  // rank-s value when every sequence sizes its tree by itself
   if (tid < 32) {
     double v[4], run = 0.0;
 #pragma unroll
@@ -868,9 +869,13 @@ __device__ __noinline__ void select_finalize_phase(const SelectParams& p, int b,
       const int s = lane * 4 + e;
       double a = 0.0;
       if (s < n) {
+        if (p.per_row) {
+          a = p.sel_value[(size_t)b * p.Ncap + s];
+        } else {
 #pragma unroll 1
-        for (int bb = 0; bb < B; ++bb) a += p.sel_value[(size_t)bb * p.Ncap + s];
-        a /= (double)B;
+          for (int bb = 0; bb < B; ++bb) a += p.sel_value[(size_t)bb * p.Ncap + s];
+          a /= (double)B;
+        }
       }
       run += a;
       v[e] = run;
@@ -1080,6 +1085,7 @@ extern "C" cast_status cast_select_nodes(cast_ctx* c, int32_t* tokens, int32_t* 
   p.P = c->P;
   p.Ncap = c->cfg.max_tree; p.words = c->words; p.m = c->cfg.total_token;
   p.pool_mode = c->cfg.pool_mode; p.enable_dr = c->cfg.enable_dr; p.C3 = c->cfg.C3;
+  p.per_row = c->cfg.enable_dr && c->cfg.rerank_per_row;
   p.tab = c->cur_table;
   p.sel_score = c->sel_score; p.sel_value = c->sel_value; p.sel_idx = c->sel_idx;
   p.tokens = tokens; p.parent = parent; p.depth = depth; p.anc = anc_mask; p.pool_idx = pool_idx;

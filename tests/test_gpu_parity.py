@@ -152,6 +152,22 @@ def test_c3_batch_sweep_cost_model(binding, name):
     check_accept_and_compact(binding, ctx, w, g, o, kv)
 
 
+@pytest.mark.parametrize("name", ["c3_llama8b_b4", "c3_llama8b_b16"])
+def test_c3_rerank_per_sequence_ragged_trees(binding, name):
+    # every sequence sizes its own tree in the rerank: n_tree differs per sequence, and the attention,
+    # acceptance and compaction that follow work on ragged trees
+    # (batch 4: the default seed puts one sequence's rerank within rounding of its threshold; the oracle's
+    # stability flag says so, and the recipe's answer to that is another seed)
+    w = wl.shrink(wl.CONFIGS[name], seed_salt=2 if name == "c3_llama8b_b4" else 0)
+    ctx, g, o, root, kv = build_tree_both(binding, w, rerank_per_row=1)
+    sizes = [int(x) for x in o["n_tree"]]
+    assert len(set(sizes)) > 1 and 1 <= min(sizes) and max(sizes) <= 64, sizes
+    check_attention(binding, ctx, w, g, o, kv, sample=24)
+    check_accept_and_compact(binding, ctx, w, g, o, kv)
+    if name == "c3_llama8b_b4":
+        _run_stochastic(binding, ctx, w, o["tokens"], o["parent"], o["n_tree"], w.depth, 1.0, 0.7)
+
+
 def test_c3_b64_tree_and_accept_reduced_vocab(binding):
     # batch 64 with the full 128k vocabulary takes the oracle minutes; the vocabulary is cut to 8k here
     # (the full-size launch is exercised by bench.py and checked there against invariants)

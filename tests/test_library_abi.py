@@ -43,4 +43,4 @@ def test_config_struct_matches_header_layout():
     from paper_2510_26577_b200.binding import CastConfig
     # 3 doubles + 14 int32 = 80 bytes, no padding (doubles first)
     assert ctypes.sizeof(CastConfig) == 80
-    assert CastConfig.max_batch.offset == 24 and CastConfig.reserved.offset == 76
+    assert CastConfig.max_batch.offset == 24 and CastConfig.rerank_per_row.offset == 76

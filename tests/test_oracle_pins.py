@@ -466,6 +466,41 @@ def test_greedy_accept_edge_cases():
     assert (al[0], bo[0]) == (1, 5)
 
 
+def test_rerank_per_row_equals_independent_single_sequence_runs():
+    """With the per-layer sizing off the expansion of a sequence does not depend on its batch, so a
+    batch reranked per sequence must give every sequence the tree it gets when run alone with the same
+    cost row (same table, same padded context); with one sequence the two modes coincide."""
+    rng = np.random.default_rng(21)
+    V, K, H, m, B = 40, 3, 3, 24, 4
+    L, M, Ntab = 64, 4, 32
+    fT = 1.0 + 0.03 * np.arange(1, Ntab + 1)[None, :] * np.ones((M, 1)) + 0.1 * np.arange(M)[:, None]
+    fD = 0.05 * fT
+    kw = dict(vocab=V, top_k=K, max_depth=H, total_token=m, max_tree=32, enable_dr=1, C3=0.6)
+    root = rng.integers(0, V, size=B)
+    kv = np.array([100, 100, 100, 100])
+    logits = [rng.normal(size=(B, K, V)) * (1.0 + np.arange(B))[:, None, None] for _ in range(H)]  # sharper rows further down
+    tabs = {B: CostTable(B, L, M, Ntab, fT, fD), 1: CostTable(1, L, M, Ntab, fT, fD)}
+
+    def run(cfg_over, rows):
+        o = CastOracle(OracleConfig(**kw, **cfg_over), tabs)
+        o.step_begin(root[rows], kv[rows])
+        for i in range(H):
+            o.expand(i + 1, logits[i][rows])
+        return o.select_nodes()
+
+    batch = run(dict(rerank_per_row=1), np.arange(B))
+    mean = run(dict(rerank_per_row=0), np.arange(B))
+    assert len(set(int(x) for x in mean["n_tree"])) == 1
+    assert len(set(int(x) for x in batch["n_tree"])) > 1  # the recipe does give ragged sizes
+    for b in range(B):
+        for mode in (0, 1):
+            solo = run(dict(rerank_per_row=mode), np.array([b]))
+            assert solo["n_tree"][0] == batch["n_tree"][b]
+            for key in ("tokens", "parent", "depth", "pool_idx"):
+                assert np.array_equal(solo[key][0], batch[key][b]), (b, key)
+            assert np.array_equal(solo["anc"][0], batch["anc"][b])
+
+
 # ------------------------------------------------------ stochastic acceptance
 def test_stochastic_accept_hand_worked_chain_and_sibling():
     """P_T = (0.5, 0.3, 0.2), P_D = (0.2, 0.5, 0.3) at the root. A child with token 1 is accepted iff
