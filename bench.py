@@ -330,6 +330,26 @@ def run_ours(args, w):
                "mean_accept_len": float(s_len.float().mean().item()), "cluster_size": plan[0], "slices_cached": plan[1]}
         del accept_stochastic
 
+    # the draft-side use of the attention kernel: layer by layer, the new layer's tokens against the prefix
+    # and the earlier layers (rows of the growing tree); one verification layer's KV buffer per call
+    dep = tr["depth"].cpu().numpy()
+    windows = []
+    for d_ in range(1, H + 1):
+        first = np.array([int(np.sum(dep[b_, : n_tree[b_]] < d_)) for b_ in range(B)], dtype=np.int32)
+        end = np.array([int(np.sum(dep[b_, : n_tree[b_]] <= d_)) for b_ in range(B)], dtype=np.int32)
+        if int((end - first).sum()) > 0:
+            windows.append((torch.from_numpy(first).to(dev), torch.from_numpy(end).to(dev)))
+
+    def draft_attention():
+        for i_, (first, end) in enumerate(windows):
+            l_ = i_ % nl
+            ctx.cast_tree_attention_rows(q[l_], kc[l_], vc[l_], B, Hq, Hkv, D, w.page_size, table, seq_cap, num_pages,
+                                         kv_len, tr["anc"], end, first, 0.0, out[l_])
+
+    draft_attn_us = None
+    if windows and not args.quick:
+        draft_attn_us = time_graph(capture(draft_attention), max(args.steps, 20), args.warmup) * 1e3 / len(windows)
+
     # ---- phase timings (each phase alone; KV working set of the attention graph exceeds 2x L2)
     kv_len.copy_(kv0)  # the capture passes ran the compaction
     sub_reps = args.steps if args.quick else max(args.steps, 20)
@@ -463,7 +483,8 @@ def run_ours(args, w):
         "gpu_launches": launches,
         "clocks": clocks,
         "phases": {"tree_build_us": ms_tree * 1e3, "attention_us_per_layer": attn_us, "accept_us": ms_acc * 1e3,
-                   "compact_us": ms_cmp * 1e3, "accept_stochastic": sto},
+                   "compact_us": ms_cmp * 1e3, "accept_stochastic": sto,
+                   "draft_attention_us_per_layer": draft_attn_us},
         "roofline": {"kernel": "cast_tree_attention (one layer)", "bound": "hbm", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_source": which, "traffic": NCU_ATTENTION_TRAFFIC.get(w.name),
                      "algorithmic_bytes": attn_bytes},

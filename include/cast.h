@@ -12,6 +12,7 @@
  *   cast_select_nodes    dynamic rerank (Sec. "Dynamic Reranking Stage"),
  *                        linearisation + ancestor mask (Sec. "Tree Reranking Phase")
  *   cast_tree_attention  verification attention under that mask
+ *   cast_tree_attention_rows  the same for the rows of one layer of the growing tree (draft side)
  *   cast_accept          greedy acceptance (Sec. "Speculative Decoding", T = 0)
  *   cast_accept_stochastic  the same section's rule at T > 0, with residual resampling
  *   cast_compact_kv      accepted KV rows made contiguous
@@ -198,6 +199,23 @@ CAST_API cast_status cast_tree_attention(cast_ctx* ctx, const void* q, const voi
                                 const int32_t* page_table, int seq_capacity, int num_pages,
                                 const int32_t* kv_len, const uint32_t* anc_mask, const int32_t* n_tree,
                                 float scale, void* out, void* stream);
+
+/*
+ * cast_tree_attention restricted to the output rows t >= first_row[b] of every sequence: the tree
+ * tokens before first_row[b] serve as context only (their K/V rows in the cache and their bits in
+ * the masks are used, their queries are not read and their output rows are left untouched). This
+ * is the draft model's attention while the tree grows (Sec. "Tree Expansion Phase"; Eq. 2 names its
+ * context sum_{j<i} n_j): the linear order of a tree is creation order, so the tree after layer i is
+ * a prefix of the final one; with n_tree[b] = tokens up to and including layer i and first_row[b] =
+ * tokens before layer i the call computes layer i's n_i query rows against the prefix and the earlier
+ * layers. first_row [B] device int32 (clamped to [0, n_tree[b]]); NULL means 0 everywhere, which is
+ * cast_tree_attention. All other arguments, layouts and errors as for cast_tree_attention.
+ */
+CAST_API cast_status cast_tree_attention_rows(cast_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
+                                     cast_dtype dtype, int B, int Hq, int Hkv, int D, int page_size,
+                                     const int32_t* page_table, int seq_capacity, int num_pages,
+                                     const int32_t* kv_len, const uint32_t* anc_mask, const int32_t* n_tree,
+                                     const int32_t* first_row, float scale, void* out, void* stream);
 
 /*
  * Greedy acceptance: g[t] = argmax of target_logits[b,t,:] (ties: lower id).

@@ -27,7 +27,7 @@ EXPORTS = [
     "cast_create", "cast_destroy", "cast_status_string", "cast_set_cost_tables", "cast_state_export",
     "cast_state_import", "cast_step_begin", "cast_tree_expand", "cast_select_nodes", "cast_tree_attention",
     "cast_accept", "cast_compact_kv", "cast_poll_status", "cast_step_info", "cast_accept_static",
-    "cast_accept_stochastic", "cast_accept_stochastic_plan",
+    "cast_accept_stochastic", "cast_accept_stochastic_plan", "cast_tree_attention_rows",
 ]
 
 
@@ -74,6 +74,8 @@ def load_library() -> C.CDLL:
         "cast_select_nodes": [vp, i32p, i32p, i32p, vp, i32p, vp, i32p, vp],
         "cast_tree_attention": [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32p, i32, i32, i32p, vp, i32p,
                                 C.c_float, vp, vp],
+        "cast_tree_attention_rows": [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32p, i32, i32, i32p, vp, i32p,
+                                     i32p, C.c_float, vp, vp],
         "cast_accept": [vp, vp, i32, i32, i32p, i32p, i32p, vp, i32p, i32p, i32p, i32p, vp],
         "cast_compact_kv": [vp, vp, vp, i32, i32, i32, C.c_size_t, i32, i32, i32, i32p, i32, i32, i32p, i32p, i32p,
                             vp],
@@ -192,6 +194,13 @@ class CastContext:
                                             Hkv, D, page_size, _ptr(page_table), seq_capacity, num_pages,
                                             _ptr(kv_len), _ptr(anc_mask), _ptr(n_tree), float(scale), _ptr(out),
                                             _stream(stream)), "cast_tree_attention")
+
+    def cast_tree_attention_rows(self, q, k_cache, v_cache, B, Hq, Hkv, D, page_size, page_table, seq_capacity,
+                                 num_pages, kv_len, anc_mask, n_tree, first_row, scale, out, stream=None):
+        _check(self.lib.cast_tree_attention_rows(self.handle, _ptr(q), _ptr(k_cache), _ptr(v_cache), _dtype_code(q), B,
+                                                 Hq, Hkv, D, page_size, _ptr(page_table), seq_capacity, num_pages,
+                                                 _ptr(kv_len), _ptr(anc_mask), _ptr(n_tree), _ptr(first_row),
+                                                 float(scale), _ptr(out), _stream(stream)), "cast_tree_attention_rows")
 
     def cast_accept(self, target_logits, B, tokens, parent, depth, anc_mask, n_tree, accept_len, accept_path,
                     bonus_token, stream=None):

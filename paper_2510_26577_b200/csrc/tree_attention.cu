@@ -18,8 +18,8 @@ namespace cast {
 // implemented in tree_attention_tc.cu; returns false when the shape is not taken there
 bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const void* v, int B, int Hq, int Hkv, int D,
                               int page_size, const int32_t* page_table, int seq_capacity, int num_pages,
-                              const int32_t* kv_len, const uint32_t* anc, const int32_t* n_tree, float scale, void* out,
-                              cudaStream_t stream, cast_status* status);
+                              const int32_t* kv_len, const uint32_t* anc, const int32_t* n_tree, const int32_t* first_row,
+                              float scale, void* out, cudaStream_t stream, cast_status* status);
 }
 
 namespace {
@@ -38,6 +38,7 @@ struct AttnParams {
   const int32_t* page_table;
   const int32_t* kv_len;
   const int32_t* n_tree;
+  const int32_t* first_row;  // [B] or null: output rows start at this tree token
   const uint32_t* anc;
   float scale;
   float* part_o;   // [B][Hq][Ncap][nsplit][D]
@@ -86,7 +87,9 @@ __global__ void __launch_bounds__(kThreads) tree_attn_cc_kernel(const AttnParams
   int L = p.kv_len[b];
   if (L < 0) L = 0;
   const int G = p.G;
-  const int rows_total = N * G;
+  int F = p.first_row != nullptr ? p.first_row[b] : 0;  // tokens before F are context only
+  F = F < 0 ? 0 : (F > N ? N : F);
+  const int rows_total = (N - F) * G;
   const int row0 = rb * kRB;
   if (row0 >= rows_total) return;
   const int max_pos = p.page_size == 0 ? p.seq_capacity : p.seq_capacity * p.page_size;
@@ -104,7 +107,7 @@ __global__ void __launch_bounds__(kThreads) tree_attn_cc_kernel(const AttnParams
     const int r = i / CPR, ch = i % CPR, row = row0 + r;
     float f[CH];
     if (row < rows_total) {
-      const int t = row / G, g = row % G;
+      const int t = F + row / G, g = row % G;
       load_chunk<T>(q + (((size_t)b * p.Ncap + t) * p.Hq + kvh * G + g) * D + ch * CH, f);
     } else {
 #pragma unroll
@@ -118,7 +121,7 @@ __global__ void __launch_bounds__(kThreads) tree_attn_cc_kernel(const AttnParams
     row_l[tid] = 0.f;
     const int row = row0 + tid;
     for (int w = 0; w < CAST_MAX_TREE / 32; ++w)
-      anc_s[tid][w] = (row < rows_total && w < p.words) ? p.anc[((size_t)b * p.Ncap + row / G) * p.words + w] : 0u;
+      anc_s[tid][w] = (row < rows_total && w < p.words) ? p.anc[((size_t)b * p.Ncap + F + row / G) * p.words + w] : 0u;
   }
   float o[4][DC];
 #pragma unroll
@@ -261,7 +264,7 @@ __global__ void __launch_bounds__(kThreads) tree_attn_cc_kernel(const AttnParams
   for (int rr = 0; rr < 4; ++rr) {
     const int r = 4 * warp + rr, row = row0 + r;
     if (row >= rows_total) continue;
-    const int t = row / G, h = kvh * G + row % G;
+    const int t = F + row / G, h = kvh * G + row % G;
     const size_t pr = (((size_t)b * p.Hq + h) * p.Ncap + t) * p.nsplit + split;
 #pragma unroll
     for (int e = 0; e < DC; ++e) p.part_o[pr * D + lane * DC + e] = o[rr][e];
@@ -279,7 +282,7 @@ __global__ void __launch_bounds__(D) attn_combine_kernel(const AttnParams p) {
   T* out = reinterpret_cast<T*>(p.out) + (((size_t)b * p.Ncap + t) * p.Hq + h) * D;
   int N = p.n_tree[b];
   N = N > p.Ncap ? p.Ncap : N;
-  if (t >= N) return;
+  if (t >= N || (p.first_row != nullptr && t < p.first_row[b])) return;
   const size_t pr = (((size_t)b * p.Hq + h) * p.Ncap + t) * p.nsplit;
   float M = -INFINITY;
   for (int s = 0; s < p.nsplit; ++s) M = fmaxf(M, p.part_ml[(pr + s) * 2]);
@@ -327,11 +330,11 @@ cast_status launch_cc(cast_ctx* c, AttnParams& p, cudaStream_t s) {
 
 }  // namespace
 
-extern "C" cast_status cast_tree_attention(cast_ctx* c, const void* q, const void* k_cache, const void* v_cache,
-                                           cast_dtype dtype, int B, int Hq, int Hkv, int D, int page_size,
-                                           const int32_t* page_table, int seq_capacity, int num_pages,
-                                           const int32_t* kv_len, const uint32_t* anc_mask, const int32_t* n_tree,
-                                           float scale, void* out, void* stream) {
+extern "C" cast_status cast_tree_attention_rows(cast_ctx* c, const void* q, const void* k_cache, const void* v_cache,
+                                                cast_dtype dtype, int B, int Hq, int Hkv, int D, int page_size,
+                                                const int32_t* page_table, int seq_capacity, int num_pages,
+                                                const int32_t* kv_len, const uint32_t* anc_mask, const int32_t* n_tree,
+                                                const int32_t* first_row, float scale, void* out, void* stream) {
   if (!c || !q || !k_cache || !v_cache || !kv_len || !anc_mask || !n_tree || !out || B < 1 || Hq < 1 || Hkv < 1 ||
       page_size < 0 || seq_capacity < 1 || (page_size > 0 && (!page_table || num_pages < 1)))
     return CAST_ERR_INVALID_ARG;
@@ -344,7 +347,7 @@ extern "C" cast_status cast_tree_attention(cast_ctx* c, const void* q, const voi
   if (dtype == CAST_BF16) {
     cast_status st = CAST_OK;
     if (tree_attention_tc_launch(c, q, k_cache, v_cache, B, Hq, Hkv, D, page_size, page_table, seq_capacity, num_pages,
-                                 kv_len, anc_mask, n_tree, scale, out, s, &st))
+                                 kv_len, anc_mask, n_tree, first_row, scale, out, s, &st))
       return st;
   }
   AttnParams p;
@@ -352,8 +355,17 @@ extern "C" cast_status cast_tree_attention(cast_ctx* c, const void* q, const voi
   p.B = B; p.Ncap = c->cfg.max_tree; p.Hq = Hq; p.Hkv = Hkv; p.G = Hq / Hkv;
   p.page_size = page_size; p.seq_capacity = seq_capacity; p.num_pages = num_pages; p.words = c->words;
   p.nsplit = 1;
-  p.page_table = page_table; p.kv_len = kv_len; p.n_tree = n_tree; p.anc = anc_mask;
+  p.page_table = page_table; p.kv_len = kv_len; p.n_tree = n_tree; p.first_row = first_row; p.anc = anc_mask;
   p.scale = scale; p.part_o = nullptr; p.part_ml = nullptr; p.st = c->state;
   if (dtype == CAST_F32) return D == 64 ? launch_cc<float, 64>(c, p, s) : launch_cc<float, 128>(c, p, s);
   return D == 64 ? launch_cc<__nv_bfloat16, 64>(c, p, s) : launch_cc<__nv_bfloat16, 128>(c, p, s);
+}
+
+extern "C" cast_status cast_tree_attention(cast_ctx* c, const void* q, const void* k_cache, const void* v_cache,
+                                           cast_dtype dtype, int B, int Hq, int Hkv, int D, int page_size,
+                                           const int32_t* page_table, int seq_capacity, int num_pages,
+                                           const int32_t* kv_len, const uint32_t* anc_mask, const int32_t* n_tree,
+                                           float scale, void* out, void* stream) {
+  return cast_tree_attention_rows(c, q, k_cache, v_cache, dtype, B, Hq, Hkv, D, page_size, page_table, seq_capacity,
+                                  num_pages, kv_len, anc_mask, n_tree, nullptr, scale, out, stream);
 }

@@ -98,6 +98,7 @@ struct TcParams {
   const int32_t* page_table;
   const int32_t* kv_len;
   const int32_t* n_tree;
+  const int32_t* first_row;  // [B] or null: output rows start at this tree token (the tokens before it are context only)
   const uint32_t* anc;
   float scale_log2;
   DevState* st;
@@ -280,7 +281,7 @@ __device__ __forceinline__ int clampi(int x, int lo, int hi) { return x < lo ? l
 // same time. Clusters past the count exit at once. Every warp computes the same values (all 32
 // lanes must call).
 struct WorkItem {
-  int b, kvh, rb, split, nsplit, N, L;
+  int b, kvh, rb, split, nsplit, N, L, F;
   bool valid;   // the cluster has work
   bool active;  // this CTA has a row block (an inactive CTA of a valid cluster only keeps the barriers in step)
 };
@@ -289,20 +290,22 @@ __device__ __forceinline__ WorkItem decode_work(const TcParams& p, int cid, int 
   constexpr int KB = CAST_MAX_BATCH / 32;
   const int lane = threadIdx.x & 31;
   const int max_pos = p.page_size == 0 ? p.seq_capacity : p.seq_capacity * p.page_size;
-  int Nv[KB], Lv[KB], tl[KB], nr[KB], cnt[KB], off[KB];
+  int Nv[KB], Lv[KB], Fv[KB], tl[KB], nr[KB], cnt[KB], off[KB];
 #pragma unroll
   for (int k = 0; k < KB; ++k) {  // all loads first: one memory round trip
     const int bb = k * 32 + lane;
     Nv[k] = bb < p.B ? p.n_tree[bb] : 0;
     Lv[k] = bb < p.B ? p.kv_len[bb] : 0;
+    Fv[k] = (p.first_row != nullptr && bb < p.B) ? p.first_row[bb] : 0;
   }
 #pragma unroll
   for (int k = 0; k < KB; ++k) {
     Nv[k] = clampi(Nv[k], 0, p.Nmax);
+    Fv[k] = clampi(Fv[k], 0, Nv[k]);
     Lv[k] = Lv[k] < 0 ? 0 : Lv[k];
     int total = Lv[k] + Nv[k];
     total = total > max_pos ? max_pos : total;
-    nr[k] = (Nv[k] * p.G + kBM - 1) / kBM;
+    nr[k] = ((Nv[k] - Fv[k]) * p.G + kBM - 1) / kBM;
     tl[k] = nr[k] > 0 ? (total + kBN - 1) / kBN : 0;
     cnt[k] = p.Hkv * ((nr[k] + p.rpc - 1) / p.rpc);
     off[k] = 0;
@@ -328,7 +331,7 @@ __device__ __forceinline__ WorkItem decode_work(const TcParams& p, int cid, int 
   }
   WorkItem w;
   w.valid = w.active = false;
-  w.b = w.kvh = w.rb = w.split = w.N = w.L = 0;
+  w.b = w.kvh = w.rb = w.split = w.N = w.L = w.F = 0;
   w.nsplit = 1;
 #pragma unroll
   for (int k = 0; k < KB; ++k) {
@@ -338,6 +341,7 @@ __device__ __forceinline__ WorkItem decode_work(const TcParams& p, int cid, int 
       const int local = cid - __shfl_sync(0xffffffffu, off[k], bl);
       const int nrb = __shfl_sync(0xffffffffu, nr[k], bl);
       w.N = __shfl_sync(0xffffffffu, Nv[k], bl);
+      w.F = __shfl_sync(0xffffffffu, Fv[k], bl);
       w.L = __shfl_sync(0xffffffffu, Lv[k], bl);
       w.b = k * 32 + bl;
       w.kvh = local % p.Hkv;
@@ -465,21 +469,23 @@ __device__ __forceinline__ WorkItem decode_work_chunked(const TcParams& p, int i
   constexpr int KB = CAST_MAX_BATCH / 32;
   const int lane = threadIdx.x & 31;
   const int max_pos = p.page_size == 0 ? p.seq_capacity : p.seq_capacity * p.page_size;
-  int Nv[KB], Lv[KB], tl[KB], nr[KB];
+  int Nv[KB], Lv[KB], Fv[KB], tl[KB], nr[KB];
 #pragma unroll
   for (int k = 0; k < KB; ++k) {  // all loads first: one memory round trip
     const int bb = k * 32 + lane;
     Nv[k] = bb < p.B ? p.n_tree[bb] : 0;
     Lv[k] = bb < p.B ? p.kv_len[bb] : 0;
+    Fv[k] = (p.first_row != nullptr && bb < p.B) ? p.first_row[bb] : 0;
   }
   int base = 0, T = 0, tmax = 0;
 #pragma unroll
   for (int k = 0; k < KB; ++k) {
     Nv[k] = clampi(Nv[k], 0, p.Nmax);
+    Fv[k] = clampi(Fv[k], 0, Nv[k]);
     Lv[k] = Lv[k] < 0 ? 0 : Lv[k];
     int total = Lv[k] + Nv[k];
     total = total > max_pos ? max_pos : total;
-    nr[k] = (Nv[k] * p.G + kBM - 1) / kBM;
+    nr[k] = ((Nv[k] - Fv[k]) * p.G + kBM - 1) / kBM;
     tl[k] = nr[k] > 0 ? (total + kBN - 1) / kBN : 0;
     base += p.Hkv * nr[k];
     T += p.Hkv * nr[k] * tl[k];
@@ -551,7 +557,7 @@ __device__ __forceinline__ WorkItem decode_work_chunked(const TcParams& p, int i
   }
   WorkItem w;
   w.valid = w.active = false;
-  w.b = w.kvh = w.rb = w.split = w.N = w.L = 0;
+  w.b = w.kvh = w.rb = w.split = w.N = w.L = w.F = 0;
   w.nsplit = 1;
 #pragma unroll
   for (int k = 0; k < KB; ++k) {
@@ -561,6 +567,7 @@ __device__ __forceinline__ WorkItem decode_work_chunked(const TcParams& p, int i
       const int local = idx - __shfl_sync(0xffffffffu, off[k], bl);
       w.nsplit = __shfl_sync(0xffffffffu, ns[k], bl);
       w.N = __shfl_sync(0xffffffffu, Nv[k], bl);
+      w.F = __shfl_sync(0xffffffffu, Fv[k], bl);
       w.L = __shfl_sync(0xffffffffu, Lv[k], bl);
       w.b = k * 32 + bl;
       w.kvh = local % p.Hkv;
@@ -660,7 +667,8 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
   if (!wk.valid) return;  // the whole cluster leaves
   const int b = wk.b, kvh = wk.kvh, rb = wk.rb, split = wk.split, N = wk.N, L = wk.L;
   const int nsplit = wk.nsplit;
-  const int G = p.G, rows_total = N * G, row0 = rb * kBM;
+  const int G = p.G, F = wk.F, rows_total = (N - F) * G, row0 = rb * kBM;
+  const int grow0 = F * G + row0;  // the row block's first row counted from tree token 0
   const int max_pos = p.page_size == 0 ? p.seq_capacity : p.seq_capacity * p.page_size;
   int total = L + N;
   if (total > max_pos) {
@@ -690,7 +698,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
   const int r = tid & (kBM - 1);  // softmax role: the query row of this thread
   const int row = row0 + r;
   const bool row_ok = warp < 4 && row < rows_total;
-  const int t_tok = row_ok ? row / G : 0, h_q = kvh * G + (row_ok ? row % G : 0);
+  const int t_tok = row_ok ? F + row / G : 0, h_q = kvh * G + (row_ok ? row % G : 0);
 
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kSmemBar);
   static_assert(kStagesK <= 3 && kStagesV <= 2, "barrier slots");
@@ -1161,7 +1169,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
   const int rows_here = rows_total - row0 < kBM ? rows_total - row0 : kBM;
   if (nsplit == 1) {
     for (int rr = warp; rr < rows_here; rr += kThreadsTC / 32) {
-      const int grow = row0 + rr, tt = grow / G, hh = kvh * G + grow % G;
+      const int grow = grow0 + rr, tt = grow / G, hh = kvh * G + grow % G;
       const float4 o4 = *reinterpret_cast<const float4*>(stage_o + rr * kStageStride + lane * 4);
       const float l_tot = stage_ml[rr * 2 + 1];
       const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
@@ -1175,7 +1183,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     // global-merge mode: partials to the workspace; the last split of this row block to finish merges
     const __half* sh = reinterpret_cast<const __half*>(stage_o);
     for (int rr = warp; rr < rows_here; rr += kThreadsTC / 32) {
-      const int grow = row0 + rr, tt = grow / G, hh = kvh * G + grow % G;
+      const int grow = grow0 + rr, tt = grow / G, hh = kvh * G + grow % G;
       const size_t pr = (((size_t)b * p.Hq + hh) * p.Ncap + tt) * p.nsplit_max + split;
       __stcg(reinterpret_cast<uint2*>(p.part_o + pr * kHD + lane * 4),
              *reinterpret_cast<const uint2*>(sh + rr * kStageStrideH + lane * 4));
@@ -1196,16 +1204,16 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     }
     __syncthreads();
     if (*last_s) {
-      if (nsplit <= 2) merge_rows_global<8, 2>(p, b, kvh, row0, rows_here, nsplit);
-      else if (nsplit <= 4) merge_rows_global<4, 4>(p, b, kvh, row0, rows_here, nsplit);
-      else merge_rows_global<2, kMaxSplit>(p, b, kvh, row0, rows_here, nsplit);
+      if (nsplit <= 2) merge_rows_global<8, 2>(p, b, kvh, grow0, rows_here, nsplit);
+      else if (nsplit <= 4) merge_rows_global<4, 4>(p, b, kvh, grow0, rows_here, nsplit);
+      else merge_rows_global<2, kMaxSplit>(p, b, kvh, grow0, rows_here, nsplit);
     }
   } else {
     const uint32_t so_s = smem_u32(stage_o), sml_s = smem_u32(stage_ml);
     const int rank0 = crank - split;  // first CTA of this row block's split group
-    if (nsplit <= 2) merge_rows<8, 2>(p, so_s, sml_s, rank0, b, kvh, row0, rows_here, nsplit, split);
-    else if (nsplit <= 4) merge_rows<4, 4>(p, so_s, sml_s, rank0, b, kvh, row0, rows_here, nsplit, split);
-    else merge_rows<2, kMaxSplit>(p, so_s, sml_s, rank0, b, kvh, row0, rows_here, nsplit, split);
+    if (nsplit <= 2) merge_rows<8, 2>(p, so_s, sml_s, rank0, b, kvh, grow0, rows_here, nsplit, split);
+    else if (nsplit <= 4) merge_rows<4, 4>(p, so_s, sml_s, rank0, b, kvh, grow0, rows_here, nsplit, split);
+    else merge_rows<2, kMaxSplit>(p, so_s, sml_s, rank0, b, kvh, grow0, rows_here, nsplit, split);
   }
   TC_MARK(7);
   TC_CTA_LOG(1, gtimer());
@@ -1254,8 +1262,8 @@ bool make_kv_map(CUtensorMap* map, const void* base, int B, int Hkv, int page_si
 
 bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const void* v, int B, int Hq, int Hkv, int D,
                               int page_size, const int32_t* page_table, int seq_capacity, int num_pages,
-                              const int32_t* kv_len, const uint32_t* anc, const int32_t* n_tree, float scale, void* out,
-                              cudaStream_t stream, cast_status* status) {
+                              const int32_t* kv_len, const uint32_t* anc, const int32_t* n_tree, const int32_t* first_row,
+                              float scale, void* out, cudaStream_t stream, cast_status* status) {
   if (D != kHD || !(scale > 0.f)) return false;
   if (page_size != 0 && (page_size < 8 || page_size > kBN || (kBN % page_size) != 0 || (page_size % 8) != 0))
     return false;
@@ -1296,7 +1304,7 @@ bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const v
   p.q = (const __nv_bfloat16*)q; p.out = (__nv_bfloat16*)out;
   p.B = B; p.Ncap = Ncap; p.Nmax = Nmax; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.page_size = page_size;
   p.seq_capacity = seq_capacity; p.num_pages = num_pages; p.words = c->words;
-  p.page_table = page_table; p.kv_len = kv_len; p.n_tree = n_tree; p.anc = anc;
+  p.page_table = page_table; p.kv_len = kv_len; p.n_tree = n_tree; p.first_row = first_row; p.anc = anc;
   p.scale_log2 = scale * 1.4426950408889634f;
   p.st = c->state;
   p.num_sms = c->num_sms; p.nrb = nrb;

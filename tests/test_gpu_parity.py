@@ -361,6 +361,48 @@ def test_attention_arbitrary_trees_ragged(binding, dtype, D, Hq, Hkv, page):
         assert np.isnan(got[b, int(n_tree[b]):]).all()
 
 
+@pytest.mark.parametrize("name", ["c1_tiny", "c2_llama8b", "c4_llama70b_n128"])
+def test_attention_rows_of_the_growing_tree(binding, name):
+    """The draft-side use: layer by layer, the new layer's tokens attend to the prefix and the earlier
+    layers (the linear order is creation order, so the tree after layer d is a prefix of the final tree).
+    c1: CUDA-core path; c2, c4: tensor-core path, cluster and global-merge launches."""
+    w = wl.CONFIGS[name]
+    ctx, g, o, root, kv = build_tree_both(binding, w)
+    B, Hq = w.batch, w.q_heads
+    q = wl.query(w, 0, "cpu").cuda()
+    k, v = (t.cuda() for t in wl.kv_cache(w, 0, "cpu"))
+    table, num_pages = wl.page_table(w, "cuda")
+    tab = table.cpu().numpy() if table is not None else None
+    f32 = lambda t: t.float().cpu().numpy()
+    qf, kf, vf = f32(q), f32(k), f32(v)
+    depth = o["depth"]
+    assert all(np.all(np.diff(depth[b, : int(o["n_tree"][b])]) >= 0) for b in range(B))  # creation order is layer order
+    rng = np.random.default_rng(3)
+    for d in range(1, int(depth.max()) + 1):
+        first = np.array([int(np.sum(depth[b, : int(o["n_tree"][b])] < d)) for b in range(B)], dtype=np.int32)
+        end = np.array([int(np.sum(depth[b, : int(o["n_tree"][b])] <= d)) for b in range(B)], dtype=np.int32)
+        out = gpu_attention(ctx, w, q, k, v, table, num_pages, kv, g["dev"]["anc"], torch.from_numpy(end).cuda(),
+                            first_row=torch.from_numpy(first).cuda())
+        assert ctx.cast_poll_status()[0] == 0
+        got = to_f64(out)
+        only = set()
+        for b in range(B):
+            assert np.isnan(got[b, : first[b]]).all() and np.isnan(got[b, end[b]:]).all()  # rows outside the window: untouched
+            assert np.isfinite(got[b, first[b]: end[b]]).all()
+            if first[b] == end[b]:  # this sequence kept nothing of layer d
+                continue
+            for t in {int(first[b]), int(end[b]) - 1} | {int(x) for x in rng.integers(first[b], end[b], size=2)}:
+                for h in {0, Hq - 1, int(rng.integers(0, Hq))}:
+                    only.add((b, t, h))
+        ref = tree_attention(qf, kf, vf, w.page_size, tab, kv.cpu().numpy(), o["anc"], end, None, only)
+        err = max(np.max(np.abs(got[i] - ref[i])) for i in only)
+        assert err <= attention_tolerance(w.kv_dtype), (d, err)
+    # an empty window writes nothing; a null first_row is the plain call
+    nt = g["dev"]["n_tree"]
+    out = gpu_attention(ctx, w, q, k, v, table, num_pages, kv, g["dev"]["anc"], nt, first_row=nt.clone())
+    assert torch.isnan(out).all()
+
+
 @pytest.mark.parametrize("name,n", [("c3_llama8b_b64", 9), ("c3_llama8b_b16", 12), ("c4_llama70b_n32", 32)])
 def test_attention_full_size_launch_sampled(binding, name, n):
     """The launch shapes bench.py times (plain, global-merge and cluster mode at full cache sizes), on
