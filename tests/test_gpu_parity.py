@@ -150,6 +150,8 @@ def test_c3_batch_sweep_cost_model(binding, name):
     assert 1 <= int(o["n_tree"][0]) <= 64
     check_attention(binding, ctx, w, g, o, kv, sample=24)
     check_accept_and_compact(binding, ctx, w, g, o, kv)
+    if name == "c3_llama8b_b16":  # more sequences than clusters fit at a time
+        _run_stochastic(binding, ctx, w, o["tokens"], o["parent"], o["n_tree"], w.depth, 1.0, 0.7)
 
 
 @pytest.mark.parametrize("name", ["c3_llama8b_b4", "c3_llama8b_b16"])
@@ -200,6 +202,7 @@ def test_c5_qwen_long_context(binding):
     assert list(o["n_tree"]) == [96] * 4
     check_attention(binding, ctx, w, g, o, kv, sample=8)
     check_accept_and_compact(binding, ctx, w, g, o, kv)
+    _run_stochastic(binding, ctx, w, o["tokens"], o["parent"], o["n_tree"], w.depth, 0.9, 0.5)  # the largest cached slice
 
 
 # ------------------------------------------------------------------ tree-build variants and edge cases
