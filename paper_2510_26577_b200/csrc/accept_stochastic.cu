@@ -104,6 +104,29 @@ __device__ __forceinline__ double sto_exp(double x) {
   return xin >= -708.0 ? res : (xin != xin ? xin : 0.0);
 }
 
+// The same to the same accuracy in half the fp64 instructions, for the pass that evaluates 2 V / cluster-size
+// exponentials per node: x = (128 n + j) ln2/128 + r, |r| <= ln2/256, e^x = 2^n * tab[j] * (degree-5 Taylor
+// polynomial of e^r, remainder below 1e-18), tab[j] = 2^(j/128) from shared memory.
+__device__ __forceinline__ double sto_exp_tab(double x, const double* tab) {
+  const double xin = x;
+  x = fmax(x, -708.0);
+  const double kMagic = 6755399441055744.0;
+  const double tn = fma(x, 128.0 * 1.4426950408889634074, kMagic);
+  const int k = __double2loint(tn);  // round(x * 128 / ln2), negative or zero
+  const double kd = tn - kMagic;
+  double r = fma(kd, -6.93147180369123816490e-01 / 128.0, x);
+  r = fma(kd, -1.90821492927058770002e-10 / 128.0, r);
+  double y = 8.33333333333333333333e-03;
+  y = fma(y, r, 4.16666666666666666667e-02);
+  y = fma(y, r, 1.66666666666666666667e-01);
+  y = fma(y, r, 0.5);
+  y = fma(y, r, 1.0);
+  y = fma(y, r, 1.0);
+  y *= tab[k & 127];
+  const double res = __hiloint2double(__double2hiint(y) + (k >> 7) * 1048576, __double2loint(y));
+  return xin >= -708.0 ? res : (xin != xin ? xin : 0.0);
+}
+
 struct StoShared {
   double xch[2][kStoMaxCluster][4];  // records of the cluster's CTAs, double-buffered by exchange parity
   double wred[kStoWarps][4];
@@ -113,6 +136,7 @@ struct StoShared {
   int32_t nkids;
   int32_t pick_lo, pick_hi;
   double wscan[kStoWarps];
+  double tab[128];  // 2^(j/128)
 };
 
 // Block-wide reduction of up to four values per thread (sum, or maximum for OP_MAX); every thread returns
@@ -171,6 +195,7 @@ __global__ void __launch_bounds__(kStoThreads, 1) accept_stochastic_kernel(const
     if (rank == 0 && tid == 0) report(p.st, CAST_ERR_BAD_TREE, b);
     N = N < 1 ? 1 : p.Ncap;
   }
+  if (tid >= kStoThreads - 128) sh.tab[tid - (kStoThreads - 128)] = exp2((double)(tid - (kStoThreads - 128)) * (1.0 / 128.0));
   if (tid < CAST_MAX_TREE) {
     sh.par[tid] = tid < N ? p.parent[(size_t)b * p.Ncap + tid] : -2;
     sh.tok[tid] = tid < N ? p.tokens[(size_t)b * p.Ncap + tid] : 0;
@@ -191,10 +216,10 @@ __global__ void __launch_bounds__(kStoThreads, 1) accept_stochastic_kernel(const
 
   // unnormalised slice entries: p~(i) * cp = P_T(begin + i), q~(i) * cq = P_D(begin + i)
   auto pt = [&](int i) -> double {
-    return CACHED ? ep[i] : sto_exp((double)to_float(lp[begin + i]) * p.inv_T - (Mp_loc > -INFINITY ? Mp_loc : 0.0));
+    return CACHED ? ep[i] : sto_exp_tab((double)to_float(lp[begin + i]) * p.inv_T - (Mp_loc > -INFINITY ? Mp_loc : 0.0), sh.tab);
   };
   auto qt = [&](int i) -> double {
-    return CACHED ? eq[i] : sto_exp((double)to_float(lq[begin + i]) * p.inv_T - (Mq_loc > -INFINITY ? Mq_loc : 0.0));
+    return CACHED ? eq[i] : sto_exp_tab((double)to_float(lq[begin + i]) * p.inv_T - (Mq_loc > -INFINITY ? Mq_loc : 0.0), sh.tab);
   };
 
   for (;;) {
@@ -264,8 +289,8 @@ __global__ void __launch_bounds__(kStoThreads, 1) accept_stochastic_kernel(const
       if (has_q) {
 #pragma unroll 4
         for (int i = tid; i < len; i += kStoThreads) {
-          const double e0 = sto_exp((CACHED ? ep[i] : (double)to_float(lp[begin + i]) * p.inv_T) - ref_p);
-          const double e1 = sto_exp((CACHED ? eq[i] : (double)to_float(lq[begin + i]) * p.inv_T) - ref_q);
+          const double e0 = sto_exp_tab((CACHED ? ep[i] : (double)to_float(lp[begin + i]) * p.inv_T) - ref_p, sh.tab);
+          const double e1 = sto_exp_tab((CACHED ? eq[i] : (double)to_float(lq[begin + i]) * p.inv_T) - ref_q, sh.tab);
           if (CACHED) {
             ep[i] = e0;
             eq[i] = e1;
@@ -276,7 +301,7 @@ __global__ void __launch_bounds__(kStoThreads, 1) accept_stochastic_kernel(const
       } else {
 #pragma unroll 4
         for (int i = tid; i < len; i += kStoThreads) {
-          const double e0 = sto_exp((CACHED ? ep[i] : (double)to_float(lp[begin + i]) * p.inv_T) - ref_p);
+          const double e0 = sto_exp_tab((CACHED ? ep[i] : (double)to_float(lp[begin + i]) * p.inv_T) - ref_p, sh.tab);
           if (CACHED) ep[i] = e0;
           sm[0] += e0;
         }
