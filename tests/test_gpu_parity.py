@@ -590,6 +590,19 @@ def test_accept_stochastic_special_cases(binding):
     ol = _run_stochastic(binding, ctx, w, tokens, parent, n_tree, H, 1.0, inputs=(hot, dl, ua, ub))
     gl, gp, gb = greedy_accept(to_f64(hot), tokens, parent, n_tree, H)
     assert np.array_equal(ol, gl)
+    # what only the device can see goes to the status word: a token outside the vocabulary, a NaN logit
+    alen, apath, bonus = (torch.zeros(B, dtype=torch.int32, device="cuda"), torch.zeros((B, H + 1), dtype=torch.int32, device="cuda"),
+                          torch.zeros(B, dtype=torch.int32, device="cuda"))
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    bad_tok = tokens.copy()
+    bad_tok[1, 1] = V + 5
+    ctx.cast_accept_stochastic(tl, dl, B, 1.0, dev(bad_tok), dev(parent), dev(n_tree), ua, ub, alen, apath, bonus)
+    assert ctx.cast_poll_status()[0] == 6  # BAD_TREE
+    nan_tl = tl.clone()
+    nan_tl[2, 0, 17] = float("nan")
+    ctx.cast_accept_stochastic(nan_tl, dl, B, 1.0, dev(tokens), dev(parent), dev(n_tree), ua, ub, alen, apath, bonus)
+    assert ctx.cast_poll_status()[0] == 8  # NONFINITE
+    assert ctx.cast_poll_status()[0] == 0  # the poll cleared it
     # host-side checks
     i32 = lambda *s: torch.zeros(s, dtype=torch.int32, device="cuda")
     for bad_T in (0.0, -1.0, float("nan")):
