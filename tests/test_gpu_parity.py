@@ -179,11 +179,14 @@ def test_c3_b64_tree_and_accept_reduced_vocab(binding):
     check_accept_and_compact(binding, ctx, w, g, o, kv)
 
 
-def test_c3_b64_full_vocab_tree_build(binding):
-    # the batch-64 tree build at the full 128k vocabulary (the oracle needs about a minute for its 3000 row sorts)
+def test_c3_b64_full_vocab_tree_accept_compaction(binding):
+    # batch 64 at the full 128k vocabulary: tree build (the oracle needs half a minute for its 3000 row sorts), then
+    # acceptance and compaction on that tree
     w = wl.CONFIGS["c3_llama8b_b64"]
     ctx, g, o, root, kv = build_tree_both(binding, w)
     assert 4 <= int(o["n_tree"][0]) <= 16  # the cost model shrinks the tree at batch 64
+    # acceptance (argmax sweep over 64 x N rows of the full vocabulary) and compaction at the same size
+    check_accept_and_compact(binding, ctx, w, g, o, kv)
 
 
 @pytest.mark.parametrize("name", ["c4_llama70b_n16", "c4_llama70b_n128"])
