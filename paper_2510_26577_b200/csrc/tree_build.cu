@@ -1022,19 +1022,30 @@ extern "C" cast_status cast_tree_expand(cast_ctx* c, int layer, const void* draf
   c->next_layer = layer + 1;
   const int B = c->cur_B, V = c->cfg.vocab;
   const int rows_per_seq = layer == 1 ? 1 : c->W;
-  // A logits row is swept by one cluster of up to 8 CTAs: as many as it takes to cover the machine
-  // about four times over all rows. With few rows (small batches: latency counts) a CTA may get as
-  // little as 2048 logits; with many, at least half a pass, because a pass costs the same whether its
-  // slots are full or not.
+  // A logits row is swept by one cluster of 1 to 8 CTAs. A CTA pays for its fixed phases (prologue, chunk
+  // result, cluster barrier and row merge when there is more than one chunk: about 2.5 us, 2 without) and
+  // about 4 us per pass of kSweepSub logits, whether the pass is full or not; CTAs beyond one per SM queue
+  // up (figures fitted to the measured layer times of the benchmark shapes). The chunk count with the smallest estimate wins: few rows get many one-pass chunks (latency), many
+  // rows get few chunks of several full passes (throughput).
   const int rows = B * rows_per_seq;
-  int nchunks = (4 * c->num_sms + rows - 1) / rows;
-  const int min_chunk = rows < 16 ? 2048 : kSweepSub / 2;
-  if (nchunks > V / min_chunk) nchunks = V / min_chunk;
-  if (nchunks > kSweepMaxChunks) nchunks = kSweepMaxChunks;
-  if (nchunks < 1) nchunks = 1;
-  int chunk_elems = (V + nchunks - 1) / nchunks;
-  chunk_elems = (chunk_elems + 7) / 8 * 8;
-  nchunks = (V + chunk_elems - 1) / chunk_elems;
+  int nchunks = 1, chunk_elems = (V + 7) / 8 * 8;
+  {
+    double best = 1e30;
+    for (int n = 1; n <= kSweepMaxChunks; ++n) {
+      int ce = ((V + n - 1) / n + 7) / 8 * 8;
+      if (n > 1 && ce < 2048) break;  // below this a chunk is all overhead
+      const int ne = (V + ce - 1) / ce;
+      const int passes = (ce + kSweepSub - 1) / kSweepSub;
+      const double per_cta = (ne == 1 ? 2.0 : 2.5) + 4.0 * passes;
+      const double queue = (double)rows * ne / c->num_sms;
+      const double cost = per_cta * (queue < 1.0 ? 1.0 : queue);
+      if (cost < best - 1e-9) {
+        best = cost;
+        nchunks = ne;
+        chunk_elems = ce;
+      }
+    }
+  }
 
   ExpandParams p;
   p.logits = draft_logits;
