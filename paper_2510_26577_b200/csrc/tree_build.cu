@@ -207,7 +207,6 @@ __device__ __forceinline__ bool take_ticket(int32_t* counter, int expected, int*
 __device__ __forceinline__ void layer_tail(const ExpandParams& p, const TailState& ts, int B, int n_prev, int base,
                                         unsigned char* scratch, int* sorted /* [CAST_MAX_BATCH * CAST_MAX_WIDTH] */) {
   __shared__ double vbar[CAST_MAX_WIDTH], u[CAST_MAX_WIDTH], c[CAST_MAX_WIDTH];
-  __shared__ int mark[CAST_MAX_WIDTH];
   __shared__ int s_ni, s_next;
   const int tid = threadIdx.x, nt = blockDim.x;
   DevState* st = p.st;
@@ -311,21 +310,22 @@ __device__ __forceinline__ void layer_tail(const ExpandParams& p, const TailStat
     if (tid < n) u[tid] = a;
   }
   __syncthreads();
-  // Algorithm 1: mark[j] survives iff no earlier i has (u_j - u_i) < C1 (c_j - c_i)
-  if (tid < n) {
-    int ok = 1;
-    if (p.enable_bp)
-#pragma unroll 1
+  // Algorithm 1: mark[j] survives iff no earlier i has (u_j - u_i) < C1 (c_j - c_i); n_i = the largest
+  // marked index. n <= CAST_MAX_WIDTH <= 32: one warp, the marks as a ballot.
+  if (tid < 32) {
+    int ok = tid < n ? 1 : 0;
+    if (p.enable_bp && tid < n) {
+      const double uj = u[tid], cj = c[tid];
+#pragma unroll 4
       for (int i = 0; i < tid; ++i)
-        if ((u[tid] - u[i]) < p.C1 * (c[tid] - c[i])) ok = 0;
-    mark[tid] = ok;
+        ok &= !((uj - u[i]) < p.C1 * (cj - c[i]));
+    }
+    const unsigned marks = __ballot_sync(0xffffffffu, ok != 0);
+    if (tid == 0) s_ni = marks != 0u ? 32 - __clz(marks) : 1;
   }
   __syncthreads();
   if (tid == 0) {
-    int n_i = 1;
-#pragma unroll 1
-    for (int j = 0; j < n; ++j)
-      if (mark[j]) n_i = j + 1;
+    const int n_i = s_ni;
     bool go = true;
     if (p.enable_dp) {
       if (p.layer >= 2) {  // gain ratio of the previous layer goes into its buffer, FIFO
@@ -349,7 +349,6 @@ __device__ __forceinline__ void layer_tail(const ExpandParams& p, const TailStat
         go = (alpha * u[n_i - 1] / c[n_i - 1]) >= p.C2;
       }
     }
-    s_ni = n_i;
     s_next = (p.layer < p.H && go) ? n_i : 0;
     st->rows[p.layer + 1] = s_next;
     st->n_hist[p.layer] = n_i;
@@ -669,6 +668,7 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
   // the row's top K out of the chunks' lists (each in descending order): the rank of a key is its
   // position in its own list plus, for every other list, the number of larger keys there (a binary
   // search each; in its own list it finds its own position). Neighbouring lanes share a key slot.
+  if (p.nchunks > 1) {  // (a row of one chunk has its top K in `topk` already)
   if (tid < K) topk[tid] = 0ull;
   __syncthreads();
   {
@@ -701,6 +701,7 @@ __global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParam
     if (act && sub == 0 && cnt < K) topk[cnt] = key;
   }
   __syncthreads();
+  }
   if (warp == 0) {
     float M0 = -INFINITY, M1 = -INFINITY;
     double S0 = 0.0, S1 = 0.0;
