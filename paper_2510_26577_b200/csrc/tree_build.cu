@@ -379,8 +379,10 @@ __device__ __forceinline__ void layer_tail(const ExpandParams& p, const TailStat
   }
 }
 
-template <typename T>
-__global__ void __launch_bounds__(kSweepThreads) expand_kernel(const ExpandParams p) {
+// MINB = 2 compiles the same code for two CTAs per SM (half the registers): for launches with more CTAs than
+// SMs, where a second resident CTA hides the first one's latencies; MINB = 1 is for the short launches.
+template <typename T, int MINB>
+__global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const ExpandParams p) {
   __shared__ __align__(16) unsigned char scratch[kCandCap * 8];  // the warps' key lists and the short list; later the tail's arrays
   __shared__ unsigned long long topk[CAST_MAX_TOP_K];
   __shared__ float red_f[kSweepThreads / 32];
@@ -1077,8 +1079,13 @@ extern "C" cast_status cast_tree_expand(cast_ctx* c, int layer, const void* draf
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  const cudaError_t e = dtype == CAST_F32 ? cudaLaunchKernelEx(&cfg, expand_kernel<float>, p)
-                                          : cudaLaunchKernelEx(&cfg, expand_kernel<__nv_bfloat16>, p);
+  const bool queued = (long long)rows * nchunks > c->num_sms;
+  cudaError_t e;
+  if (dtype == CAST_F32)
+    e = queued ? cudaLaunchKernelEx(&cfg, expand_kernel<float, 2>, p) : cudaLaunchKernelEx(&cfg, expand_kernel<float, 1>, p);
+  else
+    e = queued ? cudaLaunchKernelEx(&cfg, expand_kernel<__nv_bfloat16, 2>, p)
+               : cudaLaunchKernelEx(&cfg, expand_kernel<__nv_bfloat16, 1>, p);
   if (e != cudaSuccess) {
     cudaGetLastError();
     return CAST_ERR_CUDA;
