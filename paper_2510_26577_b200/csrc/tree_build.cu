@@ -496,13 +496,17 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
     } else {
       thr_val = key_value(thr_key);
     }
-    // Few logits pass. One vote per logit slot keeps the common path at a compare and a vote; a slot
-    // with a passer (rare) takes the exact test on the full key and appends to the warp's list.
+    // Few logits pass. Every lane marks its passing slots in a bit mask and the warp takes the union with
+    // one reduction; only a slot with a passer somewhere (rare) takes the exact test on the full key and
+    // appends to the warp's list.
     const int have0 = have;
+    unsigned mine_mask = 0u;
+#pragma unroll
+    for (int i = 0; i < kSweepEpt; ++i) mine_mask |= (xv[i] >= thr_val) ? (1u << i) : 0u;
+    const unsigned any_mask = __reduce_or_sync(0xffffffffu, mine_mask);
 #pragma unroll
     for (int i = 0; i < kSweepEpt; ++i) {
-      const unsigned m0 = __ballot_sync(0xffffffffu, xv[i] >= thr_val);
-      if (m0 != 0u) {
+      if (any_mask & (1u << i)) {
         const int id = sub + ((i / VEC) * kSweepThreads + tid) * VEC + (i % VEC);
         const unsigned long long key = make_key(xv[i], id);
         const bool ok = xv[i] >= thr_val && id < end && key > thr_key;
