@@ -116,3 +116,61 @@ def test_attention_random_shapes_and_windows(binding, seed):
         err = max(np.max(np.abs(got[i] - ref[i])) for i in only)
         assert err <= attention_tolerance(dtype), (case, dtype, D, Hq, Hkv, page, err)
         ctx.close()
+
+
+@pytest.mark.parametrize("seed", [6, 7])
+def test_accept_and_compaction_random(binding, seed):
+    from oracle import compact_kv, greedy_accept
+    rng = np.random.default_rng(seed)
+    for case in range(16):
+        B, H = int(rng.integers(1, 7)), int(rng.integers(2, 9))
+        Ncap = int(rng.choice([32, 64, 128]))
+        V = int(rng.choice([rng.integers(50, 3000), rng.integers(3000, 70000)]))
+        dt = "bf16" if rng.random() < 0.4 else "f32"
+        page = int(rng.choice([0, 4, 16]))
+        Hkv, D, n_layers = int(rng.choice([1, 2, 4])), int(rng.choice([64, 128])), int(rng.integers(1, 4))
+        w = wl.Workload("fuzz", 400 + case, B, dt, dt, Hkv, Hkv, D, 3, 90, page, V, 2.0, H, 4, Ncap, False, n_layers,
+                        max_tree=Ncap, seed_salt=seed)
+        ctx = binding.CastContext(max_batch=B, vocab=V, top_k=4, max_depth=H, total_token=Ncap, max_tree=Ncap)
+        n_tree = rng.integers(1, Ncap + 1, size=B).astype(np.int32)
+        tokens = np.full((B, Ncap), -1, dtype=np.int32)
+        parent = np.full((B, Ncap), -1, dtype=np.int32)
+        for b in range(B):
+            N = int(n_tree[b])
+            par = _random_parents(rng, N)
+            depth = np.zeros(N, dtype=int)
+            for t in range(1, N):
+                if depth[par[t]] + 1 > H:
+                    par[t] = 0
+                depth[t] = depth[par[t]] + 1
+            parent[b, :N] = par
+            tokens[b, :N] = rng.integers(0, V, size=N)  # siblings may share a token: the lowest index wins
+        tl = wl.target_logits(w, "cpu")
+        wl.plant_acceptance(w, tl, tokens, parent, n_tree)
+        tl = tl.cuda()
+        dev = lambda a: torch.from_numpy(a).cuda()
+        alen = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+        apath = torch.full((B, H + 1), -7, dtype=torch.int32, device="cuda")
+        bonus = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+        ctx.cast_accept(tl, B, dev(tokens), dev(parent), None, None, dev(n_tree), alen, apath, bonus)
+        assert ctx.cast_poll_status()[0] == 0
+        ol, op, ob = greedy_accept(to_f64(tl[:, : int(n_tree.max())]), tokens, parent, n_tree, H)
+        assert np.array_equal(alen.cpu().numpy(), ol) and np.array_equal(apath.cpu().numpy(), op), case
+        assert np.array_equal(bonus.cpu().numpy(), ob), case
+        # compaction of all layers, compared as raw bits
+        kv = wl.kv_lengths(w, "cpu").cuda()
+        layers = [tuple(t.cuda() for t in wl.kv_cache(w, l, "cpu")) for l in range(n_layers)]
+        kk = torch.stack([a for a, _ in layers]).contiguous()
+        vv = torch.stack([c for _, c in layers]).contiguous()
+        table, num_pages = wl.page_table(w, "cuda")
+        bits = torch.int16 if dt == "bf16" else torch.int32
+        k_old, v_old = kk.view(bits).cpu().numpy(), vv.view(bits).cpu().numpy()
+        kv2 = kv.clone()
+        ctx.cast_compact_kv(kk, vv, B, n_layers, kk[0].numel() * kk.element_size(), Hkv, D, page, table,
+                            wl.seq_capacity(w) // (page or 1), num_pages, apath, alen, kv2)
+        assert ctx.cast_poll_status()[0] == 0
+        tab = table.cpu().numpy() if table is not None else None
+        nk, nv, nlen = compact_kv(k_old, v_old, page, tab, kv.cpu().numpy(), op, ol)
+        assert np.array_equal(kv2.cpu().numpy(), nlen), case
+        assert np.array_equal(kk.view(bits).cpu().numpy(), nk) and np.array_equal(vv.view(bits).cpu().numpy(), nv), case
+        ctx.close()
