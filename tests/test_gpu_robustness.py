@@ -1,7 +1,10 @@
-"""Randomised parity: many small configurations drawn from a fixed seed, each compared with the
-oracle like the hand-picked cases of test_gpu_parity.py.  The draws cover what those cases fix by
-hand: vocabulary sizes that are not multiples of anything, every K and W up to the caps, batch
-sizes, logit dtypes, the sizing switches, window starts and head groupings."""
+"""More parity through the C-ABI, beyond the hand-picked cases of test_gpu_parity.py:
+
+* many small configurations drawn from fixed seeds (vocabulary sizes that are not multiples of
+  anything, every K and W up to the caps, batch sizes, logit dtypes, the sizing switches, window starts,
+  head groupings, random trees with shared sibling tokens), each compared with the oracle;
+* the tree build at the hyper-parameters the paper reports for its own runs;
+* one whole step with sentinel bands around every tensor the library writes."""
 import numpy as np
 import pytest
 import torch
@@ -174,3 +177,127 @@ def test_accept_and_compaction_random(binding, seed):
         assert np.array_equal(kv2.cpu().numpy(), nlen), case
         assert np.array_equal(kk.view(bits).cpu().numpy(), nk) and np.array_equal(vv.view(bits).cpu().numpy(), nv), case
         ctx.close()
+
+
+# ------------------------------------------------------------------ the paper's own hyper-parameters
+@pytest.mark.parametrize("B,H,K,m,thr,V", [(1, 13, 12, 72, 3.5, 128256),   # batch 1: depth 13, top-k 12, 72 tokens
+                                           (8, 9, 12, 72, 2.5, 32000)])    # batch 8: depth 9, top-k 12, 72 tokens
+def test_tree_build_with_the_papers_settings(binding, B, H, K, m, thr, V):
+    """Depth, top-k, token budget and threshold as the paper reports them for its runs (its one threshold
+    is used for C1, C2 and C3), all three sizing switches on, peaked logits, two steps so that the
+    depth-pruning buffers carry over."""
+    w = wl.Workload("paper", 500 + B, B, "bf16", "f32", 32, 8, 128, 512, 2048, 16, V, 3.0, H, K, m, True, 1, max_tree=128)
+    kw = cfg_kwargs(w, enable_dp=1, C1=thr, C2=thr, C3=thr)
+    L, M, Ntab, fT, fD = make_tables(w, B)
+    tables = {B: CostTable(B, L, M, Ntab, fT, fD)}
+    ctx = binding.CastContext(max_batch=B, **kw)
+    ctx.cast_set_cost_tables(B, L, M, Ntab, fT, fD)
+    root, kv = wl.root_tokens(w, "cpu").cuda(), wl.kv_lengths(w, "cpu").cuda()
+    oracle = None
+    for step in range(2):
+        logits = [wl.draft_logits(w, 20 * step + l, "cpu", peaked=True).cuda() for l in range(1, H + 1)]
+        o = oracle_tree(kw, tables, root, kv, logits, oracle)
+        oracle = o["oracle"]
+        g = gpu_tree(ctx, root, kv, logits)
+        assert ctx.cast_poll_status()[0] == 0
+        assert o["min_score_gap"] >= 1e-5 and o["stable"], "a decision within rounding of its threshold: pick another seed"
+        assert_tree_equal(g, o)
+    assert 1 <= int(o["n_tree"][0]) <= m
+
+
+# ------------------------------------------------------------------ nothing is written outside the outputs
+class _Guarded:
+    """Device buffers with a band of sentinel bytes on both sides of every output tensor."""
+    BAND = 256  # bytes; a multiple of 16 so that the tensor inside keeps its alignment
+
+    def __init__(self):
+        self.items = []
+
+    def alloc(self, shape, dtype, fill=None):
+        n = int(np.prod(shape))
+        size = torch.empty((), dtype=dtype).element_size()
+        raw = torch.full((2 * self.BAND + n * size,), 0xA5, dtype=torch.uint8, device="cuda")
+        inner = raw[self.BAND: self.BAND + n * size].view(dtype).view(*shape)
+        if fill is not None:
+            inner.fill_(fill)
+        self.items.append(raw)
+        return inner
+
+    def check(self):
+        for raw in self.items:
+            assert bool((raw[: self.BAND] == 0xA5).all()) and bool((raw[-self.BAND:] == 0xA5).all())
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_guard_bands_around_every_output(binding, dtype):
+    """One whole step (tree build, attention on the full tree and on a window, greedy and stochastic
+    acceptance) with sentinel bands around every tensor the library writes: the bands stay intact and
+    the results are the oracle's."""
+    from oracle import greedy_accept
+    B, H, K, m, Ncap = 3, 3, 4, 24, 32
+    w = wl.Workload("guard", 600, B, dtype, "f32", 8, 2, 128 if dtype == "bf16" else 64, 100, 400, 16, 5000, 3.0, H, K, m, False,
+                    1, max_tree=Ncap)
+    kw = cfg_kwargs(w)
+    ctx = binding.CastContext(max_batch=B, **kw)
+    gd = _Guarded()
+    root, kv = wl.root_tokens(w, "cpu").cuda(), wl.kv_lengths(w, "cpu").cuda()
+    logits = [wl.draft_logits(w, l, "cpu").cuda() for l in range(1, H + 1)]
+    ctx.cast_step_begin(B, root, kv)
+    per_layer = []
+    for i, lg in enumerate(logits, start=1):
+        nt, npr, cnt = gd.alloc((B, K), torch.int32), gd.alloc((B, K), torch.int32), gd.alloc((1,), torch.int32)
+        ctx.cast_tree_expand(i, lg, nt, npr, cnt)
+        per_layer.append((nt, npr, cnt))
+    tr = dict(tokens=gd.alloc((B, Ncap), torch.int32), parent=gd.alloc((B, Ncap), torch.int32),
+              depth=gd.alloc((B, Ncap), torch.int32), anc=gd.alloc((B, Ncap, ctx.words), torch.int32),
+              pool_idx=gd.alloc((B, Ncap), torch.int32), scores=gd.alloc((B, Ncap), torch.float64),
+              n_tree=gd.alloc((B,), torch.int32))
+    ctx.cast_select_nodes(tr["tokens"], tr["parent"], tr["depth"], tr["anc"], tr["pool_idx"], tr["scores"], tr["n_tree"])
+    assert ctx.cast_poll_status()[0] == 0
+    o = oracle_tree(kw, None, root, kv, logits)
+    g = {k: v.cpu().numpy() for k, v in tr.items()}
+    g["anc"] = g["anc"].view(np.uint32)
+    g["per_layer"] = [(a.cpu().numpy(), b.cpu().numpy(), int(c.item())) for a, b, c in per_layer]
+    g["status"], g["info"] = (0, 0), ctx.cast_step_info()
+    assert_tree_equal(g, o)
+    # attention: the whole tree, then a window
+    q = wl.query(w, 0, "cpu").cuda()
+    k, v = (t.cuda() for t in wl.kv_cache(w, 0, "cpu"))
+    table, num_pages = wl.page_table(w, "cuda")
+    seq_cap = wl.seq_capacity(w) // w.page_size
+    tab = table.cpu().numpy()
+    f32 = lambda t: t.float().cpu().numpy()
+    for first in (None, torch.tensor([3, 0, 20], dtype=torch.int32, device="cuda")):
+        out = gd.alloc(tuple(q.shape), q.dtype, fill=float("nan"))
+        ctx.cast_tree_attention_rows(q, k, v, B, w.q_heads, w.kv_heads, w.head_dim, w.page_size, table, seq_cap, num_pages, kv,
+                                     tr["anc"], tr["n_tree"], first, 0.0, out)
+        assert ctx.cast_poll_status()[0] == 0
+        ref = tree_attention(f32(q), f32(k), f32(v), w.page_size, tab, kv.cpu().numpy(), o["anc"], o["n_tree"])
+        got = to_f64(out)
+        for b in range(B):
+            lo = int(first[b]) if first is not None else 0
+            lo = min(lo, int(o["n_tree"][b]))
+            assert np.isnan(got[b, :lo]).all() and np.isnan(got[b, int(o["n_tree"][b]):]).all()
+            err = np.max(np.abs(got[b, lo: int(o["n_tree"][b])] - ref[b, lo: int(o["n_tree"][b])])) if lo < o["n_tree"][b] else 0.0
+            assert err <= attention_tolerance(dtype)
+    # acceptance, greedy and at temperature 1
+    tl = wl.target_logits(w, "cpu")
+    wl.plant_acceptance(w, tl, o["tokens"], o["parent"], o["n_tree"])
+    tl = tl.cuda()
+    alen, apath, bonus = gd.alloc((B,), torch.int32), gd.alloc((B, H + 1), torch.int32), gd.alloc((B,), torch.int32)
+    ctx.cast_accept(tl, B, tr["tokens"], tr["parent"], tr["depth"], tr["anc"], tr["n_tree"], alen, apath, bonus)
+    ol, op, ob = greedy_accept(to_f64(tl), o["tokens"], o["parent"], o["n_tree"], H)
+    assert np.array_equal(alen.cpu().numpy(), ol) and np.array_equal(apath.cpu().numpy(), op)
+    assert np.array_equal(bonus.cpu().numpy(), ob)
+    s_tl, s_dl, ua, ub = wl.stochastic_accept_inputs(w, o["tokens"], o["parent"], o["n_tree"], "cuda", 0.7, Ncap)
+    alen2, apath2, bonus2 = gd.alloc((B,), torch.int32), gd.alloc((B, H + 1), torch.int32), gd.alloc((B,), torch.int32)
+    ctx.cast_accept_stochastic(s_tl, s_dl, B, 1.0, tr["tokens"], tr["parent"], tr["n_tree"], ua, ub, alen2, apath2, bonus2)
+    assert ctx.cast_poll_status()[0] == 0
+    from oracle import stochastic_accept
+    sl, sp, sb, margin = stochastic_accept(to_f64(s_tl), to_f64(s_dl), o["tokens"], o["parent"], o["n_tree"], H, 1.0,
+                                           ua.cpu().numpy(), ub.cpu().numpy())
+    assert margin.min() >= 1e-9
+    assert np.array_equal(alen2.cpu().numpy(), sl) and np.array_equal(apath2.cpu().numpy(), sp)
+    assert np.array_equal(bonus2.cpu().numpy(), sb)
+    torch.cuda.synchronize()
+    gd.check()
