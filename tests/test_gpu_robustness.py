@@ -301,3 +301,39 @@ def test_guard_bands_around_every_output(binding, dtype):
     assert np.array_equal(bonus2.cpu().numpy(), sb)
     torch.cuda.synchronize()
     gd.check()
+
+
+# ------------------------------------------------------------------ run-to-run determinism
+@pytest.mark.parametrize("name", ["c2_llama8b", "c3_llama8b_b16", "c4_llama70b_n64"])
+def test_repeated_calls_give_identical_bits(binding, name):
+    """No result depends on which CTA finishes first: the merges (cluster, ticket) combine their pieces in a
+    fixed order, so a repeated call reproduces every output bit for bit - tree, attention (cluster mode,
+    global-merge mode) and acceptance at temperature 1."""
+    w = wl.CONFIGS[name]
+    B, H = w.batch, w.depth
+    kw = cfg_kwargs(w)
+    ctx = binding.CastContext(max_batch=B, **kw)
+    if w.cost_model:
+        ctx.cast_set_cost_tables(B, *make_tables(w, B))
+    root, kv = wl.root_tokens(w, "cpu").cuda(), wl.kv_lengths(w, "cpu").cuda()
+    logits = [wl.draft_logits(w, l, "cuda") for l in range(1, H + 1)]
+    q = wl.query(w, 0, "cuda")
+    k, v = wl.kv_cache(w, 0, "cuda")
+    table, num_pages = wl.page_table(w, "cuda")
+    runs = []
+    for rep in range(3):
+        g = gpu_tree(ctx, root, kv, logits)
+        d = g["dev"]
+        out = gpu_attention(ctx, w, q, k, v, table, num_pages, kv, d["anc"], d["n_tree"])
+        res = [g[key].tobytes() for key in ("tokens", "parent", "depth", "anc", "pool_idx", "scores", "n_tree")]
+        res.append(out.view(torch.int16).cpu().numpy().tobytes())
+        if rep == 0:
+            sto = wl.stochastic_accept_inputs(w, g["tokens"], g["parent"], g["n_tree"], "cuda", 0.7)
+        alen = torch.empty((B,), dtype=torch.int32, device="cuda")
+        apath = torch.empty((B, H + 1), dtype=torch.int32, device="cuda")
+        bonus = torch.empty((B,), dtype=torch.int32, device="cuda")
+        ctx.cast_accept_stochastic(sto[0], sto[1], B, 1.0, d["tokens"], d["parent"], d["n_tree"], sto[2], sto[3], alen, apath, bonus)
+        res += [alen.cpu().numpy().tobytes(), apath.cpu().numpy().tobytes(), bonus.cpu().numpy().tobytes()]
+        assert ctx.cast_poll_status()[0] == 0
+        runs.append(res)
+    assert runs[0] == runs[1] == runs[2]
