@@ -337,3 +337,50 @@ def test_repeated_calls_give_identical_bits(binding, name):
         assert ctx.cast_poll_status()[0] == 0
         runs.append(res)
     assert runs[0] == runs[1] == runs[2]
+
+
+# ------------------------------------------------------------------ malformed inputs: a status, never a fault
+def test_malformed_inputs_are_reported_not_followed(binding):
+    """What the host can see is refused with a code; what only the device can see (a parent that does not
+    precede its child, a tree larger than the budget, a path entry below zero) sets the status word, first
+    error first, and the call still ends in bounds."""
+    with pytest.raises(binding.CastError) as e:  # more children per node than the vocabulary has tokens
+        binding.CastContext(max_batch=1, vocab=3, top_k=4, max_depth=2, total_token=8)
+    assert e.value.code == 3
+    with pytest.raises(binding.CastError) as e:  # token budget beyond the row stride
+        binding.CastContext(max_batch=1, vocab=100, top_k=2, max_depth=2, total_token=64, max_tree=32)
+    assert e.value.code == 3
+    H, Ncap, V, B = 4, 32, 64, 2
+    ctx = binding.CastContext(max_batch=B, vocab=V, top_k=2, max_depth=H, total_token=16, max_tree=Ncap)
+    dev = lambda a: torch.from_numpy(a).cuda()
+    tokens = np.zeros((B, Ncap), dtype=np.int32)
+    parent = np.full((B, Ncap), -1, dtype=np.int32)
+    parent[:, 1:6] = [0, 0, 1, 5, 2]  # node 4 names node 5 as its parent
+    n_tree = np.array([6, 6], dtype=np.int32)
+    logits = torch.zeros((B, Ncap, V), device="cuda")
+    alen = torch.zeros(B, dtype=torch.int32, device="cuda")
+    apath = torch.zeros((B, H + 1), dtype=torch.int32, device="cuda")
+    bonus = torch.zeros(B, dtype=torch.int32, device="cuda")
+    ctx.cast_accept(logits, B, dev(tokens), dev(parent), None, None, dev(n_tree), alen, apath, bonus)
+    st, detail = ctx.cast_poll_status()
+    assert st == 6 and detail % Ncap == 4  # BAD_TREE, at the offending node
+    assert int(alen.min()) >= 0 and int(alen.max()) <= H and ctx.cast_poll_status()[0] == 0
+    # attention with a tree larger than the context's token budget (tensor-core path)
+    w = wl.Workload("bad", 700, B, "bf16", "f32", 8, 2, 128, 50, 60, 16, V, 1.0, H, 2, 16, False, 1, max_tree=Ncap)
+    q = wl.query(w, 0, "cuda")
+    k, v = wl.kv_cache(w, 0, "cuda")
+    table, num_pages = wl.page_table(w, "cuda")
+    kv = wl.kv_lengths(w, "cuda")
+    anc = torch.zeros((B, Ncap, ctx.words), dtype=torch.int32, device="cuda")
+    out = torch.zeros_like(q)
+    ctx.cast_tree_attention(q, k, v, B, 8, 2, 128, 16, table, wl.seq_capacity(w) // 16, num_pages, kv, anc,
+                            dev(np.array([20, 4], dtype=np.int32)), 0.0, out)
+    assert ctx.cast_poll_status()[0] == 6
+    # compaction with a path entry below zero inside the accepted length
+    kk, vv = k.unsqueeze(0).contiguous(), v.unsqueeze(0).contiguous()
+    path = np.full((B, H + 1), -1, dtype=np.int32)
+    path[:, 0] = 0
+    ctx.cast_compact_kv(kk, vv, B, 1, kk[0].numel() * 2, 2, 128, 16, table, wl.seq_capacity(w) // 16, num_pages, dev(path),
+                        dev(np.array([2, 0], dtype=np.int32)), kv.clone())
+    assert ctx.cast_poll_status()[0] == 7  # BAD_PAGE
+    assert ctx.cast_poll_status()[0] == 0
