@@ -414,6 +414,11 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
   // one memory round trip for both
   float xv[kSweepEpt];
   auto load_pass = [&](int sub) {
+    if (aligned && sub + kSweepSub <= end) {  // a full pass: no per-vector checks
+#pragma unroll
+      for (int v = 0; v < NV; ++v) Vec<T>::load(x + sub + (v * kSweepThreads + tid) * VEC, xv + v * VEC);
+      return;
+    }
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
       const int idx = sub + (v * kSweepThreads + tid) * VEC;
