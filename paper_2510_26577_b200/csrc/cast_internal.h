@@ -76,6 +76,11 @@ struct cast_ctx {
   cast::DevState* state;
 
   int32_t* layer_ticket;          // [1]
+  // batched layer tail: per-sequence tickets and what every sequence hands to the batch-wide part
+  int32_t* seq_ticket;            // [max_batch]
+  double* tail_vs;                // [max_batch][CAST_MAX_WIDTH] values of the first n sorted candidates
+  int32_t* tail_sorted;           // [max_batch][CAST_MAX_WIDTH] their pool indices
+  int32_t* tail_tok;              // [max_batch][CAST_MAX_WIDTH] their tokens
 
   // depth-pruning buffers
   double* fifo_vals;   // [H-1][R]

@@ -44,7 +44,8 @@ namespace {
 __global__ void step_begin_kernel(DevState* st, int B, int P, int W, const int32_t* root_token,
                                   const int32_t* kv_len, double* pool_score, int32_t* pool_token,
                                   int32_t* pool_parent, int32_t* pool_depth, uint8_t* pool_kept,
-                                  int32_t* retained, int32_t* lsort, double* lscore, int32_t* layer_ticket) {
+                                  int32_t* retained, int32_t* lsort, double* lscore, int32_t* layer_ticket,
+                                  int32_t* seq_ticket) {
   __shared__ int s_max;
   const int tid = threadIdx.x;
   if (tid == 0) s_max = 0;
@@ -59,6 +60,7 @@ __global__ void step_begin_kernel(DevState* st, int B, int P, int W, const int32
     lsort[o] = 0;
     lscore[o] = 0.0;
     retained[b * W] = 0;
+    seq_ticket[b] = 0;
     atomicMax(&s_max, kv_len[b]);
   }
   __syncthreads();
@@ -99,6 +101,10 @@ struct ExpandParams {
   double* lscore;
   DevState* st;
   int32_t* layer_ticket;
+  int32_t* seq_ticket;
+  double* tail_vs;
+  int32_t* tail_sorted;
+  int32_t* tail_tok;
   double* fifo_vals;
   int32_t* fifo_cnt;
   int R;
@@ -203,41 +209,43 @@ __device__ __forceinline__ bool take_ticket(int32_t* counter, int expected, int*
   return *flag_s != 0;
 }
 
-// Layer tail (Eq. 1, Eq. 2, Algorithm 1, depth pruning), run by the last CTA of the layer.
-__device__ __forceinline__ void layer_tail(const ExpandParams& p, const TailState& ts, int B, int n_prev, int base,
-                                        unsigned char* scratch, int* sorted /* [CAST_MAX_BATCH * CAST_MAX_WIDTH] */) {
-  __shared__ double vbar[CAST_MAX_WIDTH], u[CAST_MAX_WIDTH], c[CAST_MAX_WIDTH];
-  __shared__ int s_ni, s_next;
-  const int tid = threadIdx.x, nt = blockDim.x;
-  DevState* st = p.st;
-  const int K = p.K, W = p.W, P = p.P;
-  const int Ni = n_prev * K;
-  const bool need_cost = p.enable_bp || p.enable_dp;
-  int n = Ni < W ? Ni : W;
-  if (need_cost && p.tab.Ntab < n) n = p.tab.Ntab;
-  // Eq. 2 needs one table row: fetch it now, its latency hides behind the ranking
-  double c_mine = 0.0;
-  if (need_cost && tid < n) {
-    const int ctx = ts.ctx_sum + (p.ctx_base_mode ? ts.n0 : 0);
-    const int g = select_grid(ctx, p.tab.L, p.tab.M);
-    c_mine = p.tab.fD[(size_t)(g - 1) * p.tab.Ntab + tid] / p.tab.fT[(size_t)(g - 1) * p.tab.Ntab];
-  }
-  const double u_last = ts.u_last;
+// Layer tail (Eq. 1, Eq. 2, Algorithm 1, depth pruning) in two parts. tail_rank orders the candidates of
+// some sequences and is what costs time with many sequences; tail_decide is the batch-wide rest. With up to
+// four sequences the last CTA of the layer runs both from shared memory; with more, the last CTA of every
+// sequence ranks that sequence (so the sequences are ranked in parallel) and leaves the first n sorted
+// nodes in global memory, and the last of those CTAs decides.
 
+// Up to this many sequences the one-CTA tail is faster than a second ticket.
+constexpr int kTailSingleMaxB = 4;
+
+// Candidates Algorithm 1 looks at: the first n of the sorted list.
+__device__ __forceinline__ int tail_width(const ExpandParams& p, int n_prev) {
+  const int Ni = n_prev * p.K;
+  int n = Ni < p.W ? Ni : p.W;
+  if ((p.enable_bp || p.enable_dp) && p.tab.Ntab < n) n = p.tab.Ntab;
+  return n;
+}
+
+// Ranks the layer's candidates of the sequences [b_begin, b_begin + b_count): writes every sequence's sorted
+// list for the rerank (lsort, lscore) and, for rank < n, pool index, token and value to sorted_o, stok_o,
+// vs_o at [b * CAST_MAX_WIDTH + rank] (shared or global memory).
+__device__ __forceinline__ void tail_rank(const ExpandParams& p, int b_begin, int b_count, int n, int n_prev, int base,
+                                          unsigned char* scratch, int* sorted_o, int* stok_o, double* vs_o) {
+  const int tid = threadIdx.x, nt = blockDim.x;
+  const int K = p.K, P = p.P;
+  const int Ni = n_prev * K;
   double* sc = reinterpret_cast<double*>(scratch);              // 1024 scores
   int* tk = reinterpret_cast<int*>(scratch + 8192);             // 1024 tokens
   unsigned short* r1s = reinterpret_cast<unsigned short*>(scratch + 12288);  // 1024: row of the candidate
   unsigned short* cis = reinterpret_cast<unsigned short*>(scratch + 14336);  // 1024: index within the sequence
-  double* vs = reinterpret_cast<double*>(scratch + 16384);      // [B][CAST_MAX_WIDTH] sorted values
-  int* stok = reinterpret_cast<int*>(scratch + 24576);          // [B][CAST_MAX_WIDTH] tokens of the sorted nodes
   const int group = 1024 / Ni;                                  // sequences ranked per pass
 #pragma unroll 1
-  for (int b0 = 0; b0 < B; b0 += group) {
-    const int nb = (B - b0) < group ? (B - b0) : group;
+  for (int b0 = 0; b0 < b_count; b0 += group) {
+    const int nb = (b_count - b0) < group ? (b_count - b0) : group;
     const int tot = nb * Ni;
     for (int i = tid; i < tot; i += nt) {
       const int bl = i / Ni, ci = i - bl * Ni;  // (the divisions hide behind the loads)
-      const size_t o = (size_t)(b0 + bl) * P + base + ci;
+      const size_t o = (size_t)(b_begin + b0 + bl) * P + base + ci;
       sc[i] = __ldcg(p.pool_score + o);
       tk[i] = __ldcg(p.pool_token + o);
       r1s[i] = (unsigned short)(ci / K);
@@ -278,24 +286,46 @@ __device__ __forceinline__ void layer_tail(const ExpandParams& p, const TailStat
       cnt += __shfl_xor_sync(0xffffffffu, cnt, 2);
       cnt += __shfl_xor_sync(0xffffffffu, cnt, 1);
       if (act && sub == 0) {
-        const int bl = sbase / Ni, rank = cnt;
-        const size_t o = (size_t)(b0 + bl) * P + base + rank;
+        const int bg = b_begin + b0 + sbase / Ni, rank = cnt;
+        const size_t o = (size_t)bg * P + base + rank;
         p.lsort[o] = base + ci;  // the layer's sorted list, for the rerank
         p.lscore[o] = s;
         if (rank < n) {
-          sorted[(b0 + bl) * CAST_MAX_WIDTH + rank] = base + ci;
-          stok[(b0 + bl) * CAST_MAX_WIDTH + rank] = t;
-          vs[(b0 + bl) * CAST_MAX_WIDTH + rank] = fast_exp_neg(s);
+          sorted_o[bg * CAST_MAX_WIDTH + rank] = base + ci;
+          stok_o[bg * CAST_MAX_WIDTH + rank] = t;
+          vs_o[bg * CAST_MAX_WIDTH + rank] = fast_exp_neg(s);
         }
       }
     }
     __syncthreads();
   }
-  // Eq. 1: batch mean of the rank-wise values, then prefix sums
+}
+
+// The batch-wide part: Eq. 1 over the sequences' first n sorted values, Eq. 2, Algorithm 1, the depth test,
+// the state for the next layer and the layer's outputs. GLOBAL: the inputs were written to global memory by
+// other CTAs (read past L1).
+template <bool GLOBAL>
+__device__ __forceinline__ void tail_decide(const ExpandParams& p, const TailState& ts, int B, int n, int n_prev, int base,
+                                            const int* sorted_i, const int* stok_i, const double* vs_i) {
+  __shared__ double vbar[CAST_MAX_WIDTH], u[CAST_MAX_WIDTH], c[CAST_MAX_WIDTH];
+  __shared__ int s_ni, s_next;
+  const int tid = threadIdx.x, nt = blockDim.x;
+  DevState* st = p.st;
+  const int K = p.K, W = p.W, P = p.P;
+  const int Ni = n_prev * K;
+  const bool need_cost = p.enable_bp || p.enable_dp;
+  const double u_last = ts.u_last;
+  // Eq. 1: batch mean of the rank-wise values, then prefix sums; Eq. 2 needs one table row
   if (tid < n) {
+    double c_mine = 0.0;
+    if (need_cost) {
+      const int ctx = ts.ctx_sum + (p.ctx_base_mode ? ts.n0 : 0);
+      const int g = select_grid(ctx, p.tab.L, p.tab.M);
+      c_mine = p.tab.fD[(size_t)(g - 1) * p.tab.Ntab + tid] / p.tab.fT[(size_t)(g - 1) * p.tab.Ntab];
+    }
     double a = 0.0;
-#pragma unroll 1
-    for (int b = 0; b < B; ++b) a += vs[b * CAST_MAX_WIDTH + tid];
+#pragma unroll 4
+    for (int b = 0; b < B; ++b) a += GLOBAL ? __ldcg(vs_i + b * CAST_MAX_WIDTH + tid) : vs_i[b * CAST_MAX_WIDTH + tid];
     vbar[tid] = a / (double)B;
     c[tid] = c_mine;
   }
@@ -368,8 +398,8 @@ __device__ __forceinline__ void layer_tail(const ExpandParams& p, const TailStat
     const int b = i / W, s = i % W;
     int tok = -1, prow = -1;
     if (s < n_i) {
-      const int idx = sorted[b * CAST_MAX_WIDTH + s];
-      tok = stok[b * CAST_MAX_WIDTH + s];
+      const int idx = GLOBAL ? __ldcg(sorted_i + b * CAST_MAX_WIDTH + s) : sorted_i[b * CAST_MAX_WIDTH + s];
+      tok = GLOBAL ? __ldcg(stok_i + b * CAST_MAX_WIDTH + s) : stok_i[b * CAST_MAX_WIDTH + s];
       prow = (idx - base) / K;
       p.retained[b * W + s] = idx;
       p.pool_kept[(size_t)b * P + idx] = 1;
@@ -387,7 +417,7 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
   __shared__ unsigned long long topk[CAST_MAX_TOP_K];
   __shared__ float red_f[kSweepThreads / 32];
   __shared__ double red_d[kSweepThreads / 32];
-  __shared__ int sorted[CAST_MAX_BATCH * CAST_MAX_WIDTH];
+  __shared__ int sorted[kTailSingleMaxB * CAST_MAX_WIDTH];  // small batches: pool indices of the first sorted candidates
   __shared__ int s_flag, short_n;
   // filled in the first CTA of the row's cluster by all CTAs of the cluster: chunk c's top-K keys
   // (descending), maximum (log2 units) and sum of 2^(. - maximum)
@@ -750,11 +780,24 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
   }
   CAST_STAMP(5);
 
-  // ---- layer tail by the last CTA of the layer
+  // ---- layer tail
   __syncthreads();
-  if (!take_ticket(p.layer_ticket, B * n_prev, &s_flag)) return;
-  CAST_STAMP(6);
-  layer_tail(p, ts, B, n_prev, base, scratch, sorted);
+  const int n_tail = tail_width(p, n_prev);
+  if (B <= kTailSingleMaxB) {  // the last CTA of the layer ranks and decides, everything in shared memory
+    if (!take_ticket(p.layer_ticket, B * n_prev, &s_flag)) return;
+    CAST_STAMP(6);
+    double* vs = reinterpret_cast<double*>(scratch + 16384);  // [B][CAST_MAX_WIDTH] sorted values
+    int* stok = reinterpret_cast<int*>(scratch + 24576);      // [B][CAST_MAX_WIDTH] tokens of the sorted nodes
+    tail_rank(p, 0, B, n_tail, n_prev, base, scratch, sorted, stok, vs);
+    tail_decide<false>(p, ts, B, n_tail, n_prev, base, sorted, stok, vs);
+  } else {  // the last CTA of every sequence ranks that sequence; the last of those decides for the batch
+    if (!take_ticket(p.seq_ticket + b, n_prev, &s_flag)) return;
+    CAST_STAMP(6);
+    tail_rank(p, b, 1, n_tail, n_prev, base, scratch, p.tail_sorted, p.tail_tok, p.tail_vs);
+    // (tail_rank ends with a CTA barrier: the ticket below releases what all threads wrote)
+    if (!take_ticket(p.layer_ticket, B, &s_flag)) return;
+    tail_decide<true>(p, ts, B, n_tail, n_prev, base, p.tail_sorted, p.tail_tok, p.tail_vs);
+  }
   CAST_STAMP(7);
   CAST_STAMP_FLUSH(0, 8);
 }
@@ -1021,7 +1064,8 @@ extern "C" cast_status cast_step_begin(cast_ctx* c, int B, const int32_t* root_t
   c->next_layer = 1;
   step_begin_kernel<<<1, 128, 0, (cudaStream_t)stream>>>(c->state, B, c->P, c->W, root_token, kv_len, c->pool_score,
                                                          c->pool_token, c->pool_parent, c->pool_depth, c->pool_kept,
-                                                         c->retained, c->lsort, c->lscore, c->layer_ticket);
+                                                         c->retained, c->lsort, c->lscore, c->layer_ticket,
+                                                         c->seq_ticket);
   return launch_status();
 }
 
@@ -1068,6 +1112,7 @@ extern "C" cast_status cast_tree_expand(cast_ctx* c, int layer, const void* draf
   p.lsort = c->lsort; p.lscore = c->lscore;
   p.st = c->state;
   p.layer_ticket = c->layer_ticket;
+  p.seq_ticket = c->seq_ticket; p.tail_vs = c->tail_vs; p.tail_sorted = c->tail_sorted; p.tail_tok = c->tail_tok;
   p.fifo_vals = c->fifo_vals; p.fifo_cnt = c->fifo_cnt; p.R = c->cfg.fifo_len;
   p.tab = c->cur_table;
   p.C1 = c->cfg.C1; p.C2 = c->cfg.C2;
