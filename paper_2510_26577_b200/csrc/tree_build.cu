@@ -323,11 +323,25 @@ __device__ __forceinline__ void tail_decide(const ExpandParams& p, const TailSta
       const int g = select_grid(ctx, p.tab.L, p.tab.M);
       c_mine = p.tab.fD[(size_t)(g - 1) * p.tab.Ntab + tid] / p.tab.fT[(size_t)(g - 1) * p.tab.Ntab];
     }
-    double a = 0.0;
-#pragma unroll 4
-    for (int b = 0; b < B; ++b) a += GLOBAL ? __ldcg(vs_i + b * CAST_MAX_WIDTH + tid) : vs_i[b * CAST_MAX_WIDTH + tid];
-    vbar[tid] = a / (double)B;
+    if (!GLOBAL) {
+      double a = 0.0;
+#pragma unroll 1
+      for (int b = 0; b < B; ++b) a += vs_i[b * CAST_MAX_WIDTH + tid];
+      vbar[tid] = a / (double)B;
+    }
     c[tid] = c_mine;
+  }
+  if (GLOBAL) {
+    // many sequences: warp j sums rank j over the sequences, two per lane, then a fixed shuffle tree
+    static_assert(kSweepThreads / 32 >= CAST_MAX_WIDTH && CAST_MAX_BATCH <= 64, "one warp per rank, two sequences per lane");
+    const int j = tid >> 5, lane = tid & 31;
+    if (j < n) {
+      double a = (lane < B ? __ldcg(vs_i + lane * CAST_MAX_WIDTH + j) : 0.0) +
+                 (lane + 32 < B ? __ldcg(vs_i + (lane + 32) * CAST_MAX_WIDTH + j) : 0.0);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+      if (lane == 0) vbar[j] = a / (double)B;
+    }
   }
   __syncthreads();
   if (tid < 32) {  // inclusive scan of at most 16 values
