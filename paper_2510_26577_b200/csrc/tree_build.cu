@@ -930,23 +930,27 @@ __device__ __noinline__ void select_finalize_phase(const SelectParams& p, int b,
   if (p.enable_dr && p.tab.Ntab < n) n = p.tab.Ntab;
   if (tid == 0) s_N = 1;
   // u_k = sum_{s<=k} v(s), v(s) = batch mean of the rank-s values (Eq. 1), or this sequence's own
-  // rank-s value when every sequence sizes its tree by itself
+  // rank-s value when every sequence sizes its tree by itself. The means first, a thread per rank with
+  // several loads in flight (u doubles as their buffer), then the prefix sums in one warp.
+#pragma unroll 1
+  for (int s = tid; s < n; s += nt) {
+    double a = 0.0;
+    if (p.per_row) {
+      a = p.sel_value[(size_t)b * p.Ncap + s];
+    } else {
+#pragma unroll 8
+      for (int bb = 0; bb < B; ++bb) a += p.sel_value[(size_t)bb * p.Ncap + s];
+      a /= (double)B;
+    }
+    u[s] = a;
+  }
+  __syncthreads();
   if (tid < 32) {
     double v[4], run = 0.0;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       const int s = lane * 4 + e;
-      double a = 0.0;
-      if (s < n) {
-        if (p.per_row) {
-          a = p.sel_value[(size_t)b * p.Ncap + s];
-        } else {
-#pragma unroll 1
-          for (int bb = 0; bb < B; ++bb) a += p.sel_value[(size_t)bb * p.Ncap + s];
-          a /= (double)B;
-        }
-      }
-      run += a;
+      run += s < n ? u[s] : 0.0;
       v[e] = run;
     }
     double incl = run;  // inclusive scan of the lane totals
