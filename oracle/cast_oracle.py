@@ -14,7 +14,12 @@ verified tokens, v(u) node value, u_k utility, c_k normalised cost.
 Pins (tests marked "not gpu"): Algorithm 1 on hand-worked cases and on the
 Theorem's linear-cost special case in exact rational arithmetic; select() on a
 hand table; expansion and rerank against brute-force enumeration of all paths
-on tiny vocabularies; attention against separately coded causal attention on a
+on tiny vocabularies; the composition of Eq. 1, Eq. 2, Algorithm 1, the depth
+test and the rerank inside expand() / select_nodes() with every sizing switch
+on against a batch-2, two-step case worked by hand in exact fractions (ragged
+prefixes, cost rows that all differ, f_D not proportional to f_T, C1 != C3),
+and the orders of exactly equal values and the ">=" of the depth test against
+hand-worked exact-tie cases (tests/golden/cast_step_*.txt); attention against separately coded causal attention on a
 chain tree and against per-path dense attention; acceptance against sequential
 token-by-token decoding; stochastic acceptance against a hand-worked case, the
 greedy rule for a one-hot target, the all-accept case P_T = P_D and the
@@ -69,26 +74,27 @@ class CostTable:
 
 def alg1_select_max_valid_index(u, c, C: float, slack: float = 0.0) -> int:
     """Algorithm 1 ("Select Maximum Valid Index").  u, c hold u[1..n], c[1..n]
-    (python index k-1 holds element k); returns max{j : mark[j] = 1} in 1..n.
+    (python index k-1 holds element k), c strictly increasing.
 
-    The test (u[j]-u[i])/(c[j]-c[i]) < C is evaluated division-free (c is
-    strictly increasing, so the denominator is positive).  The outer loop does
-    not skip indices already unmarked, as printed.  `slack` shifts every test by
-    slack*(|u[j]|+|u[i]|); it is 0 for the algorithm proper and is used only by
-    alg1_is_stable.
+    What the algorithm computes: index j is valid iff every chord from an
+    earlier index i < j has slope (u[j]-u[i])/(c[j]-c[i]) >= C (a cleared index
+    still clears later ones; index 1 has no earlier index and is always valid);
+    the result is the largest valid index.  The slope test is written
+    division-free (the denominator is positive) and strict: a slope of exactly
+    C keeps the index.  `slack` shifts every test by slack*(|u[j]|+|u[i]|); it
+    is 0 for the algorithm proper and is used only by alg1_is_stable.
     """
     n = len(u)
     assert n >= 1 and len(c) == n
-    mark = [1] * n
-    for i in range(n):
-        for j in range(i + 1, n):
-            lhs = u[j] - u[i]
-            rhs = C * (c[j] - c[i])
-            if slack != 0.0:
-                rhs = rhs + slack * (abs(u[j]) + abs(u[i]))
-            if lhs < rhs:
-                mark[j] = 0
-    return max(j + 1 for j in range(n) if mark[j] == 1)
+
+    def chord_ok(i, j):
+        bound = C * (c[j] - c[i])
+        if slack != 0.0:
+            bound = bound + slack * (abs(u[j]) + abs(u[i]))
+        return not (u[j] - u[i] < bound)
+
+    valid = [j for j in range(n) if all(chord_ok(i, j) for i in range(j))]
+    return valid[-1] + 1
 
 
 def alg1_is_stable(u, c, C: float, rel: float = 2e-6) -> bool:
@@ -343,6 +349,7 @@ class CastOracle:
                 out["scores"][b, t] = self.score[b][p]
             out["anc"][b] = ancestor_masks(out["parent"][b], N, words)
         self.last_u_sel = u_mean
+        self.last_c_sel = c if cfg.enable_dr else None
         return out
 
 

@@ -655,3 +655,90 @@ def test_compaction_is_an_out_of_place_gather(page):
     # identity path leaves the cache as it was
     nk2, _, _ = compact_kv(k, v, page, table, kv_len, np.array([[0, 1, 2, 3]] * 2), np.array([3, 3]))
     assert np.array_equal(nk2, k)
+
+
+# ------------------------------------- hand-worked steps with the sizing switches on
+def _close(got, want_fracs, tol=1e-12):
+    want = np.array([float(v) for v in want_fracs])
+    got = np.asarray(got, dtype=np.float64)
+    return got.shape == want.shape and bool(np.all(np.abs(got - want) <= tol * np.maximum(1.0, np.abs(want))))
+
+
+def _run_golden_case(case):
+    """Feeds a hand-worked case to the oracle and checks every written-out value."""
+    import golden_cases  # noqa: F401  (tests/ is on sys.path under pytest)
+
+    tables = None
+    if case.fT:
+        L, M, Ntab, fT, fD = case.table_arrays()
+        tables = {case.B: CostTable(case.B, L, M, Ntab, fT, fD)}
+    o = CastOracle(OracleConfig(**case.config_kwargs()), tables)
+    H = int(case.param["H"])
+    for step in case.steps():
+        o.step_begin(case.root, case.kv_len)
+        for layer in range(1, H + 1):
+            nt, npr, cnt = o.expand(layer, case.logits(layer))
+            if layer not in case.layers(step):
+                assert cnt == 0 and o.layers_done < layer, f"step {step}: layer {layer} should not exist"
+                continue
+            key = ("step", step, "layer", layer)
+            n_i = case.ints(*key, "n")[0][0]
+            assert o.n_hist[layer] == n_i, (key, o.n_hist)
+            assert cnt == case.ints(*key, "next_count")[0][0], (key, cnt)
+            if case.has(*key, "u"):
+                assert _close(o.last_u, case.get(*key, "u")[0]), (key, o.last_u)
+            if case.has(*key, "c"):
+                assert _close(o.last_c, case.get(*key, "c")[0]), (key, o.last_c)
+            for b in range(case.B):
+                assert list(nt[b, :n_i]) == case.ints(*key, "next_tokens")[b], (key, b, nt[b])
+                assert list(npr[b, :n_i]) == case.ints(*key, "next_parent_row")[b], (key, b, npr[b])
+        if case.has("step", step, "fifo"):
+            for i, want in enumerate(case.get("step", step, "fifo")):
+                assert _close(o.fifo[i], want), (step, i, o.fifo[i])
+        if case.has("step", step, "N"):
+            sel = o.select_nodes()
+            _check_selection(case, ("step", step), sel, o)
+    # the same expansion reranked under other budgets m (fixed-mode cases)
+    for m in case.select_budgets():
+        o.cfg.total_token = m
+        _check_selection(case, ("select", "m", m), o.select_nodes(), o)
+
+
+def _check_selection(case, key, sel, o):
+    N = case.ints(*key, "N")[0][0]
+    assert list(sel["n_tree"]) == [N] * case.B, (key, sel["n_tree"])
+    if case.has(*key, "rerank", "u"):
+        assert _close(o.last_u_sel, case.get(*key, "rerank", "u")[0]), (key, o.last_u_sel)
+        assert _close(o.last_c_sel, case.get(*key, "rerank", "c")[0]), (key, o.last_c_sel)
+    for name in ("tokens", "parent", "depth", "pool_idx"):
+        for b in range(case.B):
+            assert list(sel[name][b, :N]) == case.ints(*key, name)[b], (key, name, b, sel[name][b])
+    if case.has(*key, "anc"):
+        for b in range(case.B):
+            assert list(sel["anc"][b, :N, 0]) == case.ints(*key, "anc")[b], (key, "anc", b)
+
+
+def test_hand_worked_step_batch_two_all_switches():
+    """Eq. 1 (batch mean of per-sequence prefix sums), Eq. 2 (draft row over the
+    target's first entry, context = nodes retained so far), Algorithm 1 with C1,
+    the depth test on c_{n_i} and the rerank (target row at n_0 = longest prefix,
+    C3) composed as the paper states them: every intermediate value of two
+    consecutive steps is compared with the hand derivation in the golden file."""
+    import golden_cases
+
+    (case,) = golden_cases.load("cast_step_b2.txt")
+    _run_golden_case(case)
+
+
+def test_hand_worked_exact_ties():
+    """Order of exactly equal values (token id within a layer; depth first over
+    the whole tree, so that the kept set is a tree) and the '>=' of the depth
+    test at exact equality."""
+    import golden_cases
+
+    cases = golden_cases.load("cast_step_ties.txt")
+    assert [c.name for c in cases] == ["layer_and_global_order", "depth_test_equality"]
+    # the construction relies on these two floating-point facts
+    assert np.log(0.5) + np.log(2.0) == 0.0 and np.exp(golden_cases.ZERO_PROB_LOGIT) == 0.0
+    for case in cases:
+        _run_golden_case(case)
