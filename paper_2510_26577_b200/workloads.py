@@ -214,13 +214,24 @@ def stochastic_accept_inputs(w: Workload, tokens, parent, n_tree, device="cpu", 
 
 
 def cost_table_arrays(w: Workload, B: int, L: int = 512, M: int = 64, Ntab: int = 128,
-                      stepped: bool = False) -> Tuple[int, int, int, np.ndarray, np.ndarray]:
+                      stepped: bool = False, skewed: bool = False) -> Tuple[int, int, int, np.ndarray, np.ndarray]:
     """Synthetic stand-in for the profiled latency tables (the real ones need
     the models): f_T(B, c, n) = 1 + 0.25*B*c/(64*4096) + tau*B*n on the grid
     c = g*L, n = 1..Ntab, and f_D = 0.05 * f_T; strictly increasing in n.  The
-    `stepped` variant adds 0.02*ceil(B*n/64) (tile quantisation)."""
+    `stepped` variant adds 0.02*ceil(B*n/64) (tile quantisation).
+
+    `skewed` is a test family in which a lookup in the wrong table, the wrong
+    grid row or the wrong column changes the numbers visibly: the rows differ
+    by tens of percent (so the grid step should be small enough for the
+    contexts in play to cross rows), the slope in n grows with the row, and
+    f_D is not a multiple of f_T (own offset, convex in n)."""
     c = (np.arange(1, M + 1, dtype=np.float64) * L)[:, None]
     n = np.arange(1, Ntab + 1, dtype=np.float64)[None, :]
+    if skewed:
+        g = np.arange(1, M + 1, dtype=np.float64)[:, None]
+        fT = 1.0 + 0.35 * g + w.tau * B * n * (1.0 + 0.25 * g)
+        fD = 0.02 + 0.015 * g * g + 0.4 * w.tau * B * n ** 1.25 / (1.0 + 0.1 * g)
+        return L, M, Ntab, fT, fD
     fT = 1.0 + 0.25 * (B * c) / (64.0 * 4096.0) + w.tau * B * n
     if stepped:
         fT = fT + 0.02 * np.ceil(B * n / 64.0)

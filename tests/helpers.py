@@ -22,7 +22,9 @@ def cfg_kwargs(w: wl.Workload, **over):
     return kw
 
 
-def make_tables(w: wl.Workload, B: int, stepped=False):
+def make_tables(w: wl.Workload, B: int, stepped=False, skewed=False):
+    if skewed:  # a fine grid, so that the tree's own context (tens of nodes) and the ragged prefixes cross rows
+        return wl.cost_table_arrays(w, B, L=8, M=48, Ntab=64, skewed=True)
     L, M, Ntab, fT, fD = wl.cost_table_arrays(w, B, stepped=stepped)
     return L, M, Ntab, fT, fD
 

@@ -24,17 +24,17 @@ def binding():
     return b
 
 
-def _oracle_tables(w, B, stepped=False):
+def _oracle_tables(w, B, stepped=False, skewed=False):
     from oracle import CostTable
-    L, M, Ntab, fT, fD = make_tables(w, B, stepped)
+    L, M, Ntab, fT, fD = make_tables(w, B, stepped, skewed)
     return {B: CostTable(B, L, M, Ntab, fT, fD)}, (L, M, Ntab, fT, fD)
 
 
-def build_tree_both(binding, w, peaked=False, stepped=False, steps=1, **over):
+def build_tree_both(binding, w, peaked=False, stepped=False, steps=1, skewed=False, **over):
     kw = cfg_kwargs(w, **over)
     B = w.batch
     need = kw.get("enable_bp") or kw.get("enable_dp") or kw.get("enable_dr")
-    tables, raw = _oracle_tables(w, B, stepped) if need else (None, None)
+    tables, raw = _oracle_tables(w, B, stepped, skewed) if need else (None, None)
     ctx = binding.CastContext(max_batch=B, **kw)
     if need:
         ctx.cast_set_cost_tables(B, *raw)
@@ -265,6 +265,87 @@ def test_cost_model_switches_multi_step(binding, over):
                     tau=4e-2)
     build_tree_both(binding, w, peaked=True, steps=3, **over)
     build_tree_both(binding, w, peaked=True, stepped=True, steps=2, **over)
+
+
+@pytest.mark.parametrize("over", [
+    dict(enable_bp=1, enable_dp=1, enable_dr=1, C1=0.6, C2=0.05, C3=0.25),
+    dict(enable_bp=1, enable_dp=1, enable_dr=1, C1=0.25, C2=0.02, C3=0.6, max_width=6),
+    dict(enable_bp=1, enable_dr=1, ctx_base_mode=1, C1=0.4, C3=0.15),
+    dict(enable_dr=1, rerank_per_row=1, C3=0.3),
+])
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_cost_model_tables_where_a_wrong_lookup_shows(binding, over, seed):
+    """Tables whose rows differ by tens of percent on a grid of 8 positions, f_D not a multiple of
+    f_T, ragged prefixes that land in different rows, C1 != C3: a lookup in the wrong table, row
+    or column, or a swapped threshold, changes the tree.  Three steps, so the depth-pruning
+    buffers carry over.  A draw that sits within rounding of a threshold is skipped by the
+    oracle's margin, not reseeded."""
+    w = wl.Workload("skew", 83, 3, "f32", "f32", 4, 2, 64, 5, 300, 0, 2500, 2.0, 5, 4, 24, False, 2, max_tree=32,
+                    tau=2.5e-2, seed_salt=seed)
+    try:
+        ctx, g, o, root, kv = build_tree_both(binding, w, peaked=True, steps=3, skewed=True, **over)
+    except AssertionError as e:
+        if "decision boundary" in str(e):
+            pytest.skip(str(e))
+        raise
+    # the case must exercise the switches: some layer narrowed or stopped, and a rerank below the budget
+    assert min(o["n_hist"]) < (over.get("max_width") or w.top_k) or len(o["n_hist"]) < w.depth or \
+        int(o["n_tree"].min()) < w.total_token
+
+
+def _golden_gpu_case(binding, case):
+    kw = case.config_kwargs()
+    B = case.B
+    ctx = binding.CastContext(max_batch=B, **kw)
+    if case.fT:
+        ctx.cast_set_cost_tables(B, *case.table_arrays())
+    root = torch.tensor(case.root, dtype=torch.int32, device="cuda")
+    kv = torch.tensor(case.kv_len, dtype=torch.int32, device="cuda")
+    H = int(case.param["H"])
+    logits = [torch.from_numpy(case.logits(l)).float().cuda() for l in range(1, H + 1)]
+    for step in case.steps():
+        g = gpu_tree(ctx, root, kv, logits)
+        assert g["status"][0] == 0
+        layers = case.layers(step)
+        assert g["info"]["layers"] == len(layers)
+        for layer in layers:
+            key = ("step", step, "layer", layer)
+            n_i = case.ints(*key, "n")[0][0]
+            nt, npr, cnt = g["per_layer"][layer - 1]
+            assert g["info"]["n_hist"][layer - 1] == n_i, (key, g["info"]["n_hist"])
+            assert cnt == case.ints(*key, "next_count")[0][0], key
+            for b in range(B):
+                assert list(nt[b, :n_i]) == case.ints(*key, "next_tokens")[b], (key, b)
+                assert list(npr[b, :n_i]) == case.ints(*key, "next_parent_row")[b], (key, b)
+        N = case.ints("step", step, "N")[0][0]
+        assert list(g["n_tree"]) == [N] * B
+        for name in ("tokens", "parent", "depth", "pool_idx"):
+            for b in range(B):
+                assert list(g[name][b, :N]) == case.ints("step", step, name)[b], (step, name, b)
+        for b in range(B):
+            assert list(g["anc"][b, :N, 0]) == case.ints("step", step, "anc")[b]
+    return ctx
+
+
+def test_hand_worked_step_on_the_gpu(binding):
+    """The batch-2, two-step case derived by hand in tests/golden/cast_step_b2.txt (every sizing
+    switch on; cost rows, tables and thresholds chosen so that a wrong lookup changes a decision)
+    through the C-ABI: the library's decisions and trees against the hand-derived ones, not
+    against the oracle."""
+    import golden_cases
+
+    (case,) = golden_cases.load("cast_step_b2.txt")
+    ctx = _golden_gpu_case(binding, case)
+    # the depth-pruning buffers after the two steps, read back through the state export
+    import struct
+    blob = ctx.cast_state_export()
+    nbuf, R = struct.unpack_from("ii", blob, 0)
+    off = 8
+    for i, want in enumerate(case.get("step", 2, "fifo")):
+        cnt, = struct.unpack_from("i", blob, off)
+        vals = struct.unpack_from(f"{R}d", blob, off + 4)
+        off += 4 + 8 * R
+        assert cnt == len(want) and np.allclose(vals[:cnt], [float(v) for v in want], rtol=1e-6), (i, vals)
 
 
 def test_state_export_import_roundtrip(binding):
