@@ -24,9 +24,9 @@
  *  - `stream` is a cudaStream_t passed as void*. Compute calls only enqueue
  *    work: they never synchronise the host. Tree sizes (n_i, go/no-go, N) are
  *    decided on the device and stay there.
- *  - Compute calls allocate nothing, with one exception: cast_tree_attention
- *    grows a context-owned workspace the first time it sees a larger shape
- *    (do that call once before capturing a CUDA graph).
+ *  - Compute calls allocate nothing. The split workspace of the attention is
+ *    sized at set-up time by cast_reserve_attention; an attention call whose
+ *    shape needs more than was reserved returns CAST_ERR_CAPACITY.
  *  - The return value reports errors the host can see (bad arguments, caps).
  *    Errors only the device can see (non-finite logits, a malformed tree, a
  *    page index out of range) are written to a device status word; read it with
@@ -179,6 +179,18 @@ CAST_API cast_status cast_select_nodes(cast_ctx* ctx, int32_t* tokens, int32_t* 
                               void* stream);
 
 /*
+ * Set-up call (synchronises the device and may allocate; not a compute call): sizes the context's
+ * attention workspace for calls of cast_tree_attention / cast_tree_attention_rows with these arguments
+ * (the partial results of the KV splits; nothing in the paper corresponds to it). The workspace only
+ * grows: reserving several shapes keeps the largest. Every shape that will be used has to be reserved
+ * once, before the first attention call of that shape and before any stream capture; an attention call
+ * whose shape needs more than was reserved returns CAST_ERR_CAPACITY and launches nothing.
+ * Errors: INVALID_ARG, DTYPE, SHAPE (as for cast_tree_attention), CAPACITY (B beyond max_batch), CUDA.
+ */
+CAST_API cast_status cast_reserve_attention(cast_ctx* ctx, cast_dtype dtype, int B, int Hq, int Hkv, int D,
+                                   int page_size, int seq_capacity);
+
+/*
  * One layer of verification attention (the mask of Sec. "Tree Reranking Phase"):
  * out[b,t,h] = softmax over {prefix positions 0..kv_len[b]-1} U {tree positions
  * kv_len[b]+j : bit j of anc_mask[b,t]} of (q . k) * scale, times v, for
@@ -192,7 +204,8 @@ CAST_API cast_status cast_select_nodes(cast_ctx* ctx, int32_t* tokens, int32_t* 
  *                 seq_capacity is then the number of entries per sequence)
  *   scale         0 selects 1/sqrt(D)
  * Accumulation is fp32. Needs Hq % Hkv == 0, D in {64, 128}, 16-byte aligned
- * pointers. Device errors: BAD_PAGE.
+ * pointers, and a workspace reserved for this shape (cast_reserve_attention; else CAST_ERR_CAPACITY).
+ * Device errors: BAD_PAGE.
  */
 CAST_API cast_status cast_tree_attention(cast_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
                                 cast_dtype dtype, int B, int Hq, int Hkv, int D, int page_size,
@@ -280,7 +293,8 @@ CAST_API cast_status cast_accept_stochastic_plan(cast_ctx* ctx, cast_dtype dtype
  * K and V, with out-of-place semantics; then kv_len[b] += accept_len[b] + 1.
  * Layer l of a cache starts layer_stride_bytes * l after the base pointer.
  * Cache layout, page_size, page_table, seq_capacity, num_pages as for
- * cast_tree_attention. Device errors: BAD_PAGE (also for a path entry < 0).
+ * cast_tree_attention. Device errors: BAD_PAGE (also for a path entry < 0 or below its own place on the path,
+ * or a row past the sequence's capacity: nothing is stored and kv_len stays).
  */
 CAST_API cast_status cast_compact_kv(cast_ctx* ctx, void* k_cache, void* v_cache, cast_dtype dtype, int B,
                             int n_layers, size_t layer_stride_bytes, int Hkv, int D, int page_size,

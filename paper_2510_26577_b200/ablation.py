@@ -55,6 +55,7 @@ def run(batches, steps, thresholds):
             ctx = binding.CastContext(max_batch=B, vocab=w.vocab, top_k=K, max_depth=H, total_token=w.total_token,
                                       max_tree=Ncap, C1=C1, C2=C2, C3=C3, **flags)
             ctx.cast_set_cost_tables(B, *wl.cost_table_arrays(w, B))
+            ctx.cast_reserve_attention(q.dtype, B, w.q_heads, w.kv_heads, w.head_dim, w.page_size, seq_cap)
             nt = torch.empty((B, K), dtype=torch.int32, device=dev)
             npr = torch.empty_like(nt)
             cnt = torch.empty((1,), dtype=torch.int32, device=dev)

@@ -27,7 +27,7 @@ EXPORTS = [
     "cast_create", "cast_destroy", "cast_status_string", "cast_set_cost_tables", "cast_state_export",
     "cast_state_import", "cast_step_begin", "cast_tree_expand", "cast_select_nodes", "cast_tree_attention",
     "cast_accept", "cast_compact_kv", "cast_poll_status", "cast_step_info", "cast_accept_static",
-    "cast_accept_stochastic", "cast_accept_stochastic_plan", "cast_tree_attention_rows",
+    "cast_accept_stochastic", "cast_accept_stochastic_plan", "cast_tree_attention_rows", "cast_reserve_attention",
 ]
 
 
@@ -72,6 +72,7 @@ def load_library() -> C.CDLL:
         "cast_step_begin": [vp, i32, i32p, i32p, vp],
         "cast_tree_expand": [vp, i32, vp, i32, i32p, i32p, i32p, vp],
         "cast_select_nodes": [vp, i32p, i32p, i32p, vp, i32p, vp, i32p, vp],
+        "cast_reserve_attention": [vp, i32, i32, i32, i32, i32, i32, i32],
         "cast_tree_attention": [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32p, i32, i32, i32p, vp, i32p,
                                 C.c_float, vp, vp],
         "cast_tree_attention_rows": [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32p, i32, i32, i32p, vp, i32p,
@@ -172,6 +173,12 @@ class CastContext:
 
     def cast_state_import(self, blob: bytes):
         _check(self.lib.cast_state_import(self.handle, blob, len(blob)), "cast_state_import")
+
+    def cast_reserve_attention(self, dtype, B, Hq, Hkv, D, page_size, seq_capacity):
+        """Sizes the attention workspace for calls of this shape (set-up time; synchronises)."""
+        code = CAST_F32 if dtype == torch.float32 else CAST_BF16
+        _check(self.lib.cast_reserve_attention(self.handle, code, B, Hq, Hkv, D, page_size, seq_capacity),
+               "cast_reserve_attention")
 
     # --- compute calls (enqueue only) ----------------------------------------
     def cast_step_begin(self, B, root_token, kv_len, stream=None):

@@ -28,9 +28,12 @@ if ROOT not in sys.path:
 N_POINTS = (1, 2, 4, 8, 16, 32, 64, 128)  # tree sizes that are timed; the rest is interpolated
 
 
-def measure_attention_us(w, B: int, L: int, M: int, n_points=N_POINTS, reps: int = 10):
+def measure_attention_us(w, B: int, L: int, M: int, n_points=N_POINTS, reps: int = 10, max_bytes: int = 12 << 30):
     """t[g-1][j] = microseconds of one `cast_tree_attention` layer at context g*L and n_points[j] tree
-    tokens per sequence (chain trees; the mask's shape does not change the time)."""
+    tokens per sequence (chain trees; the mask's shape does not change the time). Successive calls read
+    different KV buffers, enough of them that a buffer has left the L2 cache (more than twice its size has
+    been read) before it is used again: the figures are HBM figures, as in a model whose layers each have
+    their own cache."""
     import torch
     from paper_2510_26577_b200 import binding, workloads as wl
 
@@ -40,9 +43,20 @@ def measure_attention_us(w, B: int, L: int, M: int, n_points=N_POINTS, reps: int
     ctx = binding.CastContext(max_batch=B, vocab=w.vocab, top_k=w.top_k, max_depth=w.depth, total_token=w.max_tree,
                               max_tree=w.max_tree)
     q = wl.query(wb, 0, dev)
-    k, v = wl.kv_cache(wb, 0, dev)
+    k0, v0 = wl.kv_cache(wb, 0, dev)
     table, num_pages = wl.page_table(wb, dev)
     seq_cap = wl.seq_capacity(wb) // (wb.page_size or 1)
+    ctx.cast_reserve_attention(q.dtype, B, w.q_heads, w.kv_heads, w.head_dim, w.page_size, seq_cap)
+    l2 = int(torch.cuda.get_device_properties(dev).L2_cache_size)
+    row_bytes = 2 * w.kv_heads * w.head_dim * k0.element_size()  # K and V of one position
+
+    def buffers_needed(ctx_len):
+        return -(-2 * l2 // max(B * ctx_len * row_bytes, 1)) + 1
+
+    buf_bytes = 2 * k0.numel() * k0.element_size()
+    nbuf = max(2, min(buffers_needed(L), 128, max_bytes // buf_bytes))
+    ks = [k0] + [torch.randn_like(k0) for _ in range(nbuf - 1)]
+    vs = [v0] + [torch.randn_like(v0) for _ in range(nbuf - 1)]
     out = torch.empty_like(q)
     words = ctx.words
     stream = torch.cuda.Stream(device=dev)
@@ -57,14 +71,16 @@ def measure_attention_us(w, B: int, L: int, M: int, n_points=N_POINTS, reps: int
             n_tree = torch.full((B,), n, dtype=torch.int32, device=dev)
             for g in range(1, M + 1):
                 kv_len = torch.full((B,), g * L, dtype=torch.int32, device=dev)
-                call = lambda: ctx.cast_tree_attention(q, k, v, B, w.q_heads, w.kv_heads, w.head_dim, w.page_size, table,
-                                                       seq_cap, num_pages, kv_len, anc_t, n_tree, 0.0, out)
-                for _ in range(3):
-                    call()
+                use = max(2, min(nbuf, buffers_needed(g * L)))
+                call = lambda i: ctx.cast_tree_attention(q, ks[i % use], vs[i % use], B, w.q_heads, w.kv_heads, w.head_dim,
+                                                         w.page_size, table, seq_cap, num_pages, kv_len, anc_t, n_tree,
+                                                         0.0, out)
+                for i in range(3):
+                    call(i)
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record(stream)
-                for _ in range(reps):
-                    call()
+                for i in range(reps):
+                    call(3 + i)
                 e1.record(stream)
                 stream.synchronize()
                 t[g - 1, j] = e0.elapsed_time(e1) * 1e3 / reps

@@ -191,7 +191,9 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const CompactP
       const int which = i / per, rem = i % per, j = rem / vpr, vv = rem % vpr;
       const int src = p.accept_path[b * p.H1 + j];
       const int pos = L + src;
-      if (src < 0 || pos >= max_pos) {
+      // a path element is a tree index no smaller than its place on the path (parents precede children), so
+      // the destination L + j never lies past the source; anything else is a malformed path
+      if (L < 0 || src < j || pos >= max_pos) {
         bad = true;
         continue;
       }

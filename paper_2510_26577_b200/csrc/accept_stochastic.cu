@@ -21,22 +21,6 @@
 
 using namespace cast;
 
-// Development aid, compiled only with -DCAST_PHASE_CLOCKS: thread 0 of the first CTA of sequence 0 records
-// the global timer at phase boundaries.
-#ifdef CAST_PHASE_CLOCKS
-__device__ long long g_sto_clock[64];
-__device__ int g_sto_clock_n;
-#define STO_STAMP() do { if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && sto_n < 64) { long long _t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(_t)); g_sto_clock[sto_n++] = _t; g_sto_clock_n = sto_n; } } while (0)
-#define STO_STAMP_DECL int sto_n = 0;
-extern "C" __attribute__((visibility("default"))) int cast_debug_read_sto_clocks(long long* out, int* n) {
-  cudaMemcpyFromSymbol(n, g_sto_clock_n, sizeof(int));
-  return (int)cudaMemcpyFromSymbol(out, g_sto_clock, sizeof(long long) * 64);
-}
-#else
-#define STO_STAMP() do {} while (0)
-#define STO_STAMP_DECL
-#endif
-
 namespace {
 
 constexpr int kStoThreads = 512;
@@ -203,8 +187,6 @@ __global__ void __launch_bounds__(kStoThreads, 1) accept_stochastic_kernel(const
   // the peers' shared memory may be written once all CTAs of the cluster run
   if (cs > 1) sto_cluster_sync(); else __syncthreads();
 
-  STO_STAMP_DECL
-  STO_STAMP();  // 0: start
   int parity = 0;
   int cur = 0, plen = 1;   // current node, nodes on the path so far
   double a = 0.0;          // the distribution that stands at `cur`: max(0, P_T - a P_D) / F(a)
@@ -280,7 +262,6 @@ __global__ void __launch_bounds__(kStoThreads, 1) accept_stochastic_kernel(const
         }
       }
       sto_block_reduce<true, 2>(sh, mx);
-    STO_STAMP();
       Mp_loc = mx[0];
       Mq_loc = mx[1];
       double sm[2] = {0.0, 0.0};
@@ -307,10 +288,8 @@ __global__ void __launch_bounds__(kStoThreads, 1) accept_stochastic_kernel(const
         }
       }
       sto_block_reduce<false, 2>(sh, sm);
-    STO_STAMP();
       const double rec[4] = {Mp_loc, sm[0], Mq_loc, sm[1]};
       sto_exchange(sh, parity, rank, cs, rec);
-    STO_STAMP();
       // fold of the ranks' records, the same in every warp of every CTA: lanes 0-15 take the target row's
       // records by rank, lanes 16-31 the draft row's; maxima and sums through a fixed shuffle tree
       {
@@ -369,10 +348,8 @@ __global__ void __launch_bounds__(kStoThreads, 1) accept_stochastic_kernel(const
 #pragma unroll 4
       for (int i = tid; i < len; i += kStoThreads) part[0] += fmax(0.0, pt(i) * cp - a2 * (qt(i) * cq));
       sto_block_reduce<false, 1>(sh, part);
-    STO_STAMP();
       const double rec[4] = {part[0], 0.0, 0.0, 0.0};
       sto_exchange(sh, parity, rank, cs, rec);
-      STO_STAMP();
       double F2 = 0.0;
       for (int r = 0; r < cs; ++r) F2 += sh.xch[parity][r][0];
       parity ^= 1;
@@ -397,7 +374,6 @@ __global__ void __launch_bounds__(kStoThreads, 1) accept_stochastic_kernel(const
   }
   double total = 0.0;
   for (int r = 0; r < cs; ++r) total += sh.xch[parity][r][0];
-  STO_STAMP();
   const double goal = p.u_bonus[b] * total;
   // the slice in which the cumulative sum reaches the goal (rounding may leave none: the last non-empty one)
   int owner = -1, last_nonempty = 0;

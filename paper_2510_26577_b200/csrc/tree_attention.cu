@@ -20,6 +20,8 @@ bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const v
                               int page_size, const int32_t* page_table, int seq_capacity, int num_pages,
                               const int32_t* kv_len, const uint32_t* anc, const int32_t* n_tree, const int32_t* first_row,
                               float scale, void* out, cudaStream_t stream, cast_status* status);
+size_t tree_attention_tc_workspace(const cast_ctx* c, int B, int Hq, int Hkv, int D, int page_size, int seq_capacity);
+cast_status tree_attention_tc_reserve(cast_ctx* c, size_t bytes);
 }
 
 namespace {
@@ -298,27 +300,30 @@ __global__ void __launch_bounds__(D) attn_combine_kernel(const AttnParams p) {
   store_out(out + d, l > 0.f ? acc / l : 0.f);
 }
 
-template <typename T, int D>
-cast_status launch_cc(cast_ctx* c, AttnParams& p, cudaStream_t s) {
-  const int nrowblk = (p.Ncap * p.G + kRB - 1) / kRB;
-  const int base = p.B * p.Hkv * ((c->cfg.total_token * p.G + kRB - 1) / kRB);
+// KV splits of a CUDA-core launch and the partial rows its workspace holds.
+int cc_splits(const cast_ctx* c, int B, int Hkv, int G, int page_size, int seq_capacity) {
+  const int base = B * Hkv * ((c->cfg.total_token * G + kRB - 1) / kRB);
   int nsplit = (2 * c->num_sms + base - 1) / base;
-  const int max_pos = p.page_size == 0 ? p.seq_capacity : p.seq_capacity * p.page_size;
+  const int max_pos = page_size == 0 ? seq_capacity : seq_capacity * page_size;
   const int max_tiles = (max_pos + kPT - 1) / kPT;
   if (nsplit > max_tiles) nsplit = max_tiles;
   if (nsplit > kMaxSplit) nsplit = kMaxSplit;
   if (nsplit < 1) nsplit = 1;
+  return nsplit;
+}
+size_t cc_workspace(const cast_ctx* c, int B, int Hq, int Hkv, int D, int page_size, int seq_capacity) {
+  const size_t rows = (size_t)B * Hq * c->cfg.max_tree * cc_splits(c, B, Hkv, Hq / Hkv, page_size, seq_capacity);
+  return rows * (D + 2) * sizeof(float);
+}
+
+template <typename T, int D>
+cast_status launch_cc(cast_ctx* c, AttnParams& p, cudaStream_t s) {
+  const int nrowblk = (p.Ncap * p.G + kRB - 1) / kRB;
+  const int nsplit = cc_splits(c, p.B, p.Hkv, p.G, p.page_size, p.seq_capacity);
   p.nsplit = nsplit;
   const size_t rows = (size_t)p.B * p.Hq * p.Ncap * nsplit;
-  const size_t need = rows * (D + 2) * sizeof(float);
-  if (need > c->attn_ws_bytes) {  // grow the workspace (synchronises; not legal during graph capture)
-    CAST_CUDA_OK(cudaDeviceSynchronize());
-    if (c->attn_ws) cudaFree(c->attn_ws);
-    c->attn_ws = nullptr;
-    c->attn_ws_bytes = 0;
-    CAST_CUDA_OK(cudaMalloc(&c->attn_ws, need));
-    c->attn_ws_bytes = need;
-  }
+  // compute calls never allocate: the workspace comes from cast_reserve_attention
+  if (rows * (D + 2) * sizeof(float) > c->attn_ws_bytes) return CAST_ERR_CAPACITY;
   p.part_o = reinterpret_cast<float*>(c->attn_ws);
   p.part_ml = p.part_o + rows * D;
   const size_t smem = (size_t)(kRB * (D + 4) + kPT * (D + 4) + kPT * D + kRB * (kPT + 1)) * sizeof(float);
@@ -329,6 +334,30 @@ cast_status launch_cc(cast_ctx* c, AttnParams& p, cudaStream_t s) {
 }
 
 }  // namespace
+
+extern "C" cast_status cast_reserve_attention(cast_ctx* c, cast_dtype dtype, int B, int Hq, int Hkv, int D, int page_size,
+                                              int seq_capacity) {
+  if (!c || B < 1 || Hq < 1 || Hkv < 1 || page_size < 0 || seq_capacity < 1) return CAST_ERR_INVALID_ARG;
+  if (dtype != CAST_F32 && dtype != CAST_BF16) return CAST_ERR_DTYPE;
+  if (B > c->cfg.max_batch) return CAST_ERR_CAPACITY;
+  if (Hq % Hkv != 0 || (D != 64 && D != 128)) return CAST_ERR_SHAPE;
+  // a bf16 call takes the tensor-core path when shape and pointer alignment allow and the CUDA-core path
+  // otherwise: both workspaces are sized, so the choice at call time never needs memory
+  if (dtype == CAST_BF16) {
+    const cast_status st = tree_attention_tc_reserve(c, tree_attention_tc_workspace(c, B, Hq, Hkv, D, page_size, seq_capacity));
+    if (st != CAST_OK) return st;
+  }
+  const size_t need = cc_workspace(c, B, Hq, Hkv, D, page_size, seq_capacity);
+  if (need > c->attn_ws_bytes) {
+    CAST_CUDA_OK(cudaDeviceSynchronize());
+    if (c->attn_ws) cudaFree(c->attn_ws);
+    c->attn_ws = nullptr;
+    c->attn_ws_bytes = 0;
+    CAST_CUDA_OK(cudaMalloc(&c->attn_ws, need));
+    c->attn_ws_bytes = need;
+  }
+  return CAST_OK;
+}
 
 extern "C" cast_status cast_tree_attention_rows(cast_ctx* c, const void* q, const void* k_cache, const void* v_cache,
                                                 cast_dtype dtype, int B, int Hq, int Hkv, int D, int page_size,

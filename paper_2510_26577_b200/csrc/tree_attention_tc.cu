@@ -32,30 +32,9 @@
 #include <cuda.h>
 #include <cuda_fp16.h>
 #include <math.h>
-#include <stdlib.h>
 
 #include "cast_internal.h"
 
-#ifdef CAST_PHASE_CLOCKS
-__device__ long long g_attn_clock[256];
-extern "C" __attribute__((visibility("default"))) int cast_debug_read_attn_clocks(long long* out) {
-  return (int)cudaMemcpyFromSymbol(out, g_attn_clock, sizeof(long long) * 256);
-}
-#define TC_STAMP(role, it, k) do { if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (it) >= 2 && (it) < 6 && \
-    (threadIdx.x == ((role) ? 160 : 0))) g_attn_clock[(role) * 128 + ((it) - 2) * 16 + (k)] = clock64(); } while (0)
-#define TC_MARK(k) do { if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) g_attn_clock[240 + (k)] = clock64(); } while (0)
-__device__ unsigned long long g_cta_log[4 * 16384];
-extern "C" __attribute__((visibility("default"))) int cast_debug_read_cta_log(unsigned long long* out) {
-  return (int)cudaMemcpyFromSymbol(out, g_cta_log, sizeof(unsigned long long) * 4 * 16384);
-}
-__device__ __forceinline__ unsigned long long gtimer() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-__device__ __forceinline__ unsigned smid() { unsigned s; asm volatile("mov.u32 %0, %smid;" : "=r"(s)); return s; }
-#define TC_CTA_LOG(k, v) do { if (threadIdx.x == 0) { unsigned _id = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z); if (_id < 16384) g_cta_log[_id * 4 + (k)] = (v); } } while (0)
-#else
-#define TC_CTA_LOG(k, v) do {} while (0)
-#define TC_STAMP(role, it, k) do {} while (0)
-#define TC_MARK(k) do {} while (0)
-#endif
 
 namespace cast {
 
@@ -646,11 +625,6 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
   extern __shared__ __align__(1024) unsigned char smem[];  // no static shared memory: the base is 1 KB aligned
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  TC_MARK(0);
-  TC_CTA_LOG(0, gtimer());
-  TC_CTA_LOG(1, 0ull);
-  TC_CTA_LOG(3, 0ull);
-  TC_CTA_LOG(2, (unsigned long long)smid());
   const int cs = p.cs;
   const int crank = cs > 1 ? (int)cluster_ctarank() : 0;
   if (warp == 4 && lane == 0) {
@@ -662,7 +636,6 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const WorkItem wk = cs == 0 ? decode_work_chunked(p, (int)blockIdx.x, (int)gridDim.x) : decode_work(p, (int)blockIdx.x / cs, crank);
-  TC_MARK(1);
   if (blockIdx.x < p.B && tid == 0 && p.n_tree[blockIdx.x] > p.Nmax) report(p.st, CAST_ERR_BAD_TREE, blockIdx.x);
   if (!wk.valid) return;  // the whole cluster leaves
   const int b = wk.b, kvh = wk.kvh, rb = wk.rb, split = wk.split, N = wk.N, L = wk.L;
@@ -813,13 +786,11 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
       *reinterpret_cast<uint4*>(smem + kSmemQ + (c >> 3) * kRegionQ + swz(r, c & 7)) = qv[c];
     fence_proxy_async();
   }
-  TC_MARK(2);
   // everyone but the producer waits here for the barrier objects, the TMEM address and Q; the producer
   // only signals that the barriers exist (it arrived right after initialising them) and keeps loading
   tc_fence_before();
   if (warp != 4) asm volatile("bar.sync 2, %0;" ::"n"(kThreadsTC) : "memory");
   tc_fence_after();
-  TC_MARK(3);
   const uint32_t tmem_base = *tmem_base_s;
   const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 2 * kBN;
 
@@ -869,21 +840,16 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
       mma_qk(0, 0);
     }
     for (int it = 0; ok && it < ntile; ++it) {
-      TC_STAMP(1, it, 0);
       if (it + 1 < ntile) {
         ok = mbar_wait(&bar_fullk[(it + 1) % kStagesK], ((it + 1) / kStagesK) & 1);
         if (!ok) break;
-        TC_STAMP(1, it, 1);
         tc_fence_after();
         mma_qk((it + 1) % kStagesK, (it + 1) & 1);
-        TC_STAMP(1, it, 2);
       }
       ok = mbar_wait(&bar_p[it & 1], (it >> 1) & 1) && mbar_wait(&bar_fullv[it % kStagesV], (it / kStagesV) & 1);
       if (!ok) break;
-      TC_STAMP(1, it, 3);
       tc_fence_after();
       mma_pv(it % kStagesV, it & 1, it == 0);
-      TC_STAMP(1, it, 4);
     }
     if (!ok && lane == 0) report(p.st, CAST_ERR_TIMEOUT, b);
   } else if (warp < 4) {
@@ -899,13 +865,12 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     for (int it = 0; it < ntile; ++it) {
       const int buf = it & 1, stage = it % kStagesV;
       const int pos0 = (t0 + it) * kBN;
-      TC_STAMP(0, it, 0);
       float mx = -INFINITY;
       uint32_t v0 = 0xffffffffu, v1 = 0xffffffffu;  // visibility of this row's 64 columns
       // Fast path (every tile but the first, as a rule): one pass over the scores with the reference
       // maximum of the earlier tiles. P = 2^((s - m) * scale) is then not bounded by 1, but bf16 and the
-      // fp32 accumulators have the range for it; a row whose sum of P outgrows 2^60 moves its reference
-      // afterwards (P, the row sum and O are scaled by a power of two: exact).
+      // fp32 accumulators have the range for it; a row whose P would outgrow 2^60 in a half tile moves its
+      // reference before that half is written (see below).
       // P is written over the scores it came from, in tensor memory: 64 bf16 = 32 columns of this row's
       // lane; P V takes its A operand from there.
       bool done = false;
@@ -925,72 +890,101 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
             }
             if (!row_ok) v0 = v1 = 0u;
           }
-          const float neg_ms = row_ok ? -m_used * sc : 0.f;
-          const unsigned long long sc2 = pack_f2(sc, sc), neg2 = pack_f2(neg_ms, neg_ms);
+          float neg_ms = row_ok ? -m_used * sc : 0.f;
+          const unsigned long long sc2 = pack_f2(sc, sc);
+          uint32_t pk[2][16];
           unsigned long long lacc = pack_f2(0.f, 0.f);
+          {
+            const unsigned long long neg2 = pack_f2(neg_ms, neg_ms);
 #pragma unroll
-          for (int hh = 0; hh < 2; ++hh) {
-            uint32_t sr[32], pk[16];
-            tmem_ld32(tp + hh * 32, sr);
-            tmem_wait_ld();
-            const uint32_t vv = hh ? v1 : v0;
+            for (int hh = 0; hh < 2; ++hh) {
+              uint32_t sr[32];
+              tmem_ld32(tp + hh * 32, sr);
+              tmem_wait_ld();
+              const uint32_t vv = hh ? v1 : v0;
 #pragma unroll
-            for (int e = 0; e < 16; ++e) {
-              const int c = 2 * e;
-              float x0, x1;
-              unpack_f2(fma_f2(pack_f2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, neg2), x0, x1);
-              float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
-              if (!plain) {
-                p0 = ((vv >> c) & 1u) ? p0 : 0.f;
-                p1 = ((vv >> (c + 1)) & 1u) ? p1 : 0.f;
+              for (int e = 0; e < 16; ++e) {
+                const int c = 2 * e;
+                float x0, x1;
+                unpack_f2(fma_f2(pack_f2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, neg2), x0, x1);
+                float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+                if (!plain) {
+                  p0 = ((vv >> c) & 1u) ? p0 : 0.f;
+                  p1 = ((vv >> (c + 1)) & 1u) ? p1 : 0.f;
+                }
+                lacc = add_f2(lacc, pack_f2(p0, p1));
+                const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+                pk[hh][e] = *reinterpret_cast<const uint32_t*>(&pb);
               }
-              lacc = add_f2(lacc, pack_f2(p0, p1));
-              const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
-              pk[e] = *reinterpret_cast<const uint32_t*>(&pb);
             }
-            tmem_st16(tp + hh * 16, pk);
           }
           float l0, l1;
           unpack_f2(lacc, l0, l1);
-          const float lt = l0 + l1;  // every P of the row is at most this
-          if (__any_sync(0xffffffffu, lt >= 1.15e18f) &&  // 2^60: rare. Move the reference of the rows concerned
-              mbar_wait(&bar_freev[(it - 1) % kStagesV], ((it - 1) / kStagesV) & 1)) {  // (O must be at rest)
-            tc_fence_after();
-            tmem_wait_st();
-            float alpha = 1.f;
-            if (lt >= 1.15e18f && lt < INFINITY) {
-              int e2;
-              frexpf(lt, &e2);
-              alpha = ldexpf(1.f, 1 - e2);  // 2^-floor(log2 of the row sum)
-            }
+          // A score far above the reference (a P beyond 2^60, or past the range of the exponential: the sum is
+          // then inf) is rare. Nothing of this tile has been written yet, so its scores are intact in tensor
+          // memory: the rows concerned move their reference up by a whole number of powers of two (what is
+          // already accumulated - O and the running sum - is scaled by 2^-k, which is exact) and the tile is
+          // evaluated again.
+          const bool far = !(l0 + l1 < 1.15e18f);
+          if (__any_sync(0xffffffffu, far)) {
+            ok = mbar_wait(&bar_freev[(it - 1) % kStagesV], ((it - 1) / kStagesV) & 1);  // O must be at rest
+            if (ok) {
+              tc_fence_after();
+              float alpha = 1.f, mxt = -INFINITY;
 #pragma unroll 1
-            for (int hh = 0; hh < 2; ++hh) {
-              uint32_t pk[16];
-              tmem_ld16(tp + hh * 16, pk);
-              tmem_wait_ld();
+              for (int hh = 0; hh < 2; ++hh) {
+                uint32_t sr[32];
+                tmem_ld32(tp + hh * 32, sr);
+                tmem_wait_ld();
+                const uint32_t vv = hh ? v1 : v0;
 #pragma unroll
-              for (int e = 0; e < 16; ++e) {
-                const float lo = __uint_as_float(pk[e] << 16) * alpha, hi = __uint_as_float(pk[e] & 0xffff0000u) * alpha;
-                const __nv_bfloat162 pb = __floats2bfloat162_rn(lo, hi);
-                pk[e] = *reinterpret_cast<const uint32_t*>(&pb);
+                for (int c = 0; c < 32; ++c)
+                  mxt = fmaxf(mxt, (plain || ((vv >> c) & 1u)) ? __uint_as_float(sr[c]) : -INFINITY);
               }
-              tmem_st16(tp + hh * 16, pk);
-            }
+              if (far && mxt > -INFINITY && mxt < INFINITY) {
+                float kf = ceilf(fmaf(mxt, sc, neg_ms));  // the tile's largest exponent, rounded up
+                kf = kf < 0.f ? 0.f : (kf > 1.0e9f ? 1.0e9f : kf);
+                alpha = ldexpf(1.f, -(int)kf);  // 0 beyond the range: what came before no longer counts
+                neg_ms -= kf;
+                m_used += kf / sc;
+              }
 #pragma unroll 1
-            for (int hh = 0; hh < 4; ++hh) {  // O and the running sum follow (P V of tile it-1 is over)
-              uint32_t orr[32];
-              const uint32_t ta = tmem_o + lane_sel + hh * 32;
-              tmem_ld32(ta, orr);
-              tmem_wait_ld();
+              for (int q4 = 0; q4 < 4; ++q4) {  // O and the running sum follow (P V of tile it-1 is over)
+                uint32_t orr[32];
+                const uint32_t ta = tmem_o + lane_sel + q4 * 32;
+                tmem_ld32(ta, orr);
+                tmem_wait_ld();
 #pragma unroll
-              for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
-              tmem_st32(ta, orr);
+                for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
+                tmem_st32(ta, orr);
+              }
+              l_run *= alpha;
+              l0 = l1 = 0.f;
+#pragma unroll
+              for (int hh = 0; hh < 2; ++hh) {  // the tile again (rows that did not move get the same values)
+                uint32_t sr[32];
+                tmem_ld32(tp + hh * 32, sr);
+                tmem_wait_ld();
+                const uint32_t vv = hh ? v1 : v0;
+#pragma unroll
+                for (int e = 0; e < 16; ++e) {
+                  const int c = 2 * e;
+                  float p0 = fast_exp2(fmaf(__uint_as_float(sr[c]), sc, neg_ms));
+                  float p1 = fast_exp2(fmaf(__uint_as_float(sr[c + 1]), sc, neg_ms));
+                  if (!plain) {
+                    p0 = ((vv >> c) & 1u) ? p0 : 0.f;
+                    p1 = ((vv >> (c + 1)) & 1u) ? p1 : 0.f;
+                  }
+                  l0 += p0;
+                  l1 += p1;
+                  const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+                  pk[hh][e] = *reinterpret_cast<const uint32_t*>(&pb);
+                }
+              }
             }
-            l0 *= alpha;
-            l1 *= alpha;
-            l_run *= alpha;
-            if (alpha < 1.f) m_used -= log2f(alpha) / sc;
           }
+          tmem_st16(tp, pk[0]);
+          tmem_st16(tp + 16, pk[1]);
           tmem_wait_st();
           l_run += l0 + l1;
           done = true;
@@ -998,7 +992,6 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
       }
       if (warp_live && !done) {
         if (ok) ok = mbar_wait(&bar_s[buf], (it >> 1) & 1);
-        TC_STAMP(0, it, 1);
         if (ok) {
           tc_fence_after();
           if (pos0 + kBN > L) {  // the tile reaches past the prefix: ancestor mask
@@ -1024,9 +1017,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
             }
             mx = fmaxf(mx, fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)));
           }
-          TC_STAMP(0, it, 2);
         }
-        TC_STAMP(0, it, 3);
       }
       // The two-pass path may rescale O, which P V of tile it-1 must have left. A warp without live rows
       // only has to stay in step: it waits for this tile's scores like the others, so that it cannot
@@ -1035,7 +1026,6 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
         ok = warp_live ? mbar_wait(&bar_freev[(it - 1) % kStagesV], ((it - 1) / kStagesV) & 1)
                        : mbar_wait(&bar_s[buf], (it >> 1) & 1);
       }
-      TC_STAMP(0, it, 5);
       if (warp_live && !done) {
         if (ok) {
           // lazy maximum: move the reference only when the row maximum outgrows it by 2^8
@@ -1060,7 +1050,6 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
             }
             tmem_wait_st();
           }
-          TC_STAMP(0, it, 6);
           // pass 2: P = 2^((s - m) * scale) as bf16 over the scores in tensor memory; row sum in fp32
           const bool live = m_used > -INFINITY;
           const float neg_ms = live ? -m_used * sc : 0.f;
@@ -1101,18 +1090,14 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
           }
         }
       }
-      TC_STAMP(0, it, 7);
       fence_proxy_async();
       tc_fence_before();
       mbar_arrive(&bar_p[it & 1]);
-      TC_STAMP(0, it, 9);
     }
     // epilogue: wait for the last P V, then stage O (fp32, unnormalised) and (max, sum) per row in
     // shared memory (the K/V rings, P and Q are idle now): the output rows are written, or merged
     // across the splits, from there in contiguous pieces
-    TC_MARK(4);
     if (ok && ntile > 0) ok = mbar_wait(&bar_freev[(ntile - 1) % kStagesV], ((ntile - 1) / kStagesV) & 1);
-    TC_MARK(5);
     if (!ok) {  // a wait ran out: this split contributes nothing
       m_used = -INFINITY;
       l_run = 0.f;
@@ -1157,7 +1142,6 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     stage_ml[r * 2] = m_used * sc * 0.69314718055994531f;  // natural-log units (-inf: nothing visible)
     stage_ml[r * 2 + 1] = l_run;
   }
-  TC_MARK(6);
   tc_fence_before();
   __syncthreads();
   if (warp == 0) {  // every TMEM access of this CTA is over
@@ -1165,7 +1149,6 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols));
   }
   if (cs > 1) cluster_sync_all();  // every CTA of the cluster has staged its rows
-  TC_CTA_LOG(3, gtimer());
   const int rows_here = rows_total - row0 < kBM ? rows_total - row0 : kBM;
   if (nsplit == 1) {
     for (int rr = warp; rr < rows_here; rr += kThreadsTC / 32) {
@@ -1215,8 +1198,6 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     else if (nsplit <= 4) merge_rows<4, 4>(p, so_s, sml_s, rank0, b, kvh, grow0, rows_here, nsplit, split);
     else merge_rows<2, kMaxSplit>(p, so_s, sml_s, rank0, b, kvh, grow0, rows_here, nsplit, split);
   }
-  TC_MARK(7);
-  TC_CTA_LOG(1, gtimer());
   if (cs > 1) cluster_sync_all();  // nobody leaves while a peer may still read its shared memory
 }
 
@@ -1257,21 +1238,21 @@ bool make_kv_map(CUtensorMap* map, const void* base, int B, int Hkv, int page_si
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-}  // namespace
+// What the host decides for one launch shape: the launch mode, the grid and the workspace it needs.
+struct TcPlan {
+  int nrb, splits, rpc, cs, nsplit_max;
+  bool cluster_mode;
+  long long grid;
+  size_t ws_bytes, rows;  // global-merge mode: workspace size and partial rows (0: none)
+};
+constexpr size_t kTicketBytes = (size_t)CAST_MAX_BATCH * 256 * sizeof(int32_t);
 
+bool tc_shape_ok(int D, int page_size) {
+  if (D != kHD) return false;
+  return page_size == 0 || (page_size >= 8 && page_size <= kBN && (kBN % page_size) == 0 && (page_size % 8) == 0);
+}
 
-bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const void* v, int B, int Hq, int Hkv, int D,
-                              int page_size, const int32_t* page_table, int seq_capacity, int num_pages,
-                              const int32_t* kv_len, const uint32_t* anc, const int32_t* n_tree, const int32_t* first_row,
-                              float scale, void* out, cudaStream_t stream, cast_status* status) {
-  if (D != kHD || !(scale > 0.f)) return false;
-  if (page_size != 0 && (page_size < 8 || page_size > kBN || (kBN % page_size) != 0 || (page_size % 8) != 0))
-    return false;
-  if ((((uintptr_t)k | (uintptr_t)v) & 127) != 0) return false;
-  CUtensorMap map_k, map_v;
-  if (!make_kv_map(&map_k, k, B, Hkv, page_size, seq_capacity, num_pages) ||
-      !make_kv_map(&map_v, v, B, Hkv, page_size, seq_capacity, num_pages))
-    return false;
+bool tc_plan(const cast_ctx* c, int B, int Hq, int Hkv, int page_size, int seq_capacity, TcPlan* pl) {
   const int G = Hq / Hkv, Ncap = c->cfg.max_tree;
   // no tree of this context has more than total_token nodes: row blocks past that are never launched
   const int Nmax = c->cfg.total_token < Ncap ? c->cfg.total_token : Ncap;
@@ -1287,19 +1268,72 @@ bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const v
   while (splits < kMaxSplit && (long long)B * Hkv * nrb * splits * 2 <= slots && max_tiles / (splits * 2) >= 2) splits *= 2;
   int rpc = 1;
   while (rpc * 2 * splits <= kMaxSplit && rpc * 2 <= nrb) rpc *= 2;
-#ifdef CAST_PHASE_CLOCKS
-  if (const char* e = getenv("CAST_TC_SPLITS")) splits = atoi(e);
-  if (const char* e = getenv("CAST_TC_RPC")) rpc = atoi(e);
-#endif
   // Clusters pay when CTAs are short (the merge through distributed shared memory is cheap and the
   // splits are what fills the machine). With long CTAs, or so many sequences that nothing needs
   // splitting on average, an even load matters more: no clusters, pieces sized on the device.
   // (with B * Hkv items or more than the machine has slots, nothing is ever split: plain launch, cs = 1)
-  bool cluster_mode = (splits > 1 && max_tiles / splits <= 64) || (long long)B * Hkv >= slots;
+  const bool cluster_mode = (splits > 1 && max_tiles / splits <= 64) || (long long)B * Hkv >= slots;
   if ((long long)B * Hkv >= slots) splits = rpc = 1;
-#ifdef CAST_PHASE_CLOCKS
-  if (const char* e = getenv("CAST_TC_FORCE_CLUSTER")) cluster_mode = atoi(e) != 0;
-#endif
+  pl->nrb = nrb; pl->splits = splits; pl->rpc = rpc; pl->cluster_mode = cluster_mode;
+  pl->ws_bytes = 0; pl->rows = 0;
+  if (cluster_mode) {
+    pl->cs = splits * rpc;
+    const int groups = (nrb + rpc - 1) / rpc;
+    pl->grid = (long long)B * Hkv * groups * pl->cs;
+    pl->nsplit_max = 1;
+  } else {
+    pl->cs = 1;
+    int nsplit_max = kMaxSplit < max_tiles ? kMaxSplit : max_tiles;
+    if (nsplit_max < 1) nsplit_max = 1;
+    const long long waves = ((long long)B * Hkv * nrb + slots - 1) / slots;
+    pl->grid = (long long)slots * (waves < 1 ? 1 : waves);
+    pl->nsplit_max = nsplit_max;
+    if (nsplit_max > 1) {
+      // workspace: a fixed ticket region (B * Hkv * nrb <= 64 * Hq entries), then the partials
+      if ((size_t)B * Hkv * nrb * sizeof(int32_t) > kTicketBytes) return false;
+      pl->rows = (size_t)B * Hq * Ncap * nsplit_max;
+      pl->ws_bytes = kTicketBytes + pl->rows * (kHD * sizeof(__half) + 2 * sizeof(float));
+    }
+  }
+  return pl->grid <= 0x7fffffffll;
+}
+
+}  // namespace
+
+// Workspace bytes a tensor-core launch of this shape needs (0: none, or the shape is not the tensor path's).
+size_t tree_attention_tc_workspace(const cast_ctx* c, int B, int Hq, int Hkv, int D, int page_size, int seq_capacity) {
+  TcPlan pl;
+  if (!tc_shape_ok(D, page_size) || !tc_plan(c, B, Hq, Hkv, page_size, seq_capacity, &pl)) return 0;
+  return pl.ws_bytes;
+}
+// Grows the tensor path's workspace to `bytes` (set-up time only: synchronises and allocates).
+cast_status tree_attention_tc_reserve(cast_ctx* c, size_t bytes) {
+  if (bytes <= c->attn_tc_ws_bytes) return CAST_OK;
+  CAST_CUDA_OK(cudaDeviceSynchronize());
+  if (c->attn_tc_ws) cudaFree(c->attn_tc_ws);
+  c->attn_tc_ws = nullptr;
+  c->attn_tc_ws_bytes = 0;
+  CAST_CUDA_OK(cudaMalloc(&c->attn_tc_ws, bytes));
+  // tickets start at zero; every merge leaves its ticket at zero again
+  CAST_CUDA_OK(cudaMemset(c->attn_tc_ws, 0, kTicketBytes));
+  c->attn_tc_ws_bytes = bytes;
+  return CAST_OK;
+}
+
+bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const void* v, int B, int Hq, int Hkv, int D,
+                              int page_size, const int32_t* page_table, int seq_capacity, int num_pages,
+                              const int32_t* kv_len, const uint32_t* anc, const int32_t* n_tree, const int32_t* first_row,
+                              float scale, void* out, cudaStream_t stream, cast_status* status) {
+  if (!tc_shape_ok(D, page_size) || !(scale > 0.f)) return false;
+  if ((((uintptr_t)k | (uintptr_t)v) & 127) != 0) return false;
+  TcPlan pl;
+  if (!tc_plan(c, B, Hq, Hkv, page_size, seq_capacity, &pl)) return false;
+  CUtensorMap map_k, map_v;
+  if (!make_kv_map(&map_k, k, B, Hkv, page_size, seq_capacity, num_pages) ||
+      !make_kv_map(&map_v, v, B, Hkv, page_size, seq_capacity, num_pages))
+    return false;
+  const int G = Hq / Hkv, Ncap = c->cfg.max_tree;
+  const int Nmax = c->cfg.total_token < Ncap ? c->cfg.total_token : Ncap;
   TcParams p;
   p.q = (const __nv_bfloat16*)q; p.out = (__nv_bfloat16*)out;
   p.B = B; p.Ncap = Ncap; p.Nmax = Nmax; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.page_size = page_size;
@@ -1307,45 +1341,23 @@ bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const v
   p.page_table = page_table; p.kv_len = kv_len; p.n_tree = n_tree; p.first_row = first_row; p.anc = anc;
   p.scale_log2 = scale * 1.4426950408889634f;
   p.st = c->state;
-  p.num_sms = c->num_sms; p.nrb = nrb;
+  p.num_sms = c->num_sms; p.nrb = pl.nrb;
   p.part_o = nullptr; p.part_ml = nullptr; p.ticket = nullptr;
   *status = CAST_OK;
-  long long grid;
-  int cs;
-  if (cluster_mode) {
-    cs = splits * rpc;
-    const int groups = (nrb + rpc - 1) / rpc;
-    grid = (long long)B * Hkv * groups * cs;
-    p.cs = cs; p.rpc = rpc; p.nsplit_max = 1;
-  } else {
-    cs = 1;
-    int nsplit_max = kMaxSplit < max_tiles ? kMaxSplit : max_tiles;
-    if (nsplit_max < 1) nsplit_max = 1;
-    const long long waves = ((long long)B * Hkv * nrb + slots - 1) / slots;
-    grid = (long long)slots * (waves < 1 ? 1 : waves);
-    p.cs = 0; p.rpc = 1; p.nsplit_max = nsplit_max;
-    if (nsplit_max > 1) {
-      // workspace: a fixed ticket region (B * Hkv * nrb <= 64 * Hq entries), then the partials
-      constexpr size_t kTicketBytes = (size_t)CAST_MAX_BATCH * 256 * sizeof(int32_t);
-      const size_t rows = (size_t)B * Hq * Ncap * nsplit_max;
-      if ((size_t)B * Hkv * nrb * sizeof(int32_t) > kTicketBytes) return false;
-      const size_t need = kTicketBytes + rows * (kHD * sizeof(__half) + 2 * sizeof(float));
-      if (need > c->attn_tc_ws_bytes) {  // grows the workspace (synchronises; not legal during graph capture)
-        if (cudaDeviceSynchronize() != cudaSuccess) { *status = CAST_ERR_CUDA; return true; }
-        if (c->attn_tc_ws) cudaFree(c->attn_tc_ws);
-        c->attn_tc_ws = nullptr;
-        c->attn_tc_ws_bytes = 0;
-        if (cudaMalloc(&c->attn_tc_ws, need) != cudaSuccess) { *status = CAST_ERR_CUDA; return true; }
-        // tickets start at zero; every merge leaves its ticket at zero again
-        if (cudaMemset(c->attn_tc_ws, 0, kTicketBytes) != cudaSuccess) { *status = CAST_ERR_CUDA; return true; }
-        c->attn_tc_ws_bytes = need;
-      }
-      p.ticket = reinterpret_cast<int32_t*>(c->attn_tc_ws);
-      p.part_o = reinterpret_cast<__half*>(reinterpret_cast<char*>(c->attn_tc_ws) + kTicketBytes);
-      p.part_ml = reinterpret_cast<float*>(p.part_o + rows * kHD);
+  const long long grid = pl.grid;
+  const int cs = pl.cs;
+  p.rpc = pl.rpc; p.nsplit_max = pl.nsplit_max;
+  p.cs = pl.cluster_mode ? cs : 0;
+  if (pl.ws_bytes > 0) {
+    // compute calls never allocate: the workspace comes from cast_reserve_attention
+    if (pl.ws_bytes > c->attn_tc_ws_bytes) {
+      *status = CAST_ERR_CAPACITY;
+      return true;
     }
+    p.ticket = reinterpret_cast<int32_t*>(c->attn_tc_ws);
+    p.part_o = reinterpret_cast<__half*>(reinterpret_cast<char*>(c->attn_tc_ws) + kTicketBytes);
+    p.part_ml = reinterpret_cast<float*>(p.part_o + pl.rows * kHD);
   }
-  if (grid > 0x7fffffffll) return false;
   static bool attr_done = false;
   if (!attr_done) {
     if (cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) !=

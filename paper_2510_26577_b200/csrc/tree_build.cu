@@ -21,23 +21,6 @@
 
 using namespace cast;
 
-// Development aid, compiled only with -DCAST_PHASE_CLOCKS: thread 0 of the CTA that ends up running
-// the layer tail / the rerank records clock64() at phase boundaries.
-#ifdef CAST_PHASE_CLOCKS
-__device__ long long g_phase_clock[64];
-#define CAST_STAMP(k) do { if (threadIdx.x == 0) stamp_s[k] = clock64(); } while (0)
-#define CAST_STAMP_DECL
-__shared__ long long stamp_s[32];
-#define CAST_STAMP_FLUSH(off, n) do { if (threadIdx.x == 0) for (int _i = 0; _i < (n); ++_i) g_phase_clock[(off) + _i] = stamp_s[_i]; } while (0)
-extern "C" __attribute__((visibility("default"))) int cast_debug_read_clocks(long long* out) {
-  return (int)cudaMemcpyFromSymbol(out, g_phase_clock, sizeof(long long) * 64);
-}
-#else
-#define CAST_STAMP(k) do {} while (0)
-#define CAST_STAMP_DECL
-#define CAST_STAMP_FLUSH(off, n) do {} while (0)
-#endif
-
 namespace {
 
 // ------------------------------------------------------------------ step begin
@@ -438,8 +421,6 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
   __shared__ unsigned long long row_keys[kSweepMaxChunks * CAST_MAX_TOP_K];
   __shared__ float row_max[kSweepMaxChunks];
   __shared__ double row_sum[kSweepMaxChunks];
-  CAST_STAMP_DECL
-  CAST_STAMP(0);
   unsigned long long* cand = reinterpret_cast<unsigned long long*>(scratch);
 
   const int chunk = blockIdx.x, r = blockIdx.y, b = blockIdx.z, B = gridDim.z;
@@ -507,7 +488,6 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
   unsigned long long* wlist = cand + warp * kWarpCap;
   int have = 0;
   unsigned long long thr_key = 0ull;
-  CAST_STAMP(1);
 
   for (int sub = begin; sub < end; sub += kSweepSub) {
     if (sub != begin) load_pass(sub);
@@ -620,7 +600,6 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
     }
     thr_key = have == K ? wlist[K - 1] : 0ull;
   }
-  CAST_STAMP(2);
 
   // chunk result: the top K of the warps' lists (each in descending order; the rank of a key is the
   // number of larger keys, list by list: a lower-bound search each, two lanes per key slot), the
@@ -709,7 +688,6 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
       }
     }
   }
-  CAST_STAMP(3);
 
   // ---- row merge by the first CTA of the row's cluster
   if (p.nchunks > 1) {
@@ -719,7 +697,6 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
   } else {
     __syncthreads();
   }
-  CAST_STAMP(4);
   // the row's top K out of the chunks' lists (each in descending order): the rank of a key is its
   // position in its own list plus, for every other list, the number of larger keys there (a binary
   // search each; in its own list it finds its own position). Neighbouring lanes share a key slot.
@@ -792,28 +769,23 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
       p.pool_kept[o + idx] = 0;
     }
   }
-  CAST_STAMP(5);
 
   // ---- layer tail
   __syncthreads();
   const int n_tail = tail_width(p, n_prev);
   if (B <= kTailSingleMaxB) {  // the last CTA of the layer ranks and decides, everything in shared memory
     if (!take_ticket(p.layer_ticket, B * n_prev, &s_flag)) return;
-    CAST_STAMP(6);
     double* vs = reinterpret_cast<double*>(scratch + 16384);  // [B][CAST_MAX_WIDTH] sorted values
     int* stok = reinterpret_cast<int*>(scratch + 24576);      // [B][CAST_MAX_WIDTH] tokens of the sorted nodes
     tail_rank(p, 0, B, n_tail, n_prev, base, scratch, sorted, stok, vs);
     tail_decide<false>(p, ts, B, n_tail, n_prev, base, sorted, stok, vs);
   } else {  // the last CTA of every sequence ranks that sequence; the last of those decides for the batch
     if (!take_ticket(p.seq_ticket + b, n_prev, &s_flag)) return;
-    CAST_STAMP(6);
     tail_rank(p, b, 1, n_tail, n_prev, base, scratch, p.tail_sorted, p.tail_tok, p.tail_vs);
     // (tail_rank ends with a CTA barrier: the ticket below releases what all threads wrote)
     if (!take_ticket(p.layer_ticket, B, &s_flag)) return;
     tail_decide<true>(p, ts, B, n_tail, n_prev, base, p.tail_sorted, p.tail_tok, p.tail_vs);
   }
-  CAST_STAMP(7);
-  CAST_STAMP_FLUSH(0, 8);
 }
 
 // ------------------------------------------------------------------ rerank + linearise
@@ -1052,15 +1024,10 @@ __global__ void __launch_bounds__(512) select_finalize_kernel(const SelectParams
 }
 __global__ void __launch_bounds__(512) select_fused_kernel(const SelectParams p) {  // batch 1: one launch
   extern __shared__ __align__(16) unsigned char smem[];
-  CAST_STAMP_DECL
-  CAST_STAMP(0);
   grid_dependency_wait();
   select_rank_phase(p, 0, smem);
   __syncthreads();
-  CAST_STAMP(1);
   select_finalize_phase(p, 0, 1);
-  CAST_STAMP(2);
-  CAST_STAMP_FLUSH(32, 3);
 }
 
 }  // namespace

@@ -107,6 +107,8 @@ def assert_tree_equal(g, o, score_tol=5e-6):
 def gpu_attention(ctx, w, q, k, v, table, num_pages, kv_len, anc, n_tree, scale=0.0, first_row=None):
     out = torch.full_like(q, float("nan"))
     anc_t = anc if torch.is_tensor(anc) else torch.from_numpy(anc.view(np.int32)).cuda()
+    ctx.cast_reserve_attention(q.dtype, q.shape[0], w.q_heads, w.kv_heads, w.head_dim, w.page_size,
+                               wl.seq_capacity(w) // (w.page_size or 1))
     if first_row is None:
         ctx.cast_tree_attention(q, k, v, q.shape[0], w.q_heads, w.kv_heads, w.head_dim, w.page_size, table,
                                 wl.seq_capacity(w) // (w.page_size or 1), num_pages, kv_len, anc_t, n_tree, scale, out)

@@ -53,7 +53,10 @@ def build_tree_both(binding, w, peaked=False, stepped=False, steps=1, skewed=Fal
     return ctx, g, o, root, kv
 
 
-def check_attention(binding, ctx, w, g, o, kv, layer=0, sample=None):
+def check_attention(binding, ctx, w, g, o, kv, layer=0, sample=None, dense=()):
+    """sample: that many random (sequence, token, head) outputs; dense: (sequence, kv-head) pairs of which
+    EVERY output is compared - all tree tokens times all heads of the group, i.e. every row of every 128-row
+    block of that pair (the full ones and the ragged last one), every tile and every KV split it has."""
     q = wl.query(w, layer, "cpu").cuda()
     k, v = (t.cuda() for t in wl.kv_cache(w, layer, "cpu"))
     table, num_pages = wl.page_table(w, "cuda")
@@ -70,6 +73,9 @@ def check_attention(binding, ctx, w, g, o, kv, layer=0, sample=None):
             only.add((b, int(rng.integers(0, o["n_tree"][b])), int(rng.integers(0, w.q_heads))))
         for b in range(B):  # always include the last tree token (deepest mask) of head 0
             only.add((b, int(o["n_tree"][b]) - 1, 0))
+        G = w.q_heads // w.kv_heads
+        for b, kvh in dense:
+            only |= {(b, t, h) for t in range(int(o["n_tree"][b])) for h in range(kvh * G, (kvh + 1) * G)}
     ref = tree_attention(f32(q), f32(k), f32(v), w.page_size, tab, kv.cpu().numpy(), o["anc"], o["n_tree"], None, only)
     got = to_f64(out)
     tol = attention_tolerance(w.kv_dtype)
@@ -83,6 +89,7 @@ def check_attention(binding, ctx, w, g, o, kv, layer=0, sample=None):
         err = max(np.max(np.abs(got[b, t, h] - ref[b, t, h])) for (b, t, h) in only)
         for b in range(B):  # rows beyond the tree are left untouched (the helper pre-fills NaN)
             assert np.isnan(got[b, int(o["n_tree"][b]):]).all()
+    print(f"{w.name}: attention max-abs error {err:.3e} over {'all' if only is None else len(only)} outputs")
     assert err <= tol, f"attention max-abs error {err:.3e} > {tol}"
     return err
 
@@ -148,7 +155,12 @@ def test_c3_batch_sweep_cost_model(binding, name):
     w = wl.CONFIGS[name]
     ctx, g, o, root, kv = build_tree_both(binding, w)
     assert 1 <= int(o["n_tree"][0]) <= 64
-    check_attention(binding, ctx, w, g, o, kv, sample=24)
+    # every output of the longest, the shortest and one more sequence for two kv-heads each (global-merge
+    # launch at batch 16: all splits and the merge of those pairs), and of every (sequence, kv-head) pair below
+    lens = kv.cpu().numpy()
+    seqs = sorted({int(np.argmax(lens)), int(np.argmin(lens)), w.batch // 2})
+    dense = [(b, h) for b in seqs for h in (0, w.kv_heads - 1)] if w.batch > 1 else [(0, h) for h in range(w.kv_heads)]
+    check_attention(binding, ctx, w, g, o, kv, sample=24, dense=dense)
     check_accept_and_compact(binding, ctx, w, g, o, kv)
     if name == "c3_llama8b_b16":  # more sequences than clusters fit at a time
         _run_stochastic(binding, ctx, w, o["tokens"], o["parent"], o["n_tree"], w.depth, 1.0, 0.7)
@@ -189,12 +201,14 @@ def test_c3_b64_full_vocab_tree_accept_compaction(binding):
     check_accept_and_compact(binding, ctx, w, g, o, kv)
 
 
-@pytest.mark.parametrize("name", ["c4_llama70b_n16", "c4_llama70b_n128"])
+@pytest.mark.parametrize("name", ["c4_llama70b_n16", "c4_llama70b_n32", "c4_llama70b_n128"])
 def test_c4_llama70b(binding, name):
     w = wl.CONFIGS[name]
     ctx, g, o, root, kv = build_tree_both(binding, w)
     assert list(o["n_tree"]) == [w.total_token] * 8
-    check_attention(binding, ctx, w, g, o, kv, sample=16)
+    # every output of two (sequence, kv-head) pairs: with 128 tokens x 8 heads that is eight full 128-row
+    # blocks each, the tree spanning two 64-position tiles, and every KV split of the global-merge launch
+    check_attention(binding, ctx, w, g, o, kv, sample=16, dense=[(0, 0), (5, 7)])
     check_accept_and_compact(binding, ctx, w, g, o, kv)
     _run_stochastic(binding, ctx, w, o["tokens"], o["parent"], o["n_tree"], w.depth, 1.0, 0.7)
 
@@ -203,7 +217,9 @@ def test_c5_qwen_long_context(binding):
     w = wl.CONFIGS["c5_qwen_long"]
     ctx, g, o, root, kv = build_tree_both(binding, w)
     assert list(o["n_tree"]) == [96] * 4
-    check_attention(binding, ctx, w, g, o, kv, sample=8)
+    # every output of one (sequence, kv-head) pair: 96 tokens x 7 heads = five full 128-row blocks and a
+    # ragged one of 32 rows, 515 tiles in 8 splits each
+    check_attention(binding, ctx, w, g, o, kv, sample=8, dense=[(1, 2)])
     check_accept_and_compact(binding, ctx, w, g, o, kv)
     _run_stochastic(binding, ctx, w, o["tokens"], o["parent"], o["n_tree"], w.depth, 0.9, 0.5)  # the largest cached slice
 
@@ -510,14 +526,77 @@ def test_attention_full_size_launch_sampled(binding, name, n):
     assert ctx.cast_poll_status()[0] == 0
     only = {(int(b), int(rng.integers(0, n)), int(rng.integers(0, w.q_heads))) for b in rng.integers(0, B, size=24)}
     only |= {(b, n - 1, w.q_heads - 1) for b in (0, B - 1)}
+    # and every output (all tokens, all heads of the group) of the longest, the shortest and one more sequence
+    # for the first and the last kv-head: every row block, tile and split of those pairs
+    lens, G = kv.cpu().numpy(), w.q_heads // w.kv_heads
+    for b in sorted({int(np.argmax(lens)), int(np.argmin(lens)), B // 2}):
+        for kvh in (0, w.kv_heads - 1):
+            only |= {(b, t, h) for t in range(n) for h in range(kvh * G, (kvh + 1) * G)}
     f32 = lambda t: t.float().cpu().numpy()
     tab = table.cpu().numpy() if table is not None else None
     ref = tree_attention(f32(q), f32(k), f32(v), w.page_size, tab, kv.cpu().numpy(), anc, n_tree, None, only)
     got = to_f64(out)
     err = max(np.max(np.abs(got[i] - ref[i])) for i in only)
+    print(f"{name}: attention max-abs error {err:.3e} over {len(only)} outputs")
     assert err <= attention_tolerance(w.kv_dtype), err
     for b in (0, B - 1):
         assert np.isnan(got[b, n:]).all()
+
+
+@pytest.mark.parametrize("name,factor", [("c2_llama8b", 12.0), ("c4_llama70b_n128", 12.0), ("c3_llama8b_b64", 12.0),
+                                         ("c2_llama8b", 60.0)])
+def test_attention_score_far_above_the_earlier_tiles(binding, name, factor):
+    """A key far better than anything before it, met late: in the last prefix tile, in a tree tile and in
+    the middle of the prefix (the scores of the tiles before it are ordinary, so the running reference of
+    the single-pass softmax is ~100 to ~700 nats too low when the key arrives). Cluster, global-merge and
+    plain launches; compared with the oracle on the planted rows and on their neighbours."""
+    rng = np.random.default_rng(11)
+    w = wl.CONFIGS[name]
+    B, Ncap, Hq, G = w.batch, w.max_tree, w.q_heads, w.q_heads // w.kv_heads
+    n = min(w.total_token, 16) if name.startswith("c3") else w.total_token
+    ctx = binding.CastContext(max_batch=B, **cfg_kwargs(w, enable_bp=0, enable_dr=0))
+    kv = wl.kv_lengths(w, "cpu").cuda()
+    kvh_ = kv.cpu().numpy()
+    n_tree = np.full(B, n, dtype=np.int32)
+    anc = np.zeros((B, Ncap, 4), dtype=np.uint32)
+    for b in range(B):
+        anc[b, :n] = ancestor_masks(_random_tree(rng, n, "random"), n, 4)
+    q = wl.query(w, 0, "cpu")
+    k, v = wl.kv_cache(w, 0, "cpu")
+    table, num_pages = wl.page_table(w, "cpu")
+    only = set()
+
+    def plant(b, t, h, pos):
+        row = (q[b, t, h].float() * factor).to(k.dtype)
+        if w.page_size:
+            k[int(table[b, pos // w.page_size]), pos % w.page_size, h // G] = row
+        else:
+            k[b, pos, h // G] = row
+        for tt in {t, max(t - 1, 0), min(t + 1, n - 1)}:
+            for hh in range(h // G * G, h // G * G + G):
+                only.add((b, tt, hh))
+
+    bs = sorted({0, B - 1, B // 2})
+    for i, b in enumerate(bs):
+        L = int(kvh_[b])
+        t = n - 1 - i  # a late tree token: its own tree position is in the last tile
+        plant(b, t, (3 * i) % Hq, L - 1 - 5 * i)          # last prefix tile
+        plant(b, t, (G + 1 + 3 * i) % Hq, L + t)          # its own position in the tree (always visible)
+        plant(b, 1 + i, (2 * G + 2 + i) % Hq, L // 2 + 7)  # middle of the prefix: a later split's first tiles
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    td = table.cuda() if table is not None else None
+    out = gpu_attention(ctx, w, qd, kd, vd, td, num_pages, kv, anc, torch.from_numpy(n_tree).cuda(), scale=0.0)
+    assert ctx.cast_poll_status()[0] == 0
+    f32 = lambda t_: t_.float().numpy()
+    tab = table.numpy() if table is not None else None
+    if len(only) > 400:
+        keep = sorted(only)
+        only = {keep[i] for i in rng.permutation(len(keep))[:400]}
+    ref = tree_attention(f32(q), f32(k), f32(v), w.page_size, tab, kvh_, anc, n_tree, None, only)
+    got = to_f64(out)
+    assert np.isfinite(got[:, :n]).all()
+    err = max(np.max(np.abs(got[i] - ref[i])) for i in only)
+    assert err <= attention_tolerance(w.kv_dtype), err
 
 
 def test_attention_bad_page_sets_status(binding):
@@ -694,3 +773,68 @@ def test_accept_stochastic_special_cases(binding):
             ctx.cast_accept_stochastic(tl, dl, B, bad_T, i32(B, Ncap), i32(B, Ncap), i32(B), ua, ub, i32(B), i32(B, H + 1), i32(B))
     with pytest.raises(binding.CastError):
         ctx.cast_accept_stochastic(tl, dl, B + 1, 1.0, i32(B, Ncap), i32(B, Ncap), i32(B), ua, ub, i32(B), i32(B, H + 1), i32(B))
+
+
+# ------------------------------------------------ cost tables measured on the device (Sec. "Method")
+def test_measured_cost_tables_size_the_same_tree_on_both_sides(binding):
+    """The paper fills S_T(B), S_D(B) by timing the models on the device in use. The profiler here times this
+    library's attention over a small (context, tree size) grid on distinct cache buffers, adds the linear
+    stand-in for the layer's GEMMs and hands the tables to the library and to the oracle: both must size the
+    same tree from them, over two steps, with every sizing switch on."""
+    from oracle import CostTable
+    from paper_2510_26577_b200 import cost_profile
+
+    B, L, M, Ntab = 2, 256, 3, 24
+    w = wl.Workload("prof", 84, B, "bf16", "f32", 8, 2, 128, 40, 600, 16, 3000, 2.0, 5, 4, 20, False, 2, max_tree=32,
+                    seed_salt=1)
+    t, pts = cost_profile.measure_attention_us(w, B, L, M, n_points=(1, 4, 16, 32), reps=4)
+    assert t.shape == (M, 4) and np.isfinite(t).all() and (t > 0).all()
+    # a target of 4 layers, a draft head of 1; a GEMM term that makes every further token cost a visible share
+    fT, fD = cost_profile.tables_from_measurement(t, pts, B, Ntab, n_layers=4, gemm_us=(5.0, 2.0))
+    assert (np.diff(fT, axis=1) > 0).all() and (np.diff(fD, axis=1) > 0).all()
+    over = dict(enable_bp=1, enable_dp=1, enable_dr=1, C1=2.0, C2=0.5, C3=0.25)
+    kw = cfg_kwargs(w, **over)
+    tables = {B: CostTable(B, L, M, Ntab, fT, fD)}
+    ctx = binding.CastContext(max_batch=B, **kw)
+    ctx.cast_set_cost_tables(B, L, M, Ntab, fT, fD)
+    root = wl.root_tokens(w, "cpu").cuda()
+    kv = wl.kv_lengths(w, "cpu").cuda()
+    oracle = None
+    narrowed = False
+    for step in range(2):
+        logits = [wl.draft_logits(w, 10 * step + l, "cpu", peaked=True).cuda() for l in range(1, w.depth + 1)]
+        o = oracle_tree(kw, tables, root, kv, logits, oracle)
+        oracle = o["oracle"]
+        g = gpu_tree(ctx, root, kv, logits)
+        if not (o["min_score_gap"] >= 1e-5 and o["stable"]):
+            pytest.skip("a measured table put a decision within rounding of its threshold")
+        assert_tree_equal(g, o)
+        narrowed |= min(o["n_hist"]) < w.top_k or len(o["n_hist"]) < w.depth or int(o["n_tree"].min()) < w.total_token
+    assert narrowed, "the measured tables never narrowed, stopped or trimmed the tree: thresholds out of range"
+
+
+def test_attention_without_a_reserved_workspace_is_refused(binding):
+    """Compute calls never allocate: a shape that needs a split workspace larger than what was reserved
+    returns CAST_ERR_CAPACITY and launches nothing; after cast_reserve_attention the same call runs."""
+    w = wl.shrink(wl.CONFIGS["c1_tiny"])
+    ctx = binding.CastContext(max_batch=1, **cfg_kwargs(w))
+    q = wl.query(w, 0, "cuda")
+    k, v = wl.kv_cache(w, 0, "cuda")
+    kv = wl.kv_lengths(w, "cuda")
+    anc = torch.zeros((1, w.max_tree, ctx.words), dtype=torch.int32, device="cuda")
+    anc[0, 0, 0] = 1
+    nt = torch.ones(1, dtype=torch.int32, device="cuda")
+    out = torch.full_like(q, float("nan"))
+    args = (q, k, v, 1, w.q_heads, w.kv_heads, w.head_dim, 0, None, wl.seq_capacity(w), 0, kv, anc, nt, 0.0, out)
+    with pytest.raises(binding.CastError) as e:
+        ctx.cast_tree_attention(*args)
+    assert e.value.code == 3
+    torch.cuda.synchronize()
+    assert torch.isnan(out).all()
+    free0 = torch.cuda.mem_get_info()[0]
+    ctx.cast_reserve_attention(q.dtype, 1, w.q_heads, w.kv_heads, w.head_dim, 0, wl.seq_capacity(w))
+    free1 = torch.cuda.mem_get_info()[0]
+    ctx.cast_tree_attention(*args)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free1 <= free0  # the compute call moved no device memory
+    assert torch.isfinite(out[0, 0]).all() and ctx.cast_poll_status()[0] == 0

@@ -267,6 +267,7 @@ def test_guard_bands_around_every_output(binding, dtype):
     seq_cap = wl.seq_capacity(w) // w.page_size
     tab = table.cpu().numpy()
     f32 = lambda t: t.float().cpu().numpy()
+    ctx.cast_reserve_attention(q.dtype, B, w.q_heads, w.kv_heads, w.head_dim, w.page_size, seq_cap)
     for first in (None, torch.tensor([3, 0, 20], dtype=torch.int32, device="cuda")):
         out = gd.alloc(tuple(q.shape), q.dtype, fill=float("nan"))
         ctx.cast_tree_attention_rows(q, k, v, B, w.q_heads, w.kv_heads, w.head_dim, w.page_size, table, seq_cap, num_pages, kv,
@@ -373,6 +374,7 @@ def test_malformed_inputs_are_reported_not_followed(binding):
     kv = wl.kv_lengths(w, "cuda")
     anc = torch.zeros((B, Ncap, ctx.words), dtype=torch.int32, device="cuda")
     out = torch.zeros_like(q)
+    ctx.cast_reserve_attention(q.dtype, B, 8, 2, 128, 16, wl.seq_capacity(w) // 16)
     ctx.cast_tree_attention(q, k, v, B, 8, 2, 128, 16, table, wl.seq_capacity(w) // 16, num_pages, kv, anc,
                             dev(np.array([20, 4], dtype=np.int32)), 0.0, out)
     assert ctx.cast_poll_status()[0] == 6
@@ -384,3 +386,15 @@ def test_malformed_inputs_are_reported_not_followed(binding):
                         dev(np.array([2, 0], dtype=np.int32)), kv.clone())
     assert ctx.cast_poll_status()[0] == 7  # BAD_PAGE
     assert ctx.cast_poll_status()[0] == 0
+    # a path that does not climb (entry j below j) next to the end of the sequence's capacity: the sources are
+    # in range, the destinations would not be. Reported, nothing stored, the length left alone.
+    cap = wl.seq_capacity(w)
+    near_end = torch.tensor([cap - 1, cap - 1], dtype=torch.int32, device="cuda")
+    path = np.zeros((B, H + 1), dtype=np.int32)  # 0, 0, 0
+    k0, v0 = kk.clone(), vv.clone()
+    lens = near_end.clone()
+    ctx.cast_compact_kv(kk, vv, B, 1, kk[0].numel() * 2, 2, 128, 16, table, cap // 16, num_pages, dev(path),
+                        dev(np.array([2, 2], dtype=np.int32)), lens)
+    assert ctx.cast_poll_status()[0] == 7
+    assert torch.equal(kk.view(torch.int16), k0.view(torch.int16)) and torch.equal(vv.view(torch.int16), v0.view(torch.int16))
+    assert torch.equal(lens, near_end)

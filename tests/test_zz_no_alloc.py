@@ -4,8 +4,10 @@ Such callers (an engine whose device memory is a fixed arena, a process whose al
 after start-up, a plug-in that receives device pointers but no allocator) cannot create a context,
 because a context allocates.  The static entry point keeps its only scratch in an array inside the
 library image.  This test calls it through the C-ABI twice in a row, on different inputs, and
-requires the same results as the context-based cast_accept: the shared array keeps the first
-call's contents, so the second call also shows that nothing stale is read.
+requires the same results as the context-based cast_accept and as the CPU oracle's greedy
+acceptance: the shared array keeps the first call's contents, so the second call also shows that
+nothing stale is read.  It also reads the device's free memory before and after the static call:
+the call must leave it unchanged.
 
 The file name makes pytest collect it last: if it fails, every other test has already run.
 """
@@ -65,12 +67,25 @@ def test_static_accept_matches_context_accept_twice(dtype):
             bonus = torch.full((B,), -7, dtype=torch.int32, device="cuda")
             if which == 0:
                 ctx.cast_accept(lg, B, tk_d, pr_d, None, None, nt_d, alen, apath, bonus)
+                torch.cuda.synchronize()
             else:
+                if call == 0:  # the very first call looks up the scratch array's address (and loads the kernels)
+                    binding.cast_accept_static(lg, B, Ncap, V, H, tk_d, pr_d, nt_d, alen, apath, bonus)
+                    torch.cuda.synchronize()
+                    alen.fill_(-7); apath.fill_(-7); bonus.fill_(-7)
+                    torch.cuda.synchronize()
+                free_before = torch.cuda.mem_get_info()[0]
                 binding.cast_accept_static(lg, B, Ncap, V, H, tk_d, pr_d, nt_d, alen, apath, bonus)
-            torch.cuda.synchronize()
+                torch.cuda.synchronize()
+                assert torch.cuda.mem_get_info()[0] == free_before  # no device memory was taken or returned
             outs.append((alen.cpu().numpy(), apath.cpu().numpy(), bonus.cpu().numpy()))
         assert ctx.cast_poll_status()[0] == 0
         for ref, got in zip(outs[0], outs[1]):  # integer outputs: bit-exact, as in the other accept tests
+            assert np.array_equal(ref, got)
+        # and both equal the oracle (token-by-token greedy decoding down the tree)
+        from oracle import greedy_accept
+        ol, op, ob = greedy_accept(logits.double().numpy(), tokens, parent, n_tree, H)
+        for ref, got in zip((ol, op, ob), outs[1]):
             assert np.array_equal(ref, got)
         assert outs[0][0].max() >= 1  # the walk did accept something
 
