@@ -75,6 +75,10 @@ struct cast_ctx {
 
   cast::DevState* state;
 
+  // what the step's first expand call reads (set by cast_step_begin)
+  const int32_t* step_root;
+  const int32_t* step_kv_len;
+
   int32_t* layer_ticket;          // [1]
   // batched layer tail: per-sequence tickets and what every sequence hands to the batch-wide part
   int32_t* seq_ticket;            // [max_batch]

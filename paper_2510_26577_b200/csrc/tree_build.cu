@@ -23,53 +23,6 @@ using namespace cast;
 
 namespace {
 
-// ------------------------------------------------------------------ step begin
-__global__ void step_begin_kernel(DevState* st, int B, int P, int W, const int32_t* root_token,
-                                  const int32_t* kv_len, double* pool_score, int32_t* pool_token,
-                                  int32_t* pool_parent, int32_t* pool_depth, uint8_t* pool_kept,
-                                  int32_t* retained, int32_t* lsort, double* lscore, int32_t* layer_ticket,
-                                  int32_t* seq_ticket) {
-  __shared__ int s_max;
-  const int tid = threadIdx.x;
-  if (tid == 0) s_max = 0;
-  __syncthreads();
-  for (int b = tid; b < B; b += blockDim.x) {
-    const size_t o = (size_t)b * P;
-    pool_score[o] = 0.0;  // root: value 1
-    pool_token[o] = root_token[b];
-    pool_parent[o] = -1;
-    pool_depth[o] = 0;
-    pool_kept[o] = 1;
-    lsort[o] = 0;
-    lscore[o] = 0.0;
-    retained[b * W] = 0;
-    seq_ticket[b] = 0;
-    atomicMax(&s_max, kv_len[b]);
-  }
-  __syncthreads();
-  if (tid == 0) {
-    *layer_ticket = 0;
-    st->B = B;
-    st->pool_size = 1;
-    st->ctx_sum = 0;
-    st->n0 = s_max;
-    st->layers_done = 0;
-    st->n_tree = 0;
-    st->kept_total = 1;
-    st->u_last = 1.0;
-    st->n_hist[0] = 1;
-    st->layer_base[0] = 0;
-    st->layer_n[0] = 1;
-    for (int i = 1; i <= CAST_MAX_DEPTH; ++i) {
-      st->n_hist[i] = 0;
-      st->layer_base[i] = 0;
-      st->layer_n[i] = 0;
-    }
-    for (int i = 0; i < CAST_MAX_DEPTH + 2; ++i) st->rows[i] = 0;
-    st->rows[1] = 1;
-  }
-}
-
 // ------------------------------------------------------------------ expand
 struct ExpandParams {
   const void* logits;
@@ -97,6 +50,9 @@ struct ExpandParams {
   int32_t* next_tokens;
   int32_t* next_parent_row;
   int32_t* next_count;
+  // the step's root tokens and prefix lengths (read by layer 1, which also resets the per-step state)
+  const int32_t* root_token;
+  const int32_t* kv_len;
 };
 
 template <typename T> struct Vec;
@@ -291,18 +247,42 @@ template <bool GLOBAL>
 __device__ __forceinline__ void tail_decide(const ExpandParams& p, const TailState& ts, int B, int n, int n_prev, int base,
                                             const int* sorted_i, const int* stok_i, const double* vs_i) {
   __shared__ double vbar[CAST_MAX_WIDTH], u[CAST_MAX_WIDTH], c[CAST_MAX_WIDTH];
-  __shared__ int s_ni, s_next;
+  __shared__ int s_ni, s_next, s_n0;
   const int tid = threadIdx.x, nt = blockDim.x;
   DevState* st = p.st;
   const int K = p.K, W = p.W, P = p.P;
   const int Ni = n_prev * K;
   const bool need_cost = p.enable_bp || p.enable_dp;
   const double u_last = ts.u_last;
+  int n0 = ts.n0;
+  if (p.layer == 1) {
+    // The first layer of a step also starts the step (cast_step_begin launches nothing): the padded context
+    // length n_0 = max_b kv_len[b] and every sequence's root node (value 1, depth 0) at pool index 0.
+    static_assert(CAST_MAX_BATCH <= 64, "two sequences per lane");
+    if (tid < 32) {
+      int m = max(tid < B ? p.kv_len[tid] : 0, tid + 32 < B ? p.kv_len[tid + 32] : 0);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+      if (tid == 0) s_n0 = m;
+    }
+    for (int b = tid; b < B; b += nt) {
+      const size_t o = (size_t)b * P;
+      p.pool_score[o] = 0.0;
+      p.pool_token[o] = p.root_token[b];
+      p.pool_parent[o] = -1;
+      p.pool_depth[o] = 0;
+      p.pool_kept[o] = 1;
+      p.lsort[o] = 0;
+      p.lscore[o] = 0.0;
+    }
+    __syncthreads();
+    n0 = s_n0;
+  }
   // Eq. 1: batch mean of the rank-wise values, then prefix sums; Eq. 2 needs one table row
   if (tid < n) {
     double c_mine = 0.0;
     if (need_cost) {
-      const int ctx = ts.ctx_sum + (p.ctx_base_mode ? ts.n0 : 0);
+      const int ctx = ts.ctx_sum + (p.ctx_base_mode ? n0 : 0);
       const int g = select_grid(ctx, p.tab.L, p.tab.M);
       c_mine = p.tab.fD[(size_t)(g - 1) * p.tab.Ntab + tid] / p.tab.fT[(size_t)(g - 1) * p.tab.Ntab];
     }
@@ -377,6 +357,20 @@ __device__ __forceinline__ void tail_decide(const ExpandParams& p, const TailSta
       }
     }
     s_next = (p.layer < p.H && go) ? n_i : 0;
+    if (p.layer == 1) {  // per-step state (rows[]: a later layer that is never reached must read 0)
+      st->B = B;
+      st->n0 = n0;
+      st->n_tree = 0;
+      st->n_hist[0] = 1;
+      st->layer_base[0] = 0;
+      st->layer_n[0] = 1;
+      for (int i = 2; i <= CAST_MAX_DEPTH; ++i) {
+        st->n_hist[i] = 0;
+        st->layer_base[i] = 0;
+        st->layer_n[i] = 0;
+      }
+      for (int i = 0; i < CAST_MAX_DEPTH + 2; ++i) st->rows[i] = (i == 1) ? 1 : 0;
+    }
     st->rows[p.layer + 1] = s_next;
     st->n_hist[p.layer] = n_i;
     st->layer_base[p.layer] = base;
@@ -461,14 +455,22 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
   grid_dependency_wait();
   grid_launch_dependents();  // the next grid may now take the SMs this one leaves idle
   load_pass(begin);
-  // what the layer tail needs of the state is read now, together with the row count: one round trip
-  const int n_prev = st->rows[p.layer];
+  // what the layer tail needs of the state is read now, together with the row count: one round trip.
+  // (Layer 1 starts the step: one row per sequence, the root at pool index 0 with value 1.)
+  int n_prev = 1, base = 1;
   TailState ts;
-  ts.ctx_sum = st->ctx_sum;
-  ts.n0 = st->n0;
-  ts.kept_total = st->kept_total;
-  ts.u_last = st->u_last;
-  const int base = st->pool_size;
+  ts.ctx_sum = 0;
+  ts.n0 = 0;  // layer 1: the deciding CTA works it out from kv_len
+  ts.kept_total = 1;
+  ts.u_last = 1.0;
+  if (p.layer > 1) {
+    n_prev = st->rows[p.layer];
+    ts.ctx_sum = st->ctx_sum;
+    ts.n0 = st->n0;
+    ts.kept_total = st->kept_total;
+    ts.u_last = st->u_last;
+    base = st->pool_size;
+  }
   if (n_prev == 0) {
     if (chunk == 0 && r == 0 && b == 0 && tid == 0) *p.next_count = 0;
     return;
@@ -476,8 +478,12 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
   if (r >= n_prev) return;
   // the parent of this row's children and its log-value (only the row's last CTA uses them: fetched now,
   // off the critical path)
-  const int parent = p.layer == 1 ? 0 : p.retained[b * p.W + r];
-  const double parent_score = p.pool_score[(size_t)b * p.P + parent];
+  int parent = 0;
+  double parent_score = 0.0;
+  if (p.layer > 1) {
+    parent = p.retained[b * p.W + r];
+    parent_score = p.pool_score[(size_t)b * p.P + parent];
+  }
 
   float M2 = -INFINITY, s_run = 0.f;  // running maximum (log2 units) and sum of 2^(x log2e - M2)
   // Every warp keeps the exact top K of the logits it has seen, as a descending list in shared memory;
@@ -848,6 +854,8 @@ __device__ __noinline__ void select_rank_phase(const SelectParams& p, int b, uns
   }
   __syncthreads();
   const int n_out = min(min(peff, p.m), p.Ncap);
+  int half0 = 1;  // first stride of the searches: positions up to 2 half0 - 1 >= the longest list are reachable
+  while (2 * half0 - 1 < p.m && half0 < CAST_MAX_TREE) half0 <<= 1;
 #pragma unroll 1
   for (int i = tid; i < total; i += nt) {
     int l = 0;
@@ -867,8 +875,8 @@ __device__ __noinline__ void select_rank_phase(const SelectParams& p, int b, uns
         len4[q] = valid ? llen[l2] : 0;
         off4[q] = valid ? loff[l2] : 0;
       }
-#pragma unroll
-      for (int half = CAST_MAX_TREE; half >= 1; half >>= 1) {
+#pragma unroll 1
+      for (int half = half0; half >= 1; half >>= 1) {
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
           const int idx = pos[q] + half - 1;
@@ -1047,11 +1055,12 @@ extern "C" cast_status cast_step_begin(cast_ctx* c, int B, const int32_t* root_t
   }
   c->cur_B = B;
   c->next_layer = 1;
-  step_begin_kernel<<<1, 128, 0, (cudaStream_t)stream>>>(c->state, B, c->P, c->W, root_token, kv_len, c->pool_score,
-                                                         c->pool_token, c->pool_parent, c->pool_depth, c->pool_kept,
-                                                         c->retained, c->lsort, c->lscore, c->layer_ticket,
-                                                         c->seq_ticket);
-  return launch_status();
+  // Nothing is launched here: the first cast_tree_expand of the step reads root_token and kv_len and resets
+  // the per-step state in its own kernel (one launch and one dependent round trip fewer per step).
+  c->step_root = root_token;
+  c->step_kv_len = kv_len;
+  (void)stream;
+  return CAST_OK;
 }
 
 extern "C" cast_status cast_tree_expand(cast_ctx* c, int layer, const void* draft_logits, cast_dtype dtype,
@@ -1103,6 +1112,7 @@ extern "C" cast_status cast_tree_expand(cast_ctx* c, int layer, const void* draf
   p.C1 = c->cfg.C1; p.C2 = c->cfg.C2;
   p.enable_bp = c->cfg.enable_bp; p.enable_dp = c->cfg.enable_dp; p.ctx_base_mode = c->cfg.ctx_base_mode;
   p.next_tokens = next_tokens; p.next_parent_row = next_parent_row; p.next_count = next_count;
+  p.root_token = c->step_root; p.kv_len = c->step_kv_len;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(nchunks, rows_per_seq, B);
   cfg.blockDim = dim3(kSweepThreads, 1, 1);
@@ -1136,7 +1146,7 @@ extern "C" cast_status cast_select_nodes(cast_ctx* c, int32_t* tokens, int32_t* 
                                          uint32_t* anc_mask, int32_t* pool_idx, double* scores, int32_t* n_tree,
                                          void* stream) {
   if (!c || !tokens || !parent || !depth || !anc_mask || !pool_idx || !n_tree) return CAST_ERR_INVALID_ARG;
-  if (c->cur_B < 1) return CAST_ERR_INVALID_ARG;
+  if (c->cur_B < 1 || c->next_layer < 2) return CAST_ERR_INVALID_ARG;  // a step with at least one layer
   SelectParams p;
   p.pool_score = c->pool_score; p.pool_token = c->pool_token; p.pool_parent = c->pool_parent;
   p.pool_depth = c->pool_depth; p.lsort = c->lsort; p.lscore = c->lscore; p.st = c->state;
