@@ -38,6 +38,8 @@ __global__ void __launch_bounds__(kArgThreads) argmax_sweep_kernel(const T* __re
                                                                    unsigned long long* __restrict__ part) {
   __shared__ unsigned long long red[kArgThreads / 32];
   const int chunk = blockIdx.x, t = blockIdx.y, b = blockIdx.z;
+  // the walk kernel that follows may become resident now (it waits for this grid before it reads the winners)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (t >= n_tree[b]) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const size_t row = (size_t)b * Ncap + t;
@@ -99,6 +101,14 @@ __global__ void __launch_bounds__(CAST_MAX_TREE) accept_walk_kernel(
     }
     return;
   }
+  // the tree arrays were written before the sweep was launched; the sweep's winners are read after the wait
+  // (programmatic dependent launch: this grid may be resident while the sweep still runs; a no-op otherwise)
+  int tok_mine = 0, par_mine = -1;
+  if (t < N) {
+    tok_mine = tokens[(size_t)b * Ncap + t];
+    par_mine = parent[(size_t)b * Ncap + t];
+  }
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (t < N) {
     unsigned long long key = 0ull;
     for (int c = 0; c < nchunks; ++c) {
@@ -106,8 +116,8 @@ __global__ void __launch_bounds__(CAST_MAX_TREE) accept_walk_kernel(
       key = k > key ? k : key;
     }
     g[t] = key ? key_token(key) : 0;
-    tok[t] = tokens[(size_t)b * Ncap + t];
-    par[t] = parent[(size_t)b * Ncap + t];
+    tok[t] = tok_mine;
+    par[t] = par_mine;
     if ((t == 0 && par[t] != -1) || (t > 0 && (par[t] < 0 || par[t] >= t))) report(st, CAST_ERR_BAD_TREE, b * Ncap + t);
   }
   __syncthreads();
@@ -258,8 +268,25 @@ extern "C" cast_status cast_accept(cast_ctx* c, const void* target_logits, cast_
   else
     argmax_sweep_kernel<__nv_bfloat16><<<grid, kArgThreads, 0, s>>>((const __nv_bfloat16*)target_logits, V, Ncap,
                                                                     chunk_elems, n_tree, c->acc_part);
-  accept_walk_kernel<<<B, CAST_MAX_TREE, 0, s>>>(c->acc_part, nchunks, Ncap, c->cfg.max_depth, tokens, parent, n_tree,
-                                                 accept_len, accept_path, bonus_token, c->state);
+  {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(B, 1, 1);
+    cfg.blockDim = dim3(CAST_MAX_TREE, 1, 1);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // resident while the sweep drains
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const unsigned long long* part = c->acc_part;
+    const int H = c->cfg.max_depth;
+    DevState* st = c->state;
+    if (cudaLaunchKernelEx(&cfg, accept_walk_kernel, part, nchunks, Ncap, H, tokens, parent, n_tree, accept_len,
+                           accept_path, bonus_token, st) != cudaSuccess) {
+      cudaGetLastError();
+      return CAST_ERR_CUDA;
+    }
+  }
   return launch_status();
 }
 

@@ -45,7 +45,8 @@ class Workload:
     n_layers: int  # verification layers timed per step (distinct KV buffers)
     max_tree: int = 128
     tau: float = 1.4e-4  # slope of the synthetic cost table in B*n
-    seed_salt: int = 0  # bumped when a seed puts a tree decision within rounding of its threshold
+    seed_salt: int = 0  # the first salt whose seed keeps every tree decision of the ORACLE clear of its threshold
+    # (tests/seed_margin_audit.py prints the margins of the salts passed over)
 
     @property
     def seed(self) -> int:
@@ -71,7 +72,7 @@ CONFIGS: Dict[str, Workload] = {
     for w in [
         Workload("c1_tiny", 1, 1, "f32", "f32", 8, 8, 64, 256, 256, 0, 4096, 2.0, 4, 4, 16, False, 2),
         Workload("c2_llama8b", 2, 1, "bf16", "f32", 32, 8, 128, 2048, 2048, 0, 128256, 3.0, 6, 10, 60, False, 32),
-        _c3(1, 0, 2), _c3(4, 1), _c3(16, 2), _c3(64, 3, 7),
+        _c3(1, 0, 2), _c3(4, 1), _c3(16, 2), _c3(64, 3, 4),
         _c4(16, 0), _c4(32, 1), _c4(64, 2), _c4(128, 3),
         Workload("c5_qwen_long", 5, 4, "bf16", "f32", 28, 4, 128, 32768, 32768, 16, 152064, 3.0, 8, 8, 96, False, 2,
                  seed_salt=1),

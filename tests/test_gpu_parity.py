@@ -838,3 +838,28 @@ def test_attention_without_a_reserved_workspace_is_refused(binding):
     torch.cuda.synchronize()
     assert torch.cuda.mem_get_info()[0] == free1 <= free0  # the compute call moved no device memory
     assert torch.isfinite(out[0, 0]).all() and ctx.cast_poll_status()[0] == 0
+
+
+# ------------------------------------------------ the seeds the benchmark configurations pass over
+@pytest.mark.parametrize("name,salt", [("c3_llama8b_b1", 0), ("c3_llama8b_b1", 1), ("c5_qwen_long", 0), ("c3_llama8b_b64", 0)])
+def test_seeds_passed_over_for_their_margin_still_match(binding, name, salt):
+    """A configuration's seed_salt skips seeds on which the ORACLE has a decision within rounding of its
+    threshold (a gap below 1e-5 between neighbouring values, or a test that flips under a relative 2e-6):
+    there a bit-exact comparison with fp32 device arithmetic is not well posed. They were not skipped because
+    the device disagreed: on these seeds it builds the oracle's tree as well (tests/seed_margin_audit.py lists
+    the margins; the smallest gap here is 5e-6)."""
+    w = wl.shrink(wl.CONFIGS[name], seed_salt=salt)
+    kw = cfg_kwargs(w)
+    B = w.batch
+    tables, raw = _oracle_tables(w, B) if w.cost_model else (None, None)
+    ctx = binding.CastContext(max_batch=B, **kw)
+    if raw is not None:
+        ctx.cast_set_cost_tables(B, *raw)
+    root = wl.root_tokens(w, "cpu").cuda()
+    kv = wl.kv_lengths(w, "cpu").cuda()
+    logits = [wl.draft_logits(w, l, "cpu").cuda() for l in range(1, w.depth + 1)]
+    o = oracle_tree(kw, tables, root, kv, logits)
+    assert not (o["min_score_gap"] >= 1e-5 and o["stable"]), "this seed is not a marginal one any more"
+    g = gpu_tree(ctx, root, kv, logits)
+    print(f"{name} salt {salt}: oracle gap {o['min_score_gap']:.2e}, stable {o['stable']}")
+    assert_tree_equal(g, o)
