@@ -211,6 +211,8 @@ def measure(args, w, rep, full):
     seq_cap = wl.seq_capacity(w) // (w.page_size or 1)
     ctx.cast_reserve_attention(torch.bfloat16 if w.kv_dtype == "bf16" else torch.float32, B, Hq, Hkv, D, w.page_size,
                                seq_cap)
+    # a decoding loop: between two attention layers nothing writes the tree, the lengths or the prefix rows
+    ctx.cast_set_attention_early_reads(True)
     l2_bytes = int(torch.cuda.get_device_properties(dev).L2_cache_size)
 
     # ---- synthetic inputs, resident in HBM

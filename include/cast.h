@@ -191,6 +191,22 @@ CAST_API cast_status cast_reserve_attention(cast_ctx* ctx, cast_dtype dtype, int
                                    int page_size, int seq_capacity);
 
 /*
+ * Set-up call (nothing in the paper corresponds to it). The attention kernels are launched with programmatic
+ * dependent launch and by default read nothing before the operation that precedes them on the stream has
+ * completed. With promise != 0 the caller promises, for every later attention call of this context, that of the
+ * call's inputs ONLY q and the cache rows of the tree tokens (positions >= kv_len[b]) can have been written by the
+ * operation that immediately precedes the call on the stream; kv_len, n_tree, first_row, anc_mask, page_table and
+ * the cache rows of the prefix (positions < kv_len[b]) were complete before that operation started (as they are in
+ * a decoding loop: the tree is fixed for all layers of a step, and between two layers run the model's own kernels).
+ * The kernel then decodes its work, reads the masks and fetches its first prefix tiles while its predecessor still
+ * runs, and waits only before it loads q, a tile that reaches the tree tokens' rows, or writes output. Calls of
+ * this library that write those inputs (cast_select_nodes, cast_compact_kv) are accounted for by the library: the
+ * attention call that follows one of them takes no early reads. Needs bf16, D = 128 and a GQA group size that
+ * divides 128; other shapes ignore the promise. promise = 0 (the default) restores the conservative behaviour.
+ */
+CAST_API cast_status cast_set_attention_early_reads(cast_ctx* ctx, int promise);
+
+/*
  * One layer of verification attention (the mask of Sec. "Tree Reranking Phase"):
  * out[b,t,h] = softmax over {prefix positions 0..kv_len[b]-1} U {tree positions
  * kv_len[b]+j : bit j of anc_mask[b,t]} of (q . k) * scale, times v, for

@@ -28,6 +28,7 @@ EXPORTS = [
     "cast_state_import", "cast_step_begin", "cast_tree_expand", "cast_select_nodes", "cast_tree_attention",
     "cast_accept", "cast_compact_kv", "cast_poll_status", "cast_step_info", "cast_accept_static",
     "cast_accept_stochastic", "cast_accept_stochastic_plan", "cast_tree_attention_rows", "cast_reserve_attention",
+    "cast_set_attention_early_reads",
 ]
 
 
@@ -73,6 +74,7 @@ def load_library() -> C.CDLL:
         "cast_tree_expand": [vp, i32, vp, i32, i32p, i32p, i32p, vp],
         "cast_select_nodes": [vp, i32p, i32p, i32p, vp, i32p, vp, i32p, vp],
         "cast_reserve_attention": [vp, i32, i32, i32, i32, i32, i32, i32],
+        "cast_set_attention_early_reads": [vp, i32],
         "cast_tree_attention": [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32p, i32, i32, i32p, vp, i32p,
                                 C.c_float, vp, vp],
         "cast_tree_attention_rows": [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32p, i32, i32, i32p, vp, i32p,
@@ -179,6 +181,11 @@ class CastContext:
         code = CAST_F32 if dtype == torch.float32 else CAST_BF16
         _check(self.lib.cast_reserve_attention(self.handle, code, B, Hq, Hkv, D, page_size, seq_capacity),
                "cast_reserve_attention")
+
+    def cast_set_attention_early_reads(self, promise: bool):
+        """The caller's promise that only q and the tree tokens' cache rows come from the operation right before an
+        attention call (see include/cast.h)."""
+        _check(self.lib.cast_set_attention_early_reads(self.handle, 1 if promise else 0), "cast_set_attention_early_reads")
 
     # --- compute calls (enqueue only) ----------------------------------------
     def cast_step_begin(self, B, root_token, kv_len, stream=None):

@@ -375,6 +375,7 @@ extern "C" cast_status cast_compact_kv(cast_ctx* c, void* k_cache, void* v_cache
   if (((uintptr_t)k_cache | (uintptr_t)v_cache | layer_stride_bytes) & 15) return CAST_ERR_SHAPE;
   const int H1 = c->cfg.max_depth + 1;
   if (2 * H1 * (row_bytes / 16) > kCompactThreads * kCompactItems) return CAST_ERR_CAPACITY;
+  c->tree_inputs_fresh = 1;  // kv_len and cache rows: an attention call that follows reads them after its dependency wait
   CompactParams p;
   p.k = (char*)k_cache; p.v = (char*)v_cache; p.layer_stride = layer_stride_bytes;
   p.Hkv = Hkv; p.row_bytes = row_bytes; p.page_size = page_size; p.seq_capacity = seq_capacity;

@@ -111,6 +111,11 @@ struct cast_ctx {
   int sto_cs[2];
   int sto_cached[2];
 
+  // cast_set_attention_early_reads: the caller's promise, and whether the last call of this library on the
+  // context wrote something the attention reads early (n_tree, masks: cast_select_nodes; kv_len: cast_compact_kv)
+  int attn_early;
+  int tree_inputs_fresh;
+
   std::map<int, cast::HostTable>* tables;
   cast::DevTable cur_table;   // table of the current step's batch size (zeros if none)
   int cur_B;

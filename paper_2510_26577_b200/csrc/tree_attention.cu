@@ -335,6 +335,12 @@ cast_status launch_cc(cast_ctx* c, AttnParams& p, cudaStream_t s) {
 
 }  // namespace
 
+extern "C" cast_status cast_set_attention_early_reads(cast_ctx* c, int promise) {
+  if (!c) return CAST_ERR_INVALID_ARG;
+  c->attn_early = promise ? 1 : 0;
+  return CAST_OK;
+}
+
 extern "C" cast_status cast_reserve_attention(cast_ctx* c, cast_dtype dtype, int B, int Hq, int Hkv, int D, int page_size,
                                               int seq_capacity) {
   if (!c || B < 1 || Hq < 1 || Hkv < 1 || page_size < 0 || seq_capacity < 1) return CAST_ERR_INVALID_ARG;
@@ -373,11 +379,15 @@ extern "C" cast_status cast_tree_attention_rows(cast_ctx* c, const void* q, cons
   if (((uintptr_t)q | (uintptr_t)k_cache | (uintptr_t)v_cache | (uintptr_t)out) & 15) return CAST_ERR_SHAPE;
   if (scale == 0.f) scale = 1.0f / sqrtf((float)D);
   cudaStream_t s = (cudaStream_t)stream;
+  const int fresh = c->tree_inputs_fresh;
+  c->tree_inputs_fresh = 0;  // whatever is launched below waits for its predecessor before it releases its own dependents
   if (dtype == CAST_BF16) {
     cast_status st = CAST_OK;
-    if (tree_attention_tc_launch(c, q, k_cache, v_cache, B, Hq, Hkv, D, page_size, page_table, seq_capacity, num_pages,
-                                 kv_len, anc_mask, n_tree, first_row, scale, out, s, &st))
-      return st;
+    c->tree_inputs_fresh = fresh;
+    const bool taken = tree_attention_tc_launch(c, q, k_cache, v_cache, B, Hq, Hkv, D, page_size, page_table, seq_capacity,
+                                                num_pages, kv_len, anc_mask, n_tree, first_row, scale, out, s, &st);
+    c->tree_inputs_fresh = 0;
+    if (taken) return st;
   }
   AttnParams p;
   p.q = q; p.k = k_cache; p.v = v_cache; p.out = out;

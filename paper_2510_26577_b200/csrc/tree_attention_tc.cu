@@ -68,6 +68,8 @@ struct TcParams {
   const __nv_bfloat16* q;
   __nv_bfloat16* out;
   int B, Ncap, Nmax, Hq, Hkv, G, page_size, seq_capacity, num_pages, words;
+  int q_tma;  // Q row blocks are fetched by TMA (the group size divides 128)
+  int early;  // the tree arrays, lengths, page table and prefix rows may be read before the dependency wait
   int cs;   // CTAs per cluster (1..8); 0: no clusters, splits sized on the device and merged through global memory
   int rpc;  // cluster mode: row blocks a cluster covers at most (cs is a multiple of it)
   int nsplit_max, num_sms, nrb;  // global-merge mode
@@ -621,7 +623,8 @@ __device__ __forceinline__ void merge_rows_global(const TcParams& p, int b, int 
 }
 
 __global__ void __launch_bounds__(kThreadsTC, 2)
-tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
+tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                    const __grid_constant__ CUtensorMap map_q) {
   extern __shared__ __align__(1024) unsigned char smem[];  // no static shared memory: the base is 1 KB aligned
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -630,14 +633,25 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
   if (warp == 4 && lane == 0) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_k)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_v)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_q)) : "memory");
   }
   // Programmatic dependent launch: this grid may become resident while the previous kernel of the
   // stream drains; nothing written by earlier kernels is read before this point. (No-ops for a plain launch.)
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // In the default mode nothing is read before the wait. In "early" mode (a promise of the caller, see
+  // cast_set_attention_early_reads) only Q and the cache rows of the tree tokens can come from the previous
+  // kernel: the work decode, the ancestor masks, the page ids and the K/V tiles that lie wholly inside the
+  // prefix are fetched while that kernel still runs, and every warp waits just before the first thing it does
+  // that depends on it (the Q load, a tile that reaches the tree rows, the output rows). The dependents are
+  // released only after this CTA's own wait, so "everything before my predecessor is complete" keeps holding
+  // down the chain.
+  const bool early = p.early != 0;
+  if (!early) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  }
   const WorkItem wk = cs == 0 ? decode_work_chunked(p, (int)blockIdx.x, (int)gridDim.x) : decode_work(p, (int)blockIdx.x / cs, crank);
   if (blockIdx.x < p.B && tid == 0 && p.n_tree[blockIdx.x] > p.Nmax) report(p.st, CAST_ERR_BAD_TREE, blockIdx.x);
-  if (!wk.valid) return;  // the whole cluster leaves
+  if (!wk.valid) return;  // the whole cluster leaves (a CTA that exits counts as having released its dependents)
   const int b = wk.b, kvh = wk.kvh, rb = wk.rb, split = wk.split, N = wk.N, L = wk.L;
   const int nsplit = wk.nsplit;
   const int G = p.G, F = wk.F, rows_total = (N - F) * G, row0 = rb * kBM;
@@ -682,7 +696,8 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
   uint64_t* bar_s = bars + 10;         // [2]
   uint64_t* bar_p = bars + 12;         // [2]: tile it uses bar_p[it & 1], phase it >> 1
   uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(bars + 14);
-  int* last_s = reinterpret_cast<int*>(bars + 15);
+  int* last_s = reinterpret_cast<int*>(bars + 14) + 1;
+  uint64_t* bar_q = bars + 15;         // the Q row block has landed (TMA)
 
   // ---- producer helper (warp 4; all 32 lanes call it): which = 0: K tile j, which = 1: V tile j
   auto issue_tile = [&](int j, int which) -> bool {
@@ -723,14 +738,19 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
   };
   // a producer warp fills its ring tile by tile (K: warp 4, V: warp 6); after an expired wait it reports,
   // then waits (bounded) for its copies in flight, which must land before the CTA's shared memory is released
-  auto produce = [&](int which, int first) {
+  auto produce = [&](int which, int first, bool waited) {
     const int stages = which ? kStagesV : kStagesK;
     int armed = first;
     bool ok = true;
     for (int j = first; j < ntile && ok; ++j) {
+      if (!waited && (t0 + j + 1) * kBN > L) {  // the first tile that reaches the tree tokens' rows
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        waited = true;
+      }
       ok = issue_tile(j, which);
       if (ok) armed = j + 1;
     }
+    if (!waited) asm volatile("griddepcontrol.wait;" ::: "memory");  // (this warp writes output rows in the merge)
     if (!ok) {
       if (lane == 0) report(p.st, CAST_ERR_TIMEOUT, b);
       for (int j = (armed > stages ? armed - stages : 0); j < armed; ++j) {
@@ -757,13 +777,28 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
       mbar_init(&bar_s[1], 1);
       mbar_init(&bar_p[0], kSoftmaxThreads);
       mbar_init(&bar_p[1], kSoftmaxThreads);
+      mbar_init(bar_q, 1);
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       fence_proxy_async();
     }
     __syncwarp();
     __threadfence_block();
     asm volatile("bar.arrive 2, %0;" ::"n"(kThreadsTC) : "memory");
-    // the first K tiles need no stage wait: the ring fills while the other warps stage Q
+    // The Q row block: rows are (tree token, head of the group) pairs, so a block is 128 / G consecutive
+    // tokens x the group's G heads x 128 dims: one 3-D box per 64-dim half, 128-byte swizzled like K. (Rows
+    // past the tree hold whatever the caller's buffer holds: their P is masked to exact zeros.)
+    if (early) {  // prefix tiles first, then the wait, then Q (the previous kernel may have written it)
+      for (; k_issued < kStagesK && k_issued < ntile && (t0 + k_issued + 1) * kBN <= L; ++k_issued) issue_tile(k_issued, 0);
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    }
+    if (p.q_tma) {
+      if (lane == 0) mbar_expect_tx(bar_q, 2 * kRegionQ);
+      __syncwarp();
+      if (lane < 2)
+        tma_load_3d(&map_q, smem + kSmemQ + lane * kRegionQ, bar_q, lane * 64, kvh * G, b * p.Ncap + F + row0 / G);
+    }
+    // the first K tiles need no stage wait: the ring fills while Q is on its way
     for (; k_issued < kStagesK && k_issued < ntile; ++k_issued) issue_tile(k_issued, 0);
   } else if (warp < 4) {
     if (warp == 0) {  // TMEM: two S buffers and O
@@ -771,35 +806,40 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
                    "n"(kTmemCols));
       asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
     }
-    // Q row -> swizzled shared memory (rows past the tree are zero); ancestor mask -> registers
-    const __nv_bfloat16* qrow = p.q + (((size_t)b * p.Ncap + t_tok) * p.Hq + h_q) * kHD;
-    uint4 qv[16];
-#pragma unroll
-    for (int c = 0; c < 16; ++c) qv[c] = row_ok ? *reinterpret_cast<const uint4*>(qrow + c * 8) : make_uint4(0u, 0u, 0u, 0u);
+    // ancestor mask -> registers; without TMA for Q: the Q row -> swizzled shared memory (rows past the tree zero)
     if (row_ok) {
 #pragma unroll
       for (int w = 0; w < 4; ++w)
         if (w < p.words) aw[w] = p.anc[((size_t)b * p.Ncap + t_tok) * p.words + w];
     }
+    if (!p.q_tma) {
+      const __nv_bfloat16* qrow = p.q + (((size_t)b * p.Ncap + t_tok) * p.Hq + h_q) * kHD;
+      uint4 qv[16];
 #pragma unroll
-    for (int c = 0; c < 16; ++c)
-      *reinterpret_cast<uint4*>(smem + kSmemQ + (c >> 3) * kRegionQ + swz(r, c & 7)) = qv[c];
-    fence_proxy_async();
+      for (int c = 0; c < 16; ++c) qv[c] = row_ok ? *reinterpret_cast<const uint4*>(qrow + c * 8) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+      for (int c = 0; c < 16; ++c)
+        *reinterpret_cast<uint4*>(smem + kSmemQ + (c >> 3) * kRegionQ + swz(r, c & 7)) = qv[c];
+      fence_proxy_async();
+    }
   }
   // everyone but the producer waits here for the barrier objects, the TMEM address and Q; the producer
   // only signals that the barriers exist (it arrived right after initialising them) and keeps loading
   tc_fence_before();
   if (warp != 4) asm volatile("bar.sync 2, %0;" ::"n"(kThreadsTC) : "memory");
   tc_fence_after();
+  // early mode: the softmax warps, the MMA issuer and the spare warp have nothing to do before Q arrives,
+  // which is after the wait anyway; the producers wait inside produce()
+  if (early && warp != 4 && warp != 6) asm volatile("griddepcontrol.wait;" ::: "memory");
   const uint32_t tmem_base = *tmem_base_s;
   const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 2 * kBN;
 
   if (warp == 4) {
     // =========================== TMA producer: K ring ===========================
-    produce(0, k_issued);
+    produce(0, k_issued, true);  // (this warp has waited, at the latest before the Q load)
   } else if (warp == 6) {
     // =========================== TMA producer: V ring ===========================
-    produce(1, 0);
+    produce(1, 0, !early);
   } else if (warp == 5) {
     // =========================== MMA issuer ===========================
     const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
@@ -834,7 +874,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     };
     // next scores first: Q K^T of tile it+1 runs while the softmax of tile `it` does; the other CTA on
     // this SM covers the moments when a K tile is late
-    bool ok = ntile == 0 || mbar_wait(&bar_fullk[0], 0);
+    bool ok = ntile == 0 || ((!p.q_tma || mbar_wait(bar_q, 0)) && mbar_wait(&bar_fullk[0], 0));
     if (ok && ntile > 0) {
       tc_fence_after();
       mma_qk(0, 0);
@@ -1216,6 +1256,19 @@ EncodeTiledFn get_encode() {
   return fn;
 }
 
+// Q [B * Ncap tokens][Hq heads][128 dims]: a box is 128 / G tokens x G heads x 64 dims (one row block, one half)
+bool make_q_map(CUtensorMap* map, const void* base, int B, int Ncap, int Hq, int G) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return false;
+  const cuuint64_t dims[3] = {kHD, (cuuint64_t)Hq, (cuuint64_t)B * Ncap};
+  const cuuint64_t strides[2] = {kHD * 2, (cuuint64_t)Hq * kHD * 2};
+  const cuuint32_t box[3] = {64, (cuuint32_t)G, (cuuint32_t)(kBM / G)};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool make_kv_map(CUtensorMap* map, const void* base, int B, int Hkv, int page_size, int seq_capacity, int num_pages) {
   EncodeTiledFn enc = get_encode();
   if (!enc) return false;
@@ -1334,7 +1387,11 @@ bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const v
     return false;
   const int G = Hq / Hkv, Ncap = c->cfg.max_tree;
   const int Nmax = c->cfg.total_token < Ncap ? c->cfg.total_token : Ncap;
+  CUtensorMap map_q = map_k;  // (a valid descriptor either way; used only when q_tma is set)
+  const bool q_tma = G <= kBM && (kBM % G) == 0 && make_q_map(&map_q, q, B, Ncap, Hq, G);
   TcParams p;
+  p.q_tma = q_tma ? 1 : 0;
+  p.early = (c->attn_early && !c->tree_inputs_fresh && q_tma) ? 1 : 0;
   p.q = (const __nv_bfloat16*)q; p.out = (__nv_bfloat16*)out;
   p.B = B; p.Ncap = Ncap; p.Nmax = Nmax; p.Hq = Hq; p.Hkv = Hkv; p.G = G; p.page_size = page_size;
   p.seq_capacity = seq_capacity; p.num_pages = num_pages; p.words = c->words;
@@ -1384,7 +1441,7 @@ bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const v
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  if (cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel, p, map_k, map_v) != cudaSuccess) {
+  if (cudaLaunchKernelEx(&cfg, tree_attn_tc_kernel, p, map_k, map_v, map_q) != cudaSuccess) {
     cudaGetLastError();
     *status = CAST_ERR_CUDA;
     return true;

@@ -1147,6 +1147,7 @@ extern "C" cast_status cast_select_nodes(cast_ctx* c, int32_t* tokens, int32_t* 
                                          void* stream) {
   if (!c || !tokens || !parent || !depth || !anc_mask || !pool_idx || !n_tree) return CAST_ERR_INVALID_ARG;
   if (c->cur_B < 1 || c->next_layer < 2) return CAST_ERR_INVALID_ARG;  // a step with at least one layer
+  c->tree_inputs_fresh = 1;  // n_tree and the masks: the next attention call reads them after its dependency wait
   SelectParams p;
   p.pool_score = c->pool_score; p.pool_token = c->pool_token; p.pool_parent = c->pool_parent;
   p.pool_depth = c->pool_depth; p.lsort = c->lsort; p.lscore = c->lscore; p.st = c->state;

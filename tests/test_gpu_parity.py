@@ -9,7 +9,7 @@ import torch
 from oracle import ancestor_masks, compact_kv, greedy_accept, stochastic_accept, tree_attention
 from paper_2510_26577_b200 import workloads as wl
 
-from helpers import (assert_tree_equal, attention_tolerance, cfg_kwargs, gpu_attention, gpu_tree, make_tables,
+from helpers import (alloc_tree_outputs, assert_tree_equal, attention_tolerance, cfg_kwargs, gpu_attention, gpu_tree, make_tables,
                      oracle_tree, to_f64)
 
 pytestmark = pytest.mark.gpu
@@ -863,3 +863,62 @@ def test_seeds_passed_over_for_their_margin_still_match(binding, name, salt):
     g = gpu_tree(ctx, root, kv, logits)
     print(f"{name} salt {salt}: oracle gap {o['min_score_gap']:.2e}, stable {o['stable']}")
     assert_tree_equal(g, o)
+
+
+# ------------------------------------------------ attention with early reads (the caller's promise)
+@pytest.mark.parametrize("name", ["c2_llama8b", "c3_llama8b_b4", "c3_llama8b_b16", "c4_llama70b_n32"])
+def test_attention_early_reads_give_the_same_bits(binding, name):
+    """With cast_set_attention_early_reads the kernel decodes its work, reads the masks and fetches prefix tiles
+    before its predecessor on the stream has finished. Two whole steps (tree build, four attention layers back
+    to back on different caches, acceptance, compaction - which moves kv_len and cache rows that the next step's
+    attention reads) run without any host synchronisation in between, once per mode: every attention output,
+    the accepted paths and the lengths must be bit-identical to the default mode's, which the tests above
+    compare with the oracle."""
+    w = wl.CONFIGS[name]
+    B, H, nl = w.batch, w.depth, 4
+    kw = cfg_kwargs(w)
+    tabs = wl.cost_table_arrays(w, B) if w.cost_model else None
+    root = wl.root_tokens(w, "cpu").cuda()
+    kv0 = wl.kv_lengths(w, "cpu").cuda()
+    logits = [[wl.draft_logits(w, 10 * s_ + l, "cuda") for l in range(1, H + 1)] for s_ in range(2)]
+    q = [wl.query(w, l, "cuda") for l in range(nl)]
+    table, num_pages = wl.page_table(w, "cuda")
+    seq_cap = wl.seq_capacity(w) // (w.page_size or 1)
+    tl = wl.target_logits(w, "cuda")
+    results = []
+    for promise in (False, True):
+        ctx = binding.CastContext(max_batch=B, **kw)
+        if tabs is not None:
+            ctx.cast_set_cost_tables(B, *tabs)
+        ctx.cast_reserve_attention(q[0].dtype, B, w.q_heads, w.kv_heads, w.head_dim, w.page_size, seq_cap)
+        ctx.cast_set_attention_early_reads(promise)
+        kc = torch.stack([wl.kv_cache(w, l, "cuda")[0] for l in range(nl)]).contiguous()
+        vc = torch.stack([wl.kv_cache(w, l, "cuda")[1] for l in range(nl)]).contiguous()
+        kv = kv0.clone()
+        tr = alloc_tree_outputs(B, w.max_tree, ctx.words)
+        nt = torch.empty((B, w.top_k), dtype=torch.int32, device="cuda")
+        npr, cnt = torch.empty_like(nt), torch.empty((1,), dtype=torch.int32, device="cuda")
+        alen = torch.empty((B,), dtype=torch.int32, device="cuda")
+        apath = torch.empty((B, H + 1), dtype=torch.int32, device="cuda")
+        bonus = torch.empty((B,), dtype=torch.int32, device="cuda")
+        outs = []
+        for s_ in range(2):
+            ctx.cast_step_begin(B, root, kv)
+            for i in range(H):
+                ctx.cast_tree_expand(i + 1, logits[s_][i], nt, npr, cnt)
+            ctx.cast_select_nodes(tr["tokens"], tr["parent"], tr["depth"], tr["anc"], tr["pool_idx"], tr["scores"], tr["n_tree"])
+            for l in range(nl):
+                out = torch.full_like(q[l], float("nan"))
+                ctx.cast_tree_attention(q[l], kc[l], vc[l], B, w.q_heads, w.kv_heads, w.head_dim, w.page_size, table, seq_cap,
+                                        num_pages, kv, tr["anc"], tr["n_tree"], 0.0, out)
+                outs.append(out)
+            ctx.cast_accept(tl, B, tr["tokens"], tr["parent"], tr["depth"], tr["anc"], tr["n_tree"], alen, apath, bonus)
+            ctx.cast_compact_kv(kc, vc, B, nl, kc[0].numel() * kc.element_size(), w.kv_heads, w.head_dim, w.page_size, table,
+                                seq_cap, num_pages, apath, alen, kv)
+            outs += [alen.clone(), apath.clone(), kv.clone()]
+        torch.cuda.synchronize()
+        assert ctx.cast_poll_status()[0] == 0
+        results.append([o.view(torch.int16) if o.dtype == torch.bfloat16 else o for o in outs] + [kc.view(torch.int16), vc.view(torch.int16)])
+    for a, b2 in zip(*results):
+        assert torch.equal(a, b2)
+    assert int(results[0][-3].min()) > int(kv0.min())  # the compaction did advance the lengths
