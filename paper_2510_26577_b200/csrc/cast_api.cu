@@ -34,6 +34,7 @@ cudaError_t dev_alloc(T** p, size_t n) {
 void free_all(cast_ctx* c) {
   cudaFree(c->pool_score); cudaFree(c->pool_token); cudaFree(c->pool_parent); cudaFree(c->pool_depth);
   cudaFree(c->pool_kept); cudaFree(c->retained); cudaFree(c->lsort); cudaFree(c->lscore); cudaFree(c->state);
+  cudaFree(c->attn_worklist);
   cudaFree(c->layer_ticket); cudaFree(c->seq_ticket); cudaFree(c->tail_vs); cudaFree(c->tail_sorted); cudaFree(c->tail_tok);
   cudaFree(c->fifo_vals); cudaFree(c->fifo_cnt); cudaFree(c->sel_score); cudaFree(c->sel_value);
   cudaFree(c->sel_idx); cudaFree(c->acc_part); cudaFree(c->compact_ticket); cudaFree(c->attn_ws); cudaFree(c->attn_tc_ws);
@@ -101,6 +102,7 @@ extern "C" cast_status cast_create(const cast_config* cfg, cast_ctx** out) {
   if (e == cudaSuccess) e = dev_alloc(&c->lsort, BP);
   if (e == cudaSuccess) e = dev_alloc(&c->lscore, BP);
   if (e == cudaSuccess) e = dev_alloc(&c->state, 1);
+  if (e == cudaSuccess) e = dev_alloc(&c->attn_worklist, (size_t)kAttnWorkListCap * 8);
   if (e == cudaSuccess) e = dev_alloc(&c->layer_ticket, 1);
   if (e == cudaSuccess) e = dev_alloc(&c->seq_ticket, cfg->max_batch);
   if (e == cudaSuccess) e = dev_alloc(&c->tail_vs, (size_t)cfg->max_batch * CAST_MAX_WIDTH);

@@ -51,6 +51,7 @@ constexpr int kSweepMaxChunks = 8;                        // CTAs per logits row
 constexpr int kCandCap = 4096;                            // 64-bit keys of shared scratch per CTA (warp lists, short list)
 constexpr int kMaxFifo = 64;
 constexpr int kAcceptMaxChunks = 32;
+constexpr int kAttnWorkListCap = 4096;                    // CTAs of an attention launch that a work list can describe
 
 }  // namespace cast
 
@@ -115,6 +116,12 @@ struct cast_ctx {
   // context wrote something the attention reads early (n_tree, masks: cast_select_nodes; kv_len: cast_compact_kv)
   int attn_early;
   int tree_inputs_fresh;
+  // work list of the tensor-core attention (one decoded item per CTA), written by a small kernel at the first
+  // attention call after the tree or the lengths changed and reused by the calls that follow while the promise
+  // above holds and the call's shape is the same (wl_key)
+  int32_t* attn_worklist;          // [kAttnWorkListCap][8]
+  int wl_valid;
+  unsigned long long wl_key[8];
 
   std::map<int, cast::HostTable>* tables;
   cast::DevTable cur_table;   // table of the current step's batch size (zeros if none)

@@ -338,6 +338,7 @@ cast_status launch_cc(cast_ctx* c, AttnParams& p, cudaStream_t s) {
 extern "C" cast_status cast_set_attention_early_reads(cast_ctx* c, int promise) {
   if (!c) return CAST_ERR_INVALID_ARG;
   c->attn_early = promise ? 1 : 0;
+  c->wl_valid = 0;
   return CAST_OK;
 }
 

@@ -69,6 +69,7 @@ struct TcParams {
   __nv_bfloat16* out;
   int B, Ncap, Nmax, Hq, Hkv, G, page_size, seq_capacity, num_pages, words;
   int q_tma;  // Q row blocks are fetched by TMA (the group size divides 128)
+  const int32_t* worklist;  // one decoded work item per CTA (8 ints each), or null: every CTA decodes for itself
   int early;  // the tree arrays, lengths, page table and prefix rows may be read before the dependency wait
   int cs;   // CTAs per cluster (1..8); 0: no clusters, splits sized on the device and merged through global memory
   int rpc;  // cluster mode: row blocks a cluster covers at most (cs is a multiple of it)
@@ -622,6 +623,32 @@ __device__ __forceinline__ void merge_rows_global(const TcParams& p, int b, int 
   }
 }
 
+// One work item as eight ints: {b | kvh << 8 | rb << 16 | valid << 24 | active << 25, split | nsplit << 16, N, L, F, 0, 0, 0}
+__device__ __forceinline__ void store_item(int32_t* dst, const WorkItem& w) {
+  dst[0] = w.b | (w.kvh << 8) | (w.rb << 16) | ((w.valid ? 1 : 0) << 24) | ((w.active ? 1 : 0) << 25);
+  dst[1] = w.split | (w.nsplit << 16);
+  dst[2] = w.N;
+  dst[3] = w.L;
+  dst[4] = w.F;
+}
+__device__ __forceinline__ WorkItem load_item(const int32_t* src) {
+  const int4 a = *reinterpret_cast<const int4*>(src);
+  const int f = src[4];
+  WorkItem w;
+  w.b = a.x & 0xff; w.kvh = (a.x >> 8) & 0xff; w.rb = (a.x >> 16) & 0xff;
+  w.valid = ((a.x >> 24) & 1) != 0; w.active = ((a.x >> 25) & 1) != 0;
+  w.split = a.y & 0xffff; w.nsplit = a.y >> 16;
+  w.N = a.z; w.L = a.w; w.F = f;
+  return w;
+}
+// The work decode of every CTA of a launch, done once: warp i decodes what CTA i would decode for itself.
+__global__ void __launch_bounds__(256) attn_worklist_kernel(const TcParams p, int grid, int32_t* list) {
+  const int idx = (int)blockIdx.x * 8 + (int)(threadIdx.x >> 5);
+  if (idx >= grid) return;
+  const WorkItem w = p.cs == 0 ? decode_work_chunked(p, idx, grid) : decode_work(p, idx / p.cs, idx % p.cs);
+  if ((threadIdx.x & 31) == 0) store_item(list + (size_t)idx * 8, w);
+}
+
 __global__ void __launch_bounds__(kThreadsTC, 2)
 tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                     const __grid_constant__ CUtensorMap map_q) {
@@ -649,7 +676,9 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   }
-  const WorkItem wk = cs == 0 ? decode_work_chunked(p, (int)blockIdx.x, (int)gridDim.x) : decode_work(p, (int)blockIdx.x / cs, crank);
+  const WorkItem wk = p.worklist != nullptr ? load_item(p.worklist + (size_t)blockIdx.x * 8)
+                      : cs == 0            ? decode_work_chunked(p, (int)blockIdx.x, (int)gridDim.x)
+                                           : decode_work(p, (int)blockIdx.x / cs, crank);
   if (blockIdx.x < p.B && tid == 0 && p.n_tree[blockIdx.x] > p.Nmax) report(p.st, CAST_ERR_BAD_TREE, blockIdx.x);
   if (!wk.valid) return;  // the whole cluster leaves (a CTA that exits counts as having released its dependents)
   const int b = wk.b, kvh = wk.kvh, rb = wk.rb, split = wk.split, N = wk.N, L = wk.L;
@@ -792,7 +821,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
       asm volatile("griddepcontrol.wait;" ::: "memory");
       asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     }
-    if (p.q_tma) {
+    if (p.q_tma && ntile > 0) {  // (a split without tiles stages its empty partial in this region right away)
       if (lane == 0) mbar_expect_tx(bar_q, 2 * kRegionQ);
       __syncwarp();
       if (lane < 2)
@@ -1414,6 +1443,28 @@ bool tree_attention_tc_launch(cast_ctx* c, const void* q, const void* k, const v
     p.ticket = reinterpret_cast<int32_t*>(c->attn_tc_ws);
     p.part_o = reinterpret_cast<__half*>(reinterpret_cast<char*>(c->attn_tc_ws) + kTicketBytes);
     p.part_ml = reinterpret_cast<float*>(p.part_o + pl.rows * kHD);
+  }
+  // The work list: under the caller's promise the lengths and tree sizes do not change between the attention
+  // calls of a step, so what every CTA would decode for itself is decoded once, by a small kernel launched in
+  // front of the first such call (or when the call's shape changes), and the calls after it read one item each.
+  p.worklist = nullptr;
+  if (c->attn_early && first_row == nullptr && grid <= kAttnWorkListCap) {  // (a window call names new sizes every time)
+    const unsigned long long key[8] = {(unsigned long long)(uintptr_t)n_tree, (unsigned long long)(uintptr_t)kv_len,
+                                       (unsigned long long)(uintptr_t)first_row,
+                                       ((unsigned long long)B << 48) | ((unsigned long long)Hq << 32) | ((unsigned long long)Hkv << 16) | (unsigned)page_size,
+                                       ((unsigned long long)seq_capacity << 32) | (unsigned)grid,
+                                       ((unsigned long long)(unsigned)p.cs << 32) | ((unsigned)p.rpc << 16) | (unsigned)p.nsplit_max,
+                                       (unsigned long long)Nmax, (unsigned long long)c->num_sms};
+    bool same = c->wl_valid && !c->tree_inputs_fresh;
+    for (int i = 0; i < 8 && same; ++i) same = c->wl_key[i] == key[i];
+    if (!same) {
+      attn_worklist_kernel<<<(unsigned)((grid + 7) / 8), 256, 0, stream>>>(p, (int)grid, c->attn_worklist);
+      if (cudaGetLastError() != cudaSuccess) { *status = CAST_ERR_CUDA; return true; }
+      for (int i = 0; i < 8; ++i) c->wl_key[i] = key[i];
+      c->wl_valid = 1;
+      p.early = 0;  // the list is the previous kernel's: read it after the wait
+    }
+    p.worklist = c->attn_worklist;
   }
   static bool attr_done = false;
   if (!attr_done) {

@@ -87,6 +87,9 @@ def test_attention_random_shapes_and_windows(binding, seed):
         hi = int(rng.choice([40, 300, 1500]))
         w = wl.Workload("fuzz", 300 + case, B, dtype, "f32", Hq, Hkv, D, 0, hi, page, 100, 1.0, 4, 2, 8, False, 1)
         ctx = binding.CastContext(max_batch=B, vocab=100, top_k=2, max_depth=8, total_token=128, max_tree=128)
+        # one seed runs with the early reads on (every input here is uploaded by a host copy that has completed
+        # before the call, which is what the promise asks for)
+        ctx.cast_set_attention_early_reads(seed == 4)
         kv = wl.kv_lengths(w, "cpu").cuda()
         n_tree = rng.integers(1, 129, size=B).astype(np.int32)
         first = np.array([int(rng.integers(0, n + 1)) if rng.random() < 0.6 else 0 for n in n_tree], dtype=np.int32)
