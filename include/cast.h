@@ -35,6 +35,11 @@
  *    dependent launch: their thread blocks may become resident while the previous kernel of the
  *    stream is still finishing, but they read no input (logits, Q, K/V, tree arrays, lengths) before
  *    that kernel has completed, so stream order keeps its usual meaning for the caller.
+ *  - Precision of the tree-sizing decisions: node values, u, c and every comparison are fp64, but a row's
+ *    log-sum-exp is accumulated in fp32 (about 3e-7 absolute per layer). The retained sets, n_i, go/stop
+ *    and N equal those of an exact evaluation whenever no two neighbouring values across a kept/dropped
+ *    boundary are closer than 1e-5 and no Algorithm 1 or depth test flips under a relative change of 2e-6
+ *    of its two sides; closer than that, either outcome may be returned.
  *  - A context must not be used from two streams at once.
  *  - Row-major layouts, innermost index last, written as [d0, d1, ...].
  */

@@ -253,7 +253,13 @@ extern "C" cast_status cast_accept(cast_ctx* c, const void* target_logits, cast_
   if (dtype != CAST_F32 && dtype != CAST_BF16) return CAST_ERR_DTYPE;
   if (B > c->cfg.max_batch) return CAST_ERR_CAPACITY;
   const int V = c->cfg.vocab, Ncap = c->cfg.max_tree;
-  int nchunks = (4 * c->num_sms + B * Ncap - 1) / (B * Ncap);
+  // Chunks per logits row: enough CTAs to keep four per SM streaming when every sequence verifies its full
+  // budget (the context's total_token; the row slots beyond a tree exit at once), and never chunks of more
+  // than 32 K logits, so that a batch whose trees came out far below the budget still has several live CTAs
+  // per SM; at least 4096 logits per chunk.
+  const int budget = c->cfg.total_token < Ncap ? c->cfg.total_token : Ncap;
+  int nchunks = (4 * c->num_sms + B * budget - 1) / (B * budget);
+  if (nchunks < (V + 32767) / 32768) nchunks = (V + 32767) / 32768;
   if (nchunks > kAcceptMaxChunks) nchunks = kAcceptMaxChunks;
   if (nchunks > V / 4096) nchunks = V / 4096;
   if (nchunks < 1) nchunks = 1;
