@@ -175,8 +175,7 @@ __device__ __forceinline__ void tail_rank(const ExpandParams& p, int b_begin, in
   const int Ni = n_prev * K;
   double* sc = reinterpret_cast<double*>(scratch);              // 1024 scores
   int* tk = reinterpret_cast<int*>(scratch + 8192);             // 1024 tokens
-  unsigned short* r1s = reinterpret_cast<unsigned short*>(scratch + 12288);  // 1024: row of the candidate
-  unsigned short* cis = reinterpret_cast<unsigned short*>(scratch + 14336);  // 1024: index within the sequence
+  int* rank_s = reinterpret_cast<int*>(scratch + 12288);        // 1024 ranks
   const int group = 1024 / Ni;                                  // sequences ranked per pass
 #pragma unroll 1
   for (int b0 = 0; b0 < b_count; b0 += group) {
@@ -187,53 +186,66 @@ __device__ __forceinline__ void tail_rank(const ExpandParams& p, int b_begin, in
       const size_t o = (size_t)(b_begin + b0 + bl) * P + base + ci;
       sc[i] = __ldcg(p.pool_score + o);
       tk[i] = __ldcg(p.pool_token + o);
-      r1s[i] = (unsigned short)(ci / K);
-      cis[i] = (unsigned short)ci;
+      rank_s[i] = 0;
     }
     __syncthreads();
     // Rank under the order (value desc, token asc, creation order). Every logits row contributed its K
-    // children already in that order, so the rank of a candidate is the number of children that come
-    // first, row by row: a lower-bound search per row (in its own row it finds its own position). Four
-    // neighbouring lanes share a candidate; a lane runs the searches of up to four rows in lockstep,
-    // branch-free, so their shared-memory loads overlap.
-    const int sub = tid & 3;
+    // children already in that order, so the rank of a candidate is, summed over the rows of its sequence,
+    // the number of that row's children that come first: one lower-bound search per (candidate, row) pair (in
+    // its own row it finds its own position). The pairs are spread densely over the threads - what this phase
+    // costs is the warp instructions it issues, so no lane works on a row or a step that does not exist - two
+    // per thread in step so that their shared-memory loads overlap; the counts meet in shared memory.
+    const int pairs = tot * n_prev;
+    int h0 = 1;
+    while (2 * h0 - 1 < K) h0 <<= 1;  // the search's first stride: positions up to 2 h0 - 1 >= K are reachable
 #pragma unroll 1
-    for (int i0 = 0; i0 < tot; i0 += nt / 4) {
-      const int i = i0 + (tid >> 2);
-      const bool act = i < tot;
-      const int ii = act ? i : 0;
-      const double s = sc[ii];
-      const int t = tk[ii];
-      const int r1 = r1s[ii], ci = cis[ii];
-      const int sbase = ii - ci;  // first candidate of the same sequence
-      int pos[4] = {0, 0, 0, 0};
+    for (int it0 = tid; it0 < pairs; it0 += 2 * nt) {
+      int ii[2], rs[2], rowb[2], r1[2], t2[2], pos[2] = {0, 0};
+      double s2[2];
+      bool act[2];
 #pragma unroll
-      for (int half = 16; half >= 1; half >>= 1) {
+      for (int q = 0; q < 2; ++q) {
+        const int it = it0 + q * nt;
+        act[q] = it < pairs;
+        const int itc = act[q] ? it : 0;
+        ii[q] = itc / n_prev;              // the candidate (index over the sequences of this pass)
+        rs[q] = itc - ii[q] * n_prev;      // the row searched
+        const int ci = ii[q] % Ni;
+        r1[q] = ci / K;                    // the candidate's own row
+        rowb[q] = ii[q] - ci + rs[q] * K;  // first child of the searched row, same sequence
+        s2[q] = sc[ii[q]];
+        t2[q] = tk[ii[q]];
+      }
+#pragma unroll 1
+      for (int half = h0; half >= 1; half >>= 1) {
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const int r2 = sub + 4 * q;
+        for (int q = 0; q < 2; ++q) {
           const int idx = pos[q] + half - 1;
-          const bool valid = r2 < n_prev && idx < K;
-          const int at = valid ? sbase + r2 * K + idx : ii;
+          const bool valid = idx < K;
+          const int at = rowb[q] + (valid ? idx : 0);
           const double sj = sc[at];
           const int tj = tk[at];
-          const bool first = valid && ((sj > s) || (sj == s && (tj < t || (tj == t && r2 < r1))));
+          const bool first = valid && ((sj > s2[q]) || (sj == s2[q] && (tj < t2[q] || (tj == t2[q] && rs[q] < r1[q]))));
           pos[q] += first ? half : 0;
         }
       }
-      int cnt = pos[0] + pos[1] + pos[2] + pos[3];
-      cnt += __shfl_xor_sync(0xffffffffu, cnt, 2);
-      cnt += __shfl_xor_sync(0xffffffffu, cnt, 1);
-      if (act && sub == 0) {
-        const int bg = b_begin + b0 + sbase / Ni, rank = cnt;
-        const size_t o = (size_t)bg * P + base + rank;
-        p.lsort[o] = base + ci;  // the layer's sorted list, for the rerank
-        p.lscore[o] = s;
-        if (rank < n) {
-          sorted_o[bg * CAST_MAX_WIDTH + rank] = base + ci;
-          stok_o[bg * CAST_MAX_WIDTH + rank] = t;
-          vs_o[bg * CAST_MAX_WIDTH + rank] = fast_exp_neg(s);
-        }
+#pragma unroll
+      for (int q = 0; q < 2; ++q)
+        if (act[q] && pos[q] != 0) atomicAdd(&rank_s[ii[q]], pos[q]);
+    }
+    __syncthreads();
+#pragma unroll 1
+    for (int i = tid; i < tot; i += nt) {
+      const int bl = i / Ni, ci = i - bl * Ni, rank = rank_s[i];
+      const int bg = b_begin + b0 + bl;
+      const double s = sc[i];
+      const size_t o = (size_t)bg * P + base + rank;
+      p.lsort[o] = base + ci;  // the layer's sorted list, for the rerank
+      p.lscore[o] = s;
+      if (rank < n) {
+        sorted_o[bg * CAST_MAX_WIDTH + rank] = base + ci;
+        stok_o[bg * CAST_MAX_WIDTH + rank] = tk[i];
+        vs_o[bg * CAST_MAX_WIDTH + rank] = fast_exp_neg(s);
       }
     }
     __syncthreads();
