@@ -204,9 +204,13 @@ CAST_API cast_status cast_reserve_attention(cast_ctx* ctx, cast_dtype dtype, int
  * the cache rows of the prefix (positions < kv_len[b]) were complete before that operation started (as they are in
  * a decoding loop: the tree is fixed for all layers of a step, and between two layers run the model's own kernels).
  * The kernel then decodes its work, reads the masks and fetches its first prefix tiles while its predecessor still
- * runs, and waits only before it loads q, a tile that reaches the tree tokens' rows, or writes output. Calls of
- * this library that write those inputs (cast_select_nodes, cast_compact_kv) are accounted for by the library: the
- * attention call that follows one of them takes no early reads. Needs bf16, D = 128 and a GQA group size that
+ * runs, and waits only before it loads q, a tile that reaches the tree tokens' rows, or writes output. It also
+ * reuses, from one attention call to the next, the work list it decoded from kv_len, n_tree and the call's shape:
+ * so the promise includes that kv_len, n_tree (and their pointers) keep their values between two attention calls
+ * unless a call of this library changed them. Calls of this library that write those inputs (cast_select_nodes,
+ * cast_compact_kv) or start a step (cast_step_begin) are accounted for by the library: the attention call that
+ * follows one of them decodes afresh and takes no early reads. A caller that changes the lengths or tree sizes by
+ * other means calls this function again (it discards the list). Needs bf16, D = 128 and a GQA group size that
  * divides 128; other shapes ignore the promise. promise = 0 (the default) restores the conservative behaviour.
  */
 CAST_API cast_status cast_set_attention_early_reads(cast_ctx* ctx, int promise);

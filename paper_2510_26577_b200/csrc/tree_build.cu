@@ -1071,6 +1071,7 @@ extern "C" cast_status cast_step_begin(cast_ctx* c, int B, const int32_t* root_t
   // the per-step state in its own kernel (one launch and one dependent round trip fewer per step).
   c->step_root = root_token;
   c->step_kv_len = kv_len;
+  c->tree_inputs_fresh = 1;  // a new step: the engine may have moved the lengths (an attention call decodes afresh)
   (void)stream;
   return CAST_OK;
 }
