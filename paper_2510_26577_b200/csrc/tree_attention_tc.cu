@@ -144,12 +144,18 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo_bytes
   return (uint64_t)((saddr & 0x3ffffu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
          (1ull << 46) | (2ull << 61);
 }
+// The MMA and commit wrappers are called by all 32 lanes of the issuing warp, converged, and elect the one
+// thread that issues inside: the operands are then warp-uniform values computed in convergent code, which the
+// compiler can keep in uniform registers. (Computed inside an `if (lane == 0)` block they took a chain of
+// vector-to-uniform moves per instruction: about 100 cycles per MMA, which made the issuing warp the
+// bottleneck of the tile loop.)
 // D[tmem] (+)= A[smem] * B[smem], bf16 inputs, fp32 accumulation.
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
+      "{\n\t.reg .pred p, q;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      "elect.sync _|q, 0xffffffff;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
       : "memory");
 }
@@ -157,15 +163,19 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
 // packed two to a 32-bit column, 8 columns per instruction) comes from tensor memory.
 __device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
+      "{\n\t.reg .pred p, q;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      "elect.sync _|q, 0xffffffff;\n\t"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
       ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(acc)
       : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-               : "memory");
+  asm volatile(
+      "{\n\t.reg .pred q;\n\t"
+      "elect.sync _|q, 0xffffffff;\n\t"
+      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(smem_u32(bar))
+      : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
   asm volatile(
@@ -224,6 +234,38 @@ __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+
+// Waits for this thread's tensor-memory loads and ties the wait to the registers they fill, so that no use of
+// them can be scheduled above it (a load may be issued long before its values are needed).
+__device__ __forceinline__ void tmem_wait_ld_regs(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+                 "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]),
+                 "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]),
+                 "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
+}
+// One half tile (32 scores of this thread's row, in registers) of the single-pass softmax: P = 2^(s * scale -
+// m * scale) as bf16 pairs, the row sum as a packed pair of partial sums. kMasked: `vv` holds the 32 visibility bits.
+template <bool kMasked>
+__device__ __forceinline__ void softmax_half(const uint32_t (&sr)[32], unsigned long long sc2, unsigned long long neg2,
+                                             uint32_t vv, unsigned long long& lacc, uint32_t (&pk)[16]) {
+#pragma unroll
+  for (int e = 0; e < 16; ++e) {
+    const int c = 2 * e;
+    float x0, x1;
+    unpack_f2(fma_f2(pack_f2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, neg2), x0, x1);
+    float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+    if (kMasked) {
+      p0 = ((vv >> c) & 1u) ? p0 : 0.f;
+      p1 = ((vv >> (c + 1)) & 1u) ? p1 : 0.f;
+    }
+    lacc = add_f2(lacc, pack_f2(p0, p1));
+    const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+    pk[e] = *reinterpret_cast<const uint32_t*>(&pb);
+  }
 }
 
 // 32 bits of the visibility vector of one query row, starting at tree index `start` (which may be
@@ -865,51 +907,61 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
     const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(kHD >> 3) << 17) |
                               ((uint32_t)(kBM >> 4) << 24);  // B operand (V) is MN-major, N = head dim
+    // Everything the issue loop computes with is made warp-uniform in the compiler's eyes (a warp reduction
+    // of values that are equal in all lanes anyway: the tile count comes from a load, the TMEM address from
+    // shared memory), and the ring positions are counters, not remainders: the loop then runs on the uniform
+    // datapath, where the MMA instructions take their operands.
+    const int ntile_u = __reduce_max_sync(0xffffffffu, ntile);
+    const uint32_t tmem_su = __reduce_or_sync(0xffffffffu, tmem_s), tmem_ou = tmem_su + 2 * kBN;
     // descriptors differ only in the start-address field (16-byte units), so they are built once
     const uint64_t dq = umma_desc(smem_u32(smem + kSmemQ), 16, 1024);
     const uint64_t dk = umma_desc(smem_u32(smem + kSmemK), 16, 1024);
     const uint64_t dv = umma_desc(smem_u32(smem + kSmemV), kRegionKV, 1024);
-    auto mma_qk = [&](int stage, int buf) {  // S[buf] = Q K^T; releases the K stage
-      if (lane == 0) {
-        const uint64_t dks = dk + (uint64_t)(stage * (kTileKV >> 4));
+    auto mma_qk = [&](int stage, int buf) {  // S[buf] = Q K^T; releases the K stage (all lanes, converged)
+      const uint64_t dks = dk + (uint64_t)(stage * (kTileKV >> 4));
 #pragma unroll
-        for (int ks = 0; ks < kHD / 16; ++ks)
-          umma_bf16(tmem_s + buf * kBN, dq + (uint64_t)((ks >> 2) * (kRegionQ >> 4) + (ks & 3) * 2),
-                    dks + (uint64_t)((ks >> 2) * (kRegionKV >> 4) + (ks & 3) * 2), idesc_qk, ks > 0);
-        umma_commit(&bar_s[buf]);
-        umma_commit(&bar_freek[stage]);
-      }
-      __syncwarp();
+      for (int ks = 0; ks < kHD / 16; ++ks)
+        umma_bf16(tmem_su + buf * kBN, dq + (uint64_t)((ks >> 2) * (kRegionQ >> 4) + (ks & 3) * 2),
+                  dks + (uint64_t)((ks >> 2) * (kRegionKV >> 4) + (ks & 3) * 2), idesc_qk, ks > 0);
+      umma_commit(&bar_s[buf]);
+      umma_commit(&bar_freek[stage]);
     };
     auto mma_pv = [&](int stage, int buf, bool first) {  // O (+)= P V, P from tensor memory; releases the V stage
-      if (lane == 0) {
-        const uint64_t dvs = dv + (uint64_t)(stage * (kTileKV >> 4));
+      const uint64_t dvs = dv + (uint64_t)(stage * (kTileKV >> 4));
 #pragma unroll
-        for (int ks = 0; ks < kBN / 16; ++ks)
-          umma_bf16_ts(tmem_o, tmem_s + buf * kBN + ks * 8, dvs + (uint64_t)(ks * (2048 >> 4)), idesc_pv,
-                       (!first || ks > 0) ? 1u : 0u);
-        umma_commit(&bar_freev[stage]);
-      }
-      __syncwarp();
+      for (int ks = 0; ks < kBN / 16; ++ks)
+        umma_bf16_ts(tmem_ou, tmem_su + buf * kBN + ks * 8, dvs + (uint64_t)(ks * (2048 >> 4)), idesc_pv,
+                     (!first || ks > 0) ? 1u : 0u);
+      umma_commit(&bar_freev[stage]);
     };
     // next scores first: Q K^T of tile it+1 runs while the softmax of tile `it` does; the other CTA on
     // this SM covers the moments when a K tile is late
-    bool ok = ntile == 0 || ((!p.q_tma || mbar_wait(bar_q, 0)) && mbar_wait(&bar_fullk[0], 0));
-    if (ok && ntile > 0) {
+    bool ok = ntile_u == 0 || ((!p.q_tma || mbar_wait(bar_q, 0)) && mbar_wait(&bar_fullk[0], 0));
+    if (ok && ntile_u > 0) {
       tc_fence_after();
       mma_qk(0, 0);
     }
-    for (int it = 0; ok && it < ntile; ++it) {
-      if (it + 1 < ntile) {
-        ok = mbar_wait(&bar_fullk[(it + 1) % kStagesK], ((it + 1) / kStagesK) & 1);
+    int ks1 = 1 % kStagesK, kp1 = (1 / kStagesK) & 1;  // K ring position and phase of tile it+1
+    int vs0 = 0, vp0 = 0;                              // V ring position and phase of tile it
+    for (int it = 0; ok && it < ntile_u; ++it) {
+      if (it + 1 < ntile_u) {
+        ok = mbar_wait(&bar_fullk[ks1], (uint32_t)kp1);
         if (!ok) break;
         tc_fence_after();
-        mma_qk((it + 1) % kStagesK, (it + 1) & 1);
+        mma_qk(ks1, (it + 1) & 1);
+        if (++ks1 == kStagesK) {
+          ks1 = 0;
+          kp1 ^= 1;
+        }
       }
-      ok = mbar_wait(&bar_p[it & 1], (it >> 1) & 1) && mbar_wait(&bar_fullv[it % kStagesV], (it / kStagesV) & 1);
+      ok = mbar_wait(&bar_p[it & 1], (it >> 1) & 1) && mbar_wait(&bar_fullv[vs0], (uint32_t)vp0);
       if (!ok) break;
       tc_fence_after();
-      mma_pv(it % kStagesV, it & 1, it == 0);
+      mma_pv(vs0, it & 1, it == 0);
+      if (++vs0 == kStagesV) {
+        vs0 = 0;
+        vp0 ^= 1;
+      }
     }
     if (!ok && lane == 0) report(p.st, CAST_ERR_TIMEOUT, b);
   } else if (warp < 4) {
@@ -922,135 +974,34 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     const float sc = p.scale_log2;
     float m_used = -INFINITY, l_run = 0.f;  // m_used: running reference maximum in raw score units
     bool ok = true;
-    for (int it = 0; it < ntile; ++it) {
-      const int buf = it & 1, stage = it % kStagesV;
+    // V rows past the end of the sequence may hold anything (0 * NaN would poison O): zero them (last tile only)
+    auto zero_v_tail = [&](int it) {
+      const int pos0 = (t0 + it) * kBN, stage = it % kStagesV;
+      if (ok && total - pos0 < kBN) {
+        ok = mbar_wait(&bar_fullv[stage], (it / kStagesV) & 1);  // the tile has landed
+        if (ok) {
+          const int valid = total - pos0;
+          unsigned char* vbase = smem + kSmemV + stage * kTileKV;
+          for (int i = tid; i < (kBN - valid) * 16; i += kSoftmaxThreads) {
+            const int rr = valid + (i >> 4), reg = (i >> 3) & 1, c = i & 7;
+            *reinterpret_cast<uint4*>(vbase + reg * kRegionKV + rr * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
+          }
+        }
+      }
+    };
+    // ---- Two-pass tiles: the first tile of a piece, and any tile while a row of the warp has seen nothing
+    // visible yet (its reference maximum is still -inf). A warp without live rows stays in this loop.
+    int it = 0;
+    for (; it < ntile; ++it) {
+      if (warp_live && ok && it > 0 && __all_sync(0xffffffffu, m_used > -INFINITY || !row_ok)) break;
+      const int buf = it & 1;
       const int pos0 = (t0 + it) * kBN;
       float mx = -INFINITY;
       uint32_t v0 = 0xffffffffu, v1 = 0xffffffffu;  // visibility of this row's 64 columns
-      // Fast path (every tile but the first, as a rule): one pass over the scores with the reference
-      // maximum of the earlier tiles. P = 2^((s - m) * scale) is then not bounded by 1, but bf16 and the
-      // fp32 accumulators have the range for it; a row whose P would outgrow 2^60 in a half tile moves its
-      // reference before that half is written (see below).
       // P is written over the scores it came from, in tensor memory: 64 bf16 = 32 columns of this row's
       // lane; P V takes its A operand from there.
-      bool done = false;
       const uint32_t tp = tmem_s + buf * kBN + lane_sel;
-      if (warp_live && ok && it > 0 && __all_sync(0xffffffffu, m_used > -INFINITY || !row_ok)) {
-        // Nothing but the scores is awaited: P goes into the score buffer it came from, and that buffer
-        // was last read by P V of tile it-2, which the tensor pipe finished before it produced these
-        // scores. So the softmax of this tile runs while P V of the previous one does.
-        ok = mbar_wait(&bar_s[buf], (it >> 1) & 1);
-        if (ok) {
-          tc_fence_after();
-          const bool plain = pos0 + kBN <= L && __all_sync(0xffffffffu, row_ok);  // nothing masked in this warp
-          if (!plain) {
-            if (pos0 + kBN > L) {
-              v0 = vis_bits32(aw, pos0 - L);
-              v1 = vis_bits32(aw, pos0 - L + 32);
-            }
-            if (!row_ok) v0 = v1 = 0u;
-          }
-          float neg_ms = row_ok ? -m_used * sc : 0.f;
-          const unsigned long long sc2 = pack_f2(sc, sc);
-          uint32_t pk[2][16];
-          unsigned long long lacc = pack_f2(0.f, 0.f);
-          {
-            const unsigned long long neg2 = pack_f2(neg_ms, neg_ms);
-#pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-              uint32_t sr[32];
-              tmem_ld32(tp + hh * 32, sr);
-              tmem_wait_ld();
-              const uint32_t vv = hh ? v1 : v0;
-#pragma unroll
-              for (int e = 0; e < 16; ++e) {
-                const int c = 2 * e;
-                float x0, x1;
-                unpack_f2(fma_f2(pack_f2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, neg2), x0, x1);
-                float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
-                if (!plain) {
-                  p0 = ((vv >> c) & 1u) ? p0 : 0.f;
-                  p1 = ((vv >> (c + 1)) & 1u) ? p1 : 0.f;
-                }
-                lacc = add_f2(lacc, pack_f2(p0, p1));
-                const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
-                pk[hh][e] = *reinterpret_cast<const uint32_t*>(&pb);
-              }
-            }
-          }
-          float l0, l1;
-          unpack_f2(lacc, l0, l1);
-          // A score far above the reference (a P beyond 2^60, or past the range of the exponential: the sum is
-          // then inf) is rare. Nothing of this tile has been written yet, so its scores are intact in tensor
-          // memory: the rows concerned move their reference up by a whole number of powers of two (what is
-          // already accumulated - O and the running sum - is scaled by 2^-k, which is exact) and the tile is
-          // evaluated again.
-          const bool far = !(l0 + l1 < 1.15e18f);
-          if (__any_sync(0xffffffffu, far)) {
-            ok = mbar_wait(&bar_freev[(it - 1) % kStagesV], ((it - 1) / kStagesV) & 1);  // O must be at rest
-            if (ok) {
-              tc_fence_after();
-              float alpha = 1.f, mxt = -INFINITY;
-#pragma unroll 1
-              for (int hh = 0; hh < 2; ++hh) {
-                uint32_t sr[32];
-                tmem_ld32(tp + hh * 32, sr);
-                tmem_wait_ld();
-                const uint32_t vv = hh ? v1 : v0;
-#pragma unroll
-                for (int c = 0; c < 32; ++c)
-                  mxt = fmaxf(mxt, (plain || ((vv >> c) & 1u)) ? __uint_as_float(sr[c]) : -INFINITY);
-              }
-              if (far && mxt > -INFINITY && mxt < INFINITY) {
-                float kf = ceilf(fmaf(mxt, sc, neg_ms));  // the tile's largest exponent, rounded up
-                kf = kf < 0.f ? 0.f : (kf > 1.0e9f ? 1.0e9f : kf);
-                alpha = ldexpf(1.f, -(int)kf);  // 0 beyond the range: what came before no longer counts
-                neg_ms -= kf;
-                m_used += kf / sc;
-              }
-#pragma unroll 1
-              for (int q4 = 0; q4 < 4; ++q4) {  // O and the running sum follow (P V of tile it-1 is over)
-                uint32_t orr[32];
-                const uint32_t ta = tmem_o + lane_sel + q4 * 32;
-                tmem_ld32(ta, orr);
-                tmem_wait_ld();
-#pragma unroll
-                for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
-                tmem_st32(ta, orr);
-              }
-              l_run *= alpha;
-              l0 = l1 = 0.f;
-#pragma unroll
-              for (int hh = 0; hh < 2; ++hh) {  // the tile again (rows that did not move get the same values)
-                uint32_t sr[32];
-                tmem_ld32(tp + hh * 32, sr);
-                tmem_wait_ld();
-                const uint32_t vv = hh ? v1 : v0;
-#pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                  const int c = 2 * e;
-                  float p0 = fast_exp2(fmaf(__uint_as_float(sr[c]), sc, neg_ms));
-                  float p1 = fast_exp2(fmaf(__uint_as_float(sr[c + 1]), sc, neg_ms));
-                  if (!plain) {
-                    p0 = ((vv >> c) & 1u) ? p0 : 0.f;
-                    p1 = ((vv >> (c + 1)) & 1u) ? p1 : 0.f;
-                  }
-                  l0 += p0;
-                  l1 += p1;
-                  const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
-                  pk[hh][e] = *reinterpret_cast<const uint32_t*>(&pb);
-                }
-              }
-            }
-          }
-          tmem_st16(tp, pk[0]);
-          tmem_st16(tp + 16, pk[1]);
-          tmem_wait_st();
-          l_run += l0 + l1;
-          done = true;
-        }
-      }
-      if (warp_live && !done) {
+      if (warp_live) {
         if (ok) ok = mbar_wait(&bar_s[buf], (it >> 1) & 1);
         if (ok) {
           tc_fence_after();
@@ -1079,80 +1030,195 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
           }
         }
       }
-      // The two-pass path may rescale O, which P V of tile it-1 must have left. A warp without live rows
+      // This path may rescale O, which P V of tile it-1 must have left. A warp without live rows
       // only has to stay in step: it waits for this tile's scores like the others, so that it cannot
       // arrive on bar_p[it & 1] before the phase of tile it-2 is over.
-      if (ok && it >= 1 && !(warp_live && done)) {
+      if (ok && it >= 1) {
         ok = warp_live ? mbar_wait(&bar_freev[(it - 1) % kStagesV], ((it - 1) / kStagesV) & 1)
                        : mbar_wait(&bar_s[buf], (it >> 1) & 1);
       }
-      if (warp_live && !done) {
-        if (ok) {
-          // lazy maximum: move the reference only when the row maximum outgrows it by 2^8
-          float alpha = 1.f;
-          const bool grow = (mx - m_used) * sc > kRescaleThreshold || (m_used == -INFINITY && mx > -INFINITY);
-          if (grow) {
-            alpha = fast_exp2((m_used - mx) * sc);  // 0 when m_used = -inf
-            m_used = mx;
-            l_run *= alpha;
-          }
-          if (it > 0 && __any_sync(0xffffffffu, grow)) {  // rescale this row of O
-            tc_fence_after();
+      if (warp_live && ok) {
+        // lazy maximum: move the reference only when the row maximum outgrows it by 2^8
+        float alpha = 1.f;
+        const bool grow = (mx - m_used) * sc > kRescaleThreshold || (m_used == -INFINITY && mx > -INFINITY);
+        if (grow) {
+          alpha = fast_exp2((m_used - mx) * sc);  // 0 when m_used = -inf
+          m_used = mx;
+          l_run *= alpha;
+        }
+        if (it > 0 && __any_sync(0xffffffffu, grow)) {  // rescale this row of O
+          tc_fence_after();
 #pragma unroll
-            for (int hh = 0; hh < 4; ++hh) {
+          for (int hh = 0; hh < 4; ++hh) {
+            uint32_t orr[32];
+            const uint32_t ta = tmem_o + lane_sel + hh * 32;
+            tmem_ld32(ta, orr);
+            tmem_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
+            tmem_st32(ta, orr);
+          }
+          tmem_wait_st();
+        }
+        // pass 2: P = 2^((s - m) * scale) as bf16 over the scores in tensor memory; row sum in fp32
+        const bool live = m_used > -INFINITY;
+        const float neg_ms = live ? -m_used * sc : 0.f;
+        float l0 = 0.f, l1 = 0.f;
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+          uint32_t sr[32], pk[16];
+          tmem_ld32(tp + hh * 32, sr);
+          tmem_wait_ld();
+          const uint32_t vv = live ? (hh ? v1 : v0) : 0u;
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const int c = 2 * e;
+            float p0 = fast_exp2(fmaf(__uint_as_float(sr[c]), sc, neg_ms));
+            float p1 = fast_exp2(fmaf(__uint_as_float(sr[c + 1]), sc, neg_ms));
+            p0 = ((vv >> c) & 1u) ? p0 : 0.f;
+            p1 = ((vv >> (c + 1)) & 1u) ? p1 : 0.f;
+            l0 += p0;
+            l1 += p1;
+            const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+            pk[e] = *reinterpret_cast<const uint32_t*>(&pb);
+          }
+          tmem_st16(tp + hh * 16, pk);
+        }
+        tmem_wait_st();
+        l_run += l0 + l1;
+      }
+      zero_v_tail(it);
+      fence_proxy_async();
+      tc_fence_before();
+      mbar_arrive(&bar_p[it & 1]);
+    }
+    // ---- Single-pass tiles (all the others, as a rule): one pass over the scores with the reference
+    // maximum of the earlier tiles. P = 2^((s - m) * scale) is then not bounded by 1, but bf16 and the
+    // fp32 accumulators have the range for it; a row whose P would outgrow 2^60 in a tile moves its
+    // reference before the tile is written (see below). Nothing but the scores is awaited: P goes into the
+    // score buffer it came from, and that buffer was last read by P V of tile it-2, which the tensor pipe
+    // finished before it produced these scores. So the softmax of this tile runs while P V of the previous
+    // one does.
+    // The second half of a tile's scores is loaded while the first half is computed. (Loading the next tile's
+    // first half ahead as well, or handing P over later, was tried in several forms and lost each time: what
+    // bounds the loop is the round trip between this hand-over and the next scores, see the MMA issuer.)
+    // Once a warp is here it stays: the reference maxima only grow.
+    if (it < ntile) {
+      const unsigned long long sc2 = pack_f2(sc, sc);
+      for (; it < ntile; ++it) {
+        uint32_t sra[32];
+        if (ok) {
+          ok = mbar_wait(&bar_s[it & 1], (it >> 1) & 1);
+          if (ok) {
+            tc_fence_after();
+            tmem_ld32(tmem_s + (it & 1) * kBN + lane_sel, sra);
+          }
+        }
+        if (!ok) {  // a wait ran out: keep the barriers in step and nothing else
+          tc_fence_before();
+          mbar_arrive(&bar_p[it & 1]);
+          continue;
+        }
+        const int buf = it & 1;
+        const int pos0 = (t0 + it) * kBN;
+        const uint32_t tp = tmem_s + buf * kBN + lane_sel;
+        const bool plain = pos0 + kBN <= L;  // wholly inside the prefix: nothing masked (rows past the tree: see neg_ms)
+        uint32_t v0 = 0xffffffffu, v1 = 0xffffffffu;  // visibility of this row's 64 columns
+        if (!plain) {
+          v0 = vis_bits32(aw, pos0 - L);
+          v1 = vis_bits32(aw, pos0 - L + 32);
+          if (!row_ok) v0 = v1 = 0u;
+        }
+        // a row past the tree takes -inf: its P is 0 for every finite score, with no masking
+        float neg_ms = row_ok ? -m_used * sc : -INFINITY;
+        uint32_t pk[2][16];
+        unsigned long long lacc = pack_f2(0.f, 0.f);
+        {
+          const unsigned long long neg2 = pack_f2(neg_ms, neg_ms);
+          uint32_t srb[32];
+          // Two copies of the arithmetic behind one warp-uniform branch: written as a test inside the loop the
+          // masking was compiled into selects that every tile paid for (two instructions per score on
+          // top of five per pair), and all tiles but the last one or two are unmasked.
+          tmem_wait_ld_regs(sra);
+          tmem_ld32(tp + 32, srb);  // in flight while the first half is computed
+          if (plain) softmax_half<false>(sra, sc2, neg2, 0u, lacc, pk[0]);
+          else softmax_half<true>(sra, sc2, neg2, v0, lacc, pk[0]);
+          tmem_wait_ld_regs(srb);
+          if (plain) softmax_half<false>(srb, sc2, neg2, 0u, lacc, pk[1]);
+          else softmax_half<true>(srb, sc2, neg2, v1, lacc, pk[1]);
+        }
+        float l0, l1;
+        unpack_f2(lacc, l0, l1);
+        // A score far above the reference (a P beyond 2^60, or past the range of the exponential: the sum is
+        // then inf) is rare. Nothing of this tile has been written yet, so its scores are intact in tensor
+        // memory: the rows concerned move their reference up by a whole number of powers of two (what is
+        // already accumulated - O and the running sum - is scaled by 2^-k, which is exact) and the tile is
+        // evaluated again.
+        const bool far = row_ok && !(l0 + l1 < 1.15e18f);
+        if (__any_sync(0xffffffffu, far)) {
+          ok = mbar_wait(&bar_freev[(it - 1) % kStagesV], ((it - 1) / kStagesV) & 1);  // O must be at rest
+          if (ok) {
+            tc_fence_after();
+            float alpha = 1.f, mxt = -INFINITY;
+#pragma unroll 1
+            for (int hh = 0; hh < 2; ++hh) {
+              uint32_t sr[32];
+              tmem_ld32(tp + hh * 32, sr);
+              tmem_wait_ld();
+              const uint32_t vv = hh ? v1 : v0;
+#pragma unroll
+              for (int c = 0; c < 32; ++c)  // (`plain ||`: v0 / v1 then stay out of the unmasked path's live registers)
+                mxt = fmaxf(mxt, (plain || ((vv >> c) & 1u)) ? __uint_as_float(sr[c]) : -INFINITY);
+            }
+            if (far && mxt > -INFINITY && mxt < INFINITY) {
+              float kf = ceilf(fmaf(mxt, sc, neg_ms));  // the tile's largest exponent, rounded up
+              kf = kf < 0.f ? 0.f : (kf > 1.0e9f ? 1.0e9f : kf);
+              alpha = ldexpf(1.f, -(int)kf);  // 0 beyond the range: what came before no longer counts
+              neg_ms -= kf;
+              m_used += kf / sc;
+            }
+#pragma unroll 1
+            for (int q4 = 0; q4 < 4; ++q4) {  // O and the running sum follow (P V of tile it-1 is over)
               uint32_t orr[32];
-              const uint32_t ta = tmem_o + lane_sel + hh * 32;
+              const uint32_t ta = tmem_o + lane_sel + q4 * 32;
               tmem_ld32(ta, orr);
               tmem_wait_ld();
 #pragma unroll
               for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
               tmem_st32(ta, orr);
             }
-            tmem_wait_st();
-          }
-          // pass 2: P = 2^((s - m) * scale) as bf16 over the scores in tensor memory; row sum in fp32
-          const bool live = m_used > -INFINITY;
-          const float neg_ms = live ? -m_used * sc : 0.f;
-          float l0 = 0.f, l1 = 0.f;
+            l_run *= alpha;
+            l0 = l1 = 0.f;
 #pragma unroll
-          for (int hh = 0; hh < 2; ++hh) {
-            uint32_t sr[32], pk[16];
-            tmem_ld32(tp + hh * 32, sr);
-            tmem_wait_ld();
-            const uint32_t vv = live ? (hh ? v1 : v0) : 0u;
+            for (int hh = 0; hh < 2; ++hh) {  // the tile again (rows that did not move get the same values)
+              uint32_t sr[32];
+              tmem_ld32(tp + hh * 32, sr);
+              tmem_wait_ld();
+              const uint32_t vv = plain ? 0xffffffffu : (hh ? v1 : v0);
 #pragma unroll
-            for (int e = 0; e < 16; ++e) {
-              const int c = 2 * e;
-              float p0 = fast_exp2(fmaf(__uint_as_float(sr[c]), sc, neg_ms));
-              float p1 = fast_exp2(fmaf(__uint_as_float(sr[c + 1]), sc, neg_ms));
-              p0 = ((vv >> c) & 1u) ? p0 : 0.f;
-              p1 = ((vv >> (c + 1)) & 1u) ? p1 : 0.f;
-              l0 += p0;
-              l1 += p1;
-              const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
-              pk[e] = *reinterpret_cast<const uint32_t*>(&pb);
+              for (int e = 0; e < 16; ++e) {
+                const int c = 2 * e;
+                float p0 = fast_exp2(fmaf(__uint_as_float(sr[c]), sc, neg_ms));
+                float p1 = fast_exp2(fmaf(__uint_as_float(sr[c + 1]), sc, neg_ms));
+                p0 = ((vv >> c) & 1u) ? p0 : 0.f;
+                p1 = ((vv >> (c + 1)) & 1u) ? p1 : 0.f;
+                l0 += p0;
+                l1 += p1;
+                const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+                pk[hh][e] = *reinterpret_cast<const uint32_t*>(&pb);
+              }
             }
-            tmem_st16(tp + hh * 16, pk);
-          }
-          tmem_wait_st();
-          l_run += l0 + l1;
-        }
-      }
-      // V rows past the end of the sequence may hold anything (0 * NaN would poison O): zero them
-      if (ok && total - pos0 < kBN) {
-        ok = mbar_wait(&bar_fullv[stage], (it / kStagesV) & 1);  // the tile has landed
-        if (ok) {
-          const int valid = total - pos0;
-          unsigned char* vbase = smem + kSmemV + stage * kTileKV;
-          for (int i = tid; i < (kBN - valid) * 16; i += kSoftmaxThreads) {
-            const int rr = valid + (i >> 4), reg = (i >> 3) & 1, c = i & 7;
-            *reinterpret_cast<uint4*>(vbase + reg * kRegionKV + rr * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
           }
         }
+        tmem_st16(tp, pk[0]);
+        tmem_st16(tp + 16, pk[1]);
+        l_run += l0 + l1;
+        tmem_wait_st();
+        zero_v_tail(it);
+        fence_proxy_async();
+        tc_fence_before();
+        mbar_arrive(&bar_p[it & 1]);
       }
-      fence_proxy_async();
-      tc_fence_before();
-      mbar_arrive(&bar_p[it & 1]);
     }
     // epilogue: wait for the last P V, then stage O (fp32, unnormalised) and (max, sum) per row in
     // shared memory (the K/V rings, P and Q are idle now): the output rows are written, or merged
