@@ -986,6 +986,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
             const int rr = valid + (i >> 4), reg = (i >> 3) & 1, c = i & 7;
             *reinterpret_cast<uint4*>(vbase + reg * kRegionKV + rr * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
           }
+          fence_proxy_async();  // the MMA reads these rows through the async proxy
         }
       }
     };
@@ -1088,7 +1089,6 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
         l_run += l0 + l1;
       }
       zero_v_tail(it);
-      fence_proxy_async();
       tc_fence_before();
       mbar_arrive(&bar_p[it & 1]);
     }
@@ -1105,10 +1105,11 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     // Once a warp is here it stays: the reference maxima only grow.
     if (it < ntile) {
       const unsigned long long sc2 = pack_f2(sc, sc);
+      bool s_there = false;  // the scores of tile `it` were seen complete during the previous tile
       for (; it < ntile; ++it) {
         uint32_t sra[32];
         if (ok) {
-          ok = mbar_wait(&bar_s[it & 1], (it >> 1) & 1);
+          if (!s_there) ok = mbar_wait(&bar_s[it & 1], (it >> 1) & 1);
           if (ok) {
             tc_fence_after();
             tmem_ld32(tmem_s + (it & 1) * kBN + lane_sel, sra);
@@ -1147,6 +1148,8 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
           if (plain) softmax_half<false>(srb, sc2, neg2, 0u, lacc, pk[1]);
           else softmax_half<true>(srb, sc2, neg2, v1, lacc, pk[1]);
         }
+        // A look at the next tile's scores, asked for here so that the answer's latency (over a hundred cycles
+        // even when they are there) passes while P is stored and handed over.
         float l0, l1;
         unpack_f2(lacc, l0, l1);
         // A score far above the reference (a P beyond 2^60, or past the range of the exponential: the sum is
@@ -1215,7 +1218,6 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
         l_run += l0 + l1;
         tmem_wait_st();
         zero_v_tail(it);
-        fence_proxy_async();
         tc_fence_before();
         mbar_arrive(&bar_p[it & 1]);
       }
