@@ -762,6 +762,10 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
   uint64_t* bar_q = bars + 15;         // the Q row block has landed (TMA)
 
   // ---- producer helper (warp 4; all 32 lanes call it): which = 0: K tile j, which = 1: V tile j
+  // Paged caches: a producer warp reads the page table 32 entries at a time (one coalesced load, lane l keeps
+  // entry win0 + l) and hands the ids of a tile's pages out by shuffle: one round trip to memory per 32 / (pages
+  // per tile) tiles instead of one per tile, which the tile's copies had to wait for.
+  int pg_win0 = -0x40000000, pg_id = 0;
   auto issue_tile = [&](int j, int which) -> bool {
     const int stages = which ? kStagesV : kStagesK, stage = j % stages;
     unsigned char* dst = smem + (which ? kSmemV : kSmemK) + stage * kTileKV;
@@ -770,12 +774,17 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     const int pos0 = (t0 + j) * kBN;
     const int ps = p.page_size;
     int npages = 0, page = 0;
-    if (ps != 0) {  // page ids are fetched before the stage is awaited: their latency hides behind the wait
-      const int ppt = kBN / ps;
+    if (ps != 0) {
+      const int ppt = kBN / ps, e0 = pos0 / ps;  // the tile's first page-table entry
       npages = (total - pos0 + ps - 1) / ps;
       npages = npages > ppt ? ppt : npages;
+      if (e0 < pg_win0 || e0 + ppt > pg_win0 + 32) {  // (warp-uniform)
+        pg_win0 = e0;
+        pg_id = e0 + lane < p.seq_capacity ? p.page_table[(size_t)b * p.seq_capacity + e0 + lane] : 0;
+      }
+      const int pg = __shfl_sync(0xffffffffu, pg_id, e0 - pg_win0 + (lane >> 1));
       if (lane < npages * 2) {
-        page = p.page_table[(size_t)b * p.seq_capacity + pos0 / ps + (lane >> 1)];
+        page = pg;
         if (page < 0 || page >= p.num_pages) {
           report(p.st, CAST_ERR_BAD_PAGE, b);
           page = 0;
