@@ -10,7 +10,8 @@
 //                  halves each) into the two rings; a K stage is released as soon as Q K^T has
 //                  consumed it, a V stage after P V. (One warp for both rings stalled the K loads
 //                  behind waits for V stages: the paged batch-64 case went from 142 to 114 us with two.)
-//   MMA issuer   : S = Q K^T by tcgen05.mma (M=128 rows, N=64 positions, K=128) into one of two
+//   MMA issuer   : (the whole warp runs the issue loop converged; every MMA / commit elects its one thread)
+//                  S = Q K^T by tcgen05.mma (M=128 rows, N=64 positions, K=128) into one of two
 //                  TMEM buffers; once the softmax warps have written P, O += P V with P taken
 //                  from tensor memory (A operand in TMEM) and V as the MN-major B operand: used
 //                  exactly as it lies in the cache, no transpose. Q K^T of tile i+1 is issued
@@ -1114,11 +1115,10 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     // Once a warp is here it stays: the reference maxima only grow.
     if (it < ntile) {
       const unsigned long long sc2 = pack_f2(sc, sc);
-      bool s_there = false;  // the scores of tile `it` were seen complete during the previous tile
       for (; it < ntile; ++it) {
         uint32_t sra[32];
         if (ok) {
-          if (!s_there) ok = mbar_wait(&bar_s[it & 1], (it >> 1) & 1);
+          ok = mbar_wait(&bar_s[it & 1], (it >> 1) & 1);
           if (ok) {
             tc_fence_after();
             tmem_ld32(tmem_s + (it & 1) * kBN + lane_sel, sra);
