@@ -449,6 +449,12 @@ def test_attention_arbitrary_trees_ragged(binding, dtype, D, Hq, Hkv, page):
         else:
             k[b, end:] = float("nan")
             v[b, end:] = float("nan")
+    # so may the query rows of tokens past the tree (they share 128-row blocks with live rows): NaN, inf, huge
+    for b in range(B):
+        nb = int(n_tree[b])
+        q[b, nb::3] = float("nan")
+        q[b, nb + 1::3] = float("inf")
+        q[b, nb + 2::3] = 3.0e38
     out = gpu_attention(ctx, w, q, k, v, table, num_pages, kv, anc, nt, scale=0.0)
     assert ctx.cast_poll_status()[0] == 0
     f32 = lambda t: t.float().cpu().numpy()
