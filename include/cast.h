@@ -221,7 +221,8 @@ CAST_API cast_status cast_set_attention_early_reads(cast_ctx* ctx, int promise);
  * kv_len[b]+j : bit j of anc_mask[b,t]} of (q . k) * scale, times v, for
  * t < n_tree[b]; rows t >= n_tree[b] of `out` are left untouched.
  * n_tree[b] must not exceed the context's total_token (device error BAD_TREE).
- *   q, out        [B, Ncap, Hq, D], dtype `dtype`
+ *   q, out        [B, Ncap, Hq, D], dtype `dtype`; rows t >= n_tree[b] of q may hold anything (NaN and
+ *                 inf included): they may be loaded with their neighbours but reach no output
  *   k_cache, v_cache  paged: [num_pages, page_size, Hkv, D]; the cache rows of
  *                 the tree tokens are already stored at positions kv_len[b]+j.
  *                 page_size = 0: contiguous [B, seq_capacity, Hkv, D].
