@@ -19,9 +19,9 @@
 //   4 softmax warps: one thread per query row reads its 64 scores with tcgen05.ld, applies the
 //                  prefix/ancestor mask (only tiles that reach past the prefix need one) and
 //                  writes P = 2^((s - m) * scale) as bf16 over the scores, in tensor memory
-//                  (tcgen05.st). The first tile takes two passes (row maximum, then P); later
-//                  tiles one pass with the reference maximum of the earlier ones (O in TMEM is
-//                  rescaled only if a row's P outgrows 2^60, by a power of two).
+//                  (tcgen05.st). Every tile takes one pass: the row's reference m starts at 0 and
+//                  moves (by a power of two, O in TMEM rescaled with it) only when a row's P would
+//                  leave the range 2^-60 .. 2^60.
 // The kernel is launched in thread-block clusters: a cluster covers the row blocks of one
 // (sequence, kv-head) and splits each one's KV range over its CTAs, the number of splits per row
 // block being decided on the device from the actual tree size (the host only knows the largest
@@ -57,7 +57,6 @@ constexpr int kSmemV = kSmemK + kStagesK * kTileKV;  // kStagesV tiles
 constexpr int kSmemBar = kSmemV + kStagesV * kTileKV;  // mbarriers and two words, 128 bytes
 constexpr int kSmemBytes = kSmemBar + 128;           // 112 KB + 128 B: two CTAs per SM
 constexpr int kTmemCols = 256;                     // S0: [0,64), S1: [64,128), O: [128,256)
-constexpr float kRescaleThreshold = 8.0f;          // log2 units
 constexpr long long kWaitCycles = 4000000000ll;    // about two seconds
 constexpr int kMaxSplit = 8;
 
@@ -982,7 +981,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     const uint32_t lane_sel = (uint32_t)(warp * 32) << 16;
     const bool warp_live = row0 + warp * 32 < rows_total;
     const float sc = p.scale_log2;
-    float m_used = -INFINITY, l_run = 0.f;  // m_used: running reference maximum in raw score units
+    float m_used = -INFINITY, l_run = 0.f;  // m_used: the row's reference in raw score units (see below)
     bool ok = true;
     // V rows past the end of the sequence may hold anything (0 * NaN would poison O): zero them (last tile only)
     auto zero_v_tail = [&](int it) {
@@ -1000,122 +999,36 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
         }
       }
     };
-    // ---- Two-pass tiles: the first tile of a piece, and any tile while a row of the warp has seen nothing
-    // visible yet (its reference maximum is still -inf). A warp without live rows stays in this loop.
-    int it = 0;
-    for (; it < ntile; ++it) {
-      if (warp_live && ok && it > 0 && __all_sync(0xffffffffu, m_used > -INFINITY || !row_ok)) break;
-      const int buf = it & 1;
-      const int pos0 = (t0 + it) * kBN;
-      float mx = -INFINITY;
-      uint32_t v0 = 0xffffffffu, v1 = 0xffffffffu;  // visibility of this row's 64 columns
-      // P is written over the scores it came from, in tensor memory: 64 bf16 = 32 columns of this row's
-      // lane; P V takes its A operand from there.
-      const uint32_t tp = tmem_s + buf * kBN + lane_sel;
-      if (warp_live) {
-        if (ok) ok = mbar_wait(&bar_s[buf], (it >> 1) & 1);
-        if (ok) {
-          tc_fence_after();
-          if (pos0 + kBN > L) {  // the tile reaches past the prefix: ancestor mask
-            v0 = vis_bits32(aw, pos0 - L);
-            v1 = vis_bits32(aw, pos0 - L + 32);
-          }
-          if (!row_ok) v0 = v1 = 0u;
-          // pass 1: the row maximum (the scores are read again from TMEM in pass 2: registers are scarce
-          // with two CTAs per SM, TMEM bandwidth is not)
-#pragma unroll
-          for (int hh = 0; hh < 2; ++hh) {
-            uint32_t sr[32];
-            tmem_ld32(tmem_s + buf * kBN + lane_sel + hh * 32, sr);
-            tmem_wait_ld();
-            const uint32_t vv = hh ? v1 : v0;
-            float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
-#pragma unroll
-            for (int c = 0; c < 32; c += 4) {
-              m0 = fmaxf(m0, ((vv >> c) & 1u) ? __uint_as_float(sr[c]) : -INFINITY);
-              m1 = fmaxf(m1, ((vv >> (c + 1)) & 1u) ? __uint_as_float(sr[c + 1]) : -INFINITY);
-              m2 = fmaxf(m2, ((vv >> (c + 2)) & 1u) ? __uint_as_float(sr[c + 2]) : -INFINITY);
-              m3 = fmaxf(m3, ((vv >> (c + 3)) & 1u) ? __uint_as_float(sr[c + 3]) : -INFINITY);
-            }
-            mx = fmaxf(mx, fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)));
-          }
-        }
+    // Every tile takes one pass over its scores: P = 2^(s * scale - m * scale) with a reference m per row that
+    // is NOT the running maximum. It starts at 0 and moves, by a whole number of powers of two, only when it has
+    // to: when a tile's row sum reaches 2^60 (a score far above the reference; also the case in which the
+    // exponential itself overflows, the sum is then inf), or when everything a row has seen so far sums to less
+    // than 2^-60 (the reference is far above the scores: their P would drop out of the bottom of the range).
+    // Either is rare (scores times scale stay within a few tens of powers of two in a trained model), and in
+    // between P is not bounded by 1, which bf16 and the fp32 accumulators have the range for: after every tile a
+    // row's sum lies in [2^-60, 2^66], 60 binades from either end. Nothing of a tile is written before its row
+    // sums are known, so when a reference has to move the tile's scores are still intact in tensor memory: the
+    // new reference is the larger of the tile's largest exponent and that of what is accumulated, both rounded
+    // up to a whole power of two; O and the running sum are scaled by 2^-k, which is exact; the tile is evaluated
+    // again. (An earlier version took two passes - row maximum, then P - over the first tile of every piece.)
+    // Nothing but the scores is awaited: P goes into the score buffer it came from, and that buffer was last
+    // read by P V of tile it-2, which the tensor pipe finished before it produced these scores. So the softmax
+    // of this tile runs while P V of the previous one does. The second half of a tile's scores is loaded while
+    // the first half is computed. (Loading the next tile's first half ahead as well, or handing P over later,
+    // was tried in several forms and lost each time.)
+    if (!warp_live) {
+      // no live rows: stay in step - wait for a tile's scores like the others, so as not to arrive on
+      // bar_p[it & 1] before the phase of tile it-2 is over
+      for (int it = 0; it < ntile; ++it) {
+        if (ok && it >= 1) ok = mbar_wait(&bar_s[it & 1], (it >> 1) & 1);
+        zero_v_tail(it);
+        tc_fence_before();
+        mbar_arrive(&bar_p[it & 1]);
       }
-      // This path may rescale O, which P V of tile it-1 must have left. A warp without live rows
-      // only has to stay in step: it waits for this tile's scores like the others, so that it cannot
-      // arrive on bar_p[it & 1] before the phase of tile it-2 is over.
-      if (ok && it >= 1) {
-        ok = warp_live ? mbar_wait(&bar_freev[(it - 1) % kStagesV], ((it - 1) / kStagesV) & 1)
-                       : mbar_wait(&bar_s[buf], (it >> 1) & 1);
-      }
-      if (warp_live && ok) {
-        // lazy maximum: move the reference only when the row maximum outgrows it by 2^8
-        float alpha = 1.f;
-        const bool grow = (mx - m_used) * sc > kRescaleThreshold || (m_used == -INFINITY && mx > -INFINITY);
-        if (grow) {
-          alpha = fast_exp2((m_used - mx) * sc);  // 0 when m_used = -inf
-          m_used = mx;
-          l_run *= alpha;
-        }
-        if (it > 0 && __any_sync(0xffffffffu, grow)) {  // rescale this row of O
-          tc_fence_after();
-#pragma unroll
-          for (int hh = 0; hh < 4; ++hh) {
-            uint32_t orr[32];
-            const uint32_t ta = tmem_o + lane_sel + hh * 32;
-            tmem_ld32(ta, orr);
-            tmem_wait_ld();
-#pragma unroll
-            for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
-            tmem_st32(ta, orr);
-          }
-          tmem_wait_st();
-        }
-        // pass 2: P = 2^((s - m) * scale) as bf16 over the scores in tensor memory; row sum in fp32
-        const bool live = m_used > -INFINITY;
-        const float neg_ms = live ? -m_used * sc : 0.f;
-        float l0 = 0.f, l1 = 0.f;
-#pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {
-          uint32_t sr[32], pk[16];
-          tmem_ld32(tp + hh * 32, sr);
-          tmem_wait_ld();
-          const uint32_t vv = live ? (hh ? v1 : v0) : 0u;
-#pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const int c = 2 * e;
-            float p0 = fast_exp2(fmaf(__uint_as_float(sr[c]), sc, neg_ms));
-            float p1 = fast_exp2(fmaf(__uint_as_float(sr[c + 1]), sc, neg_ms));
-            p0 = ((vv >> c) & 1u) ? p0 : 0.f;
-            p1 = ((vv >> (c + 1)) & 1u) ? p1 : 0.f;
-            l0 += p0;
-            l1 += p1;
-            const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
-            pk[e] = *reinterpret_cast<const uint32_t*>(&pb);
-          }
-          tmem_st16(tp + hh * 16, pk);
-        }
-        tmem_wait_st();
-        l_run += l0 + l1;
-      }
-      zero_v_tail(it);
-      tc_fence_before();
-      mbar_arrive(&bar_p[it & 1]);
-    }
-    // ---- Single-pass tiles (all the others, as a rule): one pass over the scores with the reference
-    // maximum of the earlier tiles. P = 2^((s - m) * scale) is then not bounded by 1, but bf16 and the
-    // fp32 accumulators have the range for it; a row whose P would outgrow 2^60 in a tile moves its
-    // reference before the tile is written (see below). Nothing but the scores is awaited: P goes into the
-    // score buffer it came from, and that buffer was last read by P V of tile it-2, which the tensor pipe
-    // finished before it produced these scores. So the softmax of this tile runs while P V of the previous
-    // one does.
-    // The second half of a tile's scores is loaded while the first half is computed. (Loading the next tile's
-    // first half ahead as well, or handing P over later, was tried in several forms and lost each time: what
-    // bounds the loop is the round trip between this hand-over and the next scores, see the MMA issuer.)
-    // Once a warp is here it stays: the reference maxima only grow.
-    if (it < ntile) {
+    } else {
+      m_used = 0.f;
       const unsigned long long sc2 = pack_f2(sc, sc);
-      for (; it < ntile; ++it) {
+      for (int it = 0; it < ntile; ++it) {
         uint32_t sra[32];
         if (ok) {
           ok = mbar_wait(&bar_s[it & 1], (it >> 1) & 1);
@@ -1157,21 +1070,15 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
           if (plain) softmax_half<false>(srb, sc2, neg2, 0u, lacc, pk[1]);
           else softmax_half<true>(srb, sc2, neg2, v1, lacc, pk[1]);
         }
-        // A look at the next tile's scores, asked for here so that the answer's latency (over a hundred cycles
-        // even when they are there) passes while P is stored and handed over.
         float l0, l1;
         unpack_f2(lacc, l0, l1);
-        // A score far above the reference (a P beyond 2^60, or past the range of the exponential: the sum is
-        // then inf) is rare. Nothing of this tile has been written yet, so its scores are intact in tensor
-        // memory: the rows concerned move their reference up by a whole number of powers of two (what is
-        // already accumulated - O and the running sum - is scaled by 2^-k, which is exact) and the tile is
-        // evaluated again.
-        const bool far = row_ok && !(l0 + l1 < 1.15e18f);
-        if (__any_sync(0xffffffffu, far)) {
-          ok = mbar_wait(&bar_freev[(it - 1) % kStagesV], ((it - 1) / kStagesV) & 1);  // O must be at rest
+        const bool far = row_ok && !(l0 + l1 < 1.15e18f);  // 2^60
+        const bool low = row_ok && (plain || (v0 | v1) != 0u) && (l_run + l0 + l1 < 8.6e-19f);  // 2^-60, something visible
+        if (__any_sync(0xffffffffu, far || low)) {
+          if (it > 0) ok = mbar_wait(&bar_freev[(it - 1) % kStagesV], ((it - 1) / kStagesV) & 1);  // O must be at rest
           if (ok) {
             tc_fence_after();
-            float alpha = 1.f, mxt = -INFINITY;
+            float mxt = -INFINITY;
 #pragma unroll 1
             for (int hh = 0; hh < 2; ++hh) {
               uint32_t sr[32];
@@ -1182,24 +1089,34 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
               for (int c = 0; c < 32; ++c)  // (`plain ||`: v0 / v1 then stay out of the unmasked path's live registers)
                 mxt = fmaxf(mxt, (plain || ((vv >> c) & 1u)) ? __uint_as_float(sr[c]) : -INFINITY);
             }
-            if (far && mxt > -INFINITY && mxt < INFINITY) {
-              float kf = ceilf(fmaf(mxt, sc, neg_ms));  // the tile's largest exponent, rounded up
-              kf = kf < 0.f ? 0.f : (kf > 1.0e9f ? 1.0e9f : kf);
-              alpha = ldexpf(1.f, -(int)kf);  // 0 beyond the range: what came before no longer counts
-              neg_ms -= kf;
-              m_used += kf / sc;
+            float kf = 0.f;
+            if (far || low) {
+              const float e_tile = mxt > -INFINITY ? fmaf(mxt, sc, neg_ms) : -INFINITY;  // the tile's largest exponent
+              const float e_acc = l_run > 0.f ? log2f(l_run) : -INFINITY;                // that of what is accumulated
+              const float e = fmaxf(e_tile, e_acc);
+              if (e > -INFINITY && e < INFINITY) {
+                kf = ceilf(e);
+                kf = kf < -1.0e9f ? -1.0e9f : (kf > 1.0e9f ? 1.0e9f : kf);
+              }
             }
+            // 2^-k for what is accumulated: nothing is (a sum of 0 means every P so far was exactly 0), or its
+            // exponent is at most k, so the product cannot overflow; 0 for k beyond the range (it no longer counts)
+            const float alpha = l_run > 0.f ? ldexpf(1.f, -(int)kf) : 1.f;
+            if (it > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
 #pragma unroll 1
-            for (int q4 = 0; q4 < 4; ++q4) {  // O and the running sum follow (P V of tile it-1 is over)
-              uint32_t orr[32];
-              const uint32_t ta = tmem_o + lane_sel + q4 * 32;
-              tmem_ld32(ta, orr);
-              tmem_wait_ld();
+              for (int q4 = 0; q4 < 4; ++q4) {  // O follows (P V of tile it-1 is over)
+                uint32_t orr[32];
+                const uint32_t ta = tmem_o + lane_sel + q4 * 32;
+                tmem_ld32(ta, orr);
+                tmem_wait_ld();
 #pragma unroll
-              for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
-              tmem_st32(ta, orr);
+                for (int c = 0; c < 32; ++c) orr[c] = __float_as_uint(__uint_as_float(orr[c]) * alpha);
+                tmem_st32(ta, orr);
+              }
             }
             l_run *= alpha;
+            neg_ms -= kf;
+            m_used += kf / sc;
             l0 = l1 = 0.f;
 #pragma unroll
             for (int hh = 0; hh < 2; ++hh) {  // the tile again (rows that did not move get the same values)
@@ -1276,7 +1193,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
         }
       }
     }
-    stage_ml[r * 2] = m_used * sc * 0.69314718055994531f;  // natural-log units (-inf: nothing visible)
+    stage_ml[r * 2] = l_run > 0.f ? m_used * sc * 0.69314718055994531f : -INFINITY;  // natural-log units (-inf: nothing visible)
     stage_ml[r * 2 + 1] = l_run;
   }
   tc_fence_before();

@@ -605,6 +605,59 @@ def test_attention_score_far_above_the_earlier_tiles(binding, name, factor):
     assert err <= attention_tolerance(w.kv_dtype), err
 
 
+@pytest.mark.parametrize("name", ["c2_llama8b", "c3_llama8b_b16", "c4_llama70b_n32"])
+@pytest.mark.parametrize("shift", [-3000.0, -700.0, 900.0, "mixed"])
+def test_attention_all_scores_far_from_zero(binding, name, shift):
+    """Every score of a head lies hundreds of nats below (or above) zero: the softmax's reference starts at 0
+    and has to move down (everything would underflow) or up (everything would overflow) in the first tile of
+    every piece. The keys get a component along the head's mean query, which shifts all its scores; "mixed"
+    gives the kv-heads different shifts and leaves some untouched, so that one launch has rows that move up,
+    rows that move down and rows that stay. Cluster and global-merge launches; sampled outputs vs the oracle."""
+    rng = np.random.default_rng(23)
+    w = wl.CONFIGS[name]
+    B, Ncap, Hq, Hkv = w.batch, w.max_tree, w.q_heads, w.kv_heads
+    G = Hq // Hkv
+    n = 12 if name.startswith("c3") else w.total_token
+    ctx = binding.CastContext(max_batch=B, **cfg_kwargs(w, enable_bp=0, enable_dr=0))
+    kv = wl.kv_lengths(w, "cpu").cuda()
+    kvh_ = kv.cpu().numpy()
+    n_tree = np.full(B, n, dtype=np.int32)
+    anc = np.zeros((B, Ncap, 4), dtype=np.uint32)
+    for b in range(B):
+        anc[b, :n] = ancestor_masks(_random_tree(rng, n, "random"), n, 4)
+    q = wl.query(w, 0, "cpu")
+    k, v = wl.kv_cache(w, 0, "cpu")
+    table, num_pages = wl.page_table(w, "cpu")
+    # all queries of a kv-head's group point roughly the same way (u plus noise), the keys get c * u added:
+    # every score of the group moves by about c * |u|^2 = the wanted shift in raw score units
+    scale = 1.0 / np.sqrt(w.head_dim)
+    for kvh in range(Hkv):
+        sh = shift if shift != "mixed" else [-3000.0, 0.0, 900.0, -200.0][kvh % 4]
+        if sh == 0.0:
+            continue
+        u = torch.randn(w.head_dim, generator=torch.Generator().manual_seed(100 + kvh))
+        u = u / u.norm() * 4.0
+        q[:, :, kvh * G:(kvh + 1) * G] = (u + 0.3 * q[:, :, kvh * G:(kvh + 1) * G].float()).to(q.dtype)
+        c = (sh / scale) / float(u.norm() ** 2)  # nats -> raw score units
+        if w.page_size:
+            k[:, :, kvh] = (k[:, :, kvh].float() + c * u).to(k.dtype)
+        else:
+            k[:, :, kvh] = (k[:, :, kvh].float() + c * u).to(k.dtype)
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    td = table.cuda() if table is not None else None
+    out = gpu_attention(ctx, w, qd, kd, vd, td, num_pages, kv, anc, torch.from_numpy(n_tree).cuda(), scale=0.0)
+    assert ctx.cast_poll_status()[0] == 0
+    only = {(int(rng.integers(0, B)), int(rng.integers(0, n)), int(rng.integers(0, Hq))) for _ in range(40)}
+    only |= {(b, n - 1, h) for b in (0, B - 1) for h in range(0, Hq, max(1, G))}
+    f32 = lambda t_: t_.float().numpy()
+    tab = table.numpy() if table is not None else None
+    ref = tree_attention(f32(q), f32(k), f32(v), w.page_size, tab, kvh_, anc, n_tree, None, only)
+    got = to_f64(out)
+    assert np.isfinite(got[:, :n]).all()
+    err = max(np.max(np.abs(got[i] - ref[i])) for i in only)
+    assert err <= attention_tolerance(w.kv_dtype), err
+
+
 def test_attention_bad_page_sets_status(binding):
     w = wl.Workload("attnbad", 91, 1, "bf16", "f32", 8, 2, 128, 100, 100, 16, 100, 1.0, 4, 2, 8, False, 1)
     ctx = binding.CastContext(max_batch=1, vocab=100, top_k=2, max_depth=4, total_token=8)
