@@ -29,7 +29,7 @@ template <> struct Vec<__nv_bfloat16> {
 };
 
 constexpr int kArgThreads = 256;
-constexpr int kArgUnroll = 4;
+constexpr int kArgUnroll = 8;
 
 // One CTA per (chunk, tree token, sequence): the largest (logit, lowest token id) of the chunk.
 template <typename T>
