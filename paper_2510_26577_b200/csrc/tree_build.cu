@@ -422,6 +422,9 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
   __shared__ double red_d[kSweepThreads / 32];
   __shared__ int sorted[kTailSingleMaxB * CAST_MAX_WIDTH];  // small batches: pool indices of the first sorted candidates
   __shared__ int s_flag, short_n;
+  __shared__ unsigned long long pass_heads[2][kSweepThreads / 32];  // the warps' best keys after a pass (see cta_bound)
+  __shared__ float pass_wmax[kSweepThreads / 32];                   // the warps' maxima of the first pass
+  static_assert(CAST_MAX_TOP_K <= kSweepThreads / 32, "the K-th largest of the warps' maxima needs K <= warps");
   // filled in the first CTA of the row's cluster by all CTAs of the cluster: chunk c's top-K keys
   // (descending), maximum (log2 units) and sum of 2^(. - maximum)
   __shared__ unsigned long long row_keys[kSweepMaxChunks * CAST_MAX_TOP_K];
@@ -506,9 +509,32 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
   unsigned long long* wlist = cand + warp * kWarpCap;
   int have = 0;
   unsigned long long thr_key = 0ull;
+  // A lower bound on the CTA's K-th largest key that all warps share from the second pass on: the K-th
+  // largest of the warps' best keys (K of the CTA's logits are at least that large). A warp's own K-th key
+  // only knows the warp's sixteenth of the data; against this bound few logits of a later pass reach any list
+  // at all, so the exact tests, the appends and the re-ranking below mostly do not run. (A logit of the CTA's
+  // final top K is >= every such bound, and a warp drops it only for K better ones: the chunk result is exact.)
+  unsigned long long cta_bound = 0ull;
+  int pass = 0;
 
-  for (int sub = begin; sub < end; sub += kSweepSub) {
-    if (sub != begin) load_pass(sub);
+  for (int sub = begin; sub < end; sub += kSweepSub, ++pass) {
+    if (sub != begin) {
+      load_pass(sub);
+      unsigned long long* hd = pass_heads[pass & 1];
+      if (lane == 0) hd[warp] = have > 0 ? wlist[0] : 0ull;
+      __syncthreads();
+      const unsigned long long head = lane < kWarps ? hd[lane] : 0ull;
+      int rh = 0;
+#pragma unroll
+      for (int j = 0; j < kWarps; ++j) rh += (__shfl_sync(0xffffffffu, head, j) > head);
+      unsigned long long bnd = (rh == K - 1) ? head : 0ull;  // heads are distinct unless 0 ("no entry")
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long other = __shfl_xor_sync(0xffffffffu, bnd, o);
+        bnd = other > bnd ? other : bnd;
+      }
+      cta_bound = bnd > cta_bound ? bnd : cta_bound;
+    }
     float tmax = xv[0];
 #pragma unroll
     for (int i = 1; i < kSweepEpt; ++i) tmax = fmaxf(tmax, xv[i]);
@@ -529,7 +555,27 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
     // filter threshold: the warp's exact K-th key once it has K, else the K-th largest of the lanes'
     // maxima of this pass (at least K of the warp's logits are >= it)
     float thr_val;
-    if (thr_key == 0ull) {
+    const unsigned long long gate = thr_key > cta_bound ? thr_key : cta_bound;  // keys at or below it cannot matter
+    if (pass == 0) {
+      // nothing is known yet: the K-th largest of the 16 warps' maxima (K <= 16 of the CTA's logits are at
+      // least that large). Against it one or two logits per warp pass; against the K-th largest of a warp's
+      // own lane maxima, which needs no barrier but a 15-stage sorting network, K to 2K per warp did.
+      float wm = tmax;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, o));
+      float* wmax = pass_wmax;
+      if (lane == 0) wmax[warp] = wm;
+      __syncthreads();
+      const float mine = lane < kWarps ? wmax[lane] : -INFINITY;
+      int rh = 0;
+#pragma unroll
+      for (int j = 0; j < kWarps; ++j) {
+        const float o = __shfl_sync(0xffffffffu, mine, j);
+        rh += (o > mine) || (o == mine && j < lane);  // equal maxima in lane order: ranks 0..15 are distinct
+      }
+      const unsigned who = __ballot_sync(0xffffffffu, lane < kWarps && rh == K - 1);
+      thr_val = __shfl_sync(0xffffffffu, mine, who != 0u ? __ffs(who) - 1 : 0);
+    } else if (gate == 0ull) {
       float kx = tmax;
 #pragma unroll
       for (int k = 2; k <= 32; k <<= 1)
@@ -541,7 +587,7 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
         }
       thr_val = __shfl_sync(0xffffffffu, kx, K - 1);
     } else {
-      thr_val = key_value(thr_key);
+      thr_val = key_value(gate);
     }
     // Few logits pass. Every lane marks its passing slots in a bit mask and the warp takes the union with
     // one reduction; only a slot with a passer somewhere (rare) takes the exact test on the full key and
@@ -556,7 +602,7 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
       if (any_mask & (1u << i)) {
         const int id = sub + ((i / VEC) * kSweepThreads + tid) * VEC + (i % VEC);
         const unsigned long long key = make_key(xv[i], id);
-        const bool ok = xv[i] >= thr_val && id < end && key > thr_key;
+        const bool ok = xv[i] >= thr_val && id < end && key > gate;
         const unsigned m = __ballot_sync(0xffffffffu, ok);
         const int pos = have + __popc(m & ((1u << lane) - 1u));
         if (ok && pos < kWarpCap) wlist[pos] = key;
