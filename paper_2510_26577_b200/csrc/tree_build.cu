@@ -589,20 +589,35 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
     } else {
       thr_val = key_value(gate);
     }
-    // Few logits pass. Every lane marks its passing slots in a bit mask and the warp takes the union with
-    // one reduction; only a slot with a passer somewhere (rare) takes the exact test on the full key and
-    // appends to the warp's list.
+    // Few logits pass, and against the shared thresholds most passes of a warp have none: one vote on the
+    // lanes' maxima settles that. Otherwise every lane marks its passing slots in a bit mask, the warp takes
+    // the union with one reduction and walks its set bits (a loop over the set bits only: unrolled over all 32
+    // slots, the tests and reconvergence points of the empty ones were most of the sweep's time); a slot's
+    // logit is picked out of the registers by a warp-uniform switch, takes the exact test on the full key and
+    // is appended to the warp's list.
     const int have0 = have;
-    unsigned mine_mask = 0u;
+    if (__any_sync(0xffffffffu, tmax >= thr_val)) {
+      unsigned mine_mask = 0u;
 #pragma unroll
-    for (int i = 0; i < kSweepEpt; ++i) mine_mask |= (xv[i] >= thr_val) ? (1u << i) : 0u;
-    const unsigned any_mask = __reduce_or_sync(0xffffffffu, mine_mask);
-#pragma unroll
-    for (int i = 0; i < kSweepEpt; ++i) {
-      if (any_mask & (1u << i)) {
+      for (int i = 0; i < kSweepEpt; ++i) mine_mask |= (xv[i] >= thr_val) ? (1u << i) : 0u;
+      unsigned any_mask = __reduce_or_sync(0xffffffffu, mine_mask);
+#pragma unroll 1
+      while (any_mask != 0u) {
+        const int i = __ffs(any_mask) - 1;
+        any_mask &= any_mask - 1u;
+        float xi = 0.f;
+        switch (i) {
+#define CAST_PICK(n) case n: xi = xv[n]; break;
+          CAST_PICK(0) CAST_PICK(1) CAST_PICK(2) CAST_PICK(3) CAST_PICK(4) CAST_PICK(5) CAST_PICK(6) CAST_PICK(7)
+          CAST_PICK(8) CAST_PICK(9) CAST_PICK(10) CAST_PICK(11) CAST_PICK(12) CAST_PICK(13) CAST_PICK(14) CAST_PICK(15)
+          CAST_PICK(16) CAST_PICK(17) CAST_PICK(18) CAST_PICK(19) CAST_PICK(20) CAST_PICK(21) CAST_PICK(22) CAST_PICK(23)
+          CAST_PICK(24) CAST_PICK(25) CAST_PICK(26) CAST_PICK(27) CAST_PICK(28) CAST_PICK(29) CAST_PICK(30) CAST_PICK(31)
+#undef CAST_PICK
+        }
+        static_assert(kSweepEpt == 32, "the switch above names every slot");
         const int id = sub + ((i / VEC) * kSweepThreads + tid) * VEC + (i % VEC);
-        const unsigned long long key = make_key(xv[i], id);
-        const bool ok = xv[i] >= thr_val && id < end && key > gate;
+        const unsigned long long key = make_key(xi, id);
+        const bool ok = xi >= thr_val && id < end && key > gate;
         const unsigned m = __ballot_sync(0xffffffffu, ok);
         const int pos = have + __popc(m & ((1u << lane) - 1u));
         if (ok && pos < kWarpCap) wlist[pos] = key;
