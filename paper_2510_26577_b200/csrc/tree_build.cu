@@ -422,7 +422,7 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
   __shared__ double red_d[kSweepThreads / 32];
   __shared__ int sorted[kTailSingleMaxB * CAST_MAX_WIDTH];  // small batches: pool indices of the first sorted candidates
   __shared__ int s_flag, short_n;
-  __shared__ unsigned long long pass_heads[2][kSweepThreads / 32];  // the warps' best keys after a pass (see cta_bound)
+  __shared__ float pass_heads[2][kSweepThreads / 32];  // the warps' largest logits after a pass (see cta_bound)
   __shared__ float pass_wmax[kSweepThreads / 32];                   // the warps' maxima of the first pass
   static_assert(CAST_MAX_TOP_K <= kSweepThreads / 32, "the K-th largest of the warps' maxima needs K <= warps");
   // filled in the first CTA of the row's cluster by all CTAs of the cluster: chunk c's top-K keys
@@ -509,31 +509,31 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
   unsigned long long* wlist = cand + warp * kWarpCap;
   int have = 0;
   unsigned long long thr_key = 0ull;
-  // A lower bound on the CTA's K-th largest key that all warps share from the second pass on: the K-th
-  // largest of the warps' best keys (K of the CTA's logits are at least that large). A warp's own K-th key
-  // only knows the warp's sixteenth of the data; against this bound few logits of a later pass reach any list
-  // at all, so the exact tests, the appends and the re-ranking below mostly do not run. (A logit of the CTA's
-  // final top K is >= every such bound, and a warp drops it only for K better ones: the chunk result is exact.)
-  unsigned long long cta_bound = 0ull;
+  // A lower bound on the CTA's K-th largest logit that all warps share from the second pass on: the K-th
+  // largest of the warps' best logits so far (K of the CTA's logits are at least that large). A warp's own K-th
+  // key only knows the warp's sixteenth of the data; against this bound few logits of a later pass reach any
+  // list at all, so the exact tests, the appends and the re-ranking below mostly do not run. (A logit of the
+  // CTA's final top K is >= every such bound, and a warp drops it only for K better ones: the chunk result is
+  // exact. The bound is a value, not a key: logits equal to it pass, which only lengthens a list.)
+  float cta_bound = -INFINITY;
   int pass = 0;
 
   for (int sub = begin; sub < end; sub += kSweepSub, ++pass) {
     if (sub != begin) {
       load_pass(sub);
-      unsigned long long* hd = pass_heads[pass & 1];
-      if (lane == 0) hd[warp] = have > 0 ? wlist[0] : 0ull;
+      float* hd = pass_heads[pass & 1];
+      if (lane == 0) hd[warp] = have > 0 ? key_value(wlist[0]) : -INFINITY;
       __syncthreads();
-      const unsigned long long head = lane < kWarps ? hd[lane] : 0ull;
+      const float head = lane < kWarps ? hd[lane] : -INFINITY;
       int rh = 0;
 #pragma unroll
-      for (int j = 0; j < kWarps; ++j) rh += (__shfl_sync(0xffffffffu, head, j) > head);
-      unsigned long long bnd = (rh == K - 1) ? head : 0ull;  // heads are distinct unless 0 ("no entry")
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const unsigned long long other = __shfl_xor_sync(0xffffffffu, bnd, o);
-        bnd = other > bnd ? other : bnd;
+      for (int j = 0; j < kWarps; ++j) {
+        const float o = __shfl_sync(0xffffffffu, head, j);
+        rh += (o > head) || (o == head && j < lane);  // equal heads in lane order: ranks 0..15 are distinct
       }
-      cta_bound = bnd > cta_bound ? bnd : cta_bound;
+      const unsigned who = __ballot_sync(0xffffffffu, lane < kWarps && rh == K - 1);
+      const float bnd = __shfl_sync(0xffffffffu, head, who != 0u ? __ffs(who) - 1 : 0);
+      cta_bound = fmaxf(cta_bound, bnd);
     }
     float tmax = xv[0];
 #pragma unroll
@@ -555,7 +555,7 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
     // filter threshold: the warp's exact K-th key once it has K, else the K-th largest of the lanes'
     // maxima of this pass (at least K of the warp's logits are >= it)
     float thr_val;
-    const unsigned long long gate = thr_key > cta_bound ? thr_key : cta_bound;  // keys at or below it cannot matter
+    const unsigned long long gate = thr_key;  // keys at or below the warp's own K-th cannot matter
     if (pass == 0) {
       // nothing is known yet: the K-th largest of the 16 warps' maxima (K <= 16 of the CTA's logits are at
       // least that large). Against it one or two logits per warp pass; against the K-th largest of a warp's
@@ -575,7 +575,7 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
       }
       const unsigned who = __ballot_sync(0xffffffffu, lane < kWarps && rh == K - 1);
       thr_val = __shfl_sync(0xffffffffu, mine, who != 0u ? __ffs(who) - 1 : 0);
-    } else if (gate == 0ull) {
+    } else if (gate == 0ull && !(cta_bound > -INFINITY)) {
       float kx = tmax;
 #pragma unroll
       for (int k = 2; k <= 32; k <<= 1)
@@ -587,7 +587,7 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
         }
       thr_val = __shfl_sync(0xffffffffu, kx, K - 1);
     } else {
-      thr_val = key_value(gate);
+      thr_val = gate != 0ull ? fmaxf(key_value(gate), cta_bound) : cta_bound;
     }
     // Few logits pass, and against the shared thresholds most passes of a warp have none: one vote on the
     // lanes' maxima settles that. Otherwise every lane marks its passing slots in a bit mask, the warp takes
