@@ -1161,8 +1161,10 @@ extern "C" cast_status cast_tree_expand(cast_ctx* c, int layer, const void* draf
       const int ne = (V + ce - 1) / ce;
       const int passes = (ce + kSweepSub - 1) / kSweepSub;
       const double per_cta = (ne == 1 ? 2.0 : 2.5) + 4.0 * passes;
+      // (a launch a little larger than the machine costs a good part of a second round: the few CTAs left over
+      // run while the other SMs idle)
       const double queue = (double)rows * ne / c->num_sms;
-      const double cost = per_cta * (queue < 1.0 ? 1.0 : queue);
+      const double cost = per_cta * (queue <= 1.0 ? 1.0 : (queue < 1.5 ? 1.5 : queue));
       if (cost < best - 1e-9) {
         best = cost;
         nchunks = ne;
