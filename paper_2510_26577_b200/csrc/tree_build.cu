@@ -83,6 +83,25 @@ __device__ __forceinline__ float ex2f(float x) {
 }
 // log2(e) split into a float just below it and a positive residual: x * log2(e) to better than one ulp
 // of the product, and -inf logits stay -inf through both FMAs (no inf - inf)
+// Packed fp32 pairs: one instruction, two lanes of the FMA pipe, the same IEEE results per element.
+__device__ __forceinline__ unsigned long long pack2(float a, float b) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b) {
+  unsigned long long r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
 constexpr float kLog2eHi = 1.4426950216293335f;
 constexpr float kLog2eLo = 1.925963033500011e-08f;  // log2(e) - kLog2eHi
 
@@ -544,12 +563,19 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
       M2 = t2;
     }
     if (M2 > -INFINITY) {
-      float a0 = 0.f, a1 = 0.f;
+      // x * log2(e) - M2 with log2(e) in two parts (the product is exact to fp32's last bit and beyond), two
+      // logits per instruction; NaN and +inf logits poison the sum
+      const unsigned long long hi2 = pack2(kLog2eHi, kLog2eHi), lo2 = pack2(kLog2eLo, kLog2eLo), nm2 = pack2(-M2, -M2);
+      unsigned long long acc2 = pack2(0.f, 0.f);
 #pragma unroll
       for (int i = 0; i < kSweepEpt; i += 2) {
-        a0 += ex2f(fmaf(xv[i], kLog2eHi, fmaf(xv[i], kLog2eLo, -M2)));  // NaN and +inf logits poison the sum
-        a1 += ex2f(fmaf(xv[i + 1], kLog2eHi, fmaf(xv[i + 1], kLog2eLo, -M2)));
+        const unsigned long long x2 = pack2(xv[i], xv[i + 1]);
+        float e0, e1;
+        unpack2(fma2(x2, hi2, fma2(x2, lo2, nm2)), e0, e1);
+        acc2 = add2(acc2, pack2(ex2f(e0), ex2f(e1)));
       }
+      float a0, a1;
+      unpack2(acc2, a0, a1);
       s_run += a0 + a1;
     }
     // filter threshold: the warp's exact K-th key once it has K, else the K-th largest of the lanes'
@@ -605,16 +631,18 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
       while (any_mask != 0u) {
         const int i = __ffs(any_mask) - 1;
         any_mask &= any_mask - 1u;
-        float xi = 0.f;
-        switch (i) {
-#define CAST_PICK(n) case n: xi = xv[n]; break;
-          CAST_PICK(0) CAST_PICK(1) CAST_PICK(2) CAST_PICK(3) CAST_PICK(4) CAST_PICK(5) CAST_PICK(6) CAST_PICK(7)
-          CAST_PICK(8) CAST_PICK(9) CAST_PICK(10) CAST_PICK(11) CAST_PICK(12) CAST_PICK(13) CAST_PICK(14) CAST_PICK(15)
-          CAST_PICK(16) CAST_PICK(17) CAST_PICK(18) CAST_PICK(19) CAST_PICK(20) CAST_PICK(21) CAST_PICK(22) CAST_PICK(23)
-          CAST_PICK(24) CAST_PICK(25) CAST_PICK(26) CAST_PICK(27) CAST_PICK(28) CAST_PICK(29) CAST_PICK(30) CAST_PICK(31)
-#undef CAST_PICK
-        }
-        static_assert(kSweepEpt == 32, "the switch above names every slot");
+        // xv[i] for a run-time i: five rounds of selects on the bits of i (registers cannot be indexed)
+        static_assert(kSweepEpt == 32, "five bits name a slot");
+        float s16[16], s8[8], s4[4];
+        const bool b0 = (i & 1) != 0, b1 = (i & 2) != 0, b2 = (i & 4) != 0, b3 = (i & 8) != 0, b4 = (i & 16) != 0;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) s16[j] = b0 ? xv[2 * j + 1] : xv[2 * j];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) s8[j] = b1 ? s16[2 * j + 1] : s16[2 * j];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) s4[j] = b2 ? s8[2 * j + 1] : s8[2 * j];
+        const float s2a = b3 ? s4[1] : s4[0], s2b = b3 ? s4[3] : s4[2];
+        const float xi = b4 ? s2b : s2a;
         const int id = sub + ((i / VEC) * kSweepThreads + tid) * VEC + (i % VEC);
         const unsigned long long key = make_key(xi, id);
         const bool ok = xi >= thr_val && id < end && key > gate;
