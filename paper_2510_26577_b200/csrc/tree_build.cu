@@ -3,9 +3,10 @@
 // cast_tree_expand is ONE kernel per draft layer, launched as thread-block clusters (the chunks of
 // one logits row form a cluster) with programmatic dependent launch between the layers:
 //   1. vocabulary sweep - one CTA per chunk: streaming 16-byte loads issued before anything else,
-//      online max / sum-exp in base 2, and an exact top-K kept per warp (the K-th largest of the
-//      lanes' maxima bounds the warp's K-th largest from below, so only a handful of logits
-//      survive the filter; the warps never meet during the sweep);
+//      online max / sum-exp in base 2, and a list of top-K candidates per warp, filtered against
+//      thresholds the CTA's warps share (the K-th largest of the warps' maxima in the first pass, of
+//      their best logits afterwards: lower bounds on the CTA's K-th largest, so the result is exact
+//      and only a logit or two per warp survives the filter);
 //   2. the chunk's top K, maximum and sum go straight into the shared memory of the cluster's
 //      first CTA, which merges the row after the cluster barrier (log-sum-exp in fp64, lower-bound
 //      merge of the sorted chunk lists) and appends the K children to the node pool;
