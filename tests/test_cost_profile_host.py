@@ -34,3 +34,22 @@ def test_gemm_term_adds_linearly_in_batch_times_tokens():
     f1, _ = tables_from_measurement(t, pts, 16, 8, n_layers=1, gemm_us=(7.0, 0.5))
     n = np.arange(1, 9)
     assert np.allclose(f1[0] - f0[0], 7.0 + 0.5 * 16 * n, rtol=1e-5)
+
+
+def test_measured_layer_and_head_terms_enter_where_the_method_puts_them():
+    """A measured GEMM curve replaces the linear form: the target's table is n_layers x (attention + layer),
+    the draft's one layer plus the vocabulary projection, so the two are no longer proportional."""
+    pts = (1, 4, 16)
+    t = np.array([[5.0, 6.0, 9.0], [7.0, 8.0, 12.0]])
+    layer_us = np.array([20.0, 21.0, 30.0])
+    head_us = np.array([50.0, 52.0, 70.0])
+    fT, fD = tables_from_measurement(t, pts, 3, 16, n_layers=10, layer_us=layer_us, head_us=head_us)
+    for g in range(2):
+        for j, n in enumerate(pts):
+            assert abs(fT[g, n - 1] - 10.0 * (t[g, j] + layer_us[j])) < 1e-9
+            assert abs(fD[g, n - 1] - (t[g, j] + layer_us[j] + head_us[j])) < 1e-9
+    # between measured points: linear in n for every term
+    assert abs(fT[0, 9] - 10.0 * ((6.0 + 9.0) / 2 + (21.0 + 30.0) / 2)) < 1e-9  # n = 10, halfway between 4 and 16
+    assert (np.diff(fT, axis=1) > 0).all() and (np.diff(fD, axis=1) > 0).all()
+    assert not np.allclose(fT / fT[0, 0], fD / fD[0, 0])
+    CostTable(3, 512, 2, 16, fT, fD)

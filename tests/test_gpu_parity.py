@@ -872,6 +872,39 @@ def test_measured_cost_tables_size_the_same_tree_on_both_sides(binding):
     assert narrowed, "the measured tables never narrowed, stopped or trimmed the tree: thresholds out of range"
 
 
+def test_measured_gemm_terms_give_tables_both_sides_size_alike(binding):
+    """The profiler's second measurement: the dense projections of a decoder layer and the vocabulary projection
+    at the workload's dimensions (library bf16 GEMMs on random weights). With them the draft's table is no
+    longer a multiple of the target's; the library and the oracle, given the same measured tables, must still
+    build the same tree with every sizing switch on."""
+    from oracle import CostTable
+    from paper_2510_26577_b200 import cost_profile
+
+    B, L, M, Ntab = 2, 256, 2, 24
+    w = wl.Workload("prof2", 85, B, "bf16", "f32", 8, 2, 128, 40, 400, 16, 3000, 2.0, 4, 4, 16, False, 2, max_tree=32,
+                    seed_salt=1)
+    pts = (1, 4, 16, 32)
+    t, pts = cost_profile.measure_attention_us(w, B, L, M, n_points=pts, reps=4)
+    layer_us, head_us = cost_profile.measure_layer_gemms_us(w, B, pts, reps=3)
+    assert layer_us.shape == head_us.shape == (len(pts),)
+    assert np.isfinite(layer_us).all() and (layer_us > 0).all() and np.isfinite(head_us).all() and (head_us > 0).all()
+    fT, fD = cost_profile.tables_from_measurement(t, pts, B, Ntab, n_layers=4, layer_us=layer_us, head_us=head_us)
+    assert (np.diff(fT, axis=1) > 0).all() and (np.diff(fD, axis=1) > 0).all()
+    over = dict(enable_bp=1, enable_dp=1, enable_dr=1, C1=0.05, C2=0.05, C3=0.02)
+    kw = cfg_kwargs(w, **over)
+    tables = {B: CostTable(B, L, M, Ntab, fT, fD)}
+    ctx = binding.CastContext(max_batch=B, **kw)
+    ctx.cast_set_cost_tables(B, L, M, Ntab, fT, fD)
+    root = wl.root_tokens(w, "cpu").cuda()
+    kv = wl.kv_lengths(w, "cpu").cuda()
+    logits = [wl.draft_logits(w, l, "cpu", peaked=True).cuda() for l in range(1, w.depth + 1)]
+    o = oracle_tree(kw, tables, root, kv, logits, None)
+    g = gpu_tree(ctx, root, kv, logits)
+    if not (o["min_score_gap"] >= 1e-5 and o["stable"]):
+        pytest.skip("a measured table put a decision within rounding of its threshold")
+    assert_tree_equal(g, o)
+
+
 def test_attention_without_a_reserved_workspace_is_refused(binding):
     """Compute calls never allocate: a shape that needs a split workspace larger than what was reserved
     returns CAST_ERR_CAPACITY and launches nothing; after cast_reserve_attention the same call runs."""
