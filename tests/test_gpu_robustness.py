@@ -124,6 +124,66 @@ def test_attention_random_shapes_and_windows(binding, seed):
         ctx.close()
 
 
+@pytest.mark.parametrize("seed", [8, 9])
+def test_attention_random_large_shapes(binding, seed):
+    """bf16, D = 128, at sizes that reach every launch mode of the tensor-core kernel (clusters, the merge through
+    a workspace, the plain launch): up to 48 ragged sequences, prefixes up to 20 000 positions (empty ones
+    included), page sizes 0 / 16 / 64, group sizes that do and do not divide a row block, tree budgets 16 to 128
+    with empty and full trees, early reads on for half of the cases. Rows past a tree stay untouched, live rows are
+    finite, and sampled outputs of up to three sequences match the oracle."""
+    rng = np.random.default_rng(seed)
+    for case in range(14):
+        D = 128
+        Hkv = int(rng.choice([1, 2, 4, 8]))
+        Hq = Hkv * int(rng.choice([1, 2, 4, 5, 8]))
+        page = int(rng.choice([0, 16, 64]))
+        B = int(rng.choice([1, 2, 3, 6, 12, 20, 33, 48]))
+        hi = int(rng.choice([700, 3000, 9000, 20000]))
+        while B * hi * Hkv * D > 1.2e8:  # keeps the cache to a few hundred MB and its generation to seconds
+            if B > 1 and rng.random() < 0.5:
+                B = max(1, B // 2)
+            else:
+                hi //= 2
+        lo = int(rng.choice([0, hi // 2, hi]))
+        Ncap = int(rng.choice([16, 64, 128]))
+        w = wl.Workload("fuzz", 700 + case, B, "bf16", "f32", Hq, Hkv, D, lo, hi, page, 100, 1.0, 4, 2, 8, False, 1,
+                        max_tree=Ncap)
+        ctx = binding.CastContext(max_batch=B, vocab=100, top_k=2, max_depth=8, total_token=Ncap, max_tree=Ncap)
+        ctx.cast_set_attention_early_reads(bool(rng.random() < 0.5))
+        kv = wl.kv_lengths(w, "cpu").cuda()
+        n_tree = rng.integers(0 if rng.random() < 0.2 else 1, Ncap + 1, size=B).astype(np.int32)
+        if rng.random() < 0.3:
+            n_tree[:] = Ncap
+        anc = np.zeros((B, Ncap, ctx.words), dtype=np.uint32)
+        for b in range(B):
+            N = int(n_tree[b])
+            if N:
+                anc[b, :N] = ancestor_masks(_random_parents(rng, N), N, ctx.words)
+        q = wl.query(w, 0, "cpu").cuda()
+        k, v = (t.cuda() for t in wl.kv_cache(w, 0, "cpu"))
+        table, num_pages = wl.page_table(w, "cuda")
+        out = gpu_attention(ctx, w, q, k, v, table, num_pages, kv, anc, torch.from_numpy(n_tree).cuda())
+        assert ctx.cast_poll_status()[0] == 0
+        got = to_f64(out)
+        only = set()
+        for b in range(B):
+            N = int(n_tree[b])
+            assert np.isnan(got[b, N:]).all() and np.isfinite(got[b, :N]).all(), (case, b)
+        for b in rng.choice(B, size=min(B, 3), replace=False):
+            N = int(n_tree[b])
+            if N:
+                for t in {0, N - 1, int(rng.integers(0, N))}:
+                    for h in {0, Hq - 1, int(rng.integers(0, Hq))}:
+                        only.add((int(b), t, h))
+        if only:
+            f32 = lambda t: t.float().cpu().numpy()
+            tab = table.cpu().numpy() if table is not None else None
+            ref = tree_attention(f32(q), f32(k), f32(v), page, tab, kv.cpu().numpy(), anc, n_tree, None, only)
+            err = max(np.max(np.abs(got[i] - ref[i])) for i in only)
+            assert err <= attention_tolerance("bf16"), (case, B, Hq, Hkv, page, lo, hi, Ncap, err)
+        ctx.close()
+
+
 @pytest.mark.parametrize("seed", [6, 7])
 def test_accept_and_compaction_random(binding, seed):
     from oracle import compact_kv, greedy_accept
