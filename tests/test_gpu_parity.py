@@ -905,6 +905,96 @@ def test_measured_gemm_terms_give_tables_both_sides_size_alike(binding):
     assert_tree_equal(g, o)
 
 
+# ------------------------------------------------ a decoding loop: every step starts from what the last one left
+@pytest.mark.parametrize("page", [0, 16])
+def test_decoding_loop_of_several_steps(binding, page):
+    """Five consecutive steps on one context and one cache, the library and the oracle side by side: tree build
+    (all sizing switches on, the FIFO carried along), fresh K/V rows written for the tree tokens right before the
+    attention (early reads promised, as in a decoding loop), attention over two layers, greedy acceptance,
+    compaction; the next step's root is the bonus token and its prefix the compacted cache. Every output of every
+    step is compared, so an error of a step - a row moved to the wrong place, a stale length or work list - shows
+    in the same or in a later one."""
+    from oracle import CostTable
+    B, H, NL = 3, 4, 2
+    w = wl.Workload("loop", 90 + (1 if page else 0), B, "bf16", "f32", 8, 2, 128, 60, 500, page, 3000, 2.0, H, 4, 20, True, NL,
+                    max_tree=64, seed_salt=2)
+    over = dict(enable_dp=1)
+    kw = cfg_kwargs(w, **over)
+    L, M, Ntab, fT, fD = make_tables(w, B, skewed=True)
+    tables = {B: CostTable(B, L, M, Ntab, fT, fD)}
+    ctx = binding.CastContext(max_batch=B, **kw)
+    ctx.cast_set_cost_tables(B, L, M, Ntab, fT, fD)
+    ctx.cast_set_attention_early_reads(True)
+    cap = wl.seq_capacity(w)
+    table, num_pages = wl.page_table(w, "cuda")
+    tab = table.cpu().numpy() if table is not None else None
+    layers = [wl.kv_cache(w, l, "cpu") for l in range(NL)]
+    kk = torch.stack([k for k, _ in layers]).contiguous().cuda()
+    vv = torch.stack([v for _, v in layers]).contiguous().cuda()
+    k_ref, v_ref = kk.view(torch.int16).cpu().numpy().copy(), vv.view(torch.int16).cpu().numpy().copy()
+    root = wl.root_tokens(w, "cpu").cuda()
+    kv = wl.kv_lengths(w, "cpu").cuda()
+    kv_ref = kv.cpu().numpy().copy()
+    oracle = None
+    gen = torch.Generator().manual_seed(w.seed)
+    f32 = lambda t: t.float().cpu().numpy()
+    bits_to_f32 = lambda a: torch.from_numpy(a).view(torch.bfloat16).float().numpy()
+    grew = 0
+    for step in range(5):
+        logits = [wl.draft_logits(w, 10 * step + l, "cpu", peaked=True).cuda() for l in range(1, H + 1)]
+        o = oracle_tree(kw, tables, root, torch.from_numpy(kv_ref), logits, oracle)
+        oracle = o["oracle"]
+        g = gpu_tree(ctx, root, kv, logits)
+        if not (o["min_score_gap"] >= 1e-5 and o["stable"]):
+            pytest.skip("a draw put a decision within rounding of its threshold")
+        assert_tree_equal(g, o)
+        n_tree = o["n_tree"]
+        assert (kv_ref + n_tree <= cap).all()
+        # the model's K/V rows of the tree tokens, written on both sides at positions L_b .. L_b + N_b - 1
+        rows = []
+        for b in range(B):
+            for t in range(int(n_tree[b])):
+                pos = int(kv_ref[b]) + t
+                rows.append(int(tab[b, pos // page]) * page + pos % page if page else b * cap + pos)
+        idx = torch.tensor(rows, dtype=torch.int64)
+        for l in range(NL):
+            for cache, ref in ((kk, k_ref), (vv, v_ref)):
+                fresh = torch.randn((len(rows), w.kv_heads, w.head_dim), generator=gen).to(torch.bfloat16)
+                cache[l].view(-1, w.kv_heads, w.head_dim).index_copy_(0, idx.cuda(), fresh.cuda())
+                ref[l].reshape(-1, w.kv_heads, w.head_dim)[rows] = fresh.view(torch.int16).numpy()
+        d = g["dev"]
+        for l in range(NL):
+            q = torch.randn((B, w.max_tree, w.q_heads, w.head_dim), generator=gen).to(torch.bfloat16).cuda()
+            out = gpu_attention(ctx, w, q, kk[l], vv[l], table, num_pages, kv, d["anc"], d["n_tree"])
+            ref = tree_attention(f32(q), bits_to_f32(k_ref[l]), bits_to_f32(v_ref[l]), page, tab, kv_ref, o["anc"], n_tree)
+            got = to_f64(out)
+            for b in range(B):
+                nb = int(n_tree[b])
+                assert np.isnan(got[b, nb:]).all() and np.isfinite(got[b, :nb]).all()
+                assert np.max(np.abs(got[b, :nb] - ref[b, :nb])) <= attention_tolerance("bf16"), (step, l, b)
+        tl = torch.randn((B, w.max_tree, w.vocab), generator=gen).mul_(2.0).cuda()
+        wl.plant_acceptance(w, tl, o["tokens"], o["parent"], n_tree)
+        alen = torch.empty((B,), dtype=torch.int32, device="cuda")
+        apath = torch.empty((B, H + 1), dtype=torch.int32, device="cuda")
+        bonus = torch.empty((B,), dtype=torch.int32, device="cuda")
+        ctx.cast_accept(tl, B, d["tokens"], d["parent"], d["depth"], d["anc"], d["n_tree"], alen, apath, bonus)
+        nmax = int(n_tree.max())
+        ol, op, ob = greedy_accept(to_f64(tl[:, :nmax]), o["tokens"], o["parent"], n_tree, H)
+        assert np.array_equal(alen.cpu().numpy(), ol) and np.array_equal(apath.cpu().numpy(), op)
+        assert np.array_equal(bonus.cpu().numpy(), ob)
+        ctx.cast_compact_kv(kk, vv, B, NL, kk[0].numel() * kk.element_size(), w.kv_heads, w.head_dim, page, table,
+                            cap // (page or 1), num_pages, apath, alen, kv)
+        assert ctx.cast_poll_status()[0] == 0
+        k_ref, v_ref, kv_ref = compact_kv(k_ref, v_ref, page, tab, kv_ref, op, ol)
+        assert np.array_equal(kv.cpu().numpy(), kv_ref)
+        assert np.array_equal(kk.view(torch.int16).cpu().numpy(), k_ref)
+        assert np.array_equal(vv.view(torch.int16).cpu().numpy(), v_ref)
+        grew += int(ol.sum())
+        root = bonus.clone()
+    assert grew >= 5, "the loop accepted almost nothing: the planted acceptances did not take"
+    ctx.close()
+
+
 def test_attention_without_a_reserved_workspace_is_refused(binding):
     """Compute calls never allocate: a shape that needs a split workspace larger than what was reserved
     returns CAST_ERR_CAPACITY and launches nothing; after cast_reserve_attention the same call runs."""
