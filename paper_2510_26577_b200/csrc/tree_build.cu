@@ -28,6 +28,7 @@ namespace {
 struct ExpandParams {
   const void* logits;
   int V, K, W, H, P, layer, nchunks, chunk_elems;
+  int prefetch;  // the layer's logits are small enough to be worth asking for ahead of the dependency wait
   double* pool_score;
   int32_t* pool_token;
   int32_t* pool_parent;
@@ -486,7 +487,19 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
   };
   // Programmatic dependent launch: this grid may have become resident while the previous kernel of the
   // stream was still finishing. Nothing that kernel may have written is read above this line - not the
-  // logits either: in a serving loop the previous kernel is the draft model's, and it writes them.
+  // logits either: in a serving loop the previous kernel is the draft model's, and it writes them. What a
+  // CTA may do is ask the L2 cache for its chunk: a prefetch returns no value, and a line that the previous
+  // kernel writes afterwards is written in that same cache, so the loads below see it. When the previous kernel
+  // is not the one that writes the logits (layers queued back to back) the first pass then costs a round trip
+  // to L2 instead of one to HBM; rows that turn out not to exist are fetched for nothing, hence only for small
+  // layers.
+  if (p.prefetch) {
+    const char* cb = reinterpret_cast<const char*>(x + begin);
+    const int bytes = (end - begin) * (int)sizeof(T);
+#pragma unroll 1
+    for (int off = tid * 128; off < bytes; off += kSweepThreads * 128)
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(cb + off));
+  }
   grid_dependency_wait();
   grid_launch_dependents();  // the next grid may now take the SMs this one leaves idle
   load_pass(begin);
@@ -1206,6 +1219,9 @@ extern "C" cast_status cast_tree_expand(cast_ctx* c, int layer, const void* draf
   p.logits = draft_logits;
   p.V = V; p.K = c->cfg.top_k; p.W = c->W; p.H = c->cfg.max_depth; p.P = c->P; p.layer = layer;
   p.nchunks = nchunks; p.chunk_elems = chunk_elems;
+  // every row that can exist is asked for, whether the previous layer kept it or not: worth it while the
+  // whole layer is a small part of the L2 cache
+  p.prefetch = (double)rows * V * (dtype == CAST_F32 ? 4 : 2) <= 24e6;
   p.pool_score = c->pool_score; p.pool_token = c->pool_token; p.pool_parent = c->pool_parent;
   p.pool_depth = c->pool_depth; p.pool_kept = c->pool_kept; p.retained = c->retained;
   p.lsort = c->lsort; p.lscore = c->lscore;
