@@ -603,23 +603,31 @@ __device__ __forceinline__ void merge_rows_global(const TcParams& p, int b, int 
   const int lane = threadIdx.x & 31, wv = threadIdx.x >> 5, G = p.G;
   for (int rr = wv; rr < rows_here; rr += 8 * ROWS) {
     uint2 v[ROWS][SPL];
-    float wgt[ROWS], inv[ROWS];
+    float wgt[ROWS], inv[ROWS], msv[ROWS], lsv[ROWS];
     size_t orow[ROWS];
+    // every load of every row first, then the reductions (a reduction waits for its row's loads; with the next
+    // row's loads issued behind it the rows cost one round trip to L2 each, 6-7 us for eight)
 #pragma unroll
     for (int u = 0; u < ROWS; ++u) {
       const int r2 = rr + 8 * u;
       const int grow = row0 + (r2 < rows_here ? r2 : rr), tt = grow / G, hh = kvh * G + grow % G;
       const size_t pr = (((size_t)b * p.Hq + hh) * p.Ncap + tt) * p.nsplit_max;
       orow[u] = (((size_t)b * p.Ncap + tt) * p.Hq + hh) * kHD;
-      float ms = -INFINITY, ls = 0.f;  // lane s holds split s's (max, sum)
+      msv[u] = -INFINITY;  // lane s holds split s's (max, sum)
+      lsv[u] = 0.f;
       if (lane < nsplit) {
-        ms = __ldcg(p.part_ml + (pr + lane) * 2);
-        ls = __ldcg(p.part_ml + (pr + lane) * 2 + 1);
+        const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + (pr + lane) * 2));
+        msv[u] = ml.x;
+        lsv[u] = ml.y;
       }
 #pragma unroll
       for (int s2 = 0; s2 < SPL; ++s2)
         v[u][s2] = s2 < nsplit ? __ldcg(reinterpret_cast<const uint2*>(p.part_o + (pr + s2) * kHD + lane * 4))
                                : make_uint2(0u, 0u);
+    }
+#pragma unroll
+    for (int u = 0; u < ROWS; ++u) {
+      const float ms = msv[u], ls = lsv[u];
       float M = ms;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
@@ -1241,7 +1249,7 @@ tree_attn_tc_kernel(const TcParams p, const __grid_constant__ CUtensorMap map_k,
     }
     __syncthreads();
     if (*last_s) {
-      if (nsplit <= 2) merge_rows_global<8, 2>(p, b, kvh, grow0, rows_here, nsplit);
+      if (nsplit <= 2) merge_rows_global<4, 2>(p, b, kvh, grow0, rows_here, nsplit);
       else if (nsplit <= 4) merge_rows_global<4, 4>(p, b, kvh, grow0, rows_here, nsplit);
       else merge_rows_global<2, kMaxSplit>(p, b, kvh, grow0, rows_here, nsplit);
     }
