@@ -27,7 +27,7 @@ METRIC, UNIT = "tree_verify_tokens_per_s", "tokens/s"
 
 # DRAM bytes (read + write) of one tree_attn_tc_kernel launch from the ncu captures summarised
 # under profiles/ (same launch shape as one layer of the workload).
-NCU_ATTENTION_TRAFFIC = {"c2_llama8b": 9.29e6, "c3_llama8b_b16": 144.3e6, "c3_llama8b_b64": 598.4e6,
+NCU_ATTENTION_TRAFFIC = {"c2_llama8b": 9.29e6, "c3_llama8b_b16": 144.8e6, "c3_llama8b_b64": 598.4e6,
                          "c4_llama70b_n128": 179.5e6}
 
 
