@@ -263,6 +263,26 @@ extern "C" cast_status cast_accept(cast_ctx* c, const void* target_logits, cast_
   if (nchunks > kAcceptMaxChunks) nchunks = kAcceptMaxChunks;
   if (nchunks > V / 4096) nchunks = V / 4096;
   if (nchunks < 1) nchunks = 1;
+  // A CTA sweeps its chunk in rounds of kArgThreads * kArgUnroll vectors, each a full memory latency whether
+  // the round is full or not: among the counts within two of the one above, the one whose last round is
+  // fullest (V = 128 256 fp32 at batch 1: 8 chunks of 1.96 rounds instead of 10 of 1.57, 10.3 -> 9.4 us).
+  {
+    const int round_elems = kArgThreads * kArgUnroll * (dtype == CAST_F32 ? 4 : 8);
+    const int lo = (V + 32767) / 32768 > nchunks - 2 ? (V + 32767) / 32768 : nchunks - 2;
+    int hi = nchunks + 2 < kAcceptMaxChunks ? nchunks + 2 : kAcceptMaxChunks;
+    if (hi > V / 4096) hi = V / 4096;
+    const int n0 = nchunks;
+    long long best = -1;
+    for (int n = lo < 1 ? 1 : lo; n <= hi; ++n) {
+      const int ce = ((V + n - 1) / n + 7) / 8 * 8;
+      const long long padded = (long long)((ce + round_elems - 1) / round_elems) * round_elems * n;  // logits' worth of rounds
+      const int dist = n > n0 ? n - n0 : n0 - n, dist_best = nchunks > n0 ? nchunks - n0 : n0 - nchunks;
+      if (best < 0 || padded < best || (padded == best && dist <= dist_best)) {  // ties: nearest to n0, the larger of two
+        best = padded;
+        nchunks = n;
+      }
+    }
+  }
   int chunk_elems = (V + nchunks - 1) / nchunks;
   chunk_elems = (chunk_elems + 7) / 8 * 8;
   nchunks = (V + chunk_elems - 1) / chunk_elems;
