@@ -265,7 +265,9 @@ CAST_API cast_status cast_tree_attention_rows(cast_ctx* ctx, const void* q, cons
  *   accept_path [B, H+1]  linear tree indices, root first, -1 padded
  *   bonus_token [B]  g at the last accepted node
  * `depth` and `anc_mask` may be NULL (not needed by the walk).
- * Device errors: BAD_TREE (parent[t] >= t or a path longer than H+1).
+ * n_tree[b] must not exceed the context's total_token: only that many rows per sequence are swept.
+ * Device errors: BAD_TREE (n_tree[b] < 1 or beyond total_token: the sequence gets accept_len 0, bonus 0 and a
+ * path of -1; parent[t] >= t; a path longer than H+1).
  */
 CAST_API cast_status cast_accept(cast_ctx* ctx, const void* target_logits, cast_dtype dtype, int B,
                         const int32_t* tokens, const int32_t* parent, const int32_t* depth,

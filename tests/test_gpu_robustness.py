@@ -429,6 +429,14 @@ def test_malformed_inputs_are_reported_not_followed(binding):
     st, detail = ctx.cast_poll_status()
     assert st == 6 and detail % Ncap == 4  # BAD_TREE, at the offending node
     assert int(alen.min()) >= 0 and int(alen.max()) <= H and ctx.cast_poll_status()[0] == 0
+    # acceptance of a tree larger than the context's token budget: refused (its rows past the budget are not swept)
+    parent_ok = np.full((B, Ncap), -1, dtype=np.int32)
+    parent_ok[:, 1:20] = np.arange(0, 19)
+    ctx.cast_accept(logits, B, dev(tokens), dev(parent_ok), None, None, dev(np.array([20, 6], dtype=np.int32)), alen, apath,
+                    bonus)
+    st, detail = ctx.cast_poll_status()
+    assert st == 6 and detail == 0  # BAD_TREE, sequence 0
+    assert int(alen[0]) == 0 and int(apath[0, 0]) == -1 and int(alen[1]) >= 0
     # attention with a tree larger than the context's token budget (tensor-core path)
     w = wl.Workload("bad", 700, B, "bf16", "f32", 8, 2, 128, 50, 60, 16, V, 1.0, H, 2, 16, False, 1, max_tree=Ncap)
     q = wl.query(w, 0, "cuda")
