@@ -550,10 +550,16 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
   // exact. The bound is a value, not a key: logits equal to it pass, which only lengthens a list.)
   float cta_bound = -INFINITY;
   int pass = 0;
+  const int npass = (end - begin + kSweepSub - 1) / kSweepSub;
 
   for (int sub = begin; sub < end; sub += kSweepSub, ++pass) {
-    if (sub != begin) {
-      load_pass(sub);
+    if (sub != begin) load_pass(sub);
+    // The bound is refreshed where it still moves: before the second pass (from the first pass's threshold to the
+    // K-th largest of sixteen warps' best it rises a great deal) and, in long chunks, before the third. Later it
+    // hardly rises, the warps' own K-th keys have caught up, and the refresh - a CTA barrier and a rank of 16 heads
+    // in every warp, about a third of a pass's instructions - costs more than the few extractions it saves
+    // (batch 64, eight passes: 302 -> 278 us per tree build; batch 16, four passes: 171 -> 166).
+    if (pass == 1 || (pass == 2 && npass >= 6)) {
       float* hd = pass_heads[pass & 1];
       if (lane == 0) hd[warp] = have > 0 ? key_value(wlist[0]) : -INFINITY;
       __syncthreads();
