@@ -574,9 +574,16 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
       const float bnd = __shfl_sync(0xffffffffu, head, who != 0u ? __ffs(who) - 1 : 0);
       cta_bound = fmaxf(cta_bound, bnd);
     }
-    float tmax = xv[0];
+    // (the maxima of the four groups of eight slots on the way: the extraction below looks only into the groups
+    // that hold a passer)
+    float gmax[4];
 #pragma unroll
-    for (int i = 1; i < kSweepEpt; ++i) tmax = fmaxf(tmax, xv[i]);
+    for (int g = 0; g < 4; ++g) {
+      gmax[g] = xv[8 * g];
+#pragma unroll
+      for (int j = 1; j < 8; ++j) gmax[g] = fmaxf(gmax[g], xv[8 * g + j]);
+    }
+    const float tmax = fmaxf(fmaxf(gmax[0], gmax[1]), fmaxf(gmax[2], gmax[3]));
     const float t2 = tmax * kLog2eHi;
     if (t2 > M2) {
       s_run *= ex2f(M2 - t2);
@@ -636,40 +643,41 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
       thr_val = gate != 0ull ? fmaxf(key_value(gate), cta_bound) : cta_bound;
     }
     // Few logits pass, and against the shared thresholds most passes of a warp have none: one vote on the
-    // lanes' maxima settles that. Otherwise every lane marks its passing slots in a bit mask, the warp takes
-    // the union with one reduction and walks its set bits (a loop over the set bits only: unrolled over all 32
-    // slots, the tests and reconvergence points of the empty ones were most of the sweep's time); a slot's
-    // logit is picked out of the registers by a warp-uniform switch, takes the exact test on the full key and
-    // is appended to the warp's list.
+    // lanes' maxima settles that. Otherwise the same vote per group of eight slots, and in a group with a passer
+    // every lane marks its passing slots in a bit mask, the warp takes the union with one reduction and walks its
+    // set bits (a loop over the set bits only: unrolled over all slots, the tests and reconvergence points of the
+    // empty ones were most of the sweep's time); a slot's logit is picked out of the group's registers by three
+    // rounds of warp-uniform selects, takes the exact test on the full key and is appended to the warp's list.
+    // (The order of the appends does not matter: the list is ranked afterwards.)
     const int have0 = have;
     if (__any_sync(0xffffffffu, tmax >= thr_val)) {
-      unsigned mine_mask = 0u;
+      static_assert(kSweepEpt == 32, "four groups of eight slots");
 #pragma unroll
-      for (int i = 0; i < kSweepEpt; ++i) mine_mask |= (xv[i] >= thr_val) ? (1u << i) : 0u;
-      unsigned any_mask = __reduce_or_sync(0xffffffffu, mine_mask);
+      for (int g = 0; g < 4; ++g) {
+        if (!__any_sync(0xffffffffu, gmax[g] >= thr_val)) continue;
+        unsigned mine_mask = 0u;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) mine_mask |= (xv[8 * g + j] >= thr_val) ? (1u << j) : 0u;
+        unsigned any_mask = __reduce_or_sync(0xffffffffu, mine_mask);
 #pragma unroll 1
-      while (any_mask != 0u) {
-        const int i = __ffs(any_mask) - 1;
-        any_mask &= any_mask - 1u;
-        // xv[i] for a run-time i: five rounds of selects on the bits of i (registers cannot be indexed)
-        static_assert(kSweepEpt == 32, "five bits name a slot");
-        float s16[16], s8[8], s4[4];
-        const bool b0 = (i & 1) != 0, b1 = (i & 2) != 0, b2 = (i & 4) != 0, b3 = (i & 8) != 0, b4 = (i & 16) != 0;
+        while (any_mask != 0u) {
+          const int j = __ffs(any_mask) - 1;
+          any_mask &= any_mask - 1u;
+          const bool b0 = (j & 1) != 0, b1 = (j & 2) != 0, b2 = (j & 4) != 0;
+          float s4[4];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) s16[j] = b0 ? xv[2 * j + 1] : xv[2 * j];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) s8[j] = b1 ? s16[2 * j + 1] : s16[2 * j];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) s4[j] = b2 ? s8[2 * j + 1] : s8[2 * j];
-        const float s2a = b3 ? s4[1] : s4[0], s2b = b3 ? s4[3] : s4[2];
-        const float xi = b4 ? s2b : s2a;
-        const int id = sub + ((i / VEC) * kSweepThreads + tid) * VEC + (i % VEC);
-        const unsigned long long key = make_key(xi, id);
-        const bool ok = xi >= thr_val && id < end && key > gate;
-        const unsigned m = __ballot_sync(0xffffffffu, ok);
-        const int pos = have + __popc(m & ((1u << lane) - 1u));
-        if (ok && pos < kWarpCap) wlist[pos] = key;
-        have += __popc(m);
+          for (int q = 0; q < 4; ++q) s4[q] = b0 ? xv[8 * g + 2 * q + 1] : xv[8 * g + 2 * q];
+          const float s2a = b1 ? s4[1] : s4[0], s2b = b1 ? s4[3] : s4[2];
+          const float xi = b2 ? s2b : s2a;
+          const int i = 8 * g + j;
+          const int id = sub + ((i / VEC) * kSweepThreads + tid) * VEC + (i % VEC);
+          const unsigned long long key = make_key(xi, id);
+          const bool ok = xi >= thr_val && id < end && key > gate;
+          const unsigned m = __ballot_sync(0xffffffffu, ok);
+          const int pos = have + __popc(m & ((1u << lane) - 1u));
+          if (ok && pos < kWarpCap) wlist[pos] = key;
+          have += __popc(m);
+        }
       }
     }
     __syncwarp();
@@ -706,6 +714,17 @@ __global__ void __launch_bounds__(kSweepThreads, MINB) expand_kernel(const Expan
       __syncwarp();
       if (lane < n) wlist[lane] = mine;
       have = n;
+      __syncwarp();
+    } else if (have == have0 + 1) {
+      // one newcomer (the usual case): the old entries are in order, so it is an insertion - the newcomer's rank is
+      // the number of larger keys (one vote), the smaller ones move down one place, the K-th of K falls off
+      const unsigned long long nk = wlist[have0];
+      const unsigned long long mine = lane < have0 ? wlist[lane] : 0ull;
+      const int rnk = __popc(__ballot_sync(0xffffffffu, lane < have0 && mine > nk));
+      __syncwarp();
+      if (lane < have0 && lane >= rnk && lane + 1 < K) wlist[lane + 1] = mine;
+      if (lane == 0 && rnk < K) wlist[rnk] = nk;
+      have = have < K ? have : K;
       __syncwarp();
     } else if (have > have0) {
       // exact order of the list (old entries and newcomers, at most 64): rank by counting, keys are distinct
