@@ -178,6 +178,17 @@ __device__ __forceinline__ bool take_ticket(int32_t* counter, int expected, int*
 // Up to this many sequences the one-CTA tail is faster than a second ticket.
 constexpr int kTailSingleMaxB = 4;
 
+// a / b for 0 <= a < 2^20 and 1 <= b <= 2^10 through the fp32 reciprocal (inv_b = 1.f / b) with one correction step:
+// the integer division by a run-time divisor is some twenty instructions, and the ranking below does several per
+// thread in a phase whose time is what its instructions take to issue.
+__device__ __forceinline__ int div_small(int a, int b, float inv_b) {
+  int q = (int)((float)a * inv_b);
+  const int r = a - q * b;
+  q += (r >= b) ? 1 : 0;
+  q -= (r < 0) ? 1 : 0;
+  return q;
+}
+
 // Candidates Algorithm 1 looks at: the first n of the sorted list.
 __device__ __forceinline__ int tail_width(const ExpandParams& p, int n_prev) {
   const int Ni = n_prev * p.K;
@@ -198,12 +209,13 @@ __device__ __forceinline__ void tail_rank(const ExpandParams& p, int b_begin, in
   int* tk = reinterpret_cast<int*>(scratch + 8192);             // 1024 tokens
   int* rank_s = reinterpret_cast<int*>(scratch + 12288);        // 1024 ranks
   const int group = 1024 / Ni;                                  // sequences ranked per pass
+  const float inv_Ni = 1.f / (float)Ni, inv_K = 1.f / (float)K;
 #pragma unroll 1
   for (int b0 = 0; b0 < b_count; b0 += group) {
     const int nb = (b_count - b0) < group ? (b_count - b0) : group;
     const int tot = nb * Ni;
     for (int i = tid; i < tot; i += nt) {
-      const int bl = i / Ni, ci = i - bl * Ni;  // (the divisions hide behind the loads)
+      const int bl = div_small(i, Ni, inv_Ni), ci = i - bl * Ni;
       const size_t o = (size_t)(b_begin + b0 + bl) * P + base + ci;
       sc[i] = __ldcg(p.pool_score + o);
       tk[i] = __ldcg(p.pool_token + o);
@@ -217,6 +229,7 @@ __device__ __forceinline__ void tail_rank(const ExpandParams& p, int b_begin, in
     // costs is the warp instructions it issues, so no lane works on a row or a step that does not exist - two
     // per thread in step so that their shared-memory loads overlap; the counts meet in shared memory.
     const int pairs = tot * n_prev;
+    const float inv_tot = 1.f / (float)tot;
     int h0 = 1;
     while (2 * h0 - 1 < K) h0 <<= 1;  // the search's first stride: positions up to 2 h0 - 1 >= K are reachable
 #pragma unroll 1
@@ -229,10 +242,12 @@ __device__ __forceinline__ void tail_rank(const ExpandParams& p, int b_begin, in
         const int it = it0 + q * nt;
         act[q] = it < pairs;
         const int itc = act[q] ? it : 0;
-        ii[q] = itc / n_prev;              // the candidate (index over the sequences of this pass)
-        rs[q] = itc - ii[q] * n_prev;      // the row searched
-        const int ci = ii[q] % Ni;
-        r1[q] = ci / K;                    // the candidate's own row
+        // (row-major: the lanes of a warp search one row for consecutive candidates, so their shared-memory loads
+        // fall on that row's K entries and their counts go to different words)
+        rs[q] = div_small(itc, tot, inv_tot);    // the row searched
+        ii[q] = itc - rs[q] * tot;               // the candidate (index over the sequences of this pass)
+        const int ci = ii[q] - div_small(ii[q], Ni, inv_Ni) * Ni;
+        r1[q] = div_small(ci, K, inv_K);         // the candidate's own row
         rowb[q] = ii[q] - ci + rs[q] * K;  // first child of the searched row, same sequence
         s2[q] = sc[ii[q]];
         t2[q] = tk[ii[q]];
@@ -257,7 +272,7 @@ __device__ __forceinline__ void tail_rank(const ExpandParams& p, int b_begin, in
     __syncthreads();
 #pragma unroll 1
     for (int i = tid; i < tot; i += nt) {
-      const int bl = i / Ni, ci = i - bl * Ni, rank = rank_s[i];
+      const int bl = div_small(i, Ni, inv_Ni), ci = i - bl * Ni, rank = rank_s[i];
       const int bg = b_begin + b0 + bl;
       const double s = sc[i];
       const size_t o = (size_t)bg * P + base + rank;
